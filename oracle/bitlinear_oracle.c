@@ -1,0 +1,321 @@
+/*
+ * BitLinear forward (BitNet b1.58) -- CPU ORACLE.  TEST INFRASTRUCTURE ONLY.
+ *
+ * This file is the slow, plain definition of what the BitLinear forward
+ * computes.  It exists so that tests can compare the CUDA library against it
+ * and so that the benchmark can time a CPU baseline.  Nothing in the product
+ * path may call it, and it shares no code, header, table or constant with the
+ * CUDA kernels.
+ *
+ * What follows the paper, and where:
+ *   - absmean weight quantisation  ............ Section 2, Eq. 1, Eq. 2, Eq. 3
+ *   - per-token symmetric activation quantisation to [-Qb, Qb], no zero point
+ *     ........................................... Section 2, paragraph after Eq. 3
+ *   - integer-only matrix product ................ Section 1 ("only involves integer addition")
+ *   - 2-bit storage of ternary weights ........... Section 3, "Memory and Latency"
+ *
+ * Readings taken where the paper is silent (each repeated next to its code):
+ *   R1  eps enters additively in Eq. 1 and is a caller argument.
+ *   R2  gamma (Eq. 3) is the order-free EXACT sum of |W| in 2^-64 fixed point
+ *       (each term truncated to a multiple of 2^-64), divided in double.
+ *   R3  round() is round-half-to-even.
+ *   R4  Qb = 127; clip to [-127, 127].
+ *   R5  beta_t = max_k |x_tk| over the K features of token t.
+ *   R6  beta_t is clamped below by 1e-5f; s_t = 127/beta_t is formed once and
+ *       every element takes ONE fp32 multiply before rounding.
+ *   R7  dequantisation scale is (gamma*beta_t)/127 with the plain gamma.
+ *   R8  output is round-to-nearest-even bfloat16 of float(acc)*scale.
+ *   R9  storage layout of the 2-bit codes (see oracle_pack_weights).
+ *   R10 one gamma per weight matrix.
+ *
+ * Parity pins (tests/test_oracle_pins.py): hand-worked cases for Eq. 1-3 and
+ * the activation quantiser including rounding ties, closed-form Gaussian
+ * statistics, textbook int32 matmul via numpy, brute-force double-precision
+ * matmul of the dequantised operands, algebraic invariants, exactness of gamma
+ * against math.fsum, pack/unpack round trip, and a pure-Python restatement
+ * (oracle/np_restatement.py) on small shapes.
+ * Parity unpinned: the bf16 output tolerance itself (1e-2 rel / 1e-3 abs) is
+ * not fixed by the paper.
+ *
+ * Build for parity:  gcc -O2 -fno-fast-math -ffp-contract=off -shared -fPIC
+ * Build for timing:  same source with -O3 -fopenmp (outer loops only).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <string.h>
+#include <fenv.h>
+
+#define ORACLE_OK 0
+#define ORACLE_ERR_ARG -1
+#define ORACLE_ERR_RANGE -8 /* non-finite value or |w| >= 2^24 */
+
+#define QB 127          /* R4 */
+#define BETA_FLOOR 1e-5f /* R6 */
+
+/* ---------- bfloat16 helpers (bf16 = upper 16 bits of an IEEE fp32) ---------- */
+
+static float bf16_to_float(uint16_t h)
+{
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+/* R8: round-to-nearest-even from fp32 to bf16 (finite inputs). */
+static uint16_t float_to_bf16_rne(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    uint32_t lower = u & 0xFFFFu;
+    uint32_t upper = u >> 16;
+    if (lower > 0x8000u || (lower == 0x8000u && (upper & 1u)))
+        upper += 1u;
+    return (uint16_t)upper;
+}
+
+/* ---------- Eq. 3 with reading R2: exact sum of |W| ---------- */
+
+/*
+ * floor(|v| * 2^64) as an unsigned 128-bit integer.  An fp32 magnitude is
+ * sig * 2^(e-150) with a 24-bit integer significand, so the scaled value is
+ * sig * 2^(e-86): a left shift when e >= 86, a truncating right shift below.
+ * Caller guarantees e < 151, i.e. |v| < 2^24.
+ */
+static unsigned __int128 fix64_of_magnitude(uint32_t magnitude_bits)
+{
+    uint32_t e = magnitude_bits >> 23;
+    uint32_t frac = magnitude_bits & 0x7FFFFFu;
+    uint32_t sig = e ? (frac | 0x800000u) : frac; /* subnormals: no hidden bit */
+    int shift = (int)(e ? e : 1u) - 86;
+    if (shift >= 0)
+        return ((unsigned __int128)sig) << shift;
+    if (-shift >= 24)
+        return 0;
+    return (unsigned __int128)(sig >> (-shift));
+}
+
+int oracle_absmean(const float *W, int64_t N, int64_t K, float *gamma)
+{
+    if (!W || !gamma || N <= 0 || K <= 0)
+        return ORACLE_ERR_ARG;
+    unsigned __int128 total = 0;
+    for (int64_t i = 0; i < N * K; ++i) {
+        uint32_t u;
+        memcpy(&u, &W[i], sizeof u);
+        u &= 0x7FFFFFFFu; /* |W_ij| */
+        if ((u >> 23) >= 151u)
+            return ORACLE_ERR_RANGE;
+        total += fix64_of_magnitude(u);
+    }
+    uint64_t hi = (uint64_t)(total >> 64);
+    uint64_t lo = (uint64_t)total;
+    double sum = ((double)hi * 18446744073709551616.0 + (double)lo) * (1.0 / 18446744073709551616.0);
+    double mean = sum / (double)(N * K);
+    *gamma = (float)mean;
+    return ORACLE_OK;
+}
+
+/* ---------- Eq. 1 and Eq. 2 ---------- */
+
+/* Eq. 2: RoundClip(x, a, b) = max(a, min(b, round(x))), round = half-to-even (R3). */
+static int round_clip(float x, int a, int b)
+{
+    float r = rintf(x); /* FE_TONEAREST: ties to even */
+    if (r < (float)a) return a;
+    if (r > (float)b) return b;
+    return (int)r;
+}
+
+/*
+ * Eq. 1: W~ = RoundClip(W / (gamma + eps), -1, 1), gamma from Eq. 3.
+ * T receives the ternary values row-major [N][K].
+ */
+int oracle_quantize_weights(const float *W, int64_t N, int64_t K, float eps, int8_t *T, float *gamma)
+{
+    if (!T)
+        return ORACLE_ERR_ARG;
+    int rc = oracle_absmean(W, N, K, gamma);
+    if (rc != ORACLE_OK)
+        return rc;
+    float denom = *gamma + eps; /* R1 */
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t k = 0; k < K; ++k)
+            T[n * K + k] = (int8_t)round_clip(W[n * K + k] / denom, -1, 1);
+    return ORACLE_OK;
+}
+
+/* ---------- R9: 2-bit storage ---------- */
+
+static int64_t padded_K(int64_t K) { return (K + 127) / 128 * 128; }
+
+int64_t oracle_packed_bytes(int64_t N, int64_t K)
+{
+    if (N <= 0 || K <= 0 || (N % 16) != 0)
+        return -1;
+    return N * padded_K(K) / 4;
+}
+
+/*
+ * Where weight (n, k) lives.  The matrix is cut into tiles of 16 rows by 128
+ * columns, 512 bytes each, stored one after another with the column-tile index
+ * running fastest.  A tile is 128 little-endian 32-bit words.  Within a tile,
+ * with r = n mod 16 and c = k mod 128:
+ *     word  = 4 * (4 * (r mod 8) + c / 32) + (c mod 32) / 8
+ *     field = 2 * ((c mod 8) / 4) + r / 8          (0..3)
+ *     byte  = c mod 4
+ * and the code occupies bits [8*byte + 2*field, 8*byte + 2*field + 1] of that
+ * word.  The stored code is t + 1, so it is 0, 1 or 2; 3 never appears.
+ * Columns K..padded_K(K)-1 hold code 1 (weight zero).
+ */
+static void locate(int64_t n, int64_t k, int64_t Kp, int64_t *word_index, int *bit)
+{
+    int64_t tile = (n / 16) * (Kp / 128) + (k / 128);
+    int r = (int)(n % 16), c = (int)(k % 128);
+    int word = 4 * (4 * (r % 8) + c / 32) + (c % 32) / 8;
+    int field = 2 * ((c % 8) / 4) + r / 8;
+    int byte = c % 4;
+    *word_index = tile * 128 + word;
+    *bit = 8 * byte + 2 * field;
+}
+
+int oracle_pack_weights(const int8_t *T, int64_t N, int64_t K, uint8_t *packed)
+{
+    if (!T || !packed || N <= 0 || K <= 0 || (N % 16) != 0)
+        return ORACLE_ERR_ARG;
+    int64_t Kp = padded_K(K);
+    memset(packed, 0, (size_t)(N * Kp / 4));
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t k = 0; k < Kp; ++k) {
+            int t = (k < K) ? T[n * K + k] : 0;
+            if (t < -1 || t > 1)
+                return ORACLE_ERR_ARG;
+            uint32_t code = (uint32_t)(t + 1);
+            int64_t w;
+            int bit;
+            locate(n, k, Kp, &w, &bit);
+            /* little-endian 32-bit word: bit b of the word is bit (b mod 8) of byte (b / 8) */
+            packed[w * 4 + bit / 8] |= (uint8_t)(code << (bit % 8));
+        }
+    }
+    return ORACLE_OK;
+}
+
+int oracle_unpack_weights(const uint8_t *packed, int64_t N, int64_t K, int8_t *T)
+{
+    if (!T || !packed || N <= 0 || K <= 0 || (N % 16) != 0)
+        return ORACLE_ERR_ARG;
+    int64_t Kp = padded_K(K);
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            int64_t w;
+            int bit;
+            locate(n, k, Kp, &w, &bit);
+            int code = (packed[w * 4 + bit / 8] >> (bit % 8)) & 3;
+            if (code == 3)
+                return ORACLE_ERR_ARG;
+            T[n * K + k] = (int8_t)(code - 1);
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* ---------- activation quantiser (Section 2, after Eq. 3; R4, R5, R6) ---------- */
+
+int oracle_quantize_acts(const uint16_t *X_bf16, int64_t M, int64_t K,
+                         int8_t *Xq, float *beta, int32_t *rowsum)
+{
+    if (!X_bf16 || !Xq || !beta || !rowsum || M < 0 || K <= 0)
+        return ORACLE_ERR_ARG;
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        float amax = 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            float a = fabsf(bf16_to_float(X_bf16[t * K + k]));
+            if (a > amax) amax = a;
+        }
+        float b = amax > BETA_FLOOR ? amax : BETA_FLOOR; /* R6 */
+        float s = (float)QB / b;                          /* one IEEE divide per token */
+        int32_t sum = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            float scaled = bf16_to_float(X_bf16[t * K + k]) * s; /* one multiply per element */
+            int q = round_clip(scaled, -QB, QB);
+            Xq[t * K + k] = (int8_t)q;
+            sum += q;
+        }
+        beta[t] = b;
+        rowsum[t] = sum;
+    }
+    return ORACLE_OK;
+}
+
+/* ---------- integer matrix product: the plain definition ---------- */
+
+/* acc[t][n] = sum_k Xq[t][k] * T[n][k], exact in int32 (|acc| <= 127*K). */
+int oracle_matmul_i32(const int8_t *Xq, const int8_t *T, int64_t M, int64_t K, int64_t N, int32_t *acc)
+{
+    if (!Xq || !T || !acc || M < 0 || K <= 0 || N <= 0)
+        return ORACLE_ERR_ARG;
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        for (int64_t n = 0; n < N; ++n) {
+            int32_t s = 0;
+            for (int64_t k = 0; k < K; ++k)
+                s += (int32_t)Xq[t * K + k] * (int32_t)T[n * K + k];
+            acc[t * N + n] = s;
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* ---------- dequantisation (R7, R8) ---------- */
+
+int oracle_dequant(const int32_t *acc, const float *beta, float gamma, int64_t M, int64_t N, uint16_t *Y_bf16)
+{
+    if (!acc || !beta || !Y_bf16 || M < 0 || N <= 0)
+        return ORACLE_ERR_ARG;
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        float scale = (gamma * beta[t]) / (float)QB;
+        for (int64_t n = 0; n < N; ++n)
+            Y_bf16[t * N + n] = float_to_bf16_rne((float)acc[t * N + n] * scale);
+    }
+    return ORACLE_OK;
+}
+
+/* ---------- the whole forward for an already ternarised weight matrix ---------- */
+
+/*
+ * Y = dequant( quantize_acts(X) x T^T ).  Scratch buffers are the caller's:
+ * Xq [M*K], beta [M], rowsum [M], acc [M*N].
+ */
+int oracle_forward(const int8_t *T, float gamma, const uint16_t *X_bf16,
+                   int64_t M, int64_t K, int64_t N,
+                   int8_t *Xq, float *beta, int32_t *rowsum, int32_t *acc, uint16_t *Y_bf16)
+{
+    int rc = oracle_quantize_acts(X_bf16, M, K, Xq, beta, rowsum);
+    if (rc != ORACLE_OK) return rc;
+    rc = oracle_matmul_i32(Xq, T, M, K, N, acc);
+    if (rc != ORACLE_OK) return rc;
+    return oracle_dequant(acc, beta, gamma, M, N, Y_bf16);
+}
+
+int oracle_num_threads(void)
+{
+#ifdef _OPENMP
+    extern int omp_get_max_threads(void);
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}

@@ -1,0 +1,177 @@
+"""ctypes front end of the C oracle (oracle/bitlinear_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests, by the smoke check and by the
+benchmark's CPU-baseline leg.  All arrays are numpy; bfloat16 travels as
+uint16 bit patterns.  Two builds of the same source exist: "parity" (-O2, no
+contraction, single thread) and "timing" (-O3 -fopenmp, outer loops parallel).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from pathlib import Path
+
+import numpy as np
+
+_HERE = Path(__file__).resolve().parent
+_SRC = _HERE / "bitlinear_oracle.c"
+_FLAGS = {
+    "parity": ["-O2", "-fno-fast-math", "-ffp-contract=off"],
+    "timing": ["-O3", "-fno-fast-math", "-ffp-contract=off", "-fopenmp"],
+}
+
+
+def _lib_path(kind: str) -> Path:
+    return _HERE / f"libbitlinear_oracle_{kind}.so"
+
+
+def build_oracle(kind: str = "parity", force: bool = False) -> Path:
+    """Compile the C oracle with gcc; returns the shared object's path."""
+    out = _lib_path(kind)
+    if not force and out.exists() and out.stat().st_mtime >= _SRC.stat().st_mtime:
+        return out
+    tmp = out.with_suffix(f".tmp{os.getpid()}.so")
+    cmd = ["gcc", *_FLAGS[kind], "-std=gnu11", "-shared", "-fPIC", "-o", str(tmp), str(_SRC), "-lm"]
+    subprocess.run(cmd, check=True)
+    os.replace(tmp, out)
+    return out
+
+
+_i64 = ctypes.c_int64
+_p = ctypes.c_void_p
+
+
+class Oracle:
+    """Thin numpy wrapper; every method mirrors one C function."""
+
+    def __init__(self, kind: str = "parity"):
+        self.kind = kind
+        self.lib = ctypes.CDLL(str(build_oracle(kind)))
+        L = self.lib
+        L.oracle_absmean.argtypes = [_p, _i64, _i64, _p]
+        L.oracle_quantize_weights.argtypes = [_p, _i64, _i64, ctypes.c_float, _p, _p]
+        L.oracle_packed_bytes.argtypes = [_i64, _i64]
+        L.oracle_packed_bytes.restype = _i64
+        L.oracle_pack_weights.argtypes = [_p, _i64, _i64, _p]
+        L.oracle_unpack_weights.argtypes = [_p, _i64, _i64, _p]
+        L.oracle_quantize_acts.argtypes = [_p, _i64, _i64, _p, _p, _p]
+        L.oracle_matmul_i32.argtypes = [_p, _p, _i64, _i64, _i64, _p]
+        L.oracle_dequant.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p]
+        L.oracle_forward.argtypes = [_p, ctypes.c_float, _p, _i64, _i64, _i64, _p, _p, _p, _p, _p]
+        L.oracle_num_threads.restype = ctypes.c_int
+
+    @staticmethod
+    def _c(a: np.ndarray, dtype) -> np.ndarray:
+        a = np.ascontiguousarray(a, dtype=dtype)
+        return a
+
+    @staticmethod
+    def _ptr(a: np.ndarray):
+        return a.ctypes.data_as(_p)
+
+    def _check(self, rc: int, what: str):
+        if rc != 0:
+            raise ValueError(f"oracle {what} failed with code {rc}")
+
+    def num_threads(self) -> int:
+        return int(self.lib.oracle_num_threads())
+
+    def absmean(self, W: np.ndarray) -> np.float32:
+        W = self._c(W, np.float32)
+        N, K = W.shape
+        g = np.zeros(1, np.float32)
+        self._check(self.lib.oracle_absmean(self._ptr(W), N, K, self._ptr(g)), "absmean")
+        return g[0]
+
+    def quantize_weights(self, W: np.ndarray, eps: float = 1e-5):
+        """Eq. 1-3 -> (T int8 [N,K] in {-1,0,1}, gamma float32)."""
+        W = self._c(W, np.float32)
+        N, K = W.shape
+        T = np.empty((N, K), np.int8)
+        g = np.zeros(1, np.float32)
+        rc = self.lib.oracle_quantize_weights(self._ptr(W), N, K, ctypes.c_float(eps), self._ptr(T), self._ptr(g))
+        self._check(rc, "quantize_weights")
+        return T, g[0]
+
+    def packed_bytes(self, N: int, K: int) -> int:
+        return int(self.lib.oracle_packed_bytes(N, K))
+
+    def pack_weights(self, T: np.ndarray) -> np.ndarray:
+        T = self._c(T, np.int8)
+        N, K = T.shape
+        nbytes = self.packed_bytes(N, K)
+        if nbytes < 0:
+            raise ValueError("N must be a positive multiple of 16")
+        out = np.empty(nbytes, np.uint8)
+        self._check(self.lib.oracle_pack_weights(self._ptr(T), N, K, self._ptr(out)), "pack_weights")
+        return out
+
+    def unpack_weights(self, packed: np.ndarray, N: int, K: int) -> np.ndarray:
+        packed = self._c(packed, np.uint8)
+        T = np.empty((N, K), np.int8)
+        self._check(self.lib.oracle_unpack_weights(self._ptr(packed), N, K, self._ptr(T)), "unpack_weights")
+        return T
+
+    def quantize_acts(self, X_bf16_bits: np.ndarray):
+        """-> (Xq int8 [M,K], beta float32 [M], rowsum int32 [M])."""
+        X = self._c(X_bf16_bits, np.uint16)
+        M, K = X.shape
+        Xq = np.empty((M, K), np.int8)
+        beta = np.empty(M, np.float32)
+        rs = np.empty(M, np.int32)
+        rc = self.lib.oracle_quantize_acts(self._ptr(X), M, K, self._ptr(Xq), self._ptr(beta), self._ptr(rs))
+        self._check(rc, "quantize_acts")
+        return Xq, beta, rs
+
+    def matmul_i32(self, Xq: np.ndarray, T: np.ndarray) -> np.ndarray:
+        Xq = self._c(Xq, np.int8)
+        T = self._c(T, np.int8)
+        M, K = Xq.shape
+        N, K2 = T.shape
+        assert K == K2
+        acc = np.empty((M, N), np.int32)
+        self._check(self.lib.oracle_matmul_i32(self._ptr(Xq), self._ptr(T), M, K, N, self._ptr(acc)), "matmul_i32")
+        return acc
+
+    def dequant(self, acc: np.ndarray, beta: np.ndarray, gamma) -> np.ndarray:
+        acc = self._c(acc, np.int32)
+        beta = self._c(beta, np.float32)
+        M, N = acc.shape
+        Y = np.empty((M, N), np.uint16)
+        rc = self.lib.oracle_dequant(self._ptr(acc), self._ptr(beta), ctypes.c_float(float(gamma)), M, N, self._ptr(Y))
+        self._check(rc, "dequant")
+        return Y
+
+    def forward(self, T: np.ndarray, gamma, X_bf16_bits: np.ndarray, return_all: bool = False):
+        """Whole forward for ternary T [N,K]; returns bf16 bit patterns [M,N]."""
+        T = self._c(T, np.int8)
+        X = self._c(X_bf16_bits, np.uint16)
+        N, K = T.shape
+        M, K2 = X.shape
+        assert K == K2
+        Xq = np.empty((M, K), np.int8)
+        beta = np.empty(M, np.float32)
+        rs = np.empty(M, np.int32)
+        acc = np.empty((M, N), np.int32)
+        Y = np.empty((M, N), np.uint16)
+        rc = self.lib.oracle_forward(self._ptr(T), ctypes.c_float(float(gamma)), self._ptr(X), M, K, N,
+                                     self._ptr(Xq), self._ptr(beta), self._ptr(rs), self._ptr(acc), self._ptr(Y))
+        self._check(rc, "forward")
+        if return_all:
+            return Y, acc, Xq, beta, rs
+        return Y
+
+
+_cache: dict[str, Oracle] = {}
+
+
+def load_oracle(kind: str = "parity") -> Oracle:
+    if kind not in _cache:
+        _cache[kind] = Oracle(kind)
+    return _cache[kind]
+
+
+def bf16_bits_to_float32(bits: np.ndarray) -> np.ndarray:
+    """Exact widening of bf16 bit patterns to float32 (a reinterpretation)."""
+    return (np.asarray(bits, np.uint16).astype(np.uint32) << 16).view(np.float32)

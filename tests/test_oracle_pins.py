@@ -1,0 +1,274 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix.
+
+None of these tests touches the CUDA library.  Each pin is chosen so that a
+plausible mistake in the oracle (wrong tie rule, eps dropped, transposed
+operand, wrong scale, wrong storage position) makes at least one of them fail.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from conftest import f32_to_bf16_bits
+from oracle import np_restatement as R
+from oracle.oracle import bf16_bits_to_float32
+
+
+def bits_to_f32(b):
+    return bf16_bits_to_float32(b)
+
+
+# ---------------------------------------------------------------- hand cases (Eq. 1-3, Section 2)
+
+def test_hand_cases_weights(oracle, golden):
+    for case in golden["weights"]:
+        W = np.array(case["W"], np.float32)
+        T, g = oracle.quantize_weights(W, case["eps"])
+        assert g == np.float32(case["gamma"]), case["citation"]
+        assert T.tolist() == case["T"], case["citation"]
+
+
+def test_hand_cases_activations(oracle, golden):
+    for case in golden["activations"]:
+        x = f32_to_bf16_bits(np.array([case["x"]], np.float32))
+        q, beta, rs = oracle.quantize_acts(x)
+        assert q[0].tolist() == case["q"], case["citation"]
+        assert beta[0] == np.float32(case["beta"]), case["citation"]
+        assert int(rs[0]) == case["rowsum"], case["citation"]
+
+
+def test_hand_cases_forward(oracle, golden):
+    for case in golden["forward"]:
+        T = np.array(case["T"], np.int8)
+        x = f32_to_bf16_bits(np.array([case["x"]], np.float32))
+        Y, acc, Xq, beta, rs = oracle.forward(T, case["gamma"], x, return_all=True)
+        assert acc[0].tolist() == case["acc"], case["citation"]
+        assert bits_to_f32(Y)[0].tolist() == case["y"], case["citation"]
+
+
+def test_zero_token_gives_zero_output(oracle):
+    T = np.array([[1, -1, 0, 1]] * 16, np.int8)
+    x = np.zeros((1, 4), np.uint16)
+    Y = oracle.forward(T, 0.3, x)
+    assert np.all(bits_to_f32(Y) == 0.0)
+
+
+def test_hand_cases_layout(oracle, golden):
+    lay = golden["layout"]
+    N, K = lay["N"], lay["K"]
+    base = oracle.pack_weights(np.zeros((N, K), np.int8))
+    assert base.size == N * K // 4 and np.all(base == 0x55)
+    for c in lay["cases"]:
+        T = np.zeros((N, K), np.int8)
+        T[c["n"], c["k"]] = 1
+        p = oracle.pack_weights(T)
+        diff = np.nonzero(p != 0x55)[0]
+        assert diff.tolist() == [c["byte_index"]], (c, lay["citation"])
+        assert int(p[c["byte_index"]]) == c["byte_value"], c
+
+
+# ---------------------------------------------------------------- value sets
+
+@pytest.mark.parametrize("seed", [0, 1])
+def test_value_sets(oracle, seed):
+    rng = np.random.default_rng(seed)
+    W = (rng.standard_normal((64, 320)) * 0.02).astype(np.float32)
+    T, g = oracle.quantize_weights(W)
+    assert set(np.unique(T).tolist()) <= {-1, 0, 1}
+    p = oracle.pack_weights(T)
+    codes = np.stack([(p >> s) & 3 for s in (0, 2, 4, 6)])
+    assert codes.max() <= 2, "code 3 must never be stored"
+    x = rng.standard_normal((5, 320)).astype(np.float32)
+    xbits = ((x.view(np.uint32) >> 16).astype(np.uint16))  # truncation to bf16 is fine for a value-set check
+    q, beta, rs = oracle.quantize_acts(xbits)
+    assert q.min() >= -127 and q.max() <= 127
+    assert np.all(np.abs(q).max(axis=1) == 127), "the absmax element of each token maps to +-127"
+    assert np.array_equal(rs, q.astype(np.int64).sum(axis=1).astype(np.int32))
+    xf = bits_to_f32(xbits)
+    assert np.array_equal(beta, np.abs(xf).max(axis=1))
+
+
+def test_padding_columns_hold_code_one(oracle):
+    rng = np.random.default_rng(3)
+    N, K = 32, 192  # padded to 256
+    T = rng.integers(-1, 2, (N, K)).astype(np.int8)
+    p = oracle.pack_weights(T)
+    assert p.size == N * 256 // 4
+    Tfull = np.concatenate([T, np.zeros((N, 64), np.int8)], axis=1)
+    assert np.array_equal(p, oracle.pack_weights(Tfull))
+
+
+# ---------------------------------------------------------------- closed forms on Gaussian input
+
+def test_gaussian_closed_forms(oracle):
+    sigma = 0.02
+    rng = np.random.default_rng(0)
+    N, K = 1024, 1536
+    W = (rng.standard_normal((N, K)) * sigma).astype(np.float32)
+    T, g = oracle.quantize_weights(W)
+    n = N * K
+    # E|w| = sigma*sqrt(2/pi); std of the sample mean = sigma*sqrt(1-2/pi)/sqrt(n)
+    expect_gamma = sigma * math.sqrt(2 / math.pi)
+    assert abs(float(g) - expect_gamma) < 5 * sigma * math.sqrt(1 - 2 / math.pi) / math.sqrt(n)
+    # t = 0  <=>  |w| < gamma/2
+    p0 = math.erf(0.5 * math.sqrt(2 / math.pi) / math.sqrt(2))
+    assert abs(p0 - 0.310064) < 1e-5
+    tol = 4 * math.sqrt(0.25 / n) + 2e-4  # binomial noise + the sampling noise of gamma itself
+    assert abs((T == 0).mean() - p0) < tol
+    assert abs((T == 1).mean() - (1 - p0) / 2) < tol
+    assert abs((T == -1).mean() - (1 - p0) / 2) < tol
+
+
+# ---------------------------------------------------------------- textbook reductions
+
+@pytest.mark.parametrize("M,K,N", [(1, 64, 16), (7, 200, 48), (33, 1536, 64)])
+def test_matmul_equals_numpy(oracle, M, K, N):
+    rng = np.random.default_rng(M * 1000 + K)
+    Xq = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    T = rng.integers(-1, 2, (N, K)).astype(np.int8)
+    acc = oracle.matmul_i32(Xq, T)
+    ref = Xq.astype(np.int64) @ T.astype(np.int64).T
+    assert np.array_equal(acc.astype(np.int64), ref)
+    # an asymmetric case: a transposed operand or swapped index cannot pass both checks
+    assert acc.shape == (M, N)
+
+
+def test_forward_close_to_double_precision_product(oracle):
+    """y ~= sum_k (gamma*t_nk) * (q_tk*beta_t/127) evaluated in double."""
+    rng = np.random.default_rng(11)
+    M, K, N = 6, 96, 32
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    xbits = (x.view(np.uint32) >> 16).astype(np.uint16)
+    T, g = oracle.quantize_weights(W)
+    Y, acc, Xq, beta, rs = oracle.forward(T, g, xbits, return_all=True)
+    Wd = float(g) * T.astype(np.float64)
+    Xd = Xq.astype(np.float64) * beta.astype(np.float64)[:, None] / 127.0
+    ref = Xd @ Wd.T
+    got = bits_to_f32(Y).astype(np.float64)
+    # bf16 rounding is at most half an ulp = 2^-8 relative; the fp32 scale (two roundings) and the
+    # fp32 product add a few 2^-24
+    assert np.all(np.abs(got - ref) <= np.abs(ref) * (2.0**-8 + 2.0**-20) + 1e-12)  # 1e-12: the double sum's own noise
+    # and the quantised product tracks the unquantised one (sanity of the scales' direction)
+    full = bits_to_f32(xbits).astype(np.float64) @ (float(g) * T.astype(np.float64)).T
+    assert np.corrcoef(full.ravel(), got.ravel())[0, 1] > 0.999
+
+
+# ---------------------------------------------------------------- invariants
+
+def test_invariants_weights(oracle):
+    rng = np.random.default_rng(5)
+    W = (rng.standard_normal((32, 256)) * 0.02).astype(np.float32)
+    T, g = oracle.quantize_weights(W, 0.0)
+    Tn, gn = oracle.quantize_weights(-W, 0.0)
+    assert gn == g and np.array_equal(Tn, -T)
+    for j in (-3, 2, 7):
+        Ts, gs = oracle.quantize_weights(np.ldexp(W, j), 0.0)
+        assert gs == np.ldexp(g, j) and np.array_equal(Ts, T)
+    # permuting entries leaves gamma unchanged bit for bit (order-free sum)
+    perm = rng.permutation(W.size)
+    assert oracle.absmean(W.ravel()[perm].reshape(W.shape)) == g
+
+
+def test_invariants_activations_and_product(oracle):
+    rng = np.random.default_rng(6)
+    M, K, N = 4, 128, 32
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    xbits = (x.view(np.uint32) >> 16).astype(np.uint16)
+    q, beta, rs = oracle.quantize_acts(xbits)
+    xf = bits_to_f32(xbits)
+    q2, beta2, _ = oracle.quantize_acts(f32_to_bf16_bits(np.ldexp(xf, 3)))
+    assert np.array_equal(q2, q) and np.array_equal(beta2, np.ldexp(beta, 3))
+    qn, betan, rsn = oracle.quantize_acts(f32_to_bf16_bits(-xf))
+    assert np.array_equal(qn, -q) and np.array_equal(betan, beta) and np.array_equal(rsn, -rs)
+    T = rng.integers(-1, 2, (N, K)).astype(np.int8)
+    acc = oracle.matmul_i32(q, T)
+    perm = rng.permutation(K)
+    assert np.array_equal(oracle.matmul_i32(q[:, perm], T[:, perm]), acc)
+    # a row of a batch equals the single-token run of that row
+    for t in range(M):
+        Yt = oracle.forward(T, 0.017, xbits[t:t + 1])
+        assert np.array_equal(Yt[0], oracle.forward(T, 0.017, xbits)[t])
+    # offset-code identity: sum_k (t+1)*q = acc + rowsum
+    assert np.array_equal(oracle.matmul_i32(q, (T + 1).astype(np.int8)), acc + rs[:, None])
+
+
+def test_pack_unpack_roundtrip(oracle):
+    rng = np.random.default_rng(7)
+    for N, K in [(16, 128), (48, 320), (16, 64), (32, 8640 // 8)]:
+        T = rng.integers(-1, 2, (N, K)).astype(np.int8)
+        p = oracle.pack_weights(T)
+        assert p.size == oracle.packed_bytes(N, K)
+        assert np.array_equal(oracle.unpack_weights(p, N, K), T)
+
+
+# ---------------------------------------------------------------- exactness of gamma
+
+def test_gamma_matches_exactly_rounded_sum(oracle):
+    rng = np.random.default_rng(8)
+    for i in range(120):
+        N = 16 * int(rng.integers(1, 6))
+        K = int(rng.integers(8, 400))
+        scale = 10.0 ** rng.uniform(-4, 2)
+        W = (rng.standard_normal((N, K)) * scale).astype(np.float32)
+        g = oracle.absmean(W)
+        exact = math.fsum(abs(float(v)) for v in W.ravel()) / W.size  # fsum is correctly rounded
+        assert g == np.float32(exact), (i, N, K)
+
+
+def test_gamma_large_matrix_against_float128_free_reference(oracle):
+    """A bigger matrix: compare with an exact integer sum done another way (numpy int64 on scaled values)."""
+    rng = np.random.default_rng(9)
+    # values that are exact multiples of 2^-20 and < 4 in magnitude: the exact sum fits int64
+    ints = rng.integers(-(1 << 22), 1 << 22, (512, 2048))
+    W = (ints.astype(np.float64) * 2.0**-20).astype(np.float32)
+    assert np.array_equal(W.astype(np.float64) * 2.0**20, ints)
+    exact = int(np.abs(ints).sum())
+    g = oracle.absmean(W)
+    assert g == np.float32((exact / W.size) * 2.0**-20) or g == np.float32(exact * 2.0**-20 / W.size)
+
+
+def test_rejects_out_of_range(oracle):
+    W = np.ones((16, 16), np.float32)
+    W[3, 3] = np.inf
+    with pytest.raises(ValueError):
+        oracle.quantize_weights(W)
+    W[3, 3] = 2.0**24
+    with pytest.raises(ValueError):
+        oracle.quantize_weights(W)
+
+
+# ---------------------------------------------------------------- second statement in Python
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_c_oracle_equals_python_restatement(oracle, seed):
+    rng = np.random.default_rng(100 + seed)
+    N, K, M = 32, 136 + 8 * seed, 3
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    x = rng.standard_normal((M, K)).astype(np.float32) * (1 + 19 * (rng.random(K) < 0.02))
+    xbits = R.f32_to_bf16_bits_rne(x.astype(np.float32))
+    T, g = oracle.quantize_weights(W)
+    T2, g2 = R.quantize_weights(W)
+    assert g == g2 and np.array_equal(T, T2)
+    assert np.array_equal(oracle.pack_weights(T), R.pack_weights(T))
+    q, beta, rs = oracle.quantize_acts(xbits)
+    q2, beta2, rs2 = R.quantize_acts(xbits)
+    assert np.array_equal(q, q2) and np.array_equal(beta, beta2) and np.array_equal(rs, rs2)
+    acc = oracle.matmul_i32(q, T)
+    assert np.array_equal(acc, R.matmul_i32(q, T))
+    assert np.array_equal(oracle.dequant(acc, beta, g), R.dequant(acc, beta, g))
+    assert np.array_equal(oracle.forward(T, g, xbits), R.dequant(acc, beta, g))
+
+
+def test_timing_build_equals_parity_build(oracle):
+    from oracle import load_oracle
+    fast = load_oracle("timing")
+    rng = np.random.default_rng(42)
+    N, K, M = 64, 512, 9
+    W = (rng.standard_normal((N, K)) * 0.02).astype(np.float32)
+    x = rng.standard_normal((M, K)).astype(np.float32)
+    xbits = R.f32_to_bf16_bits_rne(x)
+    T, g = oracle.quantize_weights(W)
+    T2, g2 = fast.quantize_weights(W)
+    assert g == g2 and np.array_equal(T, T2)
+    assert np.array_equal(oracle.forward(T, g, xbits), fast.forward(T, g, xbits))
