@@ -1,0 +1,177 @@
+/*
+ * bitlinear.h -- C ABI of the BitLinear forward of BitNet b1.58 on NVIDIA B200 (sm_100a).
+ *
+ * The library computes, for a weight matrix W [N out, K in] and M tokens X [M, K]:
+ *
+ *   gamma  = mean_ij |W_ij|                                     (Section 2, Eq. 3)
+ *   T_nk   = RoundClip(W_nk / (gamma + eps), -1, 1)             (Section 2, Eq. 1 and Eq. 2)
+ *   beta_t = max(max_k |x_tk|, 1e-5)                            (Section 2, per-token absmax, Qb = 127)
+ *   q_tk   = clip(round(x_tk * (127 / beta_t)), -127, 127)      (same passage; no zero point)
+ *   acc_tn = sum_k q_tk * T_nk           exact, int32           (Section 1: integer additions only)
+ *   y_tn   = bf16( float(acc_tn) * ((gamma * beta_t) / 127) )
+ *
+ * round() is round-half-to-even everywhere; all float steps are single IEEE fp32 operations in the
+ * order written, so integer results are reproducible bit for bit.  Ternary weights are stored as
+ * 2-bit codes (Section 3, "Memory and Latency": a 2-bit kernel) in the layout described at
+ * bitlinear_quantize_weights.
+ *
+ * Conventions
+ *   - Every pointer is a DEVICE pointer owned by the caller unless marked "host".  The library never
+ *     allocates or frees device memory.  Inputs are never modified.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL = default stream) and
+ *     return without synchronising, except bitlinear_poll_status.
+ *   - Argument errors are detected on the host, returned at once, and nothing is launched.
+ *     Conditions found on the device (a bounded wait that expired) are written to a status word in
+ *     the workspace and read back with bitlinear_poll_status.
+ *   - Alignment: all device pointers 16-byte aligned; workspaces 256-byte aligned.
+ *   - Shapes: N a multiple of 16, K a multiple of 16 with 16 <= K <= 131072 (so |acc| < 2^24 and
+ *     float(acc) is exact), 1 <= N <= 2^24, 0 <= M <= 2^20.  M = 0 is a successful no-op, and the
+ *     per-token pointers (X, Xq, beta, rowsum, Y, acc) may then be null.
+ *   - Only sm_100 devices are supported; other devices give BITLINEAR_ERR_ARCH.  There is no CPU path.
+ */
+#ifndef BITLINEAR_H_
+#define BITLINEAR_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int bitlinear_status;
+
+enum {
+    BITLINEAR_OK = 0,
+    BITLINEAR_ERR_ARG = -1,       /* null pointer, negative size, bad enum value */
+    BITLINEAR_ERR_SHAPE = -2,     /* N, K or M outside the limits above */
+    BITLINEAR_ERR_ALIGN = -3,     /* a pointer is not 16-byte (workspace: 256-byte) aligned */
+    BITLINEAR_ERR_WORKSPACE = -4, /* workspace smaller than bitlinear_workspace_bytes says */
+    BITLINEAR_ERR_ARCH = -5,      /* current device is not sm_100 */
+    BITLINEAR_ERR_CUDA = -6,      /* a CUDA runtime or driver call failed */
+    BITLINEAR_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (device status) */
+    BITLINEAR_ERR_RANGE = -8      /* a weight was non-finite or >= 2^24 in magnitude (reported as gamma = NaN) */
+};
+
+/* Matmul code paths selectable through the test hook bitlinear_matmul_i32. */
+enum {
+    BITLINEAR_PATH_AUTO = 0,
+    BITLINEAR_PATH_DP4A = 1,   /* scalar dp4a, M <= 8 */
+    BITLINEAR_PATH_MMA = 2,    /* warp-level integer MMA on register-unpacked weights, M <= 64 */
+    BITLINEAR_PATH_TCGEN05 = 3 /* TMA + tcgen05 int8 tensor-core GEMM with TMEM accumulators, any M */
+};
+
+/* Human-readable name of a status code; never NULL. (host) */
+const char *bitlinear_status_string(bitlinear_status s);
+
+/* Bytes of the packed 2-bit weight buffer of an [N, K] matrix, K padded to a multiple of 128.
+ * Returns 0 for shapes the library rejects. (host) */
+size_t bitlinear_packed_bytes(int64_t N, int64_t K);
+
+/* Bytes of workspace bitlinear_forward / bitlinear_matmul_i32 need for this shape
+ * (int8 activations, beta, row sums, split-K scratch, status word).  0 for rejected shapes. (host) */
+size_t bitlinear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+
+/*
+ * Weight quantisation and packing: Section 2, Eq. 1-3, plus the 2-bit storage of Section 3.
+ *   W       in   fp32 [N, K] row-major (out x in)
+ *   eps     in   the epsilon of Eq. 1, added to gamma in the denominator
+ *   packed  out  bitlinear_packed_bytes(N, K) bytes
+ *   gamma   out  one fp32
+ * gamma is the exact sum of |W_ij| (each term truncated to a multiple of 2^-64, accumulated in a
+ * 128-bit integer, so the result does not depend on summation order), divided by N*K in double and
+ * rounded once to fp32.  If any weight is non-finite or has magnitude >= 2^24, gamma is set to NaN and
+ * the packed contents are unspecified.  The first 32 bytes of `packed` serve as scratch while gamma is
+ * being computed and are overwritten with their final contents afterwards.
+ *
+ * Layout.  The code of a weight is T + 1 (0, 1 or 2; 3 never occurs).  The matrix is cut into tiles of
+ * 16 rows x 128 columns = 512 bytes = 128 little-endian 32-bit words, stored consecutively with the
+ * column-tile index fastest.  Inside a tile, weight (r, c) sits in word 4*(4*(r%8) + c/32) + (c%32)/8 at
+ * bits [8*(c%4) + 2*f, +1] with f = 2*((c%8)/4) + r/8.  A warp that loads the tile as one 16-byte
+ * vector per lane therefore gets, from each word w, the four integer-MMA operand registers
+ * (w >> 2*f) & 0x03030303.  Columns K..Kpad-1 hold code 1 (weight 0).
+ */
+bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K, float eps,
+                                            void *packed, float *gamma, void *stream);
+
+/*
+ * Activation quantisation: Section 2, paragraph after Eq. 3 (per token, symmetric, [-127, 127]).
+ *   X       in   bf16 [M, K] row-major
+ *   Xq      out  int8 [M, K]
+ *   beta    out  fp32 [M]   clamped absmax of each token
+ *   rowsum  out  int32 [M]  sum_k Xq[t, k]  (used by the offset-coded matmul)
+ */
+bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K,
+                                         int8_t *Xq, float *beta, int32_t *rowsum, void *stream);
+
+/*
+ * The BitLinear forward: activation quantisation, ternary x int8 matmul with exact int32 accumulation,
+ * dequantisation to bf16 (Section 2; no bias, "removes all biases").
+ *   packed, gamma   in   from bitlinear_quantize_weights (gamma stays on the device)
+ *   X               in   bf16 [M, K]
+ *   Y               out  bf16 [M, N]
+ *   workspace       scratch, >= bitlinear_workspace_bytes(M, N, K); contents undefined afterwards.
+ *                   Two calls that run concurrently must not share a workspace.
+ * M <= 64 runs the weight-streaming decode kernel, larger M the tensor-core GEMM.
+ */
+bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X,
+                                   int64_t M, int64_t K, int64_t N, void *Y,
+                                   void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * A list of independent BitLinear forwards executed by one persistent launch (the seven projections of
+ * every decoder layer of a decode step, Section 2 "LLaMA-alike Components").  All inputs X must be
+ * ready when the call is enqueued: entries do not depend on each other.  Every entry needs M <= 64.
+ */
+typedef struct {
+    const void *packed; /* device */
+    const float *gamma; /* device */
+    const void *X;      /* device, bf16 [M, K] */
+    void *Y;            /* device, bf16 [M, N] */
+    int64_t M, K, N;
+} bitlinear_layer_desc;
+
+/* Workspace bytes for a sequence (host array of n descriptors). 0 on invalid input. (host) */
+size_t bitlinear_sequence_workspace_bytes(const bitlinear_layer_desc *layers, int n);
+
+/*
+ * Builds the launch plan of a sequence: validates the n descriptors (`layers` is a HOST array, free to
+ * reuse afterwards), lays the workspace out and copies the descriptor table into it with a synchronous
+ * copy.  *out receives an opaque host object; the workspace must stay untouched by the caller until
+ * bitlinear_sequence_destroy.  The X and Y pointers are fixed at creation (static decode buffers).
+ */
+typedef struct bitlinear_sequence bitlinear_sequence;
+bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
+                                           size_t workspace_bytes, bitlinear_sequence **out);
+
+/* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch and one persistent
+ * matmul launch.  Calls on the same sequence must be stream-ordered, not concurrent. */
+bitlinear_status bitlinear_forward_sequence(const bitlinear_sequence *seq, void *stream);
+
+/* The same in two halves, so that a caller can put its own events between them:
+ * stage 1 = activation quantiser only (Section 2, per-token absmax), stage 2 = matmul + dequantisation
+ * only (needs stage 1 to have run on the same stream first), stage 0 = both. */
+bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq, int stage, void *stream);
+
+/* Frees the host object (no device work, no device memory involved).  NULL is allowed. */
+void bitlinear_sequence_destroy(bitlinear_sequence *seq);
+
+/*
+ * Test hooks.
+ * bitlinear_matmul_i32: acc[t, n] = sum_k Xq[t, k] * T[n, k] as int32 [M, N] through the chosen path
+ * (the integer matmul of Section 1 in isolation).  Xq int8 [M, K] with values in [-127, 127].
+ * bitlinear_unpack_weights: T int8 [N, K] in {-1, 0, 1} from the packed buffer.
+ */
+bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
+                                      int32_t *acc, int path, void *workspace, size_t workspace_bytes,
+                                      void *stream);
+bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream);
+
+/* Synchronises `stream`, then copies the workspace's status word to *device_status (host pointer):
+ * BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT.  The return value reports the success of the read itself. */
+bitlinear_status bitlinear_poll_status(const void *workspace, void *stream, int *device_status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BITLINEAR_H_ */

@@ -123,6 +123,7 @@ int oracle_absmean(const float *W, int64_t N, int64_t K, float *gamma)
 static int round_clip(float x, int a, int b)
 {
     float r = rintf(x); /* FE_TONEAREST: ties to even */
+    if (r != r) return 0; /* 0/0 (all-zero matrix with eps = 0): the weight is 0 */
     if (r < (float)a) return a;
     if (r > (float)b) return b;
     return (int)r;

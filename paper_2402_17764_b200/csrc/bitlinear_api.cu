@@ -1,0 +1,464 @@
+// C ABI of the BitLinear library: argument validation, workspace layout, dispatch.
+// No arithmetic of the method lives here; every step runs in the kernels.
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "internal.cuh"
+
+namespace bitlinear {
+
+int sm_count()
+{
+    static int cached[64] = {0};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 148;
+    if (cached[dev] == 0) {
+        int n = 0;
+        if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        cached[dev] = n;
+    }
+    return cached[dev];
+}
+
+namespace {
+
+bool device_is_sm100()
+{
+    static int cached[64] = {0}; // 0 unknown, 1 yes, 2 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (cached[dev] == 0) {
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return false;
+        cached[dev] = (major == 10) ? 1 : 2;
+    }
+    return cached[dev] == 1;
+}
+
+inline bool aligned(const void *p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+bitlinear_status check_shape(int64_t M, int64_t N, int64_t K)
+{
+    if (M < 0 || M > (1 << 20)) return BITLINEAR_ERR_SHAPE;
+    if (N < 16 || N > (1 << 24) || (N % 16) != 0) return BITLINEAR_ERR_SHAPE;
+    if (K < 16 || K > 131072 || (K % 16) != 0) return BITLINEAR_ERR_SHAPE;
+    return BITLINEAR_OK;
+}
+
+int env_int(const char *name, int fallback)
+{
+    const char *v = std::getenv(name);
+    if (!v || !*v) return fallback;
+    return std::atoi(v);
+}
+
+// Work-unit sizing of the persistent decode kernel: enough units to fill the machine, none longer
+// than `max_tiles` 128-column tiles (bounds the tail), none shorter than `min_tiles`.
+int choose_ksplit(int64_t total_row_blocks, int KB)
+{
+    static const int max_tiles = env_int("BITLINEAR_UNIT_MAX_TILES", 32);
+    static const int min_tiles = env_int("BITLINEAR_UNIT_MIN_TILES", 4);
+    const int64_t target_units = (int64_t)sm_count() * 32;
+    int split = 1;
+    if (total_row_blocks < target_units) split = (int)((target_units + total_row_blocks - 1) / total_row_blocks);
+    const int need = (KB + max_tiles - 1) / max_tiles;
+    if (split < need) split = need;
+    int cap = KB / min_tiles;
+    if (cap < 1) cap = 1;
+    if (split > cap) split = cap;
+    return split;
+}
+
+struct Layout {
+    size_t counters, acc32, table, xq, beta, rowsum, total;
+};
+
+// Workspace of one matmul: [header | counters | acc32 (M <= 64 only) | Xq | beta | rowsum]
+Layout single_layout(int64_t M, int64_t N, int64_t K)
+{
+    Layout L{};
+    size_t off = sizeof(WorkspaceHeader);
+    L.counters = off;
+    off += align_up((size_t)(N / 16) * 4, 256);
+    L.acc32 = off;
+    if (M <= kMaxDecodeM) off += align_up((size_t)M * N * 4, 256);
+    L.table = off;
+    L.xq = off;
+    off += align_up((size_t)M * K, 256);
+    L.beta = off;
+    off += align_up((size_t)M * 4, 256);
+    L.rowsum = off;
+    off += align_up((size_t)M * 4, 256);
+    L.total = off;
+    return L;
+}
+
+__global__ void rowsum_kernel(const int8_t *__restrict__ Xq, int K, int32_t *__restrict__ rowsum)
+{
+    const int t = blockIdx.x;
+    int s = 0;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) s += Xq[(size_t)t * K + k];
+    s = __reduce_add_sync(0xffffffffu, s);
+    __shared__ int part[8];
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = s;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int tot = 0;
+        for (int w = 0; w < 8; ++w) tot += part[w];
+        rowsum[t] = tot;
+    }
+}
+
+bool use_tcgen05_for(int64_t M)
+{
+    static const int disabled = env_int("BITLINEAR_NO_TCGEN05", 0);
+    static const int min_m = env_int("BITLINEAR_TCGEN05_MIN_M", kMaxDecodeM + 1);
+    return !disabled && M >= min_m;
+}
+
+// Fills one DecodeEntry for a matmul whose workspace part starts at `base`.
+void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
+                int64_t N, void *out, int out_i32, char *base, const Layout &L, int ksplit)
+{
+    e.packed = reinterpret_cast<const uint4 *>(packed);
+    e.gamma = gamma;
+    e.X = reinterpret_cast<const __nv_bfloat16 *>(X);
+    e.Xq = reinterpret_cast<int8_t *>(base + L.xq);
+    e.beta = reinterpret_cast<float *>(base + L.beta);
+    e.rowsum = reinterpret_cast<int32_t *>(base + L.rowsum);
+    e.out = out;
+    e.acc32 = reinterpret_cast<int32_t *>(base + L.acc32);
+    e.counters = reinterpret_cast<uint32_t *>(base + L.counters);
+    e.M = (int)M;
+    e.N = (int)N;
+    e.K = (int)K;
+    e.KB = (int)((K + kTileCols - 1) / kTileCols);
+    e.ksplit = ksplit;
+    e.unit_begin = 0;
+    e.token_begin = 0;
+    e.out_i32 = out_i32;
+}
+
+// Runs the matmul + epilogue of one entry whose activations are already quantised.
+bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, cudaStream_t stream)
+{
+    WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
+    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
+    if (tc) {
+        cudaError_t err = launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out, e.out_i32,
+                                         hdr, stream);
+        return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+    }
+    // Weight-streaming kernel, in slices of at most 64 tokens (one slice in the decode regime).
+    const int64_t M = e.M;
+    for (int64_t m0 = 0; m0 < M; m0 += kMaxDecodeM) {
+        DecodeEntry s = e;
+        s.M = (int)((M - m0 < kMaxDecodeM) ? (M - m0) : kMaxDecodeM);
+        s.Xq = e.Xq + m0 * e.K;
+        s.beta = e.beta + m0;
+        s.rowsum = e.rowsum + m0;
+        const size_t elt = e.out_i32 ? 4 : 2;
+        s.out = reinterpret_cast<char *>(e.out) + (size_t)m0 * e.N * elt;
+        if (M > kMaxDecodeM) s.ksplit = 1; // no split-K scratch is laid out for large M
+        if (m0 > 0) {
+            cudaError_t err = cudaMemsetAsync(&hdr->unit_counter, 0, sizeof(uint32_t), stream);
+            if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
+        }
+        InlineTable inl{};
+        inl.e[0] = s;
+        const int units = (s.N / kTileRows) * s.ksplit;
+        cudaError_t err = launch_decode(inl, nullptr, 1, units, s.M, path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA,
+                                        hdr, stream);
+        if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    }
+    return BITLINEAR_OK;
+}
+
+} // namespace
+} // namespace bitlinear
+
+using namespace bitlinear;
+
+extern "C" {
+
+const char *bitlinear_status_string(bitlinear_status s)
+{
+    switch (s) {
+    case BITLINEAR_OK: return "ok";
+    case BITLINEAR_ERR_ARG: return "invalid argument";
+    case BITLINEAR_ERR_SHAPE: return "unsupported shape";
+    case BITLINEAR_ERR_ALIGN: return "misaligned pointer";
+    case BITLINEAR_ERR_WORKSPACE: return "workspace too small";
+    case BITLINEAR_ERR_ARCH: return "device is not sm_100";
+    case BITLINEAR_ERR_CUDA: return "CUDA call failed";
+    case BITLINEAR_ERR_TIMEOUT: return "device-side wait timed out";
+    case BITLINEAR_ERR_RANGE: return "weight out of range";
+    default: return "unknown status";
+    }
+}
+
+size_t bitlinear_packed_bytes(int64_t N, int64_t K)
+{
+    if (check_shape(0, N, K) != BITLINEAR_OK) return 0;
+    const int64_t Kp = (K + kTileCols - 1) / kTileCols * kTileCols;
+    return (size_t)(N * Kp / 4);
+}
+
+size_t bitlinear_workspace_bytes(int64_t M, int64_t N, int64_t K)
+{
+    if (check_shape(M, N, K) != BITLINEAR_OK) return 0;
+    return single_layout(M, N, K).total;
+}
+
+bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K, float eps, void *packed,
+                                            float *gamma, void *stream)
+{
+    if (!W || !packed || !gamma || !(eps >= 0.0f)) return BITLINEAR_ERR_ARG;
+    bitlinear_status st = check_shape(0, N, K);
+    if (st != BITLINEAR_OK) return st;
+    if (!aligned(W, 16) || !aligned(packed, 16) || !aligned(gamma, 4)) return BITLINEAR_ERR_ALIGN;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    cudaError_t err = launch_absmean_and_pack(W, N, K, eps, packed, gamma, (cudaStream_t)stream);
+    return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K, int8_t *Xq, float *beta,
+                                         int32_t *rowsum, void *stream)
+{
+    if (M > 0 && (!X || !Xq || !beta || !rowsum)) return BITLINEAR_ERR_ARG;
+    bitlinear_status st = check_shape(M, 16, K);
+    if (st != BITLINEAR_OK) return st;
+    if (!aligned(X, 16) || !aligned(Xq, 16) || !aligned(beta, 4) || !aligned(rowsum, 4)) return BITLINEAR_ERR_ALIGN;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    if (M == 0) return BITLINEAR_OK;
+    InlineTable inl{};
+    DecodeEntry &e = inl.e[0];
+    e.X = reinterpret_cast<const __nv_bfloat16 *>(X);
+    e.Xq = Xq;
+    e.beta = beta;
+    e.rowsum = rowsum;
+    e.M = (int)M;
+    e.K = (int)K;
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, (cudaStream_t)stream);
+    return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
+                                   int64_t N, void *Y, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!packed || !gamma || !workspace || (M > 0 && (!X || !Y))) return BITLINEAR_ERR_ARG;
+    bitlinear_status st = check_shape(M, N, K);
+    if (st != BITLINEAR_OK) return st;
+    if (!aligned(packed, 16) || !aligned(X, 16) || !aligned(Y, 16) || !aligned(gamma, 4)) return BITLINEAR_ERR_ALIGN;
+    if (!aligned(workspace, 256)) return BITLINEAR_ERR_ALIGN;
+    const Layout L = single_layout(M, N, K);
+    if (workspace_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    if (M == 0) return BITLINEAR_OK;
+    char *ws = reinterpret_cast<char *>(workspace);
+    InlineTable inl{};
+    const int KB = (int)((K + kTileCols - 1) / kTileCols);
+    const bool tc = use_tcgen05_for(M);
+    const int ksplit = (M <= kMaxDecodeM && !tc) ? choose_ksplit(N / 16, KB) : 1;
+    fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L, ksplit);
+    // quantise the tokens; the same launch clears the header and (when splitting K) the scratch
+    const size_t zero_bytes = (ksplit > 1) ? L.table : sizeof(WorkspaceHeader);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
+    if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, (cudaStream_t)stream);
+}
+
+bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
+                                      int32_t *acc, int path, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (!packed || !workspace || (M > 0 && (!Xq || !acc))) return BITLINEAR_ERR_ARG;
+    if (path < BITLINEAR_PATH_AUTO || path > BITLINEAR_PATH_TCGEN05) return BITLINEAR_ERR_ARG;
+    bitlinear_status st = check_shape(M, N, K);
+    if (st != BITLINEAR_OK) return st;
+    if (path == BITLINEAR_PATH_DP4A && M > 8) return BITLINEAR_ERR_SHAPE;
+    if (path == BITLINEAR_PATH_MMA && M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE;
+    if (!aligned(packed, 16) || !aligned(Xq, 16) || !aligned(acc, 16)) return BITLINEAR_ERR_ALIGN;
+    if (!aligned(workspace, 256)) return BITLINEAR_ERR_ALIGN;
+    const Layout L = single_layout(M, N, K);
+    if (workspace_bytes < L.total) return BITLINEAR_ERR_WORKSPACE;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    if (M == 0) return BITLINEAR_OK;
+    char *ws = reinterpret_cast<char *>(workspace);
+    cudaStream_t s = (cudaStream_t)stream;
+    const int KB = (int)((K + kTileCols - 1) / kTileCols);
+    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
+    const int ksplit = (M <= kMaxDecodeM && !tc) ? choose_ksplit(N / 16, KB) : 1;
+    InlineTable inl{};
+    fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L, ksplit);
+    inl.e[0].Xq = const_cast<int8_t *>(Xq); // read only on this path
+    const size_t zero_bytes = (ksplit > 1) ? L.table : sizeof(WorkspaceHeader);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, s);
+    if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
+    if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    return run_matmul(inl.e[0], path, ws, s);
+}
+
+bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)
+{
+    if (!packed || !T) return BITLINEAR_ERR_ARG;
+    bitlinear_status st = check_shape(0, N, K);
+    if (st != BITLINEAR_OK) return st;
+    if (!aligned(packed, 16)) return BITLINEAR_ERR_ALIGN;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    cudaError_t err = launch_unpack(packed, N, K, T, (cudaStream_t)stream);
+    return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+
+bitlinear_status bitlinear_poll_status(const void *workspace, void *stream, int *device_status)
+{
+    if (!workspace || !device_status) return BITLINEAR_ERR_ARG;
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    int32_t v = 0;
+    if (cudaMemcpy(&v, workspace, sizeof v, cudaMemcpyDeviceToHost) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    *device_status = (int)v;
+    return BITLINEAR_OK;
+}
+
+// ---- sequences -------------------------------------------------------------------------------
+// Workspace: [header | all counters | all acc32 | descriptor table | per-entry Xq, beta, rowsum]
+
+struct bitlinear_sequence {
+    char *workspace;
+    int n, units, tokens, max_M;
+    size_t zero_bytes;
+    const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
+    bitlinear::InlineTable inl;
+};
+
+namespace {
+struct SeqLayout {
+    size_t counters, acc32, table, data, total;
+};
+
+bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::vector<size_t> *entry_off)
+{
+    if (!layers || n <= 0 || n > 65536) return false;
+    size_t counters = 0, acc = 0, data = 0;
+    for (int i = 0; i < n; ++i) {
+        const bitlinear_layer_desc &d = layers[i];
+        if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1 || d.M > kMaxDecodeM) return false;
+        counters += align_up((size_t)(d.N / 16) * 4, 256);
+        acc += align_up((size_t)d.M * d.N * 4, 256);
+        if (entry_off) entry_off->push_back(data);
+        data += align_up((size_t)d.M * d.K, 256) + 2 * align_up((size_t)d.M * 4, 256);
+    }
+    size_t off = sizeof(WorkspaceHeader);
+    S.counters = off;
+    off += counters;
+    S.acc32 = off;
+    off += acc;
+    S.table = off;
+    off += align_up((size_t)n * sizeof(DecodeEntry), 256);
+    S.data = off;
+    off += data;
+    S.total = off;
+    return true;
+}
+} // namespace
+
+size_t bitlinear_sequence_workspace_bytes(const bitlinear_layer_desc *layers, int n)
+{
+    SeqLayout S{};
+    if (!seq_layout(layers, n, S, nullptr)) return 0;
+    return S.total;
+}
+
+bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
+                                           size_t workspace_bytes, bitlinear_sequence **out)
+{
+    if (!layers || !workspace || !out || n <= 0) return BITLINEAR_ERR_ARG;
+    *out = nullptr;
+    SeqLayout S{};
+    std::vector<size_t> entry_off;
+    if (!seq_layout(layers, n, S, &entry_off)) return BITLINEAR_ERR_SHAPE;
+    if (!aligned(workspace, 256)) return BITLINEAR_ERR_ALIGN;
+    if (workspace_bytes < S.total) return BITLINEAR_ERR_WORKSPACE;
+    for (int i = 0; i < n; ++i) {
+        const bitlinear_layer_desc &d = layers[i];
+        if (!d.packed || !d.gamma || !d.X || !d.Y) return BITLINEAR_ERR_ARG;
+        if (!aligned(d.packed, 16) || !aligned(d.X, 16) || !aligned(d.Y, 16) || !aligned(d.gamma, 4))
+            return BITLINEAR_ERR_ALIGN;
+    }
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    char *ws = reinterpret_cast<char *>(workspace);
+
+    int64_t total_rb = 0;
+    for (int i = 0; i < n; ++i) total_rb += layers[i].N / 16;
+    std::vector<DecodeEntry> table((size_t)n);
+    size_t c_off = S.counters, a_off = S.acc32;
+    int units = 0, tokens = 0, max_M = 0;
+    bool any_split = false;
+    for (int i = 0; i < n; ++i) {
+        const bitlinear_layer_desc &d = layers[i];
+        Layout L{};
+        L.counters = c_off;
+        L.acc32 = a_off;
+        L.xq = S.data + entry_off[(size_t)i];
+        L.beta = L.xq + align_up((size_t)d.M * d.K, 256);
+        L.rowsum = L.beta + align_up((size_t)d.M * 4, 256);
+        c_off += align_up((size_t)(d.N / 16) * 4, 256);
+        a_off += align_up((size_t)d.M * d.N * 4, 256);
+        const int KB = (int)((d.K + kTileCols - 1) / kTileCols);
+        const int ksplit = choose_ksplit(total_rb, KB);
+        any_split |= ksplit > 1;
+        fill_entry(table[(size_t)i], d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L, ksplit);
+        table[(size_t)i].unit_begin = units;
+        table[(size_t)i].token_begin = tokens;
+        units += (int)(d.N / 16) * ksplit;
+        tokens += (int)d.M;
+        if ((int)d.M > max_M) max_M = (int)d.M;
+    }
+    bitlinear_sequence *seq = new (std::nothrow) bitlinear_sequence();
+    if (!seq) return BITLINEAR_ERR_ARG;
+    seq->workspace = ws;
+    seq->n = n;
+    seq->units = units;
+    seq->tokens = tokens;
+    seq->max_M = max_M;
+    seq->zero_bytes = any_split ? S.table : sizeof(WorkspaceHeader);
+    seq->dev_table = nullptr;
+    if (n <= kInlineEntries) {
+        for (int i = 0; i < n; ++i) seq->inl.e[i] = table[(size_t)i];
+    } else {
+        if (cudaMemcpy(ws + S.table, table.data(), (size_t)n * sizeof(DecodeEntry), cudaMemcpyHostToDevice) !=
+            cudaSuccess) {
+            delete seq;
+            return BITLINEAR_ERR_CUDA;
+        }
+        seq->dev_table = reinterpret_cast<const DecodeEntry *>(ws + S.table);
+    }
+    *out = seq;
+    return BITLINEAR_OK;
+}
+
+bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq, int stage, void *stream)
+{
+    if (!seq || stage < 0 || stage > 2) return BITLINEAR_ERR_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (stage != 2 &&
+        launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes, s) !=
+            cudaSuccess)
+        return BITLINEAR_ERR_CUDA;
+    if (stage != 1 &&
+        launch_decode(seq->inl, seq->dev_table, seq->n, seq->units, seq->max_M, BITLINEAR_PATH_MMA,
+                      reinterpret_cast<WorkspaceHeader *>(seq->workspace), s) != cudaSuccess)
+        return BITLINEAR_ERR_CUDA;
+    return BITLINEAR_OK;
+}
+
+bitlinear_status bitlinear_forward_sequence(const bitlinear_sequence *seq, void *stream)
+{
+    return bitlinear_forward_sequence_stage(seq, 0, stream);
+}
+
+void bitlinear_sequence_destroy(bitlinear_sequence *seq) { delete seq; }
+
+} // extern "C"

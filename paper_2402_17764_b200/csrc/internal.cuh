@@ -1,0 +1,74 @@
+// Internal declarations shared by the translation units of the BitLinear CUDA library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/bitlinear.h"
+
+namespace bitlinear {
+
+constexpr int kQb = 127;            // Section 2: activations scaled to [-Qb, Qb]
+constexpr float kBetaFloor = 1e-5f; // zero-token guard on the per-token absmax
+constexpr int kTileRows = 16;       // packed tile: 16 rows x 128 columns = 512 bytes
+constexpr int kTileCols = 128;
+constexpr int kTileBytes = 512;
+constexpr int kMaxDecodeM = 64;
+
+// Workspace header (first 256 bytes of every workspace).
+struct WorkspaceHeader {
+    int32_t status;        // BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT, written by kernels
+    uint32_t unit_counter; // dynamic work counter of the persistent decode kernel
+    uint32_t reserved[62];
+};
+static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
+
+// One matmul of a decode launch, as the kernels see it (device memory or kernel parameter).
+struct DecodeEntry {
+    const uint4 *packed;   // 2-bit weights
+    const float *gamma;    // 1 fp32 (unused when out_i32)
+    const __nv_bfloat16 *X; // bf16 [M, K] (input of the quantiser; null for the matmul hook)
+    int8_t *Xq;            // int8 [M, K]
+    float *beta;           // [M]
+    int32_t *rowsum;       // [M]
+    void *out;             // bf16 [M, N], or int32 [M, N] when out_i32
+    int32_t *acc32;        // split-K scratch [M, N] (zero before and after a launch)
+    uint32_t *counters;    // split-K arrival counters [N/16] (zero before and after a launch)
+    int M, N, K, KB;       // KB = padded K / 128
+    int ksplit;            // k splits per row block (1 = none)
+    int unit_begin;        // first work unit of this entry; units = (N/16) * ksplit
+    int token_begin;       // first token of this entry in the batched quantiser's grid
+    int out_i32;           // 1: write raw int32 accumulators instead of bf16
+};
+
+constexpr int kInlineEntries = 4;
+struct InlineTable {
+    DecodeEntry e[kInlineEntries];
+};
+
+static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// ---- kernel launchers (host side, each defined next to its kernel) ----
+
+cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
+                                    cudaStream_t stream);
+cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream);
+
+// Quantises the tokens of every entry (entries with X == nullptr are skipped) and zeroes
+// `zero_bytes` bytes at `zero_ptr` (control words and split-K scratch) in the same launch.
+cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
+                                 void *zero_ptr, size_t zero_bytes, cudaStream_t stream);
+
+// Persistent weight-streaming matmul over the entries. path: BITLINEAR_PATH_MMA or BITLINEAR_PATH_DP4A.
+cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_units, int max_M,
+                          int path, WorkspaceHeader *hdr, cudaStream_t stream);
+
+// Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) or raw int32.
+cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
+                           const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
+                           WorkspaceHeader *hdr, cudaStream_t stream);
+
+int sm_count();
+
+} // namespace bitlinear

@@ -1,0 +1,196 @@
+// Kernel (a): absmean weight quantisation (Section 2, Eq. 1-3) and 2-bit packing.
+//
+// Three launches on the caller's stream:
+//   1. clear 32 bytes of scratch (the head of the output buffer itself),
+//   2. exact sum of |W| in 2^-64 fixed point, 128-bit integer, order-free; the last block
+//      to finish turns it into gamma,
+//   3. ternarise with round-half-to-even and write the interleaved 2-bit tiles.
+// HBM-bound: two reads of the fp32 matrix (8 B per weight) and 0.25 B written per weight.
+#include "internal.cuh"
+
+namespace bitlinear {
+
+namespace {
+
+struct U128 {
+    unsigned long long lo, hi;
+};
+
+__device__ __forceinline__ void add128(U128 &a, unsigned long long lo, unsigned long long hi)
+{
+    a.lo += lo;
+    a.hi += hi + (a.lo < lo ? 1ull : 0ull);
+}
+
+// floor(|v| * 2^64) for an fp32 magnitude given as bits (sign cleared, exponent < 151).
+__device__ __forceinline__ void fix64(uint32_t mag, unsigned long long &lo, unsigned long long &hi)
+{
+    uint32_t e = mag >> 23;
+    uint32_t frac = mag & 0x7FFFFFu;
+    unsigned long long sig = e ? (frac | 0x800000u) : frac;
+    int shift = (int)(e ? e : 1u) - 86; // value = sig * 2^shift
+    if (shift >= 0) {
+        if (shift == 0) { lo = sig; hi = 0; }
+        else if (shift < 64) { lo = sig << shift; hi = sig >> (64 - shift); }
+        else { lo = 0; hi = sig << (shift - 64); }
+    } else {
+        int s = -shift;
+        lo = (s < 24) ? (sig >> s) : 0ull;
+        hi = 0;
+    }
+}
+
+// scratch words (unsigned long long): [0] sum.lo  [1] sum.hi  [2] blocks done  [3] range violation flag
+__global__ void __launch_bounds__(256) absmean_kernel(const float4 *__restrict__ W4, size_t n_vec,
+                                                      double count, unsigned long long *scratch,
+                                                      float *__restrict__ gamma)
+{
+    U128 acc = {0ull, 0ull};
+    uint32_t bad = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x) {
+        float4 v = __ldg(W4 + i);
+        const float f[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t mag = __float_as_uint(f[j]) & 0x7FFFFFFFu;
+            if ((mag >> 23) >= 151u) { bad = 1; continue; }
+            unsigned long long lo, hi;
+            fix64(mag, lo, hi);
+            add128(acc, lo, hi);
+        }
+    }
+    // warp reduction
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+        unsigned long long lo = __shfl_xor_sync(0xffffffffu, acc.lo, off);
+        unsigned long long hi = __shfl_xor_sync(0xffffffffu, acc.hi, off);
+        add128(acc, lo, hi);
+        bad |= __shfl_xor_sync(0xffffffffu, bad, off);
+    }
+    __shared__ U128 warp_sum[8];
+    __shared__ uint32_t warp_bad[8];
+    __shared__ bool is_last;
+    int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) { warp_sum[warp] = acc; warp_bad[warp] = bad; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        U128 tot = {0ull, 0ull};
+        uint32_t b = 0;
+        for (int w = 0; w < 8; ++w) { add128(tot, warp_sum[w].lo, warp_sum[w].hi); b |= warp_bad[w]; }
+        // 128-bit atomic add as two 64-bit ones: the number of carries out of the low word
+        // does not depend on the order in which blocks arrive.
+        unsigned long long old = atomicAdd(&scratch[0], tot.lo);
+        unsigned long long carry = (old + tot.lo < old) ? 1ull : 0ull;
+        atomicAdd(&scratch[1], tot.hi + carry);
+        if (b) atomicOr(&scratch[3], 1ull);
+        __threadfence();
+        unsigned long long ticket = atomicAdd(&scratch[2], 1ull);
+        is_last = (ticket == (unsigned long long)gridDim.x - 1ull);
+    }
+    __syncthreads();
+    if (is_last && threadIdx.x == 0) {
+        __threadfence();
+        unsigned long long lo = atomicAdd(&scratch[0], 0ull);
+        unsigned long long hi = atomicAdd(&scratch[1], 0ull);
+        unsigned long long flag = atomicAdd(&scratch[3], 0ull);
+        double sum = __dmul_rn(__dadd_rn(__dmul_rn(__ull2double_rn(hi), 18446744073709551616.0), __ull2double_rn(lo)),
+                               1.0 / 18446744073709551616.0);
+        double mean = __ddiv_rn(sum, count);
+        *gamma = flag ? __int_as_float(0x7FC00000) : __double2float_rn(mean);
+    }
+}
+
+// One warp per 16 x 128 tile; lane (g = lane / 4, tq = lane % 4) owns rows g and g + 8,
+// columns 32 * tq .. 32 * tq + 31 of the tile and writes its four 32-bit words as one 16-byte store.
+__global__ void __launch_bounds__(256) ternarize_pack_kernel(const float *__restrict__ W, int N, int K, int KB,
+                                                             float eps, const float *__restrict__ gamma,
+                                                             uint4 *__restrict__ packed)
+{
+    const long long n_tiles = (long long)(N / kTileRows) * KB;
+    const int lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const float denom = __fadd_rn(*gamma, eps); // Eq. 1: gamma + eps
+    for (long long tile = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < n_tiles;
+         tile += (long long)gridDim.x * (blockDim.x >> 5)) {
+        const int rb = (int)(tile / KB), kb = (int)(tile % KB);
+        uint32_t words[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+        for (int half = 0; half < 2; ++half) { // row g, then row g + 8
+            const float *row = W + (size_t)(rb * kTileRows + g + 8 * half) * K;
+            const int col0 = kb * kTileCols + 32 * tq;
+#pragma unroll
+            for (int v = 0; v < 8; ++v) { // eight float4 = 32 columns
+                const int col = col0 + 4 * v;
+                uint32_t codes = 0x01010101u; // padding: weight 0
+                if (col < K) {
+                    float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
+                    const float f[4] = {w.x, w.y, w.z, w.w};
+                    codes = 0;
+#pragma unroll
+                    for (int b = 0; b < 4; ++b) {
+                        int t = __float2int_rn(__fdiv_rn(f[b], denom)); // round half to even (Eq. 2)
+                        t = max(-1, min(1, t));
+                        codes |= (uint32_t)(t + 1) << (8 * b);
+                    }
+                }
+                // float4 v covers columns 8*i + 4*(f>>1) + b with i = v / 2, f>>1 = v % 2, and f&1 = half
+                const int i = v >> 1;
+                const int field = 2 * (v & 1) + half;
+                words[i] |= codes << (2 * field);
+            }
+        }
+        packed[tile * 32 + lane] = make_uint4(words[0], words[1], words[2], words[3]);
+    }
+}
+
+__global__ void __launch_bounds__(256) unpack_kernel(const uint32_t *__restrict__ packed, int N, int K, int KB,
+                                                     int8_t *__restrict__ T)
+{
+    const size_t total = (size_t)N * K;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const int n = (int)(idx / K), k = (int)(idx % K);
+        const size_t tile = (size_t)(n / 16) * KB + k / 128;
+        const int r = n % 16, c = k % 128;
+        const int word = 4 * (4 * (r % 8) + c / 32) + (c % 32) / 8;
+        const int field = 2 * ((c % 8) / 4) + r / 8;
+        const uint32_t w = packed[tile * 128 + word];
+        const int code = (w >> (8 * (c % 4) + 2 * field)) & 3;
+        T[idx] = (int8_t)(code - 1);
+    }
+}
+
+} // namespace
+
+cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
+                                    cudaStream_t stream)
+{
+    cudaError_t err = cudaMemsetAsync(packed, 0, 32, stream);
+    if (err != cudaSuccess) return err;
+    const size_t n_vec = (size_t)N * K / 4;
+    int blocks = (int)((n_vec + 255) / 256);
+    const int cap = sm_count() * 8;
+    if (blocks > cap) blocks = cap;
+    absmean_kernel<<<blocks, 256, 0, stream>>>(reinterpret_cast<const float4 *>(W), n_vec, (double)(N * K),
+                                               reinterpret_cast<unsigned long long *>(packed), gamma);
+    err = cudaGetLastError();
+    if (err != cudaSuccess) return err;
+    const int KB = (int)((K + kTileCols - 1) / kTileCols);
+    const long long n_tiles = (N / kTileRows) * (long long)KB;
+    long long pblocks = (n_tiles + 7) / 8;
+    if (pblocks > (long long)sm_count() * 16) pblocks = (long long)sm_count() * 16;
+    ternarize_pack_kernel<<<(int)pblocks, 256, 0, stream>>>(W, (int)N, (int)K, KB, eps, gamma,
+                                                            reinterpret_cast<uint4 *>(packed));
+    return cudaGetLastError();
+}
+
+cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream)
+{
+    const int KB = (int)((K + kTileCols - 1) / kTileCols);
+    size_t total = (size_t)N * K;
+    size_t blocks = (total + 255) / 256;
+    if (blocks > (size_t)sm_count() * 32) blocks = (size_t)sm_count() * 32;
+    unpack_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint32_t *>(packed), (int)N, (int)K, KB, T);
+    return cudaGetLastError();
+}
+
+} // namespace bitlinear

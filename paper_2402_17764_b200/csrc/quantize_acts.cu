@@ -1,0 +1,156 @@
+// Kernel (b): per-token absmax quantisation of bf16 activations to int8
+// (Section 2, paragraph after Eq. 3: scaled to [-Qb, Qb] per token, Qb = 127, no zero point).
+//
+// One CTA per token.  The token is read once with 16-byte loads and kept in registers
+// (up to kCache vectors per thread; longer rows re-read the tail, which hits L2), the absmax
+// is reduced with warp shuffles, then every element takes one fp32 multiply by 127/beta,
+// round-half-to-even, clip, and is stored as int8 together with the row sum of the codes.
+// HBM-bound: 2 B read + 1 B written per element.
+#include "internal.cuh"
+
+namespace bitlinear {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kCache = 8; // 16-byte vectors kept in registers per thread (8 * 8 * 256 = 16384 elements)
+
+__device__ __forceinline__ uint32_t absmax_bits(uint32_t m, const uint4 &v)
+{
+    // |bf16| as an unsigned 15-bit integer is monotone in the magnitude
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        m = max(m, w[i] & 0x7FFFu);
+        m = max(m, (w[i] >> 16) & 0x7FFFu);
+    }
+    return m;
+}
+
+__device__ __forceinline__ int quant1(uint32_t bf16_bits, float s)
+{
+    const float x = __uint_as_float(bf16_bits << 16);
+    int q = __float2int_rn(__fmul_rn(x, s)); // one multiply, round half to even
+    return max(-kQb, min(kQb, q));
+}
+
+// 8 bf16 -> 8 int8 (two 32-bit words), returns the sum of the eight codes
+__device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
+{
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    int q[8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        q[2 * i] = quant1(w[i] & 0xFFFFu, s);
+        q[2 * i + 1] = quant1(w[i] >> 16, s);
+    }
+    out.x = (uint32_t)(q[0] & 0xFF) | ((uint32_t)(q[1] & 0xFF) << 8) | ((uint32_t)(q[2] & 0xFF) << 16) |
+            ((uint32_t)(q[3] & 0xFF) << 24);
+    out.y = (uint32_t)(q[4] & 0xFF) | ((uint32_t)(q[5] & 0xFF) << 8) | ((uint32_t)(q[6] & 0xFF) << 16) |
+            ((uint32_t)(q[7] & 0xFF) << 24);
+    return q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+}
+
+__global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
+                                                                 const DecodeEntry *__restrict__ table, int n_entries,
+                                                                 int total_tokens, uint4 *zero_ptr, size_t zero_vecs)
+{
+    __shared__ uint32_t s_max[kThreads / 32];
+    __shared__ int s_sum[kThreads / 32];
+
+    if ((int)blockIdx.x >= total_tokens) {
+        // trailing blocks clear control words and split-K scratch for the matmul that follows
+        const size_t n_zero_blocks = gridDim.x - total_tokens;
+        for (size_t i = (size_t)(blockIdx.x - total_tokens) * kThreads + threadIdx.x; i < zero_vecs;
+             i += n_zero_blocks * kThreads)
+            zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
+        return;
+    }
+
+    const DecodeEntry *tab = table ? table : inl.e;
+    // entry that owns this token: the last one whose token_begin <= blockIdx.x
+    int lo = 0, hi = n_entries - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (tab[mid].token_begin <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
+    }
+    const DecodeEntry &e = tab[lo];
+    const int t = blockIdx.x - e.token_begin;
+    const int K = e.K;
+    const int n_vec = K >> 3;
+    const uint4 *row = reinterpret_cast<const uint4 *>(e.X + (size_t)t * K);
+    uint2 *out = reinterpret_cast<uint2 *>(e.Xq + (size_t)t * K);
+
+    uint4 cache[kCache];
+    uint32_t m = 0;
+#pragma unroll
+    for (int c = 0; c < kCache; ++c) {
+        const int i = threadIdx.x + c * kThreads;
+        if (i < n_vec) {
+            cache[c] = __ldg(row + i);
+            m = absmax_bits(m, cache[c]);
+        }
+    }
+    for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads)
+        m = absmax_bits(m, __ldg(row + i));
+
+    m = __reduce_max_sync(0xffffffffu, m);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (lane == 0) s_max[warp] = m;
+    __syncthreads();
+    m = s_max[0];
+#pragma unroll
+    for (int w = 1; w < kThreads / 32; ++w) m = max(m, s_max[w]);
+
+    const float amax = __uint_as_float(m << 16);
+    const float b = fmaxf(amax, kBetaFloor);
+    const float s = __fdiv_rn((float)kQb, b); // one IEEE divide per token
+
+    int sum = 0;
+#pragma unroll
+    for (int c = 0; c < kCache; ++c) {
+        const int i = threadIdx.x + c * kThreads;
+        if (i < n_vec) {
+            uint2 o;
+            sum += quant8(cache[c], s, o);
+            out[i] = o;
+        }
+    }
+    for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) {
+        uint2 o;
+        sum += quant8(__ldg(row + i), s, o);
+        out[i] = o;
+    }
+    sum = __reduce_add_sync(0xffffffffu, sum);
+    if (lane == 0) s_sum[warp] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int tot = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) tot += s_sum[w];
+        e.beta[t] = b;
+        e.rowsum[t] = tot;
+    }
+}
+
+} // namespace
+
+cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
+                                 void *zero_ptr, size_t zero_bytes, cudaStream_t stream)
+{
+    const size_t zero_vecs = zero_bytes / 16;
+    int zero_blocks = 0;
+    if (zero_vecs > 0) {
+        zero_blocks = (int)((zero_vecs + kThreads * 4 - 1) / (kThreads * 4));
+        const int cap = sm_count() * 4;
+        if (zero_blocks > cap) zero_blocks = cap;
+        if (zero_blocks < 1) zero_blocks = 1;
+    }
+    const int grid = total_tokens + zero_blocks;
+    if (grid == 0) return cudaSuccess;
+    quantize_acts_kernel<<<grid, kThreads, 0, stream>>>(inl, table, n_entries, total_tokens,
+                                                        reinterpret_cast<uint4 *>(zero_ptr), zero_vecs);
+    return cudaGetLastError();
+}
+
+} // namespace bitlinear
