@@ -1,0 +1,451 @@
+#!/usr/bin/env python
+"""Benchmark of the BitLinear forward (BitNet b1.58) on B200.
+
+Headline workload: the 3B-shaped decode step -- all 26 x 7 BitLinear projections of the decoder at
+M = 1 token, 805 MB of 2-bit weights resident in HBM -- run through bitlinear_forward_sequence.
+One "step" = activation quantisation + ternary matmul + dequantisation for all 182 matrices.
+Metric: packed-weight GB/s = (sum of N*K/4 bytes) / step time.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--no-extras]
+
+Prints one JSON line.  With --gpus N > 1 (under torchrun) every rank runs an independent replica of
+the workload on its own GPU ("replicas only": the path needs no exchange) and the aggregate is
+reported.  --impl reference times the CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+sys.path.insert(0, str(ROOT))
+
+METRIC = "decode BitLinear packed-weight GB/s"
+UNIT = "GB/s"
+WORKLOAD = "3b_decode"
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
+# summarised under profiles/ (null until a capture exists for the workload).
+NCU_TRAFFIC_BYTES = {"3b_decode": None}
+
+
+def measured_peaks():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        d = json.loads(p.read_text())
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# ---------------------------------------------------------------------------------------------------
+# clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": []}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                smax.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.unlink(self.file.name)
+        except OSError:
+            pass
+        if sm:
+            out["sm_mhz"] = statistics.median(sm)
+            out["sm_max_mhz"] = max(smax)
+            out["samples"] = len(sm)
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------------------------------
+# workloads (CUDA arm)
+
+class Stack:
+    """A list of BitLinear matrices with resident packed weights, one contiguous X and Y buffer."""
+
+    def __init__(self, layer_shapes, n_layers, M, outlier_frac=0.0, outlier_scale=1.0, copies=1, seed_base=0):
+        import torch
+        from paper_2402_17764_b200 import binding as B
+        from paper_2402_17764_b200 import synthetic as S
+        self.M = M
+        entries = [(li, mi, sh) for li in range(n_layers * copies) for mi, sh in enumerate(layer_shapes)]
+        a256 = lambda n: (n + 255) // 256 * 256
+        pk_sizes = [a256(B.packed_bytes(sh.N, sh.K)) for _, _, sh in entries]
+        self.packed_all = torch.empty(sum(pk_sizes), dtype=torch.uint8, device="cuda")
+        self.gammas = torch.empty(len(entries), dtype=torch.float32, device="cuda")
+        x_sizes = [a256(M * sh.K * 2) // 2 for _, _, sh in entries]
+        y_sizes = [a256(M * sh.N * 2) // 2 for _, _, sh in entries]
+        self.X_all = torch.empty(sum(x_sizes), dtype=torch.bfloat16, device="cuda")
+        self.Y_all = torch.zeros(sum(y_sizes), dtype=torch.bfloat16, device="cuda")
+        self.layers = []
+        self.algorithmic_bytes = 0
+        self.int_ops = 0
+        po = xo = yo = 0
+        for i, (li, mi, sh) in enumerate(entries):
+            seed = seed_base + li * 16 + mi
+            W = S.latent_weights(sh.N, sh.K, seed, device="cuda")
+            packed = self.packed_all[po:po + B.packed_bytes(sh.N, sh.K)]
+            gamma = self.gammas[i:i + 1]
+            B.quantize_weights(W, 1e-5, packed=packed, gamma=gamma)
+            del W
+            X = self.X_all[xo:xo + M * sh.K].view(M, sh.K)
+            X.copy_(S.activations(M, sh.K, seed, device="cuda", outlier_frac=outlier_frac, outlier_scale=outlier_scale))
+            Y = self.Y_all[yo:yo + M * sh.N].view(M, sh.N)
+            self.layers.append((packed, gamma, X, Y, sh.N))
+            self.algorithmic_bytes += S.packed_weight_bytes(sh.N, sh.K)
+            self.int_ops += 2 * M * sh.N * sh.K
+            po += pk_sizes[i]
+            xo += x_sizes[i]
+            yo += y_sizes[i]
+        torch.cuda.synchronize()
+
+
+def time_sequence(stack, steps, warmup, dist_barrier=None):
+    """-> (ms per step over the whole timed region, ms per launch of the matmul kernel alone)."""
+    import torch
+    from paper_2402_17764_b200 import binding as B
+    seq = B.Sequence(stack.layers)
+    for _ in range(warmup):
+        seq.forward()
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    mids = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+    start.record()
+    for a, b in mids:
+        seq.forward_stage(1)   # activation quantiser (all matrices)
+        a.record()
+        seq.forward_stage(2)   # persistent matmul + dequantisation (all matrices)
+        b.record()
+    end.record()
+    torch.cuda.synchronize()
+    if dist_barrier:
+        dist_barrier()
+    status = B.poll_status(seq.workspace)
+    if status != 0:
+        raise RuntimeError(f"device status {status}")
+    total = start.elapsed_time(end) / steps
+    kern = sum(a.elapsed_time(b) for a, b in mids) / steps
+    seq.close()
+    return total, kern
+
+
+def time_e2e(stack, steps, warmup):
+    """Host buffers in, host buffers out: per step one H2D copy of all X, the sequence, one D2H copy of all Y."""
+    import torch
+    from paper_2402_17764_b200 import binding as B
+    seq = B.Sequence(stack.layers)
+    x_host = stack.X_all.cpu().pin_memory()
+    y_host = torch.empty_like(stack.Y_all, device="cpu").pin_memory()
+    def step():
+        stack.X_all.copy_(x_host, non_blocking=True)
+        seq.forward()
+        y_host.copy_(stack.Y_all, non_blocking=True)
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for _ in range(steps):
+        step()
+    end.record()
+    torch.cuda.synchronize()
+    ms = start.elapsed_time(end) / steps
+    seq.close()
+    return ms, x_host.numel() * 2, y_host.numel() * 2
+
+
+def time_forward_calls(fn, iters, warmup=3):
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    s, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s.record()
+    for _ in range(iters):
+        fn()
+    e.record()
+    torch.cuda.synchronize()
+    return s.elapsed_time(e) / iters
+
+
+def extras(peaks):
+    """Other workloads of the benchmark definition, reported beside the headline (1 GPU only)."""
+    import torch
+    from paper_2402_17764_b200 import binding as B
+    from paper_2402_17764_b200 import synthetic as S
+    out = {}
+    hbm = peaks["hbm_gbs"]
+    int8_peak = peaks["bf16_tflops"] * 2.0  # dense int8 nominal ratio to bf16 is 2x
+
+    # single BitLinear, M=8, K=1536, N=4096 (fits L2: a latency number, not a bandwidth one)
+    cfg = S.CONFIGS["single"]
+    st = Stack(cfg["layers"], 1, 8, cfg["outlier_frac"], cfg["outlier_scale"])
+    packed, gamma, X, Y, N = st.layers[0]
+    ws = B.alloc_workspace(8, N, X.shape[1])
+    us = time_forward_calls(lambda: B.forward(packed, gamma, X, N, Y=Y, workspace=ws), 200) * 1e3
+    out["single_M8_K1536_N4096"] = {"us_per_call": round(us, 2), "note": "L2-resident, launch-bound"}
+    del st
+
+    # 7B-shaped batched decode: each shape as a sequence of distinct copies (> L2) so reads come from HBM
+    cfg = S.CONFIGS["7b_batched"]
+    res = {}
+    for sh in cfg["layers"]:
+        copies = max(2, int(400e6 // S.packed_weight_bytes(sh.N, sh.K)))
+        for M in cfg["M"]:
+            st = Stack([sh], 1, M, cfg["outlier_frac"], cfg["outlier_scale"], copies=copies)
+            ms, kern = time_sequence(st, 10, 3)
+            gbs = st.algorithmic_bytes / (ms * 1e-3) / 1e9
+            res[f"{sh.N}x{sh.K}_M{M}"] = {"GB/s": round(gbs, 1), "frac_hbm_measured": round(gbs / hbm, 3),
+                                          "TOPS": round(st.int_ops / (ms * 1e-3) / 1e12, 2)}
+            del st
+    out["decode_7b_shapes"] = res
+
+    # 13B-shaped prefill: bitlinear_forward (quantiser + tensor-core GEMM + epilogue)
+    cfg = S.CONFIGS["13b_prefill"]
+    res = {}
+    for sh in cfg["layers"]:
+        W = S.latent_weights(sh.N, sh.K, 0, device="cuda")
+        packed, gamma = B.quantize_weights(W)
+        del W
+        for M in cfg["M"]:
+            X = S.activations(M, sh.K, 0, device="cuda")
+            Y = torch.empty((M, sh.N), dtype=torch.bfloat16, device="cuda")
+            ws = B.alloc_workspace(M, sh.N, sh.K)
+            iters = 20 if M <= 2048 else 8
+            ms = time_forward_calls(lambda: B.forward(packed, gamma, X, sh.N, Y=Y, workspace=ws), iters)
+            ms_q = time_forward_calls(lambda: B.quantize_acts(X), iters)
+            tops = 2.0 * M * sh.N * sh.K / (ms * 1e-3) / 1e12
+            tops_gemm = 2.0 * M * sh.N * sh.K / (max(ms - ms_q, 1e-6) * 1e-3) / 1e12
+            res[f"{sh.N}x{sh.K}_M{M}"] = {"ms": round(ms, 4), "TOPS": round(tops, 1), "TOPS_gemm_only": round(tops_gemm, 1),
+                                          "frac_int8_nominal_4500": round(tops / 4500.0, 3),
+                                          "frac_2x_measured_bf16": round(tops / int8_peak, 3)}
+            del X, Y, ws
+    out["prefill_13b_shapes"] = res
+
+    # 70B-shaped full decode step: 80 layers, 17.1 GB of packed weights resident
+    cfg = S.CONFIGS["70b_decode"]
+    res = {}
+    for M in cfg["M"]:
+        st = Stack(cfg["layers"], cfg["n_layers"], M)
+        ms, kern = time_sequence(st, 5, 3)
+        gbs = st.algorithmic_bytes / (ms * 1e-3) / 1e9
+        res[f"M{M}"] = {"ms_per_step": round(ms, 3), "GB/s": round(gbs, 1), "frac_hbm_measured": round(gbs / hbm, 3),
+                        "packed_bytes": st.algorithmic_bytes}
+        del st
+        torch.cuda.empty_cache()
+    out["decode_70b_step"] = res
+    return out
+
+
+# ---------------------------------------------------------------------------------------------------
+# CPU oracle legs
+
+def _bf16_bits(t):
+    import numpy as np
+    import torch
+    return t.contiguous().view(torch.int16).numpy().view(np.uint16)
+
+
+class OracleSample:
+    def __init__(self):
+        from oracle import load_oracle
+        from paper_2402_17764_b200 import synthetic as S
+        self.orc = load_oracle("timing")
+        cfg = S.CONFIGS[WORKLOAD]
+        self.items = []
+        self.bytes = 0
+        for mi, sh in enumerate(cfg["layers"]):
+            W = S.latent_weights(sh.N, sh.K, mi)
+            T, g = self.orc.quantize_weights(W.numpy())
+            X = _bf16_bits(S.activations(1, sh.K, mi))
+            self.items.append((T, g, X))
+            self.bytes += S.packed_weight_bytes(sh.N, sh.K)
+        self.cores = self.orc.num_threads()
+        self.sample = "1 of 26 decoder layers (7 matrices, M=1): activation quantiser + int32 matmul + dequantisation"
+
+    def step(self):
+        for T, g, X in self.items:
+            self.orc.forward(T, g, X)
+
+
+def cpu_baseline(budget_s=10.0):
+    smp = OracleSample()
+    smp.step()
+    t0 = time.perf_counter()
+    smp.step()
+    one = time.perf_counter() - t0
+    reps = max(3, min(200, int(budget_s / max(one, 1e-4))))
+    t0 = time.perf_counter()
+    for _ in range(reps):
+        smp.step()
+    dt = time.perf_counter() - t0
+    return {"value": round(smp.bytes * reps / dt / 1e9, 3), "unit": UNIT, "cores": smp.cores, "kind": "oracle",
+            "sample": f"{smp.sample}, {reps} repetitions"}
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    smp = OracleSample()
+    for _ in range(args.warmup):
+        smp.step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        smp.step()
+    dt = time.perf_counter() - t0
+    value = smp.bytes * args.steps / dt / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": round(value, 3), "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": round(dt / args.steps * 1e3, 3),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "note": "CPU oracle on the host cores; each step is a bounded sample"},
+        "cpu_baseline": {"value": round(value, 3), "unit": UNIT, "cores": smp.cores, "kind": "oracle", "sample": smp.sample},
+        "e2e": {"value": round(value, 3), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        torch.cuda.set_device(0)
+    from paper_2402_17764_b200 import build, binding as B
+    from paper_2402_17764_b200 import synthetic as S
+    if rank == 0:
+        build.build()
+    if dist:
+        dist.barrier()
+    B.load_library()
+    peaks = measured_peaks()
+
+    cfg = S.CONFIGS[WORKLOAD]
+    stack = Stack(cfg["layers"], cfg["n_layers"], 1)
+    barrier = (lambda: dist.barrier()) if dist else None
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ms_step, ms_kernel = time_sequence(stack, args.steps, args.warmup, barrier)
+    clocks = sampler.stop()
+    ms_e2e, h2d, d2h = time_e2e(stack, max(10, args.steps // 4), 3)
+
+    if dist:
+        t = torch.tensor([ms_step, ms_kernel, ms_e2e], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_step, ms_kernel, ms_e2e = t.tolist()
+
+    n = world
+    value = n * stack.algorithmic_bytes / (ms_step * 1e-3) / 1e9
+    e2e_value = n * stack.algorithmic_bytes / (ms_e2e * 1e-3) / 1e9
+    achieved = stack.algorithmic_bytes / (ms_kernel * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": n, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(ms_step, 4), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "M": 1, "matrices": len(stack.layers),
+                   "packed_weight_bytes": stack.algorithmic_bytes,
+                   "launch": "bitlinear_forward_sequence: 1 quantiser launch + 1 persistent matmul launch per step",
+                   "l2": "inputs (805 MB of weights per step) larger than L2; no flush needed",
+                   "parallelism": "replicas only" if n > 1 else "1 GPU"},
+        "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel<1>", "achieved": round(achieved, 1),
+                     "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
+                     "frac": round(achieved / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(achieved / 8000.0, 4),
+                     "traffic": NCU_TRAFFIC_BYTES.get(WORKLOAD)},
+        "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": round(ms_e2e, 4)},
+        "gpu_launches": 2 * args.steps,
+        "clocks": clocks,
+    }
+    if rank == 0 and n == 1:
+        line["cpu_baseline"] = cpu_baseline()
+        if not args.no_extras:
+            del stack
+            torch.cuda.empty_cache()
+            line["extra"] = extras(peaks)
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if dist:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-extras", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()
