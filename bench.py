@@ -431,14 +431,54 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def profile_case(name: str):
+    """Small fixed cases for `ncu`: inputs larger than L2, well under a GB on the device, few launches."""
+    import torch
+    from paper_2402_17764_b200 import build, binding as B
+    from paper_2402_17764_b200 import synthetic as S
+    torch.cuda.set_device(0)
+    build.build()
+    if name.startswith("decode"):
+        # 48 distinct 11008x4096 matrices (541 MB of packed weights) at M = 1 (or M given as decode:M)
+        M = int(name.split(":")[1]) if ":" in name else 1
+        st = Stack([S.LayerShape("up", 11008, 4096)], 1, M, copies=48)
+        seq = B.Sequence(st.layers)
+        for _ in range(3):
+            seq.forward()
+        torch.cuda.synchronize()
+        ms = time_forward_calls(lambda: seq.forward_stage(2), 20)
+        print(json.dumps({"case": name, "packed_bytes_per_launch": st.algorithmic_bytes,
+                          "matmul_kernel_ms": round(ms, 4), "GB/s": round(st.algorithmic_bytes / ms / 1e6, 1)}))
+    elif name.startswith("prefill"):
+        # 13824x5120 at M = 2048 (or prefill:M): 290 G integer operations per launch
+        M = int(name.split(":")[1]) if ":" in name else 2048
+        W = S.latent_weights(13824, 5120, 0, device="cuda")
+        packed, gamma = B.quantize_weights(W)
+        X = S.activations(M, 5120, 0, device="cuda")
+        ws = B.alloc_workspace(M, 13824, 5120)
+        for _ in range(3):
+            B.forward(packed, gamma, X, 13824, workspace=ws)
+        torch.cuda.synchronize()
+        ms = time_forward_calls(lambda: B.forward(packed, gamma, X, 13824, workspace=ws), 20)
+        ops = 2 * M * 13824 * 5120
+        print(json.dumps({"case": name, "int_ops_per_launch": ops, "forward_ms": round(ms, 4),
+                          "TOPS": round(ops / ms / 1e9, 1)}))
+    else:
+        raise SystemExit(f"unknown profile case {name}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
-    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true")
+    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M] | prefill[:M]) and exit")
     args = ap.parse_args()
+    if args.profile_case:
+        profile_case(args.profile_case)
+        return
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":

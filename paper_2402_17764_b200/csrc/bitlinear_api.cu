@@ -163,7 +163,7 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, cudaStream_t stre
         s.out = reinterpret_cast<char *>(e.out) + (size_t)m0 * e.N * elt;
         if (M > kMaxDecodeM) s.ksplit = 1; // no split-K scratch is laid out for large M
         if (m0 > 0) {
-            cudaError_t err = cudaMemsetAsync(&hdr->unit_counter, 0, sizeof(uint32_t), stream);
+            cudaError_t err = cudaMemsetAsync(&hdr->unit_counter[0][0], 0, sizeof(hdr->unit_counter), stream);
             if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
         }
         InlineTable inl{};

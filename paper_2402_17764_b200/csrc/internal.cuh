@@ -16,13 +16,16 @@ constexpr int kTileCols = 128;
 constexpr int kTileBytes = 512;
 constexpr int kMaxDecodeM = 64;
 
-// Workspace header (first 256 bytes of every workspace).
+// Workspace header (start of every workspace).  Work units of the persistent decode kernel are dealt
+// out by kStripes counters, each in a 128-byte line of its own: stripe c hands out units c, c + kStripes,
+// c + 2 kStripes, ...  One shared counter would serialise every warp of the GPU on one L2 atomic.
+constexpr int kStripes = 64;
 struct WorkspaceHeader {
-    int32_t status;        // BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT, written by kernels
-    uint32_t unit_counter; // dynamic work counter of the persistent decode kernel
-    uint32_t reserved[62];
+    int32_t status; // BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT, written by kernels
+    uint32_t reserved[63];
+    uint32_t unit_counter[kStripes][32]; // [c][0] is the counter of stripe c
 };
-static_assert(sizeof(WorkspaceHeader) == 256, "header is 256 bytes");
+static_assert(sizeof(WorkspaceHeader) == 256 + kStripes * 128, "header layout");
 
 // One matmul of a decode launch, as the kernels see it (device memory or kernel parameter).
 struct DecodeEntry {
