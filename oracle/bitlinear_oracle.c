@@ -152,55 +152,55 @@ int oracle_quantize_weights(const float *W, int64_t N, int64_t K, float eps, int
 
 /* ---------- R9: 2-bit storage ---------- */
 
-static int64_t padded_K(int64_t K) { return (K + 127) / 128 * 128; }
+static int64_t col_tiles(int64_t K) { return (K + 63) / 64; }
+static int64_t row_blocks(int64_t N) { return (N + 63) / 64; }
 
 int64_t oracle_packed_bytes(int64_t N, int64_t K)
 {
     if (N <= 0 || K <= 0 || (N % 16) != 0)
         return -1;
-    return N * padded_K(K) / 4;
+    return row_blocks(N) * col_tiles(K) * 1024;
 }
 
 /*
- * Where weight (n, k) lives.  The matrix is cut into tiles of 16 rows by 128
- * columns, 512 bytes each, stored one after another with the column-tile index
- * running fastest.  A tile is 128 little-endian 32-bit words.  Within a tile,
- * with r = n mod 16 and c = k mod 128:
- *     word  = 4 * (4 * (r mod 8) + c / 32) + (c mod 32) / 8
- *     field = 2 * ((c mod 8) / 4) + r / 8          (0..3)
- *     byte  = c mod 4
- * and the code occupies bits [8*byte + 2*field, 8*byte + 2*field + 1] of that
- * word.  The stored code is t + 1, so it is 0, 1 or 2; 3 never appears.
- * Columns K..padded_K(K)-1 hold code 1 (weight zero).
+ * Where weight (n, k) lives.  The matrix is cut into tiles of 64 rows by 64
+ * columns, 1024 bytes each, stored one after another with the column-tile index
+ * running fastest.  One BYTE holds the codes of four rows at the same column.
+ * Within a tile, with r = n mod 64 and c = k mod 64, split
+ *     r = 16*f + 8*h + g        (f = 0..3, h = 0..1, g = 0..7)
+ *     c = 16*tq + 8*s + 4*hi + b  (tq = 0..3, s = 0..1, hi = 0..1, b = 0..3)
+ * and the code occupies bits [2*f, 2*f + 1] of byte
+ *     512*s + 16*(4*g + tq) + 4*(2*hi + h) + b
+ * of the tile.  The stored code is t + 1, so it is 0, 1 or 2; 3 never appears.
+ * Rows N..(multiple of 64) and columns K..(multiple of 64) hold code 1 (weight
+ * zero).
  */
-static void locate(int64_t n, int64_t k, int64_t Kp, int64_t *word_index, int *bit)
+static void locate(int64_t n, int64_t k, int64_t KB, int64_t *byte_index, int *bit)
 {
-    int64_t tile = (n / 16) * (Kp / 128) + (k / 128);
-    int r = (int)(n % 16), c = (int)(k % 128);
-    int word = 4 * (4 * (r % 8) + c / 32) + (c % 32) / 8;
-    int field = 2 * ((c % 8) / 4) + r / 8;
-    int byte = c % 4;
-    *word_index = tile * 128 + word;
-    *bit = 8 * byte + 2 * field;
+    int64_t tile = (n / 64) * KB + (k / 64);
+    int r = (int)(n % 64), c = (int)(k % 64);
+    int f = r / 16, h = (r % 16) / 8, g = r % 8;
+    int tq = c / 16, s = (c % 16) / 8, hi = (c % 8) / 4, b = c % 4;
+    *byte_index = tile * 1024 + 512 * s + 16 * (4 * g + tq) + 4 * (2 * hi + h) + b;
+    *bit = 2 * f;
 }
 
 int oracle_pack_weights(const int8_t *T, int64_t N, int64_t K, uint8_t *packed)
 {
     if (!T || !packed || N <= 0 || K <= 0 || (N % 16) != 0)
         return ORACLE_ERR_ARG;
-    int64_t Kp = padded_K(K);
-    memset(packed, 0, (size_t)(N * Kp / 4));
-    for (int64_t n = 0; n < N; ++n) {
-        for (int64_t k = 0; k < Kp; ++k) {
-            int t = (k < K) ? T[n * K + k] : 0;
+    int64_t KB = col_tiles(K), NB = row_blocks(N);
+    memset(packed, 0, (size_t)(NB * KB * 1024));
+    for (int64_t n = 0; n < NB * 64; ++n) {
+        for (int64_t k = 0; k < KB * 64; ++k) {
+            int t = (n < N && k < K) ? T[n * K + k] : 0;
             if (t < -1 || t > 1)
                 return ORACLE_ERR_ARG;
             uint32_t code = (uint32_t)(t + 1);
-            int64_t w;
+            int64_t at;
             int bit;
-            locate(n, k, Kp, &w, &bit);
-            /* little-endian 32-bit word: bit b of the word is bit (b mod 8) of byte (b / 8) */
-            packed[w * 4 + bit / 8] |= (uint8_t)(code << (bit % 8));
+            locate(n, k, KB, &at, &bit);
+            packed[at] |= (uint8_t)(code << bit);
         }
     }
     return ORACLE_OK;
@@ -210,13 +210,13 @@ int oracle_unpack_weights(const uint8_t *packed, int64_t N, int64_t K, int8_t *T
 {
     if (!T || !packed || N <= 0 || K <= 0 || (N % 16) != 0)
         return ORACLE_ERR_ARG;
-    int64_t Kp = padded_K(K);
+    int64_t KB = col_tiles(K);
     for (int64_t n = 0; n < N; ++n) {
         for (int64_t k = 0; k < K; ++k) {
-            int64_t w;
+            int64_t at;
             int bit;
-            locate(n, k, Kp, &w, &bit);
-            int code = (packed[w * 4 + bit / 8] >> (bit % 8)) & 3;
+            locate(n, k, KB, &at, &bit);
+            int code = (packed[at] >> bit) & 3;
             if (code == 3)
                 return ORACLE_ERR_ARG;
             T[n * K + k] = (int8_t)(code - 1);

@@ -81,25 +81,26 @@ def dequant(acc, beta, gamma):
 
 
 def pack_weights(T) -> np.ndarray:
-    """Walk the storage: tile -> word -> byte -> 2-bit field, and fetch the weight it holds."""
+    """Walk the storage: tile -> slab -> 16-byte slot -> word -> byte -> 2-bit field, and fetch the weight it holds."""
     T = np.asarray(T, np.int8)
     N, K = T.shape
     assert N % 16 == 0
-    Kp = (K + 127) // 128 * 128
-    tiles_per_row_block = Kp // 128
-    words = np.zeros(N * Kp // 16, np.uint32)
-    for row_block in range(N // 16):
-        for col_tile in range(tiles_per_row_block):
-            base = (row_block * tiles_per_row_block + col_tile) * 128
-            for slot in range(32):          # 32 slots of four words each
-                row_low, col_quarter = slot // 4, slot % 4
-                for i in range(4):          # the slot's four words
-                    w = 0
-                    for byte in range(4):
-                        for field in range(4):
-                            n = 16 * row_block + row_low + 8 * (field & 1)
-                            k = 128 * col_tile + 32 * col_quarter + 8 * i + 4 * (field >> 1) + byte
-                            code = int(T[n, k]) + 1 if k < K else 1
-                            w |= code << (8 * byte + 2 * field)
-                    words[base + 4 * slot + i] = w
-    return words.view(np.uint8)  # little-endian host
+    row_blocks, col_tiles = (N + 63) // 64, (K + 63) // 64
+    out = np.zeros(row_blocks * col_tiles * 1024, np.uint8)
+    at = 0
+    for row_block in range(row_blocks):
+        for col_tile in range(col_tiles):
+            for slab in range(2):               # columns 8*slab .. 8*slab+7 of every 16-column group
+                for slot in range(32):          # 32 slots of four words each
+                    row_low, col_group = slot // 4, slot % 4
+                    for word in range(4):       # word: row half = word % 2, column half = word // 2
+                        for byte in range(4):
+                            v = 0
+                            for field in range(4):
+                                n = 64 * row_block + 16 * field + 8 * (word % 2) + row_low
+                                k = 64 * col_tile + 16 * col_group + 8 * slab + 4 * (word // 2) + byte
+                                code = int(T[n, k]) + 1 if (n < N and k < K) else 1
+                                v |= code << (2 * field)
+                            out[at] = v
+                            at += 1
+    return out

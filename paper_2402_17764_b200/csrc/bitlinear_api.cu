@@ -54,36 +54,22 @@ int env_int(const char *name, int fallback)
     return std::atoi(v);
 }
 
-// Work-unit sizing of the persistent decode kernel: enough units to fill the machine, none longer
-// than `max_tiles` 128-column tiles (bounds the tail), none shorter than `min_tiles`.
-int choose_ksplit(int64_t total_row_blocks, int KB)
-{
-    static const int max_tiles = env_int("BITLINEAR_UNIT_MAX_TILES", 32);
-    static const int min_tiles = env_int("BITLINEAR_UNIT_MIN_TILES", 4);
-    const int64_t target_units = (int64_t)sm_count() * 32;
-    int split = 1;
-    if (total_row_blocks < target_units) split = (int)((target_units + total_row_blocks - 1) / total_row_blocks);
-    const int need = (KB + max_tiles - 1) / max_tiles;
-    if (split < need) split = need;
-    int cap = KB / min_tiles;
-    if (cap < 1) cap = 1;
-    if (split > cap) split = cap;
-    return split;
-}
-
 struct Layout {
     size_t counters, acc32, table, xq, beta, rowsum, total;
 };
 
-// Workspace of one matmul: [header | counters | acc32 (M <= 64 only) | Xq | beta | rowsum]
+inline int64_t row_blocks(int64_t N) { return (N + kTileRows - 1) / kTileRows; }
+inline int64_t col_tiles(int64_t K) { return (K + kTileCols - 1) / kTileCols; }
+
+// Workspace of one matmul: [header | counters | acc32 (at most 64 tokens) | Xq | beta | rowsum]
 Layout single_layout(int64_t M, int64_t N, int64_t K)
 {
     Layout L{};
     size_t off = sizeof(WorkspaceHeader);
     L.counters = off;
-    off += align_up((size_t)(N / 16) * 4, 256);
+    off += align_up((size_t)row_blocks(N) * 4, 256);
     L.acc32 = off;
-    if (M <= kMaxDecodeM) off += align_up((size_t)M * N * 4, 256);
+    off += align_up((size_t)(M < kMaxDecodeM ? M : kMaxDecodeM) * N * 4, 256);
     L.table = off;
     L.xq = off;
     off += align_up((size_t)M * K, 256);
@@ -120,7 +106,7 @@ bool use_tcgen05_for(int64_t M)
 
 // Fills one DecodeEntry for a matmul whose workspace part starts at `base`.
 void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
-                int64_t N, void *out, int out_i32, char *base, const Layout &L, int ksplit)
+                int64_t N, void *out, int out_i32, char *base, const Layout &L)
 {
     e.packed = reinterpret_cast<const uint4 *>(packed);
     e.gamma = gamma;
@@ -134,9 +120,9 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.M = (int)M;
     e.N = (int)N;
     e.K = (int)K;
-    e.KB = (int)((K + kTileCols - 1) / kTileCols);
-    e.ksplit = ksplit;
-    e.unit_begin = 0;
+    e.KB = (int)col_tiles(K);
+    e.NB = (int)row_blocks(N);
+    e.tile_begin = 0;
     e.token_begin = 0;
     e.out_i32 = out_i32;
 }
@@ -161,16 +147,10 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, cudaStream_t stre
         s.rowsum = e.rowsum + m0;
         const size_t elt = e.out_i32 ? 4 : 2;
         s.out = reinterpret_cast<char *>(e.out) + (size_t)m0 * e.N * elt;
-        if (M > kMaxDecodeM) s.ksplit = 1; // no split-K scratch is laid out for large M
-        if (m0 > 0) {
-            cudaError_t err = cudaMemsetAsync(&hdr->unit_counter[0][0], 0, sizeof(hdr->unit_counter), stream);
-            if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
-        }
         InlineTable inl{};
         inl.e[0] = s;
-        const int units = (s.N / kTileRows) * s.ksplit;
-        cudaError_t err = launch_decode(inl, nullptr, 1, units, s.M, path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA,
-                                        hdr, stream);
+        cudaError_t err = launch_decode(inl, nullptr, 1, (uint32_t)(s.NB * s.KB), s.M,
+                                        path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, stream);
         if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
     return BITLINEAR_OK;
@@ -202,8 +182,7 @@ const char *bitlinear_status_string(bitlinear_status s)
 size_t bitlinear_packed_bytes(int64_t N, int64_t K)
 {
     if (check_shape(0, N, K) != BITLINEAR_OK) return 0;
-    const int64_t Kp = (K + kTileCols - 1) / kTileCols * kTileCols;
-    return (size_t)(N * Kp / 4);
+    return (size_t)(row_blocks(N) * col_tiles(K)) * kTileBytes;
 }
 
 size_t bitlinear_workspace_bytes(int64_t M, int64_t N, int64_t K)
@@ -259,12 +238,9 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     if (M == 0) return BITLINEAR_OK;
     char *ws = reinterpret_cast<char *>(workspace);
     InlineTable inl{};
-    const int KB = (int)((K + kTileCols - 1) / kTileCols);
-    const bool tc = use_tcgen05_for(M);
-    const int ksplit = (M <= kMaxDecodeM && !tc) ? choose_ksplit(N / 16, KB) : 1;
-    fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L, ksplit);
-    // quantise the tokens; the same launch clears the header and (when splitting K) the scratch
-    const size_t zero_bytes = (ksplit > 1) ? L.table : sizeof(WorkspaceHeader);
+    fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L);
+    // quantise the tokens; the same launch clears the header and, for the streaming kernel, its scratch
+    const size_t zero_bytes = use_tcgen05_for(M) ? sizeof(WorkspaceHeader) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, (cudaStream_t)stream);
@@ -287,13 +263,11 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     if (M == 0) return BITLINEAR_OK;
     char *ws = reinterpret_cast<char *>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
-    const int KB = (int)((K + kTileCols - 1) / kTileCols);
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
-    const int ksplit = (M <= kMaxDecodeM && !tc) ? choose_ksplit(N / 16, KB) : 1;
     InlineTable inl{};
-    fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L, ksplit);
+    fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
     inl.e[0].Xq = const_cast<int8_t *>(Xq); // read only on this path
-    const size_t zero_bytes = (ksplit > 1) ? L.table : sizeof(WorkspaceHeader);
+    const size_t zero_bytes = tc ? sizeof(WorkspaceHeader) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, s);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
@@ -327,7 +301,8 @@ bitlinear_status bitlinear_poll_status(const void *workspace, void *stream, int 
 
 struct bitlinear_sequence {
     char *workspace;
-    int n, units, tokens, max_M;
+    int n, tokens, max_M;
+    uint32_t tiles;
     size_t zero_bytes;
     const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
     bitlinear::InlineTable inl;
@@ -342,14 +317,17 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
 {
     if (!layers || n <= 0 || n > 65536) return false;
     size_t counters = 0, acc = 0, data = 0;
+    uint64_t tiles = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1 || d.M > kMaxDecodeM) return false;
-        counters += align_up((size_t)(d.N / 16) * 4, 256);
+        counters += align_up((size_t)row_blocks(d.N) * 4, 256);
         acc += align_up((size_t)d.M * d.N * 4, 256);
+        tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K));
         if (entry_off) entry_off->push_back(data);
         data += align_up((size_t)d.M * d.K, 256) + 2 * align_up((size_t)d.M * 4, 256);
     }
+    if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
     size_t off = sizeof(WorkspaceHeader);
     S.counters = off;
     off += counters;
@@ -390,12 +368,10 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
     char *ws = reinterpret_cast<char *>(workspace);
 
-    int64_t total_rb = 0;
-    for (int i = 0; i < n; ++i) total_rb += layers[i].N / 16;
     std::vector<DecodeEntry> table((size_t)n);
     size_t c_off = S.counters, a_off = S.acc32;
-    int units = 0, tokens = 0, max_M = 0;
-    bool any_split = false;
+    uint32_t tiles = 0;
+    int tokens = 0, max_M = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         Layout L{};
@@ -404,15 +380,12 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
         L.xq = S.data + entry_off[(size_t)i];
         L.beta = L.xq + align_up((size_t)d.M * d.K, 256);
         L.rowsum = L.beta + align_up((size_t)d.M * 4, 256);
-        c_off += align_up((size_t)(d.N / 16) * 4, 256);
+        c_off += align_up((size_t)row_blocks(d.N) * 4, 256);
         a_off += align_up((size_t)d.M * d.N * 4, 256);
-        const int KB = (int)((d.K + kTileCols - 1) / kTileCols);
-        const int ksplit = choose_ksplit(total_rb, KB);
-        any_split |= ksplit > 1;
-        fill_entry(table[(size_t)i], d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L, ksplit);
-        table[(size_t)i].unit_begin = units;
+        fill_entry(table[(size_t)i], d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
+        table[(size_t)i].tile_begin = tiles;
         table[(size_t)i].token_begin = tokens;
-        units += (int)(d.N / 16) * ksplit;
+        tiles += (uint32_t)(table[(size_t)i].NB * table[(size_t)i].KB);
         tokens += (int)d.M;
         if ((int)d.M > max_M) max_M = (int)d.M;
     }
@@ -420,10 +393,10 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     if (!seq) return BITLINEAR_ERR_ARG;
     seq->workspace = ws;
     seq->n = n;
-    seq->units = units;
+    seq->tiles = tiles;
     seq->tokens = tokens;
     seq->max_M = max_M;
-    seq->zero_bytes = any_split ? S.table : sizeof(WorkspaceHeader);
+    seq->zero_bytes = S.table; // header, arrival counters and int32 scratch
     seq->dev_table = nullptr;
     if (n <= kInlineEntries) {
         for (int i = 0; i < n; ++i) seq->inl.e[i] = table[(size_t)i];
@@ -448,7 +421,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
             cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     if (stage != 1 &&
-        launch_decode(seq->inl, seq->dev_table, seq->n, seq->units, seq->max_M, BITLINEAR_PATH_MMA,
+        launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
                       reinterpret_cast<WorkspaceHeader *>(seq->workspace), s) != cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;

@@ -11,21 +11,17 @@ namespace bitlinear {
 
 constexpr int kQb = 127;            // Section 2: activations scaled to [-Qb, Qb]
 constexpr float kBetaFloor = 1e-5f; // zero-token guard on the per-token absmax
-constexpr int kTileRows = 16;       // packed tile: 16 rows x 128 columns = 512 bytes
-constexpr int kTileCols = 128;
-constexpr int kTileBytes = 512;
+constexpr int kTileRows = 64;       // packed tile: 64 rows x 64 columns = 1024 bytes
+constexpr int kTileCols = 64;
+constexpr int kTileBytes = 1024;
 constexpr int kMaxDecodeM = 64;
 
-// Workspace header (start of every workspace).  Work units of the persistent decode kernel are dealt
-// out by kStripes counters, each in a 128-byte line of its own: stripe c hands out units c, c + kStripes,
-// c + 2 kStripes, ...  One shared counter would serialise every warp of the GPU on one L2 atomic.
-constexpr int kStripes = 64;
+// Workspace header (start of every workspace).
 struct WorkspaceHeader {
     int32_t status; // BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT, written by kernels
     uint32_t reserved[63];
-    uint32_t unit_counter[kStripes][32]; // [c][0] is the counter of stripe c
 };
-static_assert(sizeof(WorkspaceHeader) == 256 + kStripes * 128, "header layout");
+static_assert(sizeof(WorkspaceHeader) == 256, "header layout");
 
 // One matmul of a decode launch, as the kernels see it (device memory or kernel parameter).
 struct DecodeEntry {
@@ -36,11 +32,11 @@ struct DecodeEntry {
     float *beta;           // [M]
     int32_t *rowsum;       // [M]
     void *out;             // bf16 [M, N], or int32 [M, N] when out_i32
-    int32_t *acc32;        // split-K scratch [M, N] (zero before and after a launch)
-    uint32_t *counters;    // split-K arrival counters [N/16] (zero before and after a launch)
-    int M, N, K, KB;       // KB = padded K / 128
-    int ksplit;            // k splits per row block (1 = none)
-    int unit_begin;        // first work unit of this entry; units = (N/16) * ksplit
+    int32_t *acc32;        // scratch [M, N] for row blocks shared by several warps (zero before and after a launch)
+    uint32_t *counters;    // column tiles arrived, one counter per row block (zero before and after a launch)
+    int M, N, K;
+    int KB, NB;            // column tiles = ceil(K / 64), row blocks = ceil(N / 64)
+    uint32_t tile_begin;   // index of this entry's first tile in the launch-wide tile sequence (NB * KB tiles each)
     int token_begin;       // first token of this entry in the batched quantiser's grid
     int out_i32;           // 1: write raw int32 accumulators instead of bf16
 };
@@ -63,9 +59,10 @@ cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, c
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
                                  void *zero_ptr, size_t zero_bytes, cudaStream_t stream);
 
-// Persistent weight-streaming matmul over the entries. path: BITLINEAR_PATH_MMA or BITLINEAR_PATH_DP4A.
-cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_units, int max_M,
-                          int path, WorkspaceHeader *hdr, cudaStream_t stream);
+// Persistent weight-streaming matmul over the entries (total_tiles = sum of NB * KB).
+// path: BITLINEAR_PATH_MMA, or BITLINEAR_PATH_DP4A (first entry only).
+cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
+                          int max_M, int path, WorkspaceHeader *hdr, cudaStream_t stream);
 
 // Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) or raw int32.
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,

@@ -100,62 +100,65 @@ __global__ void __launch_bounds__(256) absmean_kernel(const float4 *__restrict__
     }
 }
 
-// One warp per 16 x 128 tile; lane (g = lane / 4, tq = lane % 4) owns rows g and g + 8,
-// columns 32 * tq .. 32 * tq + 31 of the tile and writes its four 32-bit words as one 16-byte store.
-__global__ void __launch_bounds__(256) ternarize_pack_kernel(const float *__restrict__ W, int N, int K, int KB,
+// One warp per tile of 64 rows x 64 columns (1 KiB = two slabs of 512 bytes).  Lane (g = lane / 4,
+// tq = lane % 4) owns rows 16 f + 8 h + g (f = 0..3, h = 0, 1) and columns 16 tq .. 16 tq + 15 of the tile:
+// the code of row (f, h), column 16 tq + 8 s + 4 hi + b goes to slab s, word 2 hi + h, byte b, bits 2f, 2f+1
+// of the lane's 16 bytes.  Rows >= N and columns >= K hold code 1 (weight 0).
+__global__ void __launch_bounds__(256) ternarize_pack_kernel(const float *__restrict__ W, int N, int K, int NB, int KB,
                                                              float eps, const float *__restrict__ gamma,
                                                              uint4 *__restrict__ packed)
 {
-    const long long n_tiles = (long long)(N / kTileRows) * KB;
+    const long long n_tiles = (long long)NB * KB;
     const int lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
     const float denom = __fadd_rn(*gamma, eps); // Eq. 1: gamma + eps
     for (long long tile = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < n_tiles;
          tile += (long long)gridDim.x * (blockDim.x >> 5)) {
         const int rb = (int)(tile / KB), kb = (int)(tile % KB);
-        uint32_t words[4] = {0u, 0u, 0u, 0u};
+        uint32_t words[2][4] = {{0u, 0u, 0u, 0u}, {0u, 0u, 0u, 0u}};
+        const int col0 = kb * kTileCols + 16 * tq;
 #pragma unroll
-        for (int half = 0; half < 2; ++half) { // row g, then row g + 8
-            const float *row = W + (size_t)(rb * kTileRows + g + 8 * half) * K;
-            const int col0 = kb * kTileCols + 32 * tq;
+        for (int f = 0; f < 4; ++f) {
 #pragma unroll
-            for (int v = 0; v < 8; ++v) { // eight float4 = 32 columns
-                const int col = col0 + 4 * v;
-                uint32_t codes = 0x01010101u; // padding: weight 0
-                if (col < K) {
-                    float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
-                    const float f[4] = {w.x, w.y, w.z, w.w};
-                    codes = 0;
+            for (int h = 0; h < 2; ++h) {
+                const int n = rb * kTileRows + 16 * f + 8 * h + g;
+                const float *row = W + (size_t)n * K;
 #pragma unroll
-                    for (int b = 0; b < 4; ++b) {
-                        int t = __float2int_rn(__fdiv_rn(f[b], denom)); // round half to even (Eq. 2)
-                        t = max(-1, min(1, t));
-                        codes |= (uint32_t)(t + 1) << (8 * b);
+                for (int v = 0; v < 4; ++v) { // four float4 = 16 columns; v = 2 s + hi
+                    const int col = col0 + 4 * v;
+                    uint32_t codes = 0x01010101u; // padding: weight 0
+                    if (n < N && col < K) {
+                        float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
+                        const float x[4] = {w.x, w.y, w.z, w.w};
+                        codes = 0;
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            int t = __float2int_rn(__fdiv_rn(x[b], denom)); // round half to even (Eq. 2)
+                            t = max(-1, min(1, t));
+                            codes |= (uint32_t)(t + 1) << (8 * b);
+                        }
                     }
+                    words[v >> 1][2 * (v & 1) + h] |= codes << (2 * f);
                 }
-                // float4 v covers columns 8*i + 4*(f>>1) + b with i = v / 2, f>>1 = v % 2, and f&1 = half
-                const int i = v >> 1;
-                const int field = 2 * (v & 1) + half;
-                words[i] |= codes << (2 * field);
             }
         }
-        packed[tile * 32 + lane] = make_uint4(words[0], words[1], words[2], words[3]);
+        packed[tile * 64 + lane] = make_uint4(words[0][0], words[0][1], words[0][2], words[0][3]);
+        packed[tile * 64 + 32 + lane] = make_uint4(words[1][0], words[1][1], words[1][2], words[1][3]);
     }
 }
 
-__global__ void __launch_bounds__(256) unpack_kernel(const uint32_t *__restrict__ packed, int N, int K, int KB,
+__global__ void __launch_bounds__(256) unpack_kernel(const uint8_t *__restrict__ packed, int N, int K, int KB,
                                                      int8_t *__restrict__ T)
 {
     const size_t total = (size_t)N * K;
     for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
         const int n = (int)(idx / K), k = (int)(idx % K);
-        const size_t tile = (size_t)(n / 16) * KB + k / 128;
-        const int r = n % 16, c = k % 128;
-        const int word = 4 * (4 * (r % 8) + c / 32) + (c % 32) / 8;
-        const int field = 2 * ((c % 8) / 4) + r / 8;
-        const uint32_t w = packed[tile * 128 + word];
-        const int code = (w >> (8 * (c % 4) + 2 * field)) & 3;
-        T[idx] = (int8_t)(code - 1);
+        const size_t tile = (size_t)(n / kTileRows) * KB + k / kTileCols;
+        const int r = n % kTileRows, c = k % kTileCols;
+        const int f = r / 16, h = (r % 16) / 8, g = r % 8;
+        const int tq = c / 16, s = (c % 16) / 8, hi = (c % 8) / 4, b = c % 4;
+        const uint8_t byte = packed[tile * kTileBytes + s * 512 + (4 * g + tq) * 16 + 4 * (2 * hi + h) + b];
+        T[idx] = (int8_t)(((byte >> (2 * f)) & 3) - 1);
     }
 }
 
@@ -175,10 +178,11 @@ cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float 
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     const int KB = (int)((K + kTileCols - 1) / kTileCols);
-    const long long n_tiles = (N / kTileRows) * (long long)KB;
+    const int NB = (int)((N + kTileRows - 1) / kTileRows);
+    const long long n_tiles = (long long)NB * KB;
     long long pblocks = (n_tiles + 7) / 8;
     if (pblocks > (long long)sm_count() * 16) pblocks = (long long)sm_count() * 16;
-    ternarize_pack_kernel<<<(int)pblocks, 256, 0, stream>>>(W, (int)N, (int)K, KB, eps, gamma,
+    ternarize_pack_kernel<<<(int)pblocks, 256, 0, stream>>>(W, (int)N, (int)K, NB, KB, eps, gamma,
                                                             reinterpret_cast<uint4 *>(packed));
     return cudaGetLastError();
 }
@@ -189,7 +193,7 @@ cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, c
     size_t total = (size_t)N * K;
     size_t blocks = (total + 255) / 256;
     if (blocks > (size_t)sm_count() * 32) blocks = (size_t)sm_count() * 32;
-    unpack_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint32_t *>(packed), (int)N, (int)K, KB, T);
+    unpack_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint8_t *>(packed), (int)N, (int)K, KB, T);
     return cudaGetLastError();
 }
 

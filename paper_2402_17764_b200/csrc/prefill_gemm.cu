@@ -5,13 +5,16 @@
 // belongs on the tensor cores.  Per CTA tile of 128 tokens x 256 output features, per 128-wide
 // k block:
 //   producer warp  : TMA loads the int8 activation tile (128 x 128 B, 128-byte swizzle) and the
-//                    packed 2-bit weight tile (16 row blocks x 512 B) into shared memory;
-//   expander warps : turn the 2-bit codes into signed int8 (-1/0/+1) and write them K-major with the
-//                    same 128-byte swizzle the tensor core expects;
-//   MMA warp       : one thread issues four tcgen05.mma kind::i8 (128 x 256 x 32) per k block into a
-//                    TMEM accumulator; tcgen05.commit releases the stage;
-//   epilogue warps : tcgen05.ld the finished int32 accumulators, scale by gamma * beta_t / 127,
-//                    round to bf16 and store, while the MMA warp fills the second TMEM buffer.
+//                    packed 2-bit weight tiles (4 row blocks x 2 column tiles x 1 KiB) into shared memory;
+//   expander warps : turn the 2-bit codes into unsigned bytes with ONE mask per four weights -- the field
+//                    of row 16 f + r stays where it is, so the byte is code * 4^f -- and write them
+//                    K-major with the same 128-byte swizzle the tensor core expects;
+//   MMA warp       : one thread issues four tcgen05.mma kind::i8 (128 x 256 x 32, s8 x u8) per k block
+//                    into a TMEM accumulator; tcgen05.commit releases the stage;
+//   epilogue warps : tcgen05.ld the finished int32 accumulators, undo the 4^f of their output row with an
+//                    exact shift, subtract the token's sum of q (codes are T + 1), scale by
+//                    gamma * beta_t / 127, round to bf16 and store, while the MMA warp fills the second
+//                    TMEM buffer.  |acc| <= 64 * 2 * 127 * K < 2^31 for every K the library accepts.
 // All waits are bounded; on expiry the CTA sets the workspace status to BITLINEAR_ERR_TIMEOUT,
 // every role leaves its loop, TMEM is released and the kernel returns.
 //
@@ -43,7 +46,7 @@ constexpr int kThreads = (kFirstExpanderWarp + kExpanderWarps) * 32; // 448
 
 constexpr uint32_t kABytes = BM * BK;            // 16 KiB int8 activations
 constexpr uint32_t kBBytes = BN * BK;            // 32 KiB expanded weights
-constexpr uint32_t kPBytes = (BN / 16) * 512;    //  8 KiB packed weights
+constexpr uint32_t kPBytes = (BN / kTileRows) * (BK / kTileCols) * kTileBytes; //  8 KiB packed weights
 constexpr uint32_t kStageBytes = kABytes + kBBytes + kPBytes;
 constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared memory of an SM");
@@ -61,19 +64,13 @@ struct Barriers {
 struct Params {
     const float *gamma;
     const float *beta;
+    const int32_t *rowsum;
     void *out;
-    int M, N, KB; // KB = padded K / 128
+    int M, N, KB; // KB = k blocks of 128 columns
     int tiles_m, tiles_n;
     int out_i32;
     int32_t *status;
 };
-
-__device__ __forceinline__ uint32_t expand_signed(uint32_t w, int field)
-{
-    // 2-bit codes c = T + 1 in each byte's field -> bytes holding T as signed int8:
-    // (c + 0x7F) ^ 0x80 maps 0, 1, 2 to 0xFF, 0x00, 0x01 and never carries between bytes.
-    return ((((w >> (2 * field)) & 0x03030303u) + 0x7F7F7F7Fu) ^ 0x80808080u);
-}
 
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
@@ -136,12 +133,12 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint32_t p_dst = a_dst + kABytes + kBBytes;
                     mbar_arrive_expect_tx(full, kABytes + kPBytes);
                     tma_load_2d(a_dst, &tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
-                    tma_load_2d(p_dst, &tmap_w, kb * 128, n0 / 16, full); // x = 32-bit word column (multiple of 128)
+                    tma_load_3d(p_dst, &tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
                 }
             }
         }
     } else if (warp == kMmaWarp) {
-        constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/1);
+        constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
         uint32_t it = 0, tile_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
@@ -175,8 +172,13 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
         }
     } else if (warp >= kFirstExpanderWarp) {
+        // Expander warp ew owns packed tile (row block ew / 2, column tile ew % 2) of the stage.  Lane
+        // (g, tq) holds, in its 16 bytes of each slab, the codes of rows 16 f + 8 h + g at columns
+        // 16 tq + 8 s + 4 hi + b (slab s, word 2 hi + h, byte b, field f): 16 consecutive columns of a row
+        // are words (h, 2 + h) of slab 0 followed by words (h, 2 + h) of slab 1.
         const int ew = warp - kFirstExpanderWarp;
         const int g = lane >> 2, tq = lane & 3;
+        const int rbi = ew >> 1, kti = ew & 1;
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -188,29 +190,20 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     break;
                 }
                 uint8_t *stage = smem + s * kStageBytes;
-                const uint4 *packed = reinterpret_cast<const uint4 *>(stage + kABytes + kBBytes);
+                const uint4 *packed = reinterpret_cast<const uint4 *>(stage + kABytes + kBBytes) + ew * (kTileBytes / 16);
                 uint8_t *bt = stage + kABytes;
+                const uint4 w0 = packed[lane], w1 = packed[32 + lane];
+                const uint32_t lo[2][2] = {{w0.x, w0.z}, {w0.y, w0.w}}; // [h][hi], slab 0
+                const uint32_t up[2][2] = {{w1.x, w1.z}, {w1.y, w1.w}}; // slab 1
+                const int chunk = (kti * 4 + tq) ^ g; // 16-byte chunk of the 128-byte row, swizzled by row % 8 = g
 #pragma unroll
-                for (int j = 0; j < (BN / 16) / kExpanderWarps; ++j) {
-                    const int rb = ew * ((BN / 16) / kExpanderWarps) + j; // 16-row block inside the tile
-                    const uint4 w = packed[rb * 32 + lane];
-                    const uint32_t words[4] = {w.x, w.y, w.z, w.w};
+                for (int f = 0; f < 4; ++f) {
+                    const uint32_t mask = 0x03030303u << (2 * f);
 #pragma unroll
-                    for (int half = 0; half < 2; ++half) { // row g, then row g + 8
-                        const int r = rb * 16 + g + 8 * half;
-                        // 32 columns of this row = two 16-byte chunks, chunk index 2*tq and 2*tq + 1
-                        uint4 lo, hi;
-                        lo.x = expand_signed(words[0], half);
-                        lo.y = expand_signed(words[0], 2 + half);
-                        lo.z = expand_signed(words[1], half);
-                        lo.w = expand_signed(words[1], 2 + half);
-                        hi.x = expand_signed(words[2], half);
-                        hi.y = expand_signed(words[2], 2 + half);
-                        hi.z = expand_signed(words[3], half);
-                        hi.w = expand_signed(words[3], 2 + half);
-                        uint8_t *rowp = bt + r * 128;
-                        *reinterpret_cast<uint4 *>(rowp + (((2 * tq) ^ (r & 7)) << 4)) = lo;
-                        *reinterpret_cast<uint4 *>(rowp + (((2 * tq + 1) ^ (r & 7)) << 4)) = hi;
+                    for (int h = 0; h < 2; ++h) {
+                        const int r = rbi * kTileRows + 16 * f + 8 * h + g;
+                        *reinterpret_cast<uint4 *>(bt + r * 128 + (chunk << 4)) =
+                            make_uint4(lo[h][0] & mask, lo[h][1] & mask, up[h][0] & mask, up[h][1] & mask);
                     }
                 }
                 fence_proxy_async_smem(); // generic-proxy writes -> visible to the tensor core
@@ -233,19 +226,28 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const int t = m0 + 32 * q + lane;
             const bool row_ok = t < p.M;
             float scale = 0.0f;
-            if (row_ok && !p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), (float)kQb);
+            int rowsum = 0;
+            if (row_ok) {
+                rowsum = p.rowsum[t];
+                if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), (float)kQb);
+            }
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
                 tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * BN + c * 32), v);
                 tmem_ld_wait();
                 const int n = n0 + c * 32;
+                // output row n + i carries the factor 4^f, f = ((n + i) % 64) / 16 = 2 (c % 2) + i / 16
+                const int sh_lo = 4 * (c & 1), sh_hi = sh_lo + 2;
+                int a[32];
+#pragma unroll
+                for (int i = 0; i < 32; ++i) a[i] = ((int)v[i] >> (i < 16 ? sh_lo : sh_hi)) - rowsum;
                 if (row_ok) {
                     if (p.out_i32) {
                         int32_t *dst = reinterpret_cast<int32_t *>(p.out) + (size_t)t * p.N + n;
 #pragma unroll
                         for (int i = 0; i < 32; i += 4)
-                            if (n + i < p.N) *reinterpret_cast<uint4 *>(dst + i) = make_uint4(v[i], v[i + 1], v[i + 2], v[i + 3]);
+                            if (n + i < p.N) *reinterpret_cast<int4 *>(dst + i) = make_int4(a[i], a[i + 1], a[i + 2], a[i + 3]);
                     } else {
                         __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)t * p.N + n;
 #pragma unroll
@@ -254,9 +256,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                                 uint32_t o[4];
 #pragma unroll
                                 for (int h = 0; h < 4; ++h) {
-                                    const float a = __fmul_rn((float)(int)v[i + 2 * h], scale);
-                                    const float b = __fmul_rn((float)(int)v[i + 2 * h + 1], scale);
-                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(a, b);
+                                    const float x0 = __fmul_rn((float)a[i + 2 * h], scale);
+                                    const float x1 = __fmul_rn((float)a[i + 2 * h + 1], scale);
+                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
                                     o[h] = *reinterpret_cast<const uint32_t *>(&pr);
                                 }
                                 *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
@@ -313,10 +315,9 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
                            const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
                            WorkspaceHeader *hdr, cudaStream_t stream)
 {
-    (void)rowsum; // signed weight bytes: no offset to remove
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
-    const int KB = (int)((K + kTileCols - 1) / kTileCols);
+    const int KB = (int)((K + BK - 1) / BK);
 
     CUtensorMap tmap_x, tmap_w;
     {
@@ -331,12 +332,16 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
             return cudaErrorInvalidValue;
     }
     {
-        // packed weights as [N/16 row blocks][KB * 128 words]; box 128 words (one 512-byte tile) x 16 row blocks
-        const cuuint64_t dims[2] = {(cuuint64_t)KB * 128, (cuuint64_t)(N / 16)};
-        const cuuint64_t strides[1] = {(cuuint64_t)KB * 512};
-        const cuuint32_t box[2] = {128, (cuuint32_t)(BN / 16)};
-        const cuuint32_t estr[2] = {1, 1};
-        if (encode(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void *>(packed), dims, strides, box, estr,
+        // packed weights as [NB row blocks][KB column tiles][256 words]; box = 4 row blocks x 2 column tiles.
+        // Tiles past the end read as zero; the activations there are zero too (columns >= K), and output
+        // rows >= N are never stored.
+        const cuuint64_t tiles_k = (cuuint64_t)((K + kTileCols - 1) / kTileCols);
+        const cuuint64_t tiles_n = (cuuint64_t)((N + kTileRows - 1) / kTileRows);
+        const cuuint64_t dims[3] = {kTileBytes / 4, tiles_k, tiles_n};
+        const cuuint64_t strides[2] = {(cuuint64_t)kTileBytes, tiles_k * kTileBytes};
+        const cuuint32_t box[3] = {kTileBytes / 4, (cuuint32_t)(BK / kTileCols), (cuuint32_t)(BN / kTileRows)};
+        const cuuint32_t estr[3] = {1, 1, 1};
+        if (encode(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(packed), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
@@ -345,6 +350,7 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
     Params p;
     p.gamma = gamma;
     p.beta = beta;
+    p.rowsum = rowsum;
     p.out = out;
     p.M = (int)M;
     p.N = (int)N;

@@ -36,10 +36,11 @@ def test_host_only_functions(lib):
     assert B.status_string(0) == "ok"
     assert "timed out" in B.status_string(B.ERR_TIMEOUT)
     assert B.status_string(12345) == "unknown status"
-    # packed size: K padded to 128, two bits per weight
+    # packed size: N and K padded to 64, two bits per weight
     assert B.packed_bytes(4096, 1536) == 4096 * 1536 // 4 == 1572864
-    assert B.packed_bytes(3200, 8640) == 3200 * 8704 // 4
-    assert B.packed_bytes(16, 16) == 16 * 128 // 4
+    assert B.packed_bytes(3200, 8640) == 3200 * 8640 // 4
+    assert B.packed_bytes(1040, 144) == 1088 * 192 // 4
+    assert B.packed_bytes(16, 16) == 64 * 64 // 4
     assert B.packed_bytes(17, 128) == 0 and B.packed_bytes(16, 24) == 0 and B.packed_bytes(16, 131072 + 16) == 0
     assert B.workspace_bytes(8, 4096, 1536) >= 8 * 1536 + 8 * 8 + 256
     assert B.workspace_bytes(8, 4096, 1536) % 256 == 0
