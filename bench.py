@@ -148,8 +148,9 @@ class Stack:
         torch.cuda.synchronize()
 
 
-def time_sequence(stack, steps, warmup, dist_barrier=None):
-    """-> (ms per step over the whole timed region, ms per launch of the matmul kernel alone)."""
+def time_sequence(stack, steps, warmup, dist_barrier=None, kernel_steps=None):
+    """-> (ms per step over the timed region of `steps` whole steps,
+           ms per launch of the matmul kernel alone, from a second pass with events around that launch)."""
     import torch
     from paper_2402_17764_b200 import binding as B
     seq = B.Sequence(stack.layers)
@@ -159,13 +160,9 @@ def time_sequence(stack, steps, warmup, dist_barrier=None):
     if dist_barrier:
         dist_barrier()
     start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    mids = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
     start.record()
-    for a, b in mids:
-        seq.forward_stage(1)   # activation quantiser (all matrices)
-        a.record()
-        seq.forward_stage(2)   # persistent matmul + dequantisation (all matrices)
-        b.record()
+    for _ in range(steps):
+        seq.forward()          # activation quantiser + persistent matmul (which may start early) for all matrices
     end.record()
     torch.cuda.synchronize()
     if dist_barrier:
@@ -174,7 +171,16 @@ def time_sequence(stack, steps, warmup, dist_barrier=None):
     if status != 0:
         raise RuntimeError(f"device status {status}")
     total = start.elapsed_time(end) / steps
-    kern = sum(a.elapsed_time(b) for a, b in mids) / steps
+    # the same steps again with events around the matmul launch (they keep the two launches apart)
+    n = kernel_steps or min(steps, 200)
+    mids = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+    for a, b in mids:
+        seq.forward_stage(1)
+        a.record()
+        seq.forward_stage(2)
+        b.record()
+    torch.cuda.synchronize()
+    kern = sum(a.elapsed_time(b) for a, b in mids) / n
     seq.close()
     return total, kern
 
@@ -439,9 +445,11 @@ def profile_case(name: str):
     torch.cuda.set_device(0)
     build.build()
     if name.startswith("decode"):
-        # 48 distinct 11008x4096 matrices (541 MB of packed weights) at M = 1 (or M given as decode:M)
-        M = int(name.split(":")[1]) if ":" in name else 1
-        st = Stack([S.LayerShape("up", 11008, 4096)], 1, M, copies=48)
+        # 48 distinct 11008x4096 matrices (541 MB of packed weights) at M = 1; decode:M[:copies] overrides
+        parts = name.split(":")
+        M = int(parts[1]) if len(parts) > 1 else 1
+        copies = int(parts[2]) if len(parts) > 2 else 48
+        st = Stack([S.LayerShape("up", 11008, 4096)], 1, M, copies=copies)
         seq = B.Sequence(st.layers)
         for _ in range(3):
             seq.forward()

@@ -55,22 +55,22 @@ int env_int(const char *name, int fallback)
 }
 
 struct Layout {
-    size_t counters, acc32, table, xq, beta, rowsum, total;
+    size_t acc32, table, lists, xq, beta, rowsum, total;
 };
 
 inline int64_t row_blocks(int64_t N) { return (N + kTileRows - 1) / kTileRows; }
 inline int64_t col_tiles(int64_t K) { return (K + kTileCols - 1) / kTileCols; }
 
-// Workspace of one matmul: [header | counters | acc32 (at most 64 tokens) | Xq | beta | rowsum]
+// Workspace of one matmul: [header | acc32 (at most 64 tokens) | per-warp lists | Xq | beta | rowsum]
 Layout single_layout(int64_t M, int64_t N, int64_t K)
 {
     Layout L{};
     size_t off = sizeof(WorkspaceHeader);
-    L.counters = off;
-    off += align_up((size_t)row_blocks(N) * 4, 256);
     L.acc32 = off;
     off += align_up((size_t)(M < kMaxDecodeM ? M : kMaxDecodeM) * N * 4, 256);
-    L.table = off;
+    L.table = off; // end of what is cleared before every call
+    L.lists = off;
+    off += align_up(kOwnedListsBytes, 256);
     L.xq = off;
     off += align_up((size_t)M * K, 256);
     L.beta = off;
@@ -116,7 +116,6 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.rowsum = reinterpret_cast<int32_t *>(base + L.rowsum);
     e.out = out;
     e.acc32 = reinterpret_cast<int32_t *>(base + L.acc32);
-    e.counters = reinterpret_cast<uint32_t *>(base + L.counters);
     e.M = (int)M;
     e.N = (int)N;
     e.K = (int)K;
@@ -128,9 +127,10 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
 }
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
-bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, cudaStream_t stream)
+bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, cudaStream_t stream)
 {
     WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
+    OwnedList *lists = reinterpret_cast<OwnedList *>(ws + lists_offset);
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
     if (tc) {
         cudaError_t err = launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out, e.out_i32,
@@ -150,7 +150,7 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, cudaStream_t stre
         InlineTable inl{};
         inl.e[0] = s;
         cudaError_t err = launch_decode(inl, nullptr, 1, (uint32_t)(s.NB * s.KB), s.M,
-                                        path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, stream);
+                                        path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream);
         if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
     return BITLINEAR_OK;
@@ -243,7 +243,7 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     const size_t zero_bytes = use_tcgen05_for(M) ? sizeof(WorkspaceHeader) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, (cudaStream_t)stream);
+    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, (cudaStream_t)stream);
 }
 
 bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
@@ -272,7 +272,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
     if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], path, ws, s);
+    return run_matmul(inl.e[0], path, ws, L.lists, s);
 }
 
 bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)
@@ -297,10 +297,11 @@ bitlinear_status bitlinear_poll_status(const void *workspace, void *stream, int 
 }
 
 // ---- sequences -------------------------------------------------------------------------------
-// Workspace: [header | all counters | all acc32 | descriptor table | per-entry Xq, beta, rowsum]
+// Workspace: [header | all acc32 | descriptor table | per-warp lists | per-entry Xq, beta, rowsum]
 
 struct bitlinear_sequence {
     char *workspace;
+    bitlinear::OwnedList *lists;
     int n, tokens, max_M;
     uint32_t tiles;
     size_t zero_bytes;
@@ -310,18 +311,17 @@ struct bitlinear_sequence {
 
 namespace {
 struct SeqLayout {
-    size_t counters, acc32, table, data, total;
+    size_t acc32, table, lists, data, total;
 };
 
 bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::vector<size_t> *entry_off)
 {
     if (!layers || n <= 0 || n > 65536) return false;
-    size_t counters = 0, acc = 0, data = 0;
+    size_t acc = 0, data = 0;
     uint64_t tiles = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1 || d.M > kMaxDecodeM) return false;
-        counters += align_up((size_t)row_blocks(d.N) * 4, 256);
         acc += align_up((size_t)d.M * d.N * 4, 256);
         tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K));
         if (entry_off) entry_off->push_back(data);
@@ -329,12 +329,12 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
     }
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
     size_t off = sizeof(WorkspaceHeader);
-    S.counters = off;
-    off += counters;
     S.acc32 = off;
     off += acc;
     S.table = off;
     off += align_up((size_t)n * sizeof(DecodeEntry), 256);
+    S.lists = off;
+    off += align_up(kOwnedListsBytes, 256);
     S.data = off;
     off += data;
     S.total = off;
@@ -369,18 +369,16 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     char *ws = reinterpret_cast<char *>(workspace);
 
     std::vector<DecodeEntry> table((size_t)n);
-    size_t c_off = S.counters, a_off = S.acc32;
+    size_t a_off = S.acc32;
     uint32_t tiles = 0;
     int tokens = 0, max_M = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         Layout L{};
-        L.counters = c_off;
         L.acc32 = a_off;
         L.xq = S.data + entry_off[(size_t)i];
         L.beta = L.xq + align_up((size_t)d.M * d.K, 256);
         L.rowsum = L.beta + align_up((size_t)d.M * 4, 256);
-        c_off += align_up((size_t)row_blocks(d.N) * 4, 256);
         a_off += align_up((size_t)d.M * d.N * 4, 256);
         fill_entry(table[(size_t)i], d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
         table[(size_t)i].tile_begin = tiles;
@@ -392,11 +390,12 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     bitlinear_sequence *seq = new (std::nothrow) bitlinear_sequence();
     if (!seq) return BITLINEAR_ERR_ARG;
     seq->workspace = ws;
+    seq->lists = reinterpret_cast<OwnedList *>(ws + S.lists);
     seq->n = n;
     seq->tiles = tiles;
     seq->tokens = tokens;
     seq->max_M = max_M;
-    seq->zero_bytes = S.table; // header, arrival counters and int32 scratch
+    seq->zero_bytes = S.table; // header and int32 scratch
     seq->dev_table = nullptr;
     if (n <= kInlineEntries) {
         for (int i = 0; i < n; ++i) seq->inl.e[i] = table[(size_t)i];
@@ -422,7 +421,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
         return BITLINEAR_ERR_CUDA;
     if (stage != 1 &&
         launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
-                      reinterpret_cast<WorkspaceHeader *>(seq->workspace), s) != cudaSuccess)
+                      reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s) != cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;
 }

@@ -2,13 +2,22 @@
 //
 // The cost of decode is moving the weights from HBM once (Section 1: loading weights from DRAM is
 // the expensive part; Section 3: time per output token).  All matrices of a launch form ONE sequence
-// of 1 KiB tiles (64 output rows x 64 columns each, row block after row block, matrix after matrix),
-// and every warp of the grid takes an equal, contiguous share of that sequence.  A warp streams its
-// share through a private shared-memory ring filled by bulk copies (cp.async.bulk), so the HBM latency
-// is covered by the copy engine and not by registers, and the stream never drains at a row-block or
-// matrix boundary.  Row blocks that lie completely inside a share are finished by that warp alone; the
-// row blocks cut by the two ends of a share are completed through int32 atomics (exact, order-free) by
-// whichever contributor arrives last.
+// of 1 KiB tiles (64 output rows x 64 columns each, row block after row block, matrix after matrix).
+// Most of the sequence is split into one equal, contiguous share per warp; the rest is cut into small
+// pieces that the warps draw from a counter when their share is done, so that SMs that happen to run
+// faster take more (the memory system does not serve all SMs equally).  A warp streams its pieces
+// through a private shared-memory ring filled by bulk copies (cp.async.bulk), so the HBM latency is
+// covered by the copy engine and not by registers, and the stream never drains at a row-block, matrix
+// or piece boundary.  Row blocks that lie completely inside a piece are finished by that warp alone.
+// For the row blocks cut by the two ends of a piece the warp only adds its partial sums to an int32
+// scratch (fire-and-forget atomics: exact, order-free, nothing to wait for); the warp whose piece reaches
+// the END of such a row block notes it in a small list of its own.  A second, very small launch, in which
+// one warp takes over the list of one warp of this kernel, dequantises those row blocks.  No flags, no
+// scans, no waits between CTAs.
+//
+// Both launches are programmatic dependents of the launch before them: this kernel starts while the
+// activation quantiser is still running and streams weights until it needs the quantiser's outputs; the
+// finishing launch is resident, waiting, before this kernel ends.
 //
 // The inner loop is bound by integer-ALU issue, not by the tensor pipe, so the 2-bit codes are never
 // shifted into place.  One byte of the packed format holds the codes of FOUR ROWS at the same column
@@ -25,6 +34,8 @@
 // block.  Because codes are T + 1, the per-token sum of q is subtracted once at the end.
 //
 // Roofline: HBM.  Algorithmic bytes = N*K/4 per matrix (activations and outputs are < 0.1 % at M = 1).
+#include <cstdlib>
+
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -50,8 +61,19 @@ constexpr int kChunkTiles = BITLINEAR_DECODE_CHUNK_TILES;  // tiles per bulk cop
 constexpr int kChunkBytes = kChunkTiles * kTileBytes;
 constexpr int kStages = BITLINEAR_DECODE_STAGES;           // copies in flight per warp
 constexpr int kRingBytes = kWarps * kStages * kChunkBytes; // per CTA
-constexpr int kDecodeSmem = kRingBytes + kWarps * kStages * 8 + 16;
+constexpr int kBarsOffset = kRingBytes;
+constexpr int kAbortOffset = kBarsOffset + kWarps * kStages * 8;
+constexpr int kDecodeSmem = kAbortOffset + 16;
 constexpr int kCtasPerSm = BITLINEAR_DECODE_CTAS_PER_SM;
+#ifndef BITLINEAR_DECODE_STATIC_PERCENT
+#define BITLINEAR_DECODE_STATIC_PERCENT 80
+#endif
+#ifndef BITLINEAR_DECODE_PIECES_PER_WARP
+#define BITLINEAR_DECODE_PIECES_PER_WARP 3
+#endif
+constexpr uint32_t kStaticPercent = BITLINEAR_DECODE_STATIC_PERCENT; // share of the tiles split statically
+constexpr uint32_t kPiecesPerWarp = BITLINEAR_DECODE_PIECES_PER_WARP; // dynamic pieces per warp, on average
+constexpr uint32_t kMinPieceTiles = 16;
 
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1)
@@ -121,32 +143,81 @@ __device__ __forceinline__ float token_scale(const DecodeEntry &e, int token)
     return __fdiv_rn(__fmul_rn(*e.gamma, e.beta[token]), (float)kQb); // (gamma * beta_t) / Qb
 }
 
-// End of a row block.  `each(fn)` calls fn(token, row, partial row sum) for every output this lane holds;
-// `tiles` of the row block's KB column tiles went into the sums.  If that is all of them the sums are
-// final.  Otherwise partial sums meet in the int32 scratch and the contributor that brings the tile count
-// to KB finishes the row block and leaves scratch and counter clean for the next launch.
+// End of a row block.  `each(fn)` calls fn(token, row, partial row sum) for every output this lane holds.
+// If all KB column tiles went into the sums they are final; otherwise they are added to the int32 scratch.
 template <class Each>
-__device__ __forceinline__ void finish_block(const DecodeEntry &e, int rb, int tiles, int lane, Each each)
+__device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete, Each each)
 {
-    if (tiles == e.KB) {
+    if (complete)
         each([&](int token, int row, int v) { store_result(e, token, row, v, e.rowsum[token], token_scale(e, token)); });
-        return;
+    else
+        each([&](int token, int row, int v) { atomicAdd(&e.acc32[(size_t)token * e.N + row], v); });
+}
+
+// Finishing launch: dequantises the row blocks on one list from the scratch and leaves the scratch clean for
+// the next launch.  owned[i] = (entry index, row block).  Up to four row blocks are
+// handled at a time with all loads of one kind issued together, so that the pass costs two memory round
+// trips rather than two per row block.
+__device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, const uint2 *owned, int n_owned, int lane)
+{
+    constexpr int kBatch = 4;
+    for (int b0 = 0; b0 < n_owned; b0 += kBatch) {
+        const DecodeEntry *e[kBatch];
+        int32_t *acc[kBatch];
+        int r0[kBatch], N[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            const uint2 o = __ldcg(&owned[min(b0 + b, n_owned - 1)]); // slots past the end repeat the last one and store nothing
+            e[b] = tab + o.x;
+            r0[b] = (int)o.y * kTileRows + lane;
+        }
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            acc[b] = e[b]->acc32;
+            N[b] = (b0 + b < n_owned) ? e[b]->N : 0;
+        }
+        // token 0 of every row block of the batch
+        int v[kBatch][kTileRows / 32], rowsum[kBatch];
+        float scale[kBatch];
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+#pragma unroll
+            for (int h = 0; h < kTileRows / 32; ++h) v[b][h] = (r0[b] + 32 * h < N[b]) ? __ldcg(acc[b] + r0[b] + 32 * h) : 0;
+            rowsum[b] = e[b]->rowsum[0];
+            scale[b] = token_scale(*e[b], 0);
+        }
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+#pragma unroll
+            for (int h = 0; h < kTileRows / 32; ++h) {
+                const int r = r0[b] + 32 * h;
+                if (r < N[b]) {
+                    __stcg(acc[b] + r, 0);
+                    store_result(*e[b], 0, r, v[b][h], rowsum[b], scale[b]);
+                }
+            }
+        }
+        // further tokens
+#pragma unroll
+        for (int b = 0; b < kBatch; ++b) {
+            if (N[b] == 0) continue;
+            const int M = e[b]->M;
+            for (int t = 1; t < M; ++t) {
+                const int rs = e[b]->rowsum[t];
+                const float sc = token_scale(*e[b], t);
+#pragma unroll
+                for (int h = 0; h < kTileRows / 32; ++h) {
+                    const int r = r0[b] + 32 * h;
+                    if (r < N[b]) {
+                        int32_t *p = acc[b] + (size_t)t * N[b] + r;
+                        const int total = __ldcg(p);
+                        __stcg(p, 0);
+                        store_result(*e[b], t, r, total, rs, sc);
+                    }
+                }
+            }
+        }
     }
-    each([&](int token, int row, int v) { atomicAdd(&e.acc32[(size_t)token * e.N + row], v); });
-    __threadfence();
-    __syncwarp();
-    uint32_t old = 0;
-    if (lane == 0) old = atomicAdd(&e.counters[rb], (uint32_t)tiles);
-    old = __shfl_sync(0xffffffffu, old, 0);
-    if (old + (uint32_t)tiles != (uint32_t)e.KB) return;
-    __threadfence();
-    each([&](int token, int row, int) {
-        int32_t *p = &e.acc32[(size_t)token * e.N + row];
-        const int total = __ldcg(p);
-        __stcg(p, 0);
-        store_result(e, token, row, total, e.rowsum[token], token_scale(e, token));
-    });
-    if (lane == 0) e.counters[rb] = 0u;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -178,16 +249,18 @@ __device__ __forceinline__ uint4 load_x16(const int8_t *p) { return __ldg(reinte
 template <int NT>
 __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
-    uint32_t total_tiles, WorkspaceHeader *hdr)
+    uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr, OwnedList *lists)
 {
     extern __shared__ __align__(128) uint8_t dsmem[];
+    ptx::griddep_launch_dependents(); // the finishing launch may become resident; it waits for this grid to end
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
     const uint32_t ring = ptx::smem_u32(dsmem) + warp * (kStages * kChunkBytes);
     const uint32_t ring_lane = ring + lane * 16;
-    const uint32_t bars = ptx::smem_u32(dsmem + kRingBytes) + warp * (kStages * 8);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + kRingBytes + kWarps * kStages * 8);
+    const uint32_t bars = ptx::smem_u32(dsmem + kBarsOffset) + warp * (kStages * 8);
+    int n_owned = 0;
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + kAbortOffset);
 
     if (threadIdx.x == 0) *abort_flag = 0;
     if (lane == 0) {
@@ -198,32 +271,90 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     __syncthreads();
 
     const DecodeEntry *tab = table ? table : inl.e;
-    // this warp's share of the tile sequence
-    const uint64_t n_warps = (uint64_t)gridDim.x * kWarps, w = (uint64_t)blockIdx.x * kWarps + warp;
-    const uint32_t t_begin = (uint32_t)((uint64_t)total_tiles * w / n_warps);
-    const uint32_t t_end = (uint32_t)((uint64_t)total_tiles * (w + 1) / n_warps);
-    if (t_begin == t_end) return;
 
-    // Two cursors walk the share: the producer issues copies up to kStages chunks ahead of the consumer.
-    // A chunk is up to kChunkTiles tiles and never crosses the end of a row block, so both cursors cut the
-    // share into the same chunks.
-    const DecodeEntry *pe = tab + find_entry(tab, n_entries, t_begin, lane);
-    const DecodeEntry *e = pe;
-    int KB = e->KB;
-    int rb, kt;
+    // A piece is a contiguous range of the tile sequence.  Piece w (w < n_warps) is warp w's own share of
+    // `share` tiles; the tiles after the shares form pieces of `dyn` tiles dealt through hdr->piece_counter.
+    const uint32_t n_warps = gridDim.x * kWarps, w = blockIdx.x * kWarps + warp;
+    uint2 *owned = lists[w].item;
+    struct Piece {
+        const DecodeEntry *e;
+        int rb, kt, left; // first tile (row block, column tile) and number of tiles; left == 0: no piece
+    };
+    auto locate = [&](uint32_t t_begin, uint32_t t_end) {
+        Piece p;
+        p.e = tab + find_entry(tab, n_entries, t_begin, lane);
+        const uint32_t local = t_begin - p.e->tile_begin, kb = (uint32_t)p.e->KB;
+        p.rb = (int)(local / kb);
+        p.kt = (int)(local - (uint32_t)p.rb * kb);
+        p.left = (int)(t_end - t_begin);
+        return p;
+    };
+    uint32_t drawn = 0;        // lane 0: result of the draw in flight
+    bool drawing = dyn != 0;   // a draw is in flight
+    auto draw = [&]() {
+        if (lane == 0) drawn = atomicAdd(&hdr->piece_counter, 1u);
+    };
+    // The next dynamic piece (none: left == 0); normally leaves another draw in flight.  Every piece in hand can
+    // add one row block to the warp's list, so a warp whose list is nearly full stops drawing BEFORE it
+    // claims another piece; the number of pieces is far too small for every warp to get there.
+    auto next_piece = [&]() {
+        Piece p;
+        p.e = tab;
+        p.rb = p.kt = p.left = 0;
+        if (!drawing) return p;
+        drawing = false;
+        const uint64_t t0 = (uint64_t)share * n_warps + (uint64_t)__shfl_sync(0xffffffffu, drawn, 0) * dyn;
+        if (t0 >= total_tiles) return p;
+        if (n_owned + 3 <= kMaxOwned) {
+            draw();
+            drawing = true;
+        }
+        const uint64_t t1 = t0 + dyn;
+        return locate((uint32_t)t0, (uint32_t)(t1 < total_tiles ? t1 : total_tiles));
+    };
+
+    // ---- streaming phase (a lambda, so that a warp without work can leave it early)
+    [&]() {
+
+    // Two cursors walk the pieces: the producer issues copies up to kStages chunks ahead of the consumer and
+    // may already be in the next piece.  A chunk is up to kChunkTiles tiles and never crosses the end of a
+    // row block, so both cursors cut a piece into the same chunks.
+    Piece cur, nxt;
     {
-        const uint32_t local = t_begin - e->tile_begin;
-        rb = (int)(local / (uint32_t)KB);
-        kt = (int)(local - (uint32_t)rb * (uint32_t)KB);
+        // own share, clipped to the sequence (without a dynamic part the shares are rounded up)
+        const uint64_t s0 = (uint64_t)w * share, s1 = s0 + share;
+        const uint32_t lim = dyn ? share * n_warps : total_tiles;
+        if (s0 >= lim) { // no share (small launches): nothing to stream ahead of the wait
+            ptx::griddep_wait();
+            return;
+        }
+        cur = locate((uint32_t)s0, (uint32_t)(s1 < lim ? s1 : lim));
     }
-    int left = (int)(t_end - t_begin);                  // consumer: tiles left in the share
-    int p_left = left, p_kt = kt, p_KB = KB;            // producer: same, plus its place in the row block
-    int p_blocks = e->NB - rb;                          // producer: row blocks left in its matrix, this one included
-    const uint8_t *p_src = reinterpret_cast<const uint8_t *>(e->packed) + ((size_t)rb * KB + kt) * kTileBytes;
-    uint32_t issued = 0, consumed = 0;                  // chunks, over the whole kernel (ring slot = count % kStages)
+    nxt = cur;
+    nxt.left = 0; // drawn below, after the first copies have been issued
+
+    const DecodeEntry *pe;   // producer: matrix, tiles left in the piece, place in the row block,
+    int p_left, p_kt, p_KB, p_blocks; // row blocks left in the matrix (this one included)
+    const uint8_t *p_src;
+    bool p_on_next = false;  // producer already works on `nxt`
+    auto producer_start = [&](const Piece &p) {
+        pe = p.e;
+        p_left = p.left;
+        p_kt = p.kt;
+        p_KB = p.e->KB;
+        p_blocks = p.e->NB - p.rb;
+        p_src = reinterpret_cast<const uint8_t *>(p.e->packed) + ((size_t)p.rb * p_KB + p.kt) * kTileBytes;
+    };
+    producer_start(cur);
+    uint32_t issued = 0, consumed = 0; // chunks, over the whole kernel (ring slot = count % kStages)
 
     auto top_up = [&]() {
-        while (p_left > 0 && issued - consumed < (uint32_t)kStages) {
+        while (issued - consumed < (uint32_t)kStages) {
+            if (p_left == 0) {
+                if (p_on_next || nxt.left == 0) break;
+                producer_start(nxt);
+                p_on_next = true;
+            }
             const int n = min(min(kChunkTiles, p_KB - p_kt), p_left);
             if (lane == 0) {
                 const uint32_t s = issued % kStages;
@@ -246,10 +377,32 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         }
     };
     top_up();
+    // The weights above are never written by a kernel.  Everything below (the header's counters, the
+    // quantised activations, their scales and sums, the scratch) is written by the launch before this one:
+    // when this kernel was launched ahead of that launch's end, wait for it here.
+    ptx::griddep_wait();
+    if (drawing) draw();
+    nxt = next_piece();
+
+    // consumer
+    const DecodeEntry *e = cur.e;
+    int KB = e->KB, rb = cur.rb, kt = cur.kt, left = cur.left;
 
     bool alive = true;
-    while (alive && left > 0) {
-        // ---- one row block (or the part of it that lies in this share)
+    while (alive) {
+        if (left == 0) { // piece done: go on with the next one, which the producer has normally begun already
+            if (nxt.left == 0) break;
+            if (!p_on_next) producer_start(nxt);
+            p_on_next = false;
+            e = nxt.e;
+            KB = e->KB;
+            rb = nxt.rb;
+            kt = nxt.kt;
+            left = nxt.left;
+            nxt = next_piece();
+            top_up();
+        }
+        // ---- one row block (or the part of it that lies in this piece)
         const int K = e->K, M = e->M;
         int acc[NT][4][4];      // [token tile][field][C fragment]
         const int8_t *xrow[NT]; // this lane's B-fragment token: lanes whose token does not exist read the last one
@@ -313,9 +466,16 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         }
         if (!alive) break;
 
+        // A row block of which only a part was summed here goes through the scratch; the warp that reaches
+        // its end dequantises it in the final pass.
+        const bool complete = tiles == KB;
+        if (!complete && kt == KB) {
+            if (lane == 0) owned[n_owned] = make_uint2((uint32_t)(e - tab), (uint32_t)rb);
+            ++n_owned; // cannot exceed kMaxOwned: see next_piece
+        }
         // C fragment of field f: c0 (row 16f + g, token 2tq), c1 (same row, 2tq + 1), c2 (row 16f + 8 + g, 2tq), c3.
         const int N = e->N, row0 = rb * kTileRows + g;
-        finish_block(*e, rb, tiles, lane, [&](auto fn) {
+        finish_block(*e, complete, [&](auto fn) {
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
@@ -349,12 +509,29 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             }
         }
     }
+    }();
+
     if (*abort_flag) {
         if (lane == 0) atomicExch(&hdr->status, (int32_t)BITLINEAR_ERR_TIMEOUT);
         // let copies that may still be in flight land before the ring goes away
         const uint64_t t0 = ptx::globaltimer_ns();
         while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
     }
+
+    if (lane == 0) lists[w].n = (uint32_t)n_owned;
+}
+
+// The finishing launch: warp w takes the list of warp w of the kernel above.
+__global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constant__ InlineTable inl,
+                                                            const DecodeEntry *__restrict__ table,
+                                                            const OwnedList *__restrict__ lists, uint32_t n_lists)
+{
+    const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    ptx::griddep_wait(); // the lists and the scratch are written by the launch before this one
+    if (w >= n_lists) return;
+    const int n = (int)__ldcg(&lists[w].n);
+    if (n == 0) return;
+    finish_owned_blocks(table ? table : inl.e, lists[w].item, n, threadIdx.x & 31);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -415,9 +592,37 @@ __global__ void __launch_bounds__(kWarps * 32) decode_dp4a_kernel(const __grid_c
 
 } // namespace
 
+// Measurement aid: a positive integer in the environment overrides a tuning constant.
+static uint32_t tuning_from_env(const char *name, uint32_t fallback, uint32_t max_value)
+{
+    const char *v = std::getenv(name);
+    if (!v || !*v) return fallback;
+    const long x = std::atol(v);
+    return (x >= 1 && x <= (long)max_value) ? (uint32_t)x : fallback;
+}
+
+// Launches `kernel` as a programmatic dependent of the launch before it in the stream (it may start early and
+// must wait, on the device, before it reads what that launch writes).  early == false: an ordinary launch.
+static cudaError_t launch_dependent(const void *kernel, dim3 grid, dim3 block, size_t smem, void **args, bool early,
+                                    cudaStream_t stream)
+{
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cfg.attrs = &attr;
+    cfg.numAttrs = early ? 1 : 0;
+    return cudaLaunchKernelExC(&cfg, kernel, args);
+}
+
 template <int NT>
 static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, const DecodeEntry *table, int n_entries,
-                              uint32_t total_tiles, WorkspaceHeader *hdr, cudaStream_t stream)
+                              uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr,
+                              OwnedList *lists, cudaStream_t stream)
 {
     static bool attr_set[64] = {false};
     int dev = 0;
@@ -427,12 +632,18 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    decode_mma_kernel<NT><<<grid, block, kDecodeSmem, stream>>>(inl, table, n_entries, total_tiles, hdr);
-    return cudaGetLastError();
+    static const bool early = tuning_from_env("BITLINEAR_DECODE_EARLY_LAUNCH", 1, 2) == 1; // 2 = off
+    void *args[] = {(void *)&inl, (void *)&table, (void *)&n_entries, (void *)&total_tiles, (void *)&share,
+                    (void *)&dyn, (void *)&hdr, (void *)&lists};
+    cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT>, grid, block, kDecodeSmem, args, early, stream);
+    if (err != cudaSuccess) return err;
+    uint32_t n_lists = grid.x * kWarps;
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists};
+    return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
 }
 
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
-                          int max_M, int path, WorkspaceHeader *hdr, cudaStream_t stream)
+                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream)
 {
     if (total_tiles == 0) return cudaSuccess;
     const dim3 block(kWarps * 32);
@@ -446,13 +657,28 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     // every warp should have at least kMinTilesPerWarp tiles; beyond that, fill the machine
     constexpr uint32_t kMinTilesPerWarp = 4;
     uint32_t ctas = (total_tiles + kMinTilesPerWarp * kWarps - 1) / (kMinTilesPerWarp * kWarps);
-    const uint32_t cap = (uint32_t)sm_count() * (max_M <= 16 ? kCtasPerSm : 1);
+    uint32_t cap = (uint32_t)sm_count() * (max_M <= 16 ? kCtasPerSm : 1);
+    if (cap > kMaxDecodeWarps / kWarps) cap = kMaxDecodeWarps / kWarps;
     if (ctas > cap) ctas = cap;
     const dim3 grid(ctas);
-    if (max_M <= 8) return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, hdr, stream);
-    if (max_M <= 16) return launch_mma<2>(grid, block, inl, table, n_entries, total_tiles, hdr, stream);
-    if (max_M <= 32) return launch_mma<4>(grid, block, inl, table, n_entries, total_tiles, hdr, stream);
-    return launch_mma<8>(grid, block, inl, table, n_entries, total_tiles, hdr, stream);
+    // Static shares take kStaticPercent of the tiles; the rest is dealt in pieces of `dyn` tiles, about
+    // kPiecesPerWarp per warp, none shorter than kMinPieceTiles.  Small launches have no dynamic part.
+    static const uint32_t static_percent = tuning_from_env("BITLINEAR_DECODE_STATIC_PERCENT", kStaticPercent, 100);
+    static const uint32_t pieces_per_warp = tuning_from_env("BITLINEAR_DECODE_PIECES_PER_WARP", kPiecesPerWarp, 8);
+    const uint32_t n_warps = ctas * kWarps;
+    uint32_t share = total_tiles / n_warps, dyn = 0;
+    if (share >= 4 * kMinPieceTiles && static_percent < 100) {
+        share = (uint32_t)((uint64_t)total_tiles * static_percent / 100 / n_warps);
+        const uint32_t rest = total_tiles - share * n_warps;
+        dyn = rest / (n_warps * pieces_per_warp);
+        if (dyn < kMinPieceTiles) dyn = kMinPieceTiles;
+    } else {
+        share = (total_tiles + n_warps - 1) / n_warps; // all static: the last warps may get less, or nothing
+    }
+    if (max_M <= 8) return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
+    if (max_M <= 16) return launch_mma<2>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
+    if (max_M <= 32) return launch_mma<4>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
+    return launch_mma<8>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
 }
 
 } // namespace bitlinear

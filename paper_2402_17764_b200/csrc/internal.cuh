@@ -18,10 +18,23 @@ constexpr int kMaxDecodeM = 64;
 
 // Workspace header (start of every workspace).
 struct WorkspaceHeader {
-    int32_t status; // BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT, written by kernels
-    uint32_t reserved[63];
+    int32_t status;       // BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT, written by kernels
+    uint32_t reserved0[31];
+    uint32_t piece_counter; // next dynamically dealt piece of the decode kernel (a 128-byte line of its own)
+    uint32_t reserved1[31];
 };
 static_assert(sizeof(WorkspaceHeader) == 256, "header layout");
+
+// Row blocks a warp of the decode kernel leaves to the finishing launch: (entry index, row block) pairs.
+constexpr int kMaxOwned = 15;
+constexpr int kMaxDecodeWarps = 2560;
+struct OwnedList {
+    uint32_t n;
+    uint32_t pad;
+    uint2 item[kMaxOwned];
+};
+static_assert(sizeof(OwnedList) == 128, "one line per warp");
+constexpr size_t kOwnedListsBytes = sizeof(OwnedList) * kMaxDecodeWarps;
 
 // One matmul of a decode launch, as the kernels see it (device memory or kernel parameter).
 struct DecodeEntry {
@@ -33,7 +46,6 @@ struct DecodeEntry {
     int32_t *rowsum;       // [M]
     void *out;             // bf16 [M, N], or int32 [M, N] when out_i32
     int32_t *acc32;        // scratch [M, N] for row blocks shared by several warps (zero before and after a launch)
-    uint32_t *counters;    // column tiles arrived, one counter per row block (zero before and after a launch)
     int M, N, K;
     int KB, NB;            // column tiles = ceil(K / 64), row blocks = ceil(N / 64)
     uint32_t tile_begin;   // index of this entry's first tile in the launch-wide tile sequence (NB * KB tiles each)
@@ -61,8 +73,9 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
 
 // Persistent weight-streaming matmul over the entries (total_tiles = sum of NB * KB).
 // path: BITLINEAR_PATH_MMA, or BITLINEAR_PATH_DP4A (first entry only).
+// `lists` is scratch of kOwnedListsBytes (no need to clear it).
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
-                          int max_M, int path, WorkspaceHeader *hdr, cudaStream_t stream);
+                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream);
 
 // Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) or raw int32.
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,

@@ -19,6 +19,19 @@ __device__ __forceinline__ uint64_t globaltimer_ns()
     return t;
 }
 
+__device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t *p)
+{
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Programmatic dependent launch.  wait: blocks until the grid this one depends on has completed and its
+// writes are visible (returns at once for an ordinary launch).  launch_dependents: the next kernel in the
+// stream, if it was launched as a programmatic dependent, may start once every CTA has got here.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ bool elect_one()
 {
     uint32_t pred;

@@ -7,6 +7,7 @@
 // round-half-to-even, clip, and is stored as int8 together with the row sum of the codes.
 // HBM-bound: 2 B read + 1 B written per element.
 #include "internal.cuh"
+#include "ptx.cuh"
 
 namespace bitlinear {
 
@@ -57,6 +58,9 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
 {
     __shared__ uint32_t s_max[kThreads / 32];
     __shared__ int s_sum[kThreads / 32];
+
+    // The matmul that follows may be launched early: it streams weights until it needs what this kernel writes.
+    ptx::griddep_launch_dependents();
 
     if ((int)blockIdx.x >= total_tokens) {
         // trailing blocks clear control words and split-K scratch for the matmul that follows
