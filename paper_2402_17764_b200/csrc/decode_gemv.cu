@@ -331,7 +331,14 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         cur = locate((uint32_t)s0, (uint32_t)(s1 < lim ? s1 : lim));
     }
     nxt = cur;
-    nxt.left = 0; // drawn below, after the first copies have been issued
+    nxt.left = 0;            // the first dynamic piece is drawn below, after the first copies have been issued,
+    bool nxt_pending = false; // and looked at only when a cursor gets to the end of `cur`
+    auto resolve_next = [&]() {
+        if (nxt_pending) {
+            nxt_pending = false;
+            nxt = next_piece();
+        }
+    };
 
     const DecodeEntry *pe;   // producer: matrix, tiles left in the piece, place in the row block,
     int p_left, p_kt, p_KB, p_blocks; // row blocks left in the matrix (this one included)
@@ -351,6 +358,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     auto top_up = [&]() {
         while (issued - consumed < (uint32_t)kStages) {
             if (p_left == 0) {
+                resolve_next();
                 if (p_on_next || nxt.left == 0) break;
                 producer_start(nxt);
                 p_on_next = true;
@@ -381,8 +389,10 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     // quantised activations, their scales and sums, the scratch) is written by the launch before this one:
     // when this kernel was launched ahead of that launch's end, wait for it here.
     ptx::griddep_wait();
-    if (drawing) draw();
-    nxt = next_piece();
+    if (drawing) {
+        draw();
+        nxt_pending = true;
+    }
 
     // consumer
     const DecodeEntry *e = cur.e;
@@ -391,6 +401,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     bool alive = true;
     while (alive) {
         if (left == 0) { // piece done: go on with the next one, which the producer has normally begun already
+            resolve_next();
             if (nxt.left == 0) break;
             if (!p_on_next) producer_start(nxt);
             p_on_next = false;
