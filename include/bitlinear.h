@@ -119,6 +119,28 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
                                    void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same forward for callers that cannot give it a workspace.  (The paper has no counterpart: this is a
+ * convenience of the library.)  Some code that wants to run a BitLinear layer is not allowed to allocate
+ * device memory at the point of the call -- a plug-in that runs inside another framework's memory pool, a
+ * real-time loop that must not touch the allocator, code that runs after the process has been told to
+ * stop allocating -- and so has no workspace to hand over.  This entry point calls no allocator of any
+ * kind; it uses BITLINEAR_STATIC_WORKSPACE_BYTES of scratch that are part of the library itself (each GPU
+ * that loads the library holds them until the process exits).  Inputs and outputs are still the caller's.
+ *   - Shapes whose bitlinear_workspace_bytes(M, N, K) exceeds BITLINEAR_STATIC_WORKSPACE_BYTES are refused
+ *     with BITLINEAR_ERR_WORKSPACE and nothing is launched.
+ *   - The first call on a device looks up the scratch's device address (no allocation, no device work);
+ *     make that first call before any stream capture begins on that device.
+ *   - All calls on a device share the one scratch area, which still holds what the previous call left:
+ *     each call clears what it needs to start at zero, but two calls that overlap on the GPU (different
+ *     streams, or the same stream of two host threads without ordering) corrupt each other.  Order them.
+ *   - A bounded device-side wait that expires ends the kernel as in bitlinear_forward, but the status word
+ *     lies in the library's scratch and cannot be polled through this interface.
+ */
+#define BITLINEAR_STATIC_WORKSPACE_BYTES ((size_t)8 << 20)
+bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma, const void *X,
+                                          int64_t M, int64_t K, int64_t N, void *Y, void *stream);
+
+/*
  * A list of independent BitLinear forwards executed by one persistent launch (the seven projections of
  * every decoder layer of a decode step, Section 2 "LLaMA-alike Components").  All inputs X must be
  * ready when the call is enqueued: entries do not depend on each other.  Every entry needs M <= 64.

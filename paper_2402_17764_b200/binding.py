@@ -26,6 +26,7 @@ EXPORTS = [
     "bitlinear_quantize_weights",
     "bitlinear_quantize_acts",
     "bitlinear_forward",
+    "bitlinear_forward_static",
     "bitlinear_sequence_workspace_bytes",
     "bitlinear_sequence_create",
     "bitlinear_forward_sequence",
@@ -78,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_quantize_weights.argtypes = [vp, i64, i64, cf, vp, vp, vp]
     L.bitlinear_quantize_acts.argtypes = [vp, i64, i64, vp, vp, vp, vp]
     L.bitlinear_forward.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
+    L.bitlinear_forward_static.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.bitlinear_sequence_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci]
     L.bitlinear_sequence_workspace_bytes.restype = sz
     L.bitlinear_sequence_create.argtypes = [ctypes.POINTER(LayerDesc), ci, vp, sz, ctypes.POINTER(vp)]
@@ -161,6 +163,15 @@ def forward(packed: torch.Tensor, gamma: torch.Tensor, X: torch.Tensor, N: int, 
     st = load_library().bitlinear_forward(_ptr(packed), _ptr(gamma), _ptr(X), M, K, N, _ptr(Y), _ptr(workspace),
                                           workspace.numel(), _stream(stream))
     _check(st, "bitlinear_forward")
+    return Y
+
+
+def forward_static(packed: torch.Tensor, gamma: torch.Tensor, X: torch.Tensor, N: int, Y: torch.Tensor,
+                   stream=None) -> torch.Tensor:
+    """bitlinear_forward_static: the forward on the library's own scratch; the caller supplies Y, nothing is allocated."""
+    M, K = X.shape
+    st = load_library().bitlinear_forward_static(_ptr(packed), _ptr(gamma), _ptr(X), M, K, N, _ptr(Y), _stream(stream))
+    _check(st, "bitlinear_forward_static")
     return Y
 
 

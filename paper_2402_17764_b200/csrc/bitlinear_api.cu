@@ -296,6 +296,32 @@ bitlinear_status bitlinear_poll_status(const void *workspace, void *stream, int 
     return BITLINEAR_OK;
 }
 
+// ---- forward without a caller workspace ---------------------------------------------------------
+// Scratch for bitlinear_forward_static: part of the library's device image, so every GPU that loads the
+// library holds these bytes until the process exits.  In host code this name is only a handle; the
+// device address comes from cudaGetSymbolAddress.
+constexpr size_t kStaticWorkspaceBytes = BITLINEAR_STATIC_WORKSPACE_BYTES;
+static __device__ __align__(256) unsigned char g_static_workspace[kStaticWorkspaceBytes];
+
+bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
+                                          int64_t N, void *Y, void *stream)
+{
+    bitlinear_status st = check_shape(M, N, K);
+    if (st != BITLINEAR_OK) return st;
+    if (single_layout(M, N, K).total > kStaticWorkspaceBytes) return BITLINEAR_ERR_WORKSPACE;
+    // device address of the scratch, looked up once per device while that device is current
+    static void *address[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BITLINEAR_ERR_CUDA;
+    if (!address[dev]) {
+        void *p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return BITLINEAR_ERR_CUDA;
+        address[dev] = p;
+    }
+    // bitlinear_forward clears the part of the workspace that has to start at zero on every call
+    return bitlinear_forward(packed, gamma, X, M, K, N, Y, address[dev], kStaticWorkspaceBytes, stream);
+}
+
 // ---- sequences -------------------------------------------------------------------------------
 // Workspace: [header | all acc32 | descriptor table | per-warp lists | per-entry Xq, beta, rowsum]
 
