@@ -172,12 +172,17 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             __syncwarp();
         }
     } else if (warp >= kFirstExpanderWarp) {
-        // Expander warp ew owns packed tile (row block ew / 2, column tile ew % 2) of the stage.  Lane
-        // (g, tq) holds, in its 16 bytes of each slab, the codes of rows 16 f + 8 h + g at columns
+        // Expander warp ew owns packed tile (row block ew / 2, column tile ew % 2) of the stage.  The 16 bytes
+        // at slot 4 g + tq of each slab hold the codes of rows 16 f + 8 h + g at columns
         // 16 tq + 8 s + 4 hi + b (slab s, word 2 hi + h, byte b, field f): 16 consecutive columns of a row
         // are words (h, 2 + h) of slab 0 followed by words (h, 2 + h) of slab 1.
+        // Which thread takes which slot is free here.  Eight consecutive threads take g in {q, (q ^ 1) + 4}
+        // (q = lane / 8) and tq = 0..3: their 16-byte loads fall into eight different bank groups, and so do
+        // their 16-byte stores, because the swizzled chunk (4 kti + tq) ^ g then takes eight different values.
         const int ew = warp - kFirstExpanderWarp;
-        const int g = lane >> 2, tq = lane & 3;
+        const int q = lane >> 3;
+        const int g = (lane & 4) ? ((q ^ 1) + 4) : q, tq = lane & 3;
+        const int slot = 4 * g + tq;
         const int rbi = ew >> 1, kti = ew & 1;
         uint32_t it = 0;
         bool ok = true;
@@ -192,7 +197,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 uint8_t *stage = smem + s * kStageBytes;
                 const uint4 *packed = reinterpret_cast<const uint4 *>(stage + kABytes + kBBytes) + ew * (kTileBytes / 16);
                 uint8_t *bt = stage + kABytes;
-                const uint4 w0 = packed[lane], w1 = packed[32 + lane];
+                const uint4 w0 = packed[slot], w1 = packed[32 + slot];
                 const uint32_t lo[2][2] = {{w0.x, w0.z}, {w0.y, w0.w}}; // [h][hi], slab 0
                 const uint32_t up[2][2] = {{w1.x, w1.z}, {w1.y, w1.w}}; // slab 1
                 const int chunk = (kti * 4 + tq) ^ g; // 16-byte chunk of the 128-byte row, swizzled by row % 8 = g
