@@ -31,9 +31,11 @@ METRIC = "decode BitLinear packed-weight GB/s"
 UNIT = "GB/s"
 WORKLOAD = "3b_decode"
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, from the ncu capture
-# summarised under profiles/ (null until a capture exists for the workload).
-NCU_TRAFFIC_BYTES = {"3b_decode": None}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel.  The ncu capture summarised in
+# profiles/decode_mma_kernel_7b_up_x48_M1.md measured 547.77 MB on a launch of 541.07 MB of packed weights (the
+# full step is too large for a 40-pass capture); traffic grows in proportion to the packed bytes, so the figure
+# for the benchmark's launch is that ratio times its packed bytes.  Set to None when the kernel changes.
+NCU_TRAFFIC_RATIO = {"3b_decode": 547.77 / 541.07}
 
 
 def measured_peaks():
@@ -418,7 +420,8 @@ def run_ours(args):
         "roofline": {"bound": "hbm", "kernel": "decode_mma_kernel<1>", "achieved": round(achieved, 1),
                      "peak": peaks["hbm_gbs"], "peak_source": peaks["source"], "unit": "GB/s",
                      "frac": round(achieved / peaks["hbm_gbs"], 4), "frac_of_nominal_8000": round(achieved / 8000.0, 4),
-                     "traffic": NCU_TRAFFIC_BYTES.get(WORKLOAD)},
+                     "traffic": (round(NCU_TRAFFIC_RATIO[WORKLOAD] * stack.algorithmic_bytes)
+                                 if NCU_TRAFFIC_RATIO.get(WORKLOAD) else None)},
         "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": round(ms_e2e, 4)},
         "gpu_launches": 2 * args.steps,
