@@ -64,12 +64,13 @@ enum {
 /* Human-readable name of a status code; never NULL. (host) */
 const char *bitlinear_status_string(bitlinear_status s);
 
-/* Bytes of the packed 2-bit weight buffer of an [N, K] matrix, K padded to a multiple of 128.
+/* Bytes of the packed 2-bit weight buffer of an [N, K] matrix: N and K padded to multiples of 64, 4 weights per byte.
  * Returns 0 for shapes the library rejects. (host) */
 size_t bitlinear_packed_bytes(int64_t N, int64_t K);
 
 /* Bytes of workspace bitlinear_forward / bitlinear_matmul_i32 need for this shape
- * (int8 activations, beta, row sums, split-K scratch, status word).  0 for rejected shapes. (host) */
+ * (int8 activations, beta, row sums, int32 scratch and per-warp lists of the streaming kernel, status word).
+ * 0 for rejected shapes. (host) */
 size_t bitlinear_workspace_bytes(int64_t M, int64_t N, int64_t K);
 
 /*
@@ -85,11 +86,16 @@ size_t bitlinear_workspace_bytes(int64_t M, int64_t N, int64_t K);
  * being computed and are overwritten with their final contents afterwards.
  *
  * Layout.  The code of a weight is T + 1 (0, 1 or 2; 3 never occurs).  The matrix is cut into tiles of
- * 16 rows x 128 columns = 512 bytes = 128 little-endian 32-bit words, stored consecutively with the
- * column-tile index fastest.  Inside a tile, weight (r, c) sits in word 4*(4*(r%8) + c/32) + (c%32)/8 at
- * bits [8*(c%4) + 2*f, +1] with f = 2*((c%8)/4) + r/8.  A warp that loads the tile as one 16-byte
- * vector per lane therefore gets, from each word w, the four integer-MMA operand registers
- * (w >> 2*f) & 0x03030303.  Columns K..Kpad-1 hold code 1 (weight 0).
+ * 64 rows x 64 columns = 1024 bytes, stored consecutively with the column-tile index fastest; rows N.. and
+ * columns K.. up to the next multiple of 64 hold code 1 (weight 0).  One byte holds the codes of four rows at
+ * the same column.  Inside a tile, split the row r = n % 64 as 16 f + 8 h + g (f = 0..3, h = 0..1, g = 0..7)
+ * and the column c = k % 64 as 16 tq + 8 s + 4 hi + b (tq = 0..3, s = 0..1, hi = 0..1, b = 0..3): the code
+ * sits in bits [2 f, 2 f + 1] of byte 512 s + 16 (4 g + tq) + 4 (2 hi + h) + b.  A warp that loads a 512-byte
+ * half tile as one 16-byte vector per lane (lane = 4 g + tq) therefore holds, in its four 32-bit words as they
+ * are, the A operand of an m16n8k32 integer MMA over rows 8 h + g and columns 16 tq + 8 s + 4 hi + b of all
+ * four 16-row groups at once: the operand of group f is w & (0xFF << 2 f & 0xFF, in every byte), i.e. no shift
+ * and at most one AND per register (see csrc/decode_gemv.cu), and the tensor-core GEMM expands a tile to
+ * bytes with one AND per four weights.
  */
 bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K, float eps,
                                             void *packed, float *gamma, void *stream);
@@ -166,8 +172,9 @@ typedef struct bitlinear_sequence bitlinear_sequence;
 bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
                                            size_t workspace_bytes, bitlinear_sequence **out);
 
-/* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch and one persistent
- * matmul launch.  Calls on the same sequence must be stream-ordered, not concurrent. */
+/* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch, one persistent matmul
+ * launch that starts while the quantiser is still running (programmatic dependent launch) and one very small
+ * finishing launch.  Calls on the same sequence must be stream-ordered, not concurrent. */
 bitlinear_status bitlinear_forward_sequence(const bitlinear_sequence *seq, void *stream);
 
 /* The same in two halves, so that a caller can put its own events between them:
