@@ -72,7 +72,7 @@ Layout single_layout(int64_t M, int64_t N, int64_t K)
     L.lists = off;
     off += align_up(kOwnedListsBytes, 256);
     L.xq = off;
-    off += align_up((size_t)M * K, 256);
+    off += align_up((size_t)M * col_tiles(K) * kTileCols, 256); // room for either layout of the int8 activations
     L.beta = off;
     off += align_up((size_t)M * 4, 256);
     L.rowsum = off;
@@ -97,11 +97,12 @@ __global__ void rowsum_kernel(const int8_t *__restrict__ Xq, int K, int32_t *__r
     }
 }
 
+// More than 64 tokens always go to the tensor-core GEMM; BITLINEAR_TCGEN05_MIN_M (a measurement aid) lowers the
+// switch-over point.
 bool use_tcgen05_for(int64_t M)
 {
-    static const int disabled = env_int("BITLINEAR_NO_TCGEN05", 0);
     static const int min_m = env_int("BITLINEAR_TCGEN05_MIN_M", kMaxDecodeM + 1);
-    return !disabled && M >= min_m;
+    return M > kMaxDecodeM || M >= min_m;
 }
 
 // Fills one DecodeEntry for a matmul whose workspace part starts at `base`.
@@ -124,6 +125,7 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.tile_begin = 0;
     e.token_begin = 0;
     e.out_i32 = out_i32;
+    e.xq_tiled = 0;
 }
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
@@ -137,22 +139,12 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
                                          hdr, stream);
         return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }
-    // Weight-streaming kernel, in slices of at most 64 tokens (one slice in the decode regime).
-    const int64_t M = e.M;
-    for (int64_t m0 = 0; m0 < M; m0 += kMaxDecodeM) {
-        DecodeEntry s = e;
-        s.M = (int)((M - m0 < kMaxDecodeM) ? (M - m0) : kMaxDecodeM);
-        s.Xq = e.Xq + m0 * e.K;
-        s.beta = e.beta + m0;
-        s.rowsum = e.rowsum + m0;
-        const size_t elt = e.out_i32 ? 4 : 2;
-        s.out = reinterpret_cast<char *>(e.out) + (size_t)m0 * e.N * elt;
-        InlineTable inl{};
-        inl.e[0] = s;
-        cudaError_t err = launch_decode(inl, nullptr, 1, (uint32_t)(s.NB * s.KB), s.M,
-                                        path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream);
-        if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    }
+    if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
+    InlineTable inl{};
+    inl.e[0] = e;
+    cudaError_t err = launch_decode(inl, nullptr, 1, (uint32_t)(e.NB * e.KB), e.M,
+                                    path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream);
+    if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;
 }
 
@@ -239,6 +231,7 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     char *ws = reinterpret_cast<char *>(workspace);
     InlineTable inl{};
     fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L);
+    inl.e[0].xq_tiled = use_tcgen05_for(M) ? 0 : 1;
     // quantise the tokens; the same launch clears the header and, for the streaming kernel, its scratch
     const size_t zero_bytes = use_tcgen05_for(M) ? sizeof(WorkspaceHeader) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
@@ -266,10 +259,15 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
     InlineTable inl{};
     fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
-    inl.e[0].Xq = const_cast<int8_t *>(Xq); // read only on this path
     const size_t zero_bytes = tc ? sizeof(WorkspaceHeader) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, s);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    if (tc) {
+        inl.e[0].Xq = const_cast<int8_t *>(Xq); // the GEMM reads the caller's rows in place
+    } else {
+        inl.e[0].xq_tiled = 1; // the streaming kernels read tiles: copy the rows into the workspace
+        if (launch_retile_acts(Xq, M, K, inl.e[0].Xq, s) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    }
     rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
     if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return run_matmul(inl.e[0], path, ws, L.lists, s);
@@ -351,7 +349,7 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
         acc += align_up((size_t)d.M * d.N * 4, 256);
         tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K));
         if (entry_off) entry_off->push_back(data);
-        data += align_up((size_t)d.M * d.K, 256) + 2 * align_up((size_t)d.M * 4, 256);
+        data += align_up((size_t)d.M * col_tiles(d.K) * kTileCols, 256) + 2 * align_up((size_t)d.M * 4, 256);
     }
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
     size_t off = sizeof(WorkspaceHeader);
@@ -403,10 +401,11 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
         Layout L{};
         L.acc32 = a_off;
         L.xq = S.data + entry_off[(size_t)i];
-        L.beta = L.xq + align_up((size_t)d.M * d.K, 256);
+        L.beta = L.xq + align_up((size_t)d.M * col_tiles(d.K) * kTileCols, 256);
         L.rowsum = L.beta + align_up((size_t)d.M * 4, 256);
         a_off += align_up((size_t)d.M * d.N * 4, 256);
         fill_entry(table[(size_t)i], d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
+        table[(size_t)i].xq_tiled = 1;
         table[(size_t)i].tile_begin = tiles;
         table[(size_t)i].token_begin = tokens;
         tiles += (uint32_t)(table[(size_t)i].NB * table[(size_t)i].KB);

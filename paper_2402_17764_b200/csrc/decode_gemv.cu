@@ -15,6 +15,12 @@
 // one warp takes over the list of one warp of this kernel, dequantises those row blocks.  No flags, no
 // scans, no waits between CTAs.
 //
+// The quantised activations travel the same way.  The quantiser writes them tile by tile ([column tile][token]
+// [64 bytes]), so the activations a chunk of weight tiles needs are ONE contiguous range, fetched by a
+// second bulk copy into the same ring slot; the B fragments of the MMAs are then conflict-free 16-byte
+// shared-memory loads, nothing depends on L1 hit rates when many tokens and many matrices are in flight,
+// and columns past K need no special case (the quantiser writes zeros there).
+//
 // Both launches are programmatic dependents of the launch before them: this kernel starts while the
 // activation quantiser is still running and streams weights until it needs the quantiser's outputs; the
 // finishing launch is resident, waiting, before this kernel ends.
@@ -57,14 +63,22 @@ namespace {
 #define BITLINEAR_DECODE_CTAS_PER_SM 1
 #endif
 constexpr int kWarps = BITLINEAR_DECODE_WARPS;             // warps per CTA, each independent
-constexpr int kChunkTiles = BITLINEAR_DECODE_CHUNK_TILES;  // tiles per bulk copy
-constexpr int kChunkBytes = kChunkTiles * kTileBytes;
-constexpr int kStages = BITLINEAR_DECODE_STAGES;           // copies in flight per warp
-constexpr int kRingBytes = kWarps * kStages * kChunkBytes; // per CTA
-constexpr int kBarsOffset = kRingBytes;
-constexpr int kAbortOffset = kBarsOffset + kWarps * kStages * 8;
-constexpr int kDecodeSmem = kAbortOffset + 16;
+constexpr int kStages = BITLINEAR_DECODE_STAGES;           // chunks in flight per warp
 constexpr int kCtasPerSm = BITLINEAR_DECODE_CTAS_PER_SM;
+constexpr int kXTileBytes = 64;                            // int8 activations of one token for one column tile
+
+// Shared memory of the kernel for NT 8-token tiles: per warp kStages slots of
+// [kTiles weight tiles | kTiles x (up to 8 NT tokens) x 64 bytes of activations], then barriers and a flag.
+template <int NT>
+struct Ring {
+    static constexpr int kTiles = NT == 1 ? BITLINEAR_DECODE_CHUNK_TILES : (NT == 8 ? 2 : 4); // tiles per chunk
+    static constexpr int kWeightBytes = kTiles * kTileBytes;
+    static constexpr int kSlotBytes = kWeightBytes + kTiles * 8 * NT * kXTileBytes;
+    static constexpr int kBarsOffset = kWarps * kStages * kSlotBytes;
+    static constexpr int kAbortOffset = kBarsOffset + kWarps * kStages * 8;
+    static constexpr int kSmem = kAbortOffset + 16;
+    static_assert(kSmem * (NT <= 2 ? kCtasPerSm : 1) <= 227 * 1024, "ring does not fit the SM's shared memory");
+};
 #ifndef BITLINEAR_DECODE_STATIC_PERCENT
 #define BITLINEAR_DECODE_STATIC_PERCENT 80
 #endif
@@ -238,13 +252,6 @@ __device__ __forceinline__ void mma_slab(int (&acc)[4][4], const uint4 &w, uint3
     mma_u8s8(acc[3], w.x & 0xC0C0C0C0u, w.y & 0xC0C0C0C0u, w.z & 0xC0C0C0C0u, w.w & 0xC0C0C0C0u, b0, b1);
 }
 
-__device__ __forceinline__ void mma_tile(int (&acc)[4][4], uint32_t stage, const uint4 &x)
-{
-    mma_slab(acc, lds128(stage), x.x, x.y);
-    mma_slab(acc, lds128(stage + 512), x.z, x.w);
-}
-
-__device__ __forceinline__ uint4 load_x16(const int8_t *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
 
 template <int NT>
 __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
@@ -256,16 +263,18 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
-    const uint32_t ring = ptx::smem_u32(dsmem) + warp * (kStages * kChunkBytes);
-    const uint32_t ring_lane = ring + lane * 16;
-    const uint32_t bars = ptx::smem_u32(dsmem + kBarsOffset) + warp * (kStages * 8);
+    using R = Ring<NT>;
+    constexpr int kChunkTiles = R::kTiles;
+    const uint32_t ring = ptx::smem_u32(dsmem) + warp * (kStages * R::kSlotBytes);
+    const uint32_t bars = ptx::smem_u32(dsmem + R::kBarsOffset) + warp * (kStages * 8);
     int n_owned = 0;
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + kAbortOffset);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + R::kAbortOffset);
 
     if (threadIdx.x == 0) *abort_flag = 0;
     if (lane == 0) {
+        // two arrivals per phase: one announces the weight bytes of a chunk, one its activation bytes
 #pragma unroll
-        for (int s = 0; s < kStages; ++s) ptx::mbar_init(bars + 8 * s, 1);
+        for (int s = 0; s < kStages; ++s) ptx::mbar_init(bars + 8 * s, 2);
         ptx::fence_mbar_init();
     }
     __syncthreads();
@@ -343,6 +352,8 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     const DecodeEntry *pe;   // producer: matrix, tiles left in the piece, place in the row block,
     int p_left, p_kt, p_KB, p_blocks; // row blocks left in the matrix (this one included)
     const uint8_t *p_src;
+    const int8_t *p_x; // the matrix's activations, [column tile][token][64 bytes]
+    int p_xbytes;      // activation bytes per column tile = tokens * 64
     bool p_on_next = false;  // producer already works on `nxt`
     auto producer_start = [&](const Piece &p) {
         pe = p.e;
@@ -351,9 +362,18 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         p_KB = p.e->KB;
         p_blocks = p.e->NB - p.rb;
         p_src = reinterpret_cast<const uint8_t *>(p.e->packed) + ((size_t)p.rb * p_KB + p.kt) * kTileBytes;
+        p_x = p.e->Xq;
+        p_xbytes = p.e->M * kXTileBytes;
     };
     producer_start(cur);
     uint32_t issued = 0, consumed = 0; // chunks, over the whole kernel (ring slot = count % kStages)
+
+    // Activation copies must not be issued before the quantiser's results are visible; the weight copies of
+    // the first chunks are.  The activation copies of those chunks are kept here and issued after the wait.
+    bool x_ready = false;
+    const int8_t *held_x[kStages];
+    uint32_t held_bytes[kStages];
+    int n_held = 0;
 
     auto top_up = [&]() {
         while (issued - consumed < (uint32_t)kStages) {
@@ -364,10 +384,22 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
                 p_on_next = true;
             }
             const int n = min(min(kChunkTiles, p_KB - p_kt), p_left);
+            const uint32_t s = issued % kStages;
+            const int8_t *xsrc = p_x + (size_t)p_kt * p_xbytes;
+            const uint32_t xbytes = (uint32_t)(n * p_xbytes);
             if (lane == 0) {
-                const uint32_t s = issued % kStages;
+                const uint32_t slot = ring + s * R::kSlotBytes;
                 ptx::mbar_arrive_expect_tx(bars + 8 * s, (uint32_t)n * kTileBytes);
-                bulk_copy_g2s(ring + s * kChunkBytes, p_src, (uint32_t)n * kTileBytes, bars + 8 * s);
+                bulk_copy_g2s(slot, p_src, (uint32_t)n * kTileBytes, bars + 8 * s);
+                if (x_ready) {
+                    ptx::mbar_arrive_expect_tx(bars + 8 * s, xbytes);
+                    bulk_copy_g2s(slot + R::kWeightBytes, xsrc, xbytes, bars + 8 * s);
+                }
+            }
+            if (!x_ready) { // at most kStages chunks are issued before the wait, into slots 0, 1, ...
+                held_x[n_held] = xsrc;
+                held_bytes[n_held] = xbytes;
+                ++n_held;
             }
             ++issued;
             p_left -= n;
@@ -380,6 +412,8 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
                     p_KB = pe->KB;
                     p_blocks = pe->NB;
                     p_src = reinterpret_cast<const uint8_t *>(pe->packed);
+                    p_x = pe->Xq;
+                    p_xbytes = pe->M * kXTileBytes;
                 }
             }
         }
@@ -389,6 +423,16 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     // quantised activations, their scales and sums, the scratch) is written by the launch before this one:
     // when this kernel was launched ahead of that launch's end, wait for it here.
     ptx::griddep_wait();
+    x_ready = true;
+    if (lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) {
+            if (i < n_held) {
+                ptx::mbar_arrive_expect_tx(bars + 8 * i, held_bytes[i]);
+                bulk_copy_g2s(ring + i * R::kSlotBytes + R::kWeightBytes, held_x[i], held_bytes[i], bars + 8 * i);
+            }
+        }
+    }
     if (drawing) {
         draw();
         nxt_pending = true;
@@ -414,54 +458,44 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             top_up();
         }
         // ---- one row block (or the part of it that lies in this piece)
-        const int K = e->K, M = e->M;
-        int acc[NT][4][4];      // [token tile][field][C fragment]
-        const int8_t *xrow[NT]; // this lane's B-fragment token: lanes whose token does not exist read the last one
+        const int M = e->M;
+        int acc[NT][4][4]; // [token tile][field][C fragment]
+        uint32_t xlane[NT]; // offset of this lane's B-fragment token (lanes without a token read the last one) and columns
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
             for (int f = 0; f < 4; ++f) acc[nt][f][0] = acc[nt][f][1] = acc[nt][f][2] = acc[nt][f][3] = 0;
-            xrow[nt] = e->Xq + (size_t)min(8 * nt + g, M - 1) * K + 16 * tq;
+            xlane[nt] = (uint32_t)(R::kWeightBytes + min(8 * nt + g, M - 1) * kXTileBytes + 16 * tq);
         }
+        const uint32_t xtile = (uint32_t)(M * kXTileBytes); // activation bytes per column tile in the slot
         int tiles = 0; // tiles of this row block accumulated here
         while (kt < KB && left > 0) {
             const int n = min(min(kChunkTiles, KB - kt), left);
             const uint32_t s = consumed % kStages;
-            const uint32_t stage = ring_lane + s * kChunkBytes;
-            const int col0 = kt * kTileCols + 16 * tq; // this lane's first column; columns >= K read as zero
-            if (NT == 1) {
-                // activations of the whole chunk are requested before the weights are waited for
-                uint4 x[kChunkTiles];
-                const int8_t *xp = xrow[0] + kt * kTileCols;
-                // (the condition must be the same for all lanes: mma.sync needs the whole warp)
-                if (n == kChunkTiles && (kt + kChunkTiles) * kTileCols <= K) {
+            const uint32_t slot = ring + s * R::kSlotBytes;
+            if (!ptx::mbar_wait_bounded(bars + 8 * s, (consumed / kStages) & 1u, abort_flag)) { alive = false; break; }
+            // (n is the same for all lanes: mma.sync needs the whole warp)
+            if (n == kChunkTiles) {
 #pragma unroll
-                    for (int t = 0; t < kChunkTiles; ++t) x[t] = load_x16(xp + t * kTileCols);
-                    if (!ptx::mbar_wait_bounded(bars + 8 * s, (consumed / kStages) & 1u, abort_flag)) { alive = false; break; }
+                for (int t = 0; t < kChunkTiles; ++t) {
+                    const uint4 w0 = lds128(slot + t * kTileBytes + lane * 16);
+                    const uint4 w1 = lds128(slot + t * kTileBytes + 512 + lane * 16);
 #pragma unroll
-                    for (int t = 0; t < kChunkTiles; ++t) mma_tile(acc[0], stage + t * kTileBytes, x[t]);
-                } else {
-#pragma unroll
-                    for (int t = 0; t < kChunkTiles; ++t) {
-                        x[t] = make_uint4(0u, 0u, 0u, 0u);
-                        if (t < n && col0 + t * kTileCols < K) x[t] = load_x16(xp + t * kTileCols);
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const uint4 x = lds128(slot + t * xtile + xlane[nt]);
+                        mma_slab(acc[nt], w0, x.x, x.y);
+                        mma_slab(acc[nt], w1, x.z, x.w);
                     }
-                    if (!ptx::mbar_wait_bounded(bars + 8 * s, (consumed / kStages) & 1u, abort_flag)) { alive = false; break; }
-#pragma unroll
-                    for (int t = 0; t < kChunkTiles; ++t)
-                        if (t < n) mma_tile(acc[0], stage + t * kTileBytes, x[t]);
                 }
             } else {
-                if (!ptx::mbar_wait_bounded(bars + 8 * s, (consumed / kStages) & 1u, abort_flag)) { alive = false; break; }
 #pragma unroll
                 for (int t = 0; t < kChunkTiles; ++t) {
                     if (t < n) {
-                        const uint4 w0 = lds128(stage + t * kTileBytes);
-                        const uint4 w1 = lds128(stage + t * kTileBytes + 512);
+                        const uint4 w0 = lds128(slot + t * kTileBytes + lane * 16);
+                        const uint4 w1 = lds128(slot + t * kTileBytes + 512 + lane * 16);
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
-                            uint4 x = make_uint4(0u, 0u, 0u, 0u);
-                            if (col0 + t * kTileCols < K) x = load_x16(xrow[nt] + kt * kTileCols + t * kTileCols);
+                            const uint4 x = lds128(slot + t * xtile + xlane[nt]);
                             mma_slab(acc[nt], w0, x.x, x.y);
                             mma_slab(acc[nt], w1, x.z, x.w);
                         }
@@ -554,7 +588,7 @@ __global__ void __launch_bounds__(kWarps * 32) decode_dp4a_kernel(const __grid_c
     const DecodeEntry &e = inl.e[0];
     const int lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
-    const int K = e.K, M = e.M, KB = e.KB;
+    const int M = e.M, KB = e.KB;
     for (int rb = blockIdx.x * kWarps + (threadIdx.x >> 5); rb < e.NB; rb += gridDim.x * kWarps) {
         int acc[8][2][4]; // [token][row half][field]
 #pragma unroll
@@ -566,12 +600,10 @@ __global__ void __launch_bounds__(kWarps * 32) decode_dp4a_kernel(const __grid_c
             const uint4 w0 = ld_stream(wp), w1 = ld_stream(wp + 32);
             // [slab][word]: word j is row half j % 2, columns 8 slab + 4 (j / 2) .. + 3 of this lane's 16
             const uint32_t words[2][4] = {{w0.x, w0.y, w0.z, w0.w}, {w1.x, w1.y, w1.z, w1.w}};
-            const int col = kt * kTileCols + 16 * tq;
 #pragma unroll
             for (int t = 0; t < 8; ++t) {
                 if (t >= M) break;
-                uint4 xa = make_uint4(0u, 0u, 0u, 0u);
-                if (col < K) xa = __ldg(reinterpret_cast<const uint4 *>(e.Xq + (size_t)t * K + col));
+                const uint4 xa = __ldg(reinterpret_cast<const uint4 *>(e.Xq + ((size_t)kt * M + t) * kXTileBytes + 16 * tq));
                 const uint32_t xs[4] = {xa.x, xa.y, xa.z, xa.w};
 #pragma unroll
                 for (int sl = 0; sl < 2; ++sl)
@@ -639,14 +671,14 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeSmem);
+        cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Ring<NT>::kSmem);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     static const bool early = tuning_from_env("BITLINEAR_DECODE_EARLY_LAUNCH", 1, 2) == 1; // 2 = off
     void *args[] = {(void *)&inl, (void *)&table, (void *)&n_entries, (void *)&total_tiles, (void *)&share,
                     (void *)&dyn, (void *)&hdr, (void *)&lists};
-    cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT>, grid, block, kDecodeSmem, args, early, stream);
+    cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT>, grid, block, Ring<NT>::kSmem, args, early, stream);
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
     void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists};

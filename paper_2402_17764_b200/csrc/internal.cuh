@@ -41,7 +41,7 @@ struct DecodeEntry {
     const uint4 *packed;   // 2-bit weights
     const float *gamma;    // 1 fp32 (unused when out_i32)
     const __nv_bfloat16 *X; // bf16 [M, K] (input of the quantiser; null for the matmul hook)
-    int8_t *Xq;            // int8 [M, K]
+    int8_t *Xq;            // int8 activations: [M, K] row-major, or, if xq_tiled, [KB column tiles][M][64 bytes]
     float *beta;           // [M]
     int32_t *rowsum;       // [M]
     void *out;             // bf16 [M, N], or int32 [M, N] when out_i32
@@ -51,6 +51,7 @@ struct DecodeEntry {
     uint32_t tile_begin;   // index of this entry's first tile in the launch-wide tile sequence (NB * KB tiles each)
     int token_begin;       // first token of this entry in the batched quantiser's grid
     int out_i32;           // 1: write raw int32 accumulators instead of bf16
+    int xq_tiled;          // layout of Xq (the streaming kernel reads tiles, the tensor-core GEMM rows)
 };
 
 constexpr int kInlineEntries = 4;
@@ -65,6 +66,8 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
                                     cudaStream_t stream);
 cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream);
+// Copies row-major int8 activations [M, K] into the tiled layout [KB][M][64] (columns >= K become 0).
+cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *tiled, cudaStream_t stream);
 
 // Quantises the tokens of every entry (entries with X == nullptr are skipped) and zeroes
 // `zero_bytes` bytes at `zero_ptr` (control words and split-K scratch) in the same launch.

@@ -5,6 +5,9 @@
 // (up to kCache vectors per thread; longer rows re-read the tail, which hits L2), the absmax
 // is reduced with warp shuffles, then every element takes one fp32 multiply by 127/beta,
 // round-half-to-even, clip, and is stored as int8 together with the row sum of the codes.
+// The int8 row is written either as it is ([M, K], for the tensor-core GEMM) or tile by tile
+// ([column tile of 64][token][64 bytes], zero beyond K, for the weight-streaming kernel, which fetches the
+// activations of a run of column tiles with one bulk copy).
 // HBM-bound: 2 B read + 1 B written per element.
 #include "internal.cuh"
 #include "ptx.cuh"
@@ -83,7 +86,13 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
     const int K = e.K;
     const int n_vec = K >> 3;
     const uint4 *row = reinterpret_cast<const uint4 *>(e.X + (size_t)t * K);
-    uint2 *out = reinterpret_cast<uint2 *>(e.Xq + (size_t)t * K);
+    // output position of the i-th group of 8 codes of this token, in 8-byte units
+    uint2 *out_base = reinterpret_cast<uint2 *>(e.Xq);
+    const bool tiled = e.xq_tiled != 0;
+    const size_t M = (size_t)e.M;
+    auto out_at = [&](int i) -> uint2 & {
+        return out_base[tiled ? (((size_t)(i >> 3) * M + (size_t)t) * 8 + (size_t)(i & 7)) : ((size_t)t * n_vec + i)];
+    };
 
     uint4 cache[kCache];
     uint32_t m = 0;
@@ -117,14 +126,16 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
         if (i < n_vec) {
             uint2 o;
             sum += quant8(cache[c], s, o);
-            out[i] = o;
+            out_at(i) = o;
         }
     }
     for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) {
         uint2 o;
         sum += quant8(__ldg(row + i), s, o);
-        out[i] = o;
+        out_at(i) = o;
     }
+    if (tiled) // the last column tile is filled up with zeros
+        for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += kThreads) out_at(i) = make_uint2(0u, 0u);
     sum = __reduce_add_sync(0xffffffffu, sum);
     if (lane == 0) s_sum[warp] = sum;
     __syncthreads();
@@ -137,7 +148,25 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
     }
 }
 
+__global__ void __launch_bounds__(kThreads) retile_acts_kernel(const int8_t *__restrict__ Xq, int M, int K, int KB,
+                                                               int8_t *__restrict__ tiled)
+{
+    const int t = blockIdx.x;
+    const uint2 *row = reinterpret_cast<const uint2 *>(Xq + (size_t)t * K);
+    uint2 *out = reinterpret_cast<uint2 *>(tiled);
+    for (int i = threadIdx.x; i < KB * 8; i += kThreads)
+        out[((size_t)(i >> 3) * M + t) * 8 + (i & 7)] = (i < (K >> 3)) ? __ldg(row + i) : make_uint2(0u, 0u);
+}
+
 } // namespace
+
+cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *tiled, cudaStream_t stream)
+{
+    if (M == 0) return cudaSuccess;
+    const int KB = (int)((K + kTileCols - 1) / kTileCols);
+    retile_acts_kernel<<<(unsigned)M, kThreads, 0, stream>>>(Xq, (int)M, (int)K, KB, tiled);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
                                  void *zero_ptr, size_t zero_bytes, cudaStream_t stream)
