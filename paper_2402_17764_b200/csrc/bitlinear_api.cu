@@ -142,7 +142,7 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
     InlineTable inl{};
     inl.e[0] = e;
-    cudaError_t err = launch_decode(inl, nullptr, 1, (uint32_t)(e.NB * e.KB), e.M,
+    cudaError_t err = launch_decode(inl, nullptr, 1, decode_items(e.NB, e.KB, decode_is_wide(e.M)), e.M,
                                     path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;
@@ -347,7 +347,7 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
         const bitlinear_layer_desc &d = layers[i];
         if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1 || d.M > kMaxDecodeM) return false;
         acc += align_up((size_t)d.M * d.N * 4, 256);
-        tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K));
+        tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K)); // an upper bound of the work items in either mode
         if (entry_off) entry_off->push_back(data);
         data += align_up((size_t)d.M * col_tiles(d.K) * kTileCols, 256) + 2 * align_up((size_t)d.M * 4, 256);
     }
@@ -396,6 +396,9 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     size_t a_off = S.acc32;
     uint32_t tiles = 0;
     int tokens = 0, max_M = 0;
+    for (int i = 0; i < n; ++i)
+        if ((int)layers[i].M > max_M) max_M = (int)layers[i].M;
+    const bool wide = decode_is_wide(max_M); // one kernel serves the whole sequence
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         Layout L{};
@@ -408,9 +411,8 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
         table[(size_t)i].xq_tiled = 1;
         table[(size_t)i].tile_begin = tiles;
         table[(size_t)i].token_begin = tokens;
-        tiles += (uint32_t)(table[(size_t)i].NB * table[(size_t)i].KB);
+        tiles += decode_items(table[(size_t)i].NB, table[(size_t)i].KB, wide);
         tokens += (int)d.M;
-        if ((int)d.M > max_M) max_M = (int)d.M;
     }
     bitlinear_sequence *seq = new (std::nothrow) bitlinear_sequence();
     if (!seq) return BITLINEAR_ERR_ARG;

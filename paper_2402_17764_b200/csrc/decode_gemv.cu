@@ -253,6 +253,34 @@ __device__ __forceinline__ void mma_slab(int (&acc)[4][4], const uint4 &w, uint3
 }
 
 
+// Un-mixes the four scaled accumulators of every (row, token) this lane holds and hands the row sums to fn.
+// C fragment of field f: c0 (row 16f + g, token 2tq), c1 (same row, 2tq + 1), c2 (row 16f + 8 + g, 2tq), c3.
+template <int NT, class Fn>
+__device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, int N, int row0, int tq, Fn fn)
+{
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int tb = 0; tb < 2; ++tb) {
+            const int token = 8 * nt + 2 * tq + tb;
+            if (token >= M) continue;
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = 2 * h + tb;
+                const int t1 = acc[nt][1][c] >> 2; // S1 + 4 S2 + 16 S3   (exact shifts)
+                const int t2 = acc[nt][2][c] >> 4; // S2 + 4 S3
+                const int t3 = acc[nt][3][c] >> 6; // S3
+                const int S[4] = {acc[nt][0][c] - 4 * t1, t1 - 4 * t2, t2 - 4 * t3, t3};
+#pragma unroll
+                for (int f = 0; f < 4; ++f) {
+                    const int r = row0 + 16 * f + 8 * h;
+                    if (r < N) fn(token, r, S[f]);
+                }
+            }
+        }
+    }
+}
+
 template <int NT>
 __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
@@ -518,31 +546,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             if (lane == 0) owned[n_owned] = make_uint2((uint32_t)(e - tab), (uint32_t)rb);
             ++n_owned; // cannot exceed kMaxOwned: see next_piece
         }
-        // C fragment of field f: c0 (row 16f + g, token 2tq), c1 (same row, 2tq + 1), c2 (row 16f + 8 + g, 2tq), c3.
-        const int N = e->N, row0 = rb * kTileRows + g;
-        finish_block(*e, complete, [&](auto fn) {
-#pragma unroll
-            for (int nt = 0; nt < NT; ++nt) {
-#pragma unroll
-                for (int tb = 0; tb < 2; ++tb) {
-                    const int token = 8 * nt + 2 * tq + tb;
-                    if (token >= M) continue;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int c = 2 * h + tb;
-                        const int t1 = acc[nt][1][c] >> 2; // S1 + 4 S2 + 16 S3   (exact shifts)
-                        const int t2 = acc[nt][2][c] >> 4; // S2 + 4 S3
-                        const int t3 = acc[nt][3][c] >> 6; // S3
-                        const int S[4] = {acc[nt][0][c] - 4 * t1, t1 - 4 * t2, t2 - 4 * t3, t3};
-#pragma unroll
-                        for (int f = 0; f < 4; ++f) {
-                            const int r = row0 + 16 * f + 8 * h;
-                            if (r < N) fn(token, r, S[f]);
-                        }
-                    }
-                }
-            }
-        });
+        finish_block(*e, complete, [&](auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, fn); });
 
         // next row block, or next matrix
         if (kt == KB) {
@@ -563,6 +567,245 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
     }
 
+    if (lane == 0) lists[w].n = (uint32_t)n_owned;
+}
+
+// ---------------------------------------------------------------------------------------------
+// The same matmul for 9 to 64 tokens.  With many tokens the activations of a chunk are as large as, or
+// larger than, its weights, so here the eight warps of a CTA share them: the CTA walks a sequence of
+// GROUP tiles (eight consecutive row blocks x one column tile), warp i streams row block 8 * group + i
+// through its own ring exactly as above, and the activations of a chunk are fetched ONCE per CTA into a
+// shared ring.  Two barriers per activation slot keep the warps together: `xfull` (the copy has landed) and
+// `xempty` (all eight warps are done with the slot; only then does warp 0 refill it), so the warps of a CTA
+// are never more than the ring depth apart.  The CTAs take equal contiguous shares of the group-tile
+// sequence; cut row blocks go through the scratch and the per-warp lists as above.
+template <int NT>
+struct WideRing {
+    static constexpr int kTiles = 4;   // column tiles per chunk
+    static constexpr int kDepth = 3;   // chunks in flight
+    static constexpr int kWeightBytes = kTiles * kTileBytes;
+    static constexpr int kXSlotBytes = kTiles * 8 * NT * kXTileBytes;
+    static constexpr int kXOffset = kWarps * kDepth * kWeightBytes;
+    static constexpr int kBarsOffset = kXOffset + kDepth * kXSlotBytes;
+    static constexpr int kAbortOffset = kBarsOffset + (kWarps + 2) * kDepth * 8;
+    static constexpr int kSmem = kAbortOffset + 16;
+    static_assert(kSmem <= 227 * 1024, "rings do not fit the SM's shared memory");
+};
+
+template <int NT>
+__global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
+    const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
+    uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists)
+{
+    extern __shared__ __align__(128) uint8_t dsmem[];
+    ptx::griddep_launch_dependents();
+    using R = WideRing<NT>;
+    constexpr int kChunkTiles = R::kTiles, kDepth = R::kDepth;
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const uint32_t wring = ptx::smem_u32(dsmem) + warp * (kDepth * R::kWeightBytes);
+    const uint32_t xring = ptx::smem_u32(dsmem + R::kXOffset);
+    const uint32_t wbars = ptx::smem_u32(dsmem + R::kBarsOffset) + warp * (kDepth * 8); // this warp's weights have landed
+    const uint32_t xfull = ptx::smem_u32(dsmem + R::kBarsOffset) + kWarps * kDepth * 8; // the CTA's activations have landed
+    const uint32_t xempty = xfull + kDepth * 8;                                         // all warps are done with them
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + R::kAbortOffset);
+    const uint32_t w = blockIdx.x * kWarps + warp;
+    uint2 *owned = lists[w].item;
+    int n_owned = 0;
+
+    if (threadIdx.x == 0) {
+        *abort_flag = 0;
+#pragma unroll
+        for (int s = 0; s < kDepth; ++s) {
+            ptx::mbar_init(xfull + 8 * s, 1);
+            ptx::mbar_init(xempty + 8 * s, kWarps);
+        }
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int s = 0; s < kDepth; ++s) ptx::mbar_init(wbars + 8 * s, 1);
+        ptx::fence_mbar_init();
+    }
+    __syncthreads();
+
+    const DecodeEntry *tab = table ? table : inl.e;
+    const uint64_t i0 = (uint64_t)blockIdx.x * share;
+    const uint32_t i1 = (uint32_t)(i0 + share < total_items ? i0 + share : total_items);
+
+    // A walker steps through the CTA's share chunk by chunk; producer and consumer each have one.
+    struct Walker {
+        const DecodeEntry *e;
+        int KB, groups, group, kt, left;
+    };
+    struct Chunk {
+        const DecodeEntry *e;
+        int group, kt, n;
+        bool ends_group;
+    };
+    auto step = [](Walker &p) {
+        Chunk c;
+        c.e = p.e;
+        c.group = p.group;
+        c.kt = p.kt;
+        c.n = min(min(kChunkTiles, p.KB - p.kt), p.left);
+        p.kt += c.n;
+        p.left -= c.n;
+        c.ends_group = p.kt == p.KB;
+        if (c.ends_group) {
+            p.kt = 0;
+            if (++p.group == p.groups && p.left > 0) {
+                ++p.e;
+                p.KB = p.e->KB;
+                p.groups = (p.e->NB + kWarps - 1) / kWarps;
+                p.group = 0;
+            }
+        }
+        return c;
+    };
+
+    [&]() {
+    if (i0 >= i1) {
+        ptx::griddep_wait();
+        return;
+    }
+    Walker prod;
+    prod.e = tab + find_entry(tab, n_entries, (uint32_t)i0, lane);
+    prod.KB = prod.e->KB;
+    prod.groups = (prod.e->NB + kWarps - 1) / kWarps;
+    {
+        const uint32_t local = (uint32_t)i0 - prod.e->tile_begin;
+        prod.group = (int)(local / (uint32_t)prod.KB);
+        prod.kt = (int)(local - (uint32_t)prod.group * (uint32_t)prod.KB);
+    }
+    prod.left = (int)(i1 - (uint32_t)i0);
+    Walker cons = prod;
+    uint32_t issued = 0, consumed = 0;
+
+    bool x_ready = false; // see the kernel above: activation copies wait for the launch before this one
+    const int8_t *held_x[kDepth];
+    uint32_t held_bytes[kDepth];
+    int n_held = 0;
+    bool alive = true;
+
+    auto top_up = [&]() {
+        while (alive && prod.left > 0 && issued - consumed < (uint32_t)kDepth) {
+            const uint32_t s = issued % kDepth;
+            if (warp == 0 && issued >= (uint32_t)kDepth) {
+                // the slot's previous contents must have been consumed by all eight warps
+                if (!ptx::mbar_wait_bounded(xempty + 8 * s, (issued / kDepth - 1) & 1u, abort_flag)) {
+                    alive = false;
+                    break;
+                }
+            }
+            const Chunk c = step(prod);
+            const int rb = c.group * kWarps + warp;
+            const int xb = c.e->M * kXTileBytes;
+            const int8_t *xsrc = c.e->Xq + (size_t)c.kt * xb;
+            const uint32_t xbytes = (uint32_t)(c.n * xb);
+            if (lane == 0) {
+                if (rb < c.e->NB) {
+                    const uint8_t *src = reinterpret_cast<const uint8_t *>(c.e->packed) + ((size_t)rb * c.e->KB + c.kt) * kTileBytes;
+                    ptx::mbar_arrive_expect_tx(wbars + 8 * s, (uint32_t)c.n * kTileBytes);
+                    bulk_copy_g2s(wring + s * R::kWeightBytes, src, (uint32_t)c.n * kTileBytes, wbars + 8 * s);
+                } else {
+                    ptx::mbar_arrive(wbars + 8 * s); // no row block for this warp: the slot's phase still has to advance
+                }
+                if (warp == 0 && x_ready) {
+                    ptx::mbar_arrive_expect_tx(xfull + 8 * s, xbytes);
+                    bulk_copy_g2s(xring + s * R::kXSlotBytes, xsrc, xbytes, xfull + 8 * s);
+                }
+            }
+            if (!x_ready) {
+                held_x[n_held] = xsrc;
+                held_bytes[n_held] = xbytes;
+                ++n_held;
+            }
+            ++issued;
+        }
+    };
+    top_up();
+    ptx::griddep_wait();
+    x_ready = true;
+    if (warp == 0 && lane == 0) {
+#pragma unroll
+        for (int i = 0; i < kDepth; ++i) {
+            if (i < n_held) {
+                ptx::mbar_arrive_expect_tx(xfull + 8 * i, held_bytes[i]);
+                bulk_copy_g2s(xring + i * R::kXSlotBytes, held_x[i], held_bytes[i], xfull + 8 * i);
+            }
+        }
+    }
+
+    while (alive && cons.left > 0) {
+        // ---- one group of row blocks (or the part of it that lies in this share); this warp's row block is rb
+        const DecodeEntry *e = cons.e;
+        const int M = e->M, KB = cons.KB;
+        const int rb = cons.group * kWarps + warp;
+        const bool active = rb < e->NB; // the last group of a matrix may have fewer than eight row blocks
+        int acc[NT][4][4];
+        uint32_t xlane[NT];
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+            for (int f = 0; f < 4; ++f) acc[nt][f][0] = acc[nt][f][1] = acc[nt][f][2] = acc[nt][f][3] = 0;
+            xlane[nt] = (uint32_t)(min(8 * nt + g, M - 1) * kXTileBytes + 16 * tq);
+        }
+        const uint32_t xtile = (uint32_t)(M * kXTileBytes);
+        int tiles = 0;
+        bool ended = false;
+        while (!ended && cons.left > 0) {
+            const Chunk c = step(cons);
+            ended = c.ends_group;
+            const uint32_t s = consumed % kDepth;
+            const uint32_t parity = (consumed / kDepth) & 1u;
+            if (!ptx::mbar_wait_bounded(xfull + 8 * s, parity, abort_flag) ||
+                (active && !ptx::mbar_wait_bounded(wbars + 8 * s, parity, abort_flag))) {
+                alive = false;
+                break;
+            }
+            if (active) { // (the same for all lanes: mma.sync needs the whole warp)
+                const uint32_t wslot = wring + s * R::kWeightBytes + lane * 16;
+                const uint32_t xslot = xring + s * R::kXSlotBytes;
+#pragma unroll
+                for (int t = 0; t < kChunkTiles; ++t) {
+                    if (t < c.n) {
+                        const uint4 w0 = lds128(wslot + t * kTileBytes);
+                        const uint4 w1 = lds128(wslot + t * kTileBytes + 512);
+#pragma unroll
+                        for (int nt = 0; nt < NT; ++nt) {
+                            const uint4 x = lds128(xslot + t * xtile + xlane[nt]);
+                            mma_slab(acc[nt], w0, x.x, x.y);
+                            mma_slab(acc[nt], w1, x.z, x.w);
+                        }
+                    }
+                }
+            }
+            __syncwarp(); // every lane has read both slots
+            if (lane == 0) ptx::mbar_arrive(xempty + 8 * s);
+            ++consumed;
+            tiles += c.n;
+            top_up();
+        }
+        if (!alive) break;
+        if (active) {
+            const bool complete = tiles == KB;
+            if (!complete && ended) {
+                if (n_owned < kMaxOwned) {
+                    if (lane == 0) owned[n_owned] = make_uint2((uint32_t)(e - tab), (uint32_t)rb);
+                    ++n_owned;
+                }
+            }
+            finish_block(*e, complete, [&](auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, fn); });
+        }
+    }
+    }();
+
+    if (*abort_flag) {
+        if (lane == 0) atomicExch(&hdr->status, (int32_t)BITLINEAR_ERR_TIMEOUT);
+        const uint64_t t0 = ptx::globaltimer_ns();
+        while (ptx::globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+    }
     if (lane == 0) lists[w].n = (uint32_t)n_owned;
 }
 
@@ -685,11 +928,46 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
     return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
 }
 
+template <int NT>
+static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, const DecodeEntry *table, int n_entries,
+                               uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists,
+                               cudaStream_t stream)
+{
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(decode_wide_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, WideRing<NT>::kSmem);
+        if (e != cudaSuccess) return e;
+        attr_set[dev] = true;
+    }
+    static const bool early = tuning_from_env("BITLINEAR_DECODE_EARLY_LAUNCH", 1, 2) == 1; // 2 = off
+    void *args[] = {(void *)&inl, (void *)&table, (void *)&n_entries, (void *)&total_items, (void *)&share,
+                    (void *)&hdr, (void *)&lists};
+    cudaError_t err = launch_dependent((const void *)decode_wide_kernel<NT>, grid, block, WideRing<NT>::kSmem, args, early, stream);
+    if (err != cudaSuccess) return err;
+    uint32_t n_lists = grid.x * kWarps;
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists};
+    return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
+}
+
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
                           int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream)
 {
     if (total_tiles == 0) return cudaSuccess;
     const dim3 block(kWarps * 32);
+    if (path != BITLINEAR_PATH_DP4A && decode_is_wide(max_M)) {
+        // total_tiles counts group tiles here; one CTA per SM, equal contiguous shares, at least 4 items each
+        uint32_t ctas = (total_tiles + 3) / 4;
+        uint32_t cap = (uint32_t)sm_count();
+        if (cap > kMaxDecodeWarps / kWarps) cap = kMaxDecodeWarps / kWarps;
+        if (ctas > cap) ctas = cap;
+        const uint32_t share = (total_tiles + ctas - 1) / ctas;
+        const dim3 grid(ctas);
+        if (max_M <= 16) return launch_wide<2>(grid, block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+        if (max_M <= 32) return launch_wide<4>(grid, block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+        return launch_wide<8>(grid, block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+    }
     if (path == BITLINEAR_PATH_DP4A) {
         int ctas = (inl.e[0].NB + kWarps - 1) / kWarps;
         const int cap = sm_count() * 4;
@@ -700,7 +978,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     // every warp should have at least kMinTilesPerWarp tiles; beyond that, fill the machine
     constexpr uint32_t kMinTilesPerWarp = 4;
     uint32_t ctas = (total_tiles + kMinTilesPerWarp * kWarps - 1) / (kMinTilesPerWarp * kWarps);
-    uint32_t cap = (uint32_t)sm_count() * (max_M <= 16 ? kCtasPerSm : 1);
+    uint32_t cap = (uint32_t)sm_count() * kCtasPerSm;
     if (cap > kMaxDecodeWarps / kWarps) cap = kMaxDecodeWarps / kWarps;
     if (ctas > cap) ctas = cap;
     const dim3 grid(ctas);
@@ -718,10 +996,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     } else {
         share = (total_tiles + n_warps - 1) / n_warps; // all static: the last warps may get less, or nothing
     }
-    if (max_M <= 8) return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
-    if (max_M <= 16) return launch_mma<2>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
-    if (max_M <= 32) return launch_mma<4>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
-    return launch_mma<8>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
+    return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
 }
 
 } // namespace bitlinear

@@ -48,7 +48,8 @@ struct DecodeEntry {
     int32_t *acc32;        // scratch [M, N] for row blocks shared by several warps (zero before and after a launch)
     int M, N, K;
     int KB, NB;            // column tiles = ceil(K / 64), row blocks = ceil(N / 64)
-    uint32_t tile_begin;   // index of this entry's first tile in the launch-wide tile sequence (NB * KB tiles each)
+    uint32_t tile_begin;   // index of this entry's first work item in the launch-wide sequence: tiles (NB * KB per
+                           // entry) for up to 8 tokens, group tiles (ceil(NB / 8) * KB per entry) beyond: see below
     int token_begin;       // first token of this entry in the batched quantiser's grid
     int out_i32;           // 1: write raw int32 accumulators instead of bf16
     int xq_tiled;          // layout of Xq (the streaming kernel reads tiles, the tensor-core GEMM rows)
@@ -74,7 +75,13 @@ cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *t
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
                                  void *zero_ptr, size_t zero_bytes, cudaStream_t stream);
 
-// Persistent weight-streaming matmul over the entries (total_tiles = sum of NB * KB).
+// The weight-streaming matmul has two kernels: up to 8 tokens every warp streams tiles on its own; from 9
+// tokens the eight warps of a CTA share the activations and the CTA walks group tiles (8 row blocks x 1
+// column tile).  The sequence of work items of a launch is counted accordingly.
+inline bool decode_is_wide(int max_M) { return max_M > 8; }
+inline uint32_t decode_items(int NB, int KB, bool wide) { return (uint32_t)(wide ? (NB + 7) / 8 : NB) * (uint32_t)KB; }
+
+// Persistent weight-streaming matmul over the entries (total_tiles = sum of decode_items over the entries).
 // path: BITLINEAR_PATH_MMA, or BITLINEAR_PATH_DP4A (first entry only).
 // `lists` is scratch of kOwnedListsBytes (no need to clear it).
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
