@@ -211,22 +211,34 @@ __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, cons
                 }
             }
         }
-        // further tokens
+        // further tokens, eight at a time with their loads issued together
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             if (N[b] == 0) continue;
             const int M = e[b]->M;
-            for (int t = 1; t < M; ++t) {
-                const int rs = e[b]->rowsum[t];
-                const float sc = token_scale(*e[b], t);
+            for (int t0 = 1; t0 < M; t0 += 8) {
+                int tv[8][kTileRows / 32], rs[8];
+                float sc[8];
 #pragma unroll
-                for (int h = 0; h < kTileRows / 32; ++h) {
-                    const int r = r0[b] + 32 * h;
-                    if (r < N[b]) {
-                        int32_t *p = acc[b] + (size_t)t * N[b] + r;
-                        const int total = __ldcg(p);
-                        __stcg(p, 0);
-                        store_result(*e[b], t, r, total, rs, sc);
+                for (int i = 0; i < 8; ++i) {
+                    const int t = min(t0 + i, M - 1); // slots past the last token repeat it and store nothing
+#pragma unroll
+                    for (int h = 0; h < kTileRows / 32; ++h)
+                        tv[i][h] = (r0[b] + 32 * h < N[b]) ? __ldcg(acc[b] + (size_t)t * N[b] + r0[b] + 32 * h) : 0;
+                    rs[i] = e[b]->rowsum[t];
+                    sc[i] = token_scale(*e[b], t);
+                }
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const int t = t0 + i;
+                    if (t >= M) break;
+#pragma unroll
+                    for (int h = 0; h < kTileRows / 32; ++h) {
+                        const int r = r0[b] + 32 * h;
+                        if (r < N[b]) {
+                            __stcg(acc[b] + (size_t)t * N[b] + r, 0);
+                            store_result(*e[b], t, r, tv[i][h], rs[i], sc[i]);
+                        }
                     }
                 }
             }
