@@ -92,6 +92,13 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
                            const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
                            WorkspaceHeader *hdr, cudaStream_t stream);
 
+// The same GEMM on pairs of SMs (tcgen05 cta_group::2): 256 tokens x 256 features per pair tile.
+// prefill_pair_capacity: CTA pairs that can be resident at once (0: not available on this device).
+cudaError_t launch_prefill_pair(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
+                                const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
+                                WorkspaceHeader *hdr, cudaStream_t stream);
+int prefill_pair_capacity();
+
 int sm_count();
 
 } // namespace bitlinear
