@@ -188,7 +188,8 @@ def test_matmul_i32_decode_paths(oracle, M, K, N, path):
     assert B.poll_status(ws) == 0
 
 
-@pytest.mark.parametrize("M,K,N", [(16, 4096, 4096), (17, 8640, 1024), (33, 3200, 3200), (64, 1536, 4096)])
+@pytest.mark.parametrize("M,K,N", [(16, 4096, 4096), (17, 8640, 1024), (33, 3200, 3200), (64, 1536, 4096),
+                                   (9, 144, 48), (20, 16, 16), (40, 3200, 1040), (64, 32768, 16), (12, 1024, 8256)])
 def test_matmul_i32_mma_wider_batches(oracle, M, K, N):
     T, Xq, packed = make_operands(oracle, M, K, N, M * 7 + N)
     ref = oracle.matmul_i32(Xq, T)
@@ -334,3 +335,28 @@ def test_forward_sequence_matches_single_calls(oracle):
             for l, ref in zip(layers, refs):
                 assert np.array_equal(torch_bf16_to_bits(l[3]), ref)
         seq.close()
+
+
+def test_forward_sequence_with_mixed_token_counts(oracle):
+    """Entries of one sequence may have different M; one entry above 8 tokens puts the whole sequence on the
+    kernel in which the warps of a CTA share the activations.  Ragged shapes: N and K not multiples of 64."""
+    specs = [(3, 144, 48), (20, 1536, 1040), (1, 3200, 512), (64, 80, 528), (9, 8640, 16)]
+    layers, refs = [], []
+    for i, (M, K, N) in enumerate(specs):
+        W = S.latent_weights(N, K, 40 + i)
+        X = S.activations(M, K, 40 + i, outlier_frac=0.02, outlier_scale=10.0)
+        T_ref, g_ref = oracle.quantize_weights(W.numpy())
+        refs.append(oracle.forward(T_ref, g_ref, torch_bf16_to_bits(X)))
+        packed, gamma = B.quantize_weights(dev(W))
+        buf, Y, pad = guarded((M, N), torch.bfloat16)
+        layers.append((packed, gamma, dev(X), Y, N))
+        layers[-1] = layers[-1] + (buf, pad)
+    seq = B.Sequence([l[:5] for l in layers])
+    for _ in range(2):
+        seq.forward()
+        torch.cuda.synchronize()
+        assert B.poll_status(seq.workspace) == 0
+        for (packed, gamma, X, Y, N, buf, pad), ref in zip(layers, refs):
+            assert np.array_equal(torch_bf16_to_bits(Y), ref)
+            check_guards(buf, pad, Y.numel())
+    seq.close()
