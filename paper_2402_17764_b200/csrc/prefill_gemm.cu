@@ -15,6 +15,8 @@
 //                    exact shift, subtract the token's sum of q (codes are T + 1), scale by
 //                    gamma * beta_t / 127, round to bf16 and store, while the MMA warp fills the second
 //                    TMEM buffer.  |acc| <= 64 * 2 * 127 * K < 2^31 for every K the library accepts.
+// The kernel is a programmatic dependent of the activation quantiser: set-up (barriers, tensor memory,
+// descriptor prefetch) runs while the quantiser finishes; the producer waits for it before the first load.
 // All waits are bounded; on expiry the CTA sets the workspace status to BITLINEAR_ERR_TIMEOUT,
 // every role leaves its loop, TMEM is released and the kernel returns.
 //
@@ -116,6 +118,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         if (lane == 0) {
             prefetch_tensormap(&tmap_x);
             prefetch_tensormap(&tmap_w);
+            griddep_wait(); // the activations are written by the launch before this one
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
@@ -375,8 +378,19 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
     }
     int grid = p.tiles_m * p.tiles_n;
     if (grid > sm_count()) grid = sm_count();
-    prefill_gemm_kernel<<<grid, kThreads, kSmemBytes, stream>>>(tmap_x, tmap_w, p);
-    return cudaGetLastError();
+    // programmatic dependent launch: see the head of this file
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.stream = stream;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    void *args[] = {(void *)&tmap_x, (void *)&tmap_w, (void *)&p};
+    return cudaLaunchKernelExC(&cfg, (const void *)prefill_gemm_kernel, args);
 }
 
 } // namespace bitlinear
