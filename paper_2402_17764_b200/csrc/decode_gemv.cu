@@ -593,8 +593,8 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 // sequence; cut row blocks go through the scratch and the per-warp lists as above.
 template <int NT>
 struct WideRing {
-    static constexpr int kTiles = 4;   // column tiles per chunk
-    static constexpr int kDepth = 3;   // chunks in flight
+    static constexpr int kTiles = NT == 2 ? 8 : (NT == 4 ? 6 : 4); // column tiles per chunk
+    static constexpr int kDepth = NT == 8 ? 4 : 3;                  // chunks in flight
     static constexpr int kWeightBytes = kTiles * kTileBytes;
     static constexpr int kXSlotBytes = kTiles * 8 * NT * kXTileBytes;
     static constexpr int kXOffset = kWarps * kDepth * kWeightBytes;
