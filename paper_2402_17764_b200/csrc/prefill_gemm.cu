@@ -15,6 +15,10 @@
 //                    exact shift, subtract the token's sum of q (codes are T + 1), scale by
 //                    gamma * beta_t / 127, round to bf16 and store, while the MMA warp fills the second
 //                    TMEM buffer.  |acc| <= 64 * 2 * 127 * K < 2^31 for every K the library accepts.
+// With more than 128 tokens a CTA takes TWO token tiles per feature tile (MT = 2): the expanded weight
+// tile, the costly operand (written once and read once per MMA through shared memory, whose bandwidth bounds
+// this kernel), then feeds two MMAs per k step, and the two accumulators fill the tensor memory, so the
+// epilogue of a tile no longer overlaps the next tile's MMAs.
 // The kernel is a programmatic dependent of the activation quantiser: set-up (barriers, tensor memory,
 // descriptor prefetch) runs while the quantiser finishes; the producer waits for it before the first load.
 // All waits are bounded; on expiry the CTA sets the workspace status to BITLINEAR_ERR_TIMEOUT,
@@ -32,11 +36,10 @@ namespace {
 
 using namespace ptx;
 
-constexpr int BM = 128;      // tokens per tile  (MMA M, TMEM lanes)
+constexpr int BM = 128;      // tokens per MMA (MMA M, TMEM lanes); a CTA tile has MT of them
 constexpr int BN = 256;      // features per tile (MMA N, TMEM columns per accumulator)
 constexpr int BK = 128;      // int8 elements (= bytes) of K per stage
-constexpr int kStages = 4;
-constexpr int kAccBufs = 2;
+constexpr int kMaxStages = 4;
 constexpr int kTmemCols = 512;
 
 constexpr int kProducerWarp = 0;
@@ -46,19 +49,25 @@ constexpr int kFirstExpanderWarp = 6; // 8 warps
 constexpr int kExpanderWarps = 8;
 constexpr int kThreads = (kFirstExpanderWarp + kExpanderWarps) * 32; // 448
 
-constexpr uint32_t kABytes = BM * BK;            // 16 KiB int8 activations
+constexpr uint32_t kABytes = BM * BK;            // 16 KiB int8 activations per token tile
 constexpr uint32_t kBBytes = BN * BK;            // 32 KiB expanded weights
 constexpr uint32_t kPBytes = (BN / kTileRows) * (BK / kTileCols) * kTileBytes; //  8 KiB packed weights
-constexpr uint32_t kStageBytes = kABytes + kBBytes + kPBytes;
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared memory of an SM");
+
+template <int MT>
+struct Cfg {
+    static constexpr int kStages = (MT == 1) ? 4 : 3;
+    static constexpr int kAccBufs = (MT == 1) ? 2 : 1; // MT * BN * kAccBufs = all 512 TMEM columns
+    static constexpr uint32_t kStageBytes = MT * kABytes + kBBytes + kPBytes;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared memory of an SM");
+};
 
 struct Barriers {
-    uint64_t full[kStages];      // TMA bytes landed (activations + packed weights)
-    uint64_t expanded[kStages];  // int8 weight tile written
-    uint64_t empty[kStages];     // MMAs that read the stage have completed
-    uint64_t acc_full[kAccBufs]; // accumulator complete
-    uint64_t acc_empty[kAccBufs];// accumulator drained by the epilogue
+    uint64_t full[kMaxStages];      // TMA bytes landed (activations + packed weights)
+    uint64_t expanded[kMaxStages];  // int8 weight tile written
+    uint64_t empty[kMaxStages];     // MMAs that read the stage have completed
+    uint64_t acc_full[2];           // accumulator(s) of a tile complete
+    uint64_t acc_empty[2];          // drained by the epilogue
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -69,15 +78,18 @@ struct Params {
     const int32_t *rowsum;
     void *out;
     int M, N, KB; // KB = k blocks of 128 columns
-    int tiles_m, tiles_n;
+    int tiles_m, tiles_n; // CTA tiles: MT * 128 tokens x 256 features
     int out_i32;
     int32_t *status;
 };
 
+template <int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const Params p)
 {
+    constexpr int kStages = Cfg<MT>::kStages, kAccBufs = Cfg<MT>::kAccBufs;
+    constexpr uint32_t kStageBytes = Cfg<MT>::kStageBytes;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u; // swizzled tiles need 1024-byte alignment
@@ -122,8 +134,9 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.tiles_m) * BM;
+                const int m0 = (tile % p.tiles_m) * (MT * BM);
                 const int n0 = (tile / p.tiles_m) * BN;
+                const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // a second token tile past the end is left out
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t round = it / kStages;
@@ -133,9 +146,10 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                     const uint32_t full = smem_u32(&bars->full[s]);
                     const uint32_t a_dst = base + s * kStageBytes;
-                    const uint32_t p_dst = a_dst + kABytes + kBBytes;
-                    mbar_arrive_expect_tx(full, kABytes + kPBytes);
+                    const uint32_t p_dst = a_dst + MT * kABytes + kBBytes;
+                    mbar_arrive_expect_tx(full, halves * kABytes + kPBytes);
                     tma_load_2d(a_dst, &tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
+                    if (halves == 2) tma_load_2d(a_dst + kABytes, &tmap_x, kb * BK, m0 + BM, full);
                     tma_load_3d(p_dst, &tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
                 }
             }
@@ -149,7 +163,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
             const uint32_t use = tile_it / kAccBufs;
             if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
+            const bool two = MT == 2 && (tile % p.tiles_m) * (MT * BM) + BM < p.M;
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int s = it % kStages;
                 const uint32_t parity = (it / kStages) & 1;
@@ -161,11 +176,13 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                 tc_fence_after_sync();
                 if (lane == 0) {
                     const uint32_t a_addr = base + s * kStageBytes;
-                    const uint32_t b_addr = a_addr + kABytes;
+                    const uint32_t b_addr = a_addr + MT * kABytes;
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 32; ++k4) {
-                        mma_i8_ss(d_tmem, smem_desc_k_sw128(a_addr + 32 * k4), smem_desc_k_sw128(b_addr + 32 * k4),
-                                  idesc, (kb > 0 || k4 > 0) ? 1u : 0u);
+                        const uint64_t b_desc = smem_desc_k_sw128(b_addr + 32 * k4);
+                        const uint32_t accumulate = (kb > 0 || k4 > 0) ? 1u : 0u;
+                        mma_i8_ss(d_tmem, smem_desc_k_sw128(a_addr + 32 * k4), b_desc, idesc, accumulate);
+                        if (two) mma_i8_ss(d_tmem + BN, smem_desc_k_sw128(a_addr + kABytes + 32 * k4), b_desc, idesc, accumulate);
                     }
                     mma_commit(smem_u32(&bars->empty[s])); // stage reusable once these MMAs have read it
                 }
@@ -198,8 +215,8 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     break;
                 }
                 uint8_t *stage = smem + s * kStageBytes;
-                const uint4 *packed = reinterpret_cast<const uint4 *>(stage + kABytes + kBBytes) + ew * (kTileBytes / 16);
-                uint8_t *bt = stage + kABytes;
+                const uint4 *packed = reinterpret_cast<const uint4 *>(stage + MT * kABytes + kBBytes) + ew * (kTileBytes / 16);
+                uint8_t *bt = stage + MT * kABytes;
                 const uint4 w0 = packed[slot], w1 = packed[32 + slot];
                 const uint32_t lo[2][2] = {{w0.x, w0.z}, {w0.y, w0.w}}; // [h][hi], slab 0
                 const uint32_t up[2][2] = {{w1.x, w1.z}, {w1.y, w1.w}}; // slab 1
@@ -225,13 +242,17 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         uint32_t tile_it = 0;
         const float gamma = p.out_i32 ? 0.0f : *p.gamma;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_it) {
-            const int m0 = (tile % p.tiles_m) * BM;
+            const int m0 = (tile % p.tiles_m) * (MT * BM);
             const int n0 = (tile / p.tiles_m) * BN;
             const int buf = tile_it % kAccBufs;
             const uint32_t parity = (tile_it / kAccBufs) & 1;
             if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), parity, abort_flag)) break;
             tc_fence_after_sync();
-            const int t = m0 + 32 * q + lane;
+#pragma unroll 1
+            for (int half = 0; half < MT; ++half) {
+            if (half == 1 && m0 + BM >= p.M) break; // no MMA wrote that accumulator
+            const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
+            const int t = m0 + half * BM + 32 * q + lane;
             const bool row_ok = t < p.M;
             float scale = 0.0f;
             int rowsum = 0;
@@ -242,7 +263,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * BN + c * 32), v);
+                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
                 tmem_ld_wait();
                 const int n = n0 + c * 32;
                 // output row n + i carries the factor 4^f, f = ((n + i) % 64) / 16 = 2 (c % 2) + i / 16
@@ -275,6 +296,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     }
                 }
             }
+            } // token tiles
             tc_fence_before_sync();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
@@ -363,16 +385,23 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
     p.M = (int)M;
     p.N = (int)N;
     p.KB = KB;
-    p.tiles_m = (int)((M + BM - 1) / BM);
+    const int mt = (M > BM) ? 2 : 1; // token tiles per CTA tile
+    p.tiles_m = (int)((M + mt * BM - 1) / (mt * BM));
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.out_i32 = out_i32;
     p.status = &hdr->status;
+    const void *kernel = (mt == 2) ? (const void *)prefill_gemm_kernel<2> : (const void *)prefill_gemm_kernel<1>;
+    const uint32_t smem_bytes = (mt == 2) ? Cfg<2>::kSmemBytes : Cfg<1>::kSmemBytes;
 
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)Cfg<1>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)Cfg<2>::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
@@ -385,12 +414,12 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3((unsigned)grid);
     cfg.blockDim = dim3(kThreads);
-    cfg.dynamicSmemBytes = kSmemBytes;
+    cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     void *args[] = {(void *)&tmap_x, (void *)&tmap_w, (void *)&p};
-    return cudaLaunchKernelExC(&cfg, (const void *)prefill_gemm_kernel, args);
+    return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
 } // namespace bitlinear
