@@ -59,7 +59,8 @@ enum {
     BITLINEAR_PATH_DP4A = 1,   /* scalar dp4a, M <= 8 */
     BITLINEAR_PATH_MMA = 2,    /* warp-level integer MMA on register-unpacked weights, M <= 64 */
     BITLINEAR_PATH_TCGEN05 = 3,     /* TMA + tcgen05 int8 tensor-core GEMM with TMEM accumulators, any M */
-    BITLINEAR_PATH_TCGEN05_PAIR = 4 /* the same GEMM on pairs of SMs (tcgen05 cta_group::2), any M */
+    BITLINEAR_PATH_TCGEN05_PAIR = 4, /* the same GEMM on pairs of SMs (tcgen05 cta_group::2), any M */
+    BITLINEAR_PATH_TCGEN05_TS = 5    /* the same GEMM with the expanded weights in tensor memory, any M */
 };
 
 /* Human-readable name of a status code; never NULL. (host) */

@@ -17,7 +17,7 @@ LIB_PATH = _PKG / "libbitlinear_b200.so"
 
 OK = 0
 ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(-1, -9, -1)
-PATH_AUTO, PATH_DP4A, PATH_MMA, PATH_TCGEN05, PATH_TCGEN05_PAIR = 0, 1, 2, 3, 4
+PATH_AUTO, PATH_DP4A, PATH_MMA, PATH_TCGEN05, PATH_TCGEN05_PAIR, PATH_TCGEN05_TS = 0, 1, 2, 3, 4, 5
 
 EXPORTS = [
     "bitlinear_status_string",

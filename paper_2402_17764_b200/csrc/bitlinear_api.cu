@@ -134,8 +134,14 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
     WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
     OwnedList *lists = reinterpret_cast<OwnedList *>(ws + lists_offset);
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
-                    (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
+                    (path == BITLINEAR_PATH_TCGEN05_TS) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
     if (tc) {
+        static const int ts_tokens = env_int("BITLINEAR_PREFILL_TS_TOKENS", 0); // 192 or 256 (a measurement aid)
+        if (path == BITLINEAR_PATH_TCGEN05_TS || (path == BITLINEAR_PATH_AUTO && ts_tokens > 0)) {
+            cudaError_t err = launch_prefill_ts(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out, e.out_i32,
+                                                ts_tokens > 0 ? ts_tokens : 256, hdr, stream);
+            return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+        }
         // The two-SM form of the GEMM is correct (the tests run it) but measured slower than the one-SM form on
         // B200 (1.15 against 2.2 POP/s), so it is not chosen unless asked for.
         static const int pair_min_m = env_int("BITLINEAR_PREFILL_PAIR_MIN_M", 1 << 30);
@@ -251,7 +257,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                                       int32_t *acc, int path, void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!packed || !workspace || (M > 0 && (!Xq || !acc))) return BITLINEAR_ERR_ARG;
-    if (path < BITLINEAR_PATH_AUTO || path > BITLINEAR_PATH_TCGEN05_PAIR) return BITLINEAR_ERR_ARG;
+    if (path < BITLINEAR_PATH_AUTO || path > BITLINEAR_PATH_TCGEN05_TS) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, N, K);
     if (st != BITLINEAR_OK) return st;
     if (path == BITLINEAR_PATH_DP4A && M > 8) return BITLINEAR_ERR_SHAPE;
@@ -265,7 +271,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     char *ws = reinterpret_cast<char *>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
-                    (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
+                    (path == BITLINEAR_PATH_TCGEN05_TS) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
     InlineTable inl{};
     fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
     const size_t zero_bytes = tc ? sizeof(WorkspaceHeader) : L.table;

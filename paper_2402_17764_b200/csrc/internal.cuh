@@ -99,6 +99,12 @@ cudaError_t launch_prefill_pair(const void *packed, const float *gamma, const in
                                 WorkspaceHeader *hdr, cudaStream_t stream);
 int prefill_pair_capacity();
 
+// The same GEMM with the expanded weights in tensor memory: 128 features x tokens_per_tile (192 or 256)
+// tokens per CTA tile.
+cudaError_t launch_prefill_ts(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
+                              const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
+                              int tokens_per_tile, WorkspaceHeader *hdr, cudaStream_t stream);
+
 int sm_count();
 
 } // namespace bitlinear

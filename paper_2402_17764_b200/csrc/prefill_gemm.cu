@@ -80,6 +80,7 @@ struct Params {
     int M, N, KB; // KB = k blocks of 128 columns
     int tiles_m, tiles_n; // CTA tiles: MT * 128 tokens x 256 features
     int out_i32;
+    int out_32b_aligned; // rows of the bf16 output start on 32-byte boundaries
     int32_t *status;
 };
 
@@ -280,17 +281,22 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     } else {
                         __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)t * p.N + n;
 #pragma unroll
-                        for (int i = 0; i < 32; i += 8) {
+                        for (int i = 0; i < 32; i += 16) { // N is a multiple of 16: 16 features are in or out together
                             if (n + i < p.N) {
-                                uint32_t o[4];
+                                uint32_t o[8];
 #pragma unroll
-                                for (int h = 0; h < 4; ++h) {
+                                for (int h = 0; h < 8; ++h) {
                                     const float x0 = __fmul_rn((float)a[i + 2 * h], scale);
                                     const float x1 = __fmul_rn((float)a[i + 2 * h + 1], scale);
                                     const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
                                     o[h] = *reinterpret_cast<const uint32_t *>(&pr);
                                 }
-                                *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+                                if (p.out_32b_aligned) {
+                                    st_global_v8(dst + i, o);
+                                } else {
+                                    *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+                                    *reinterpret_cast<uint4 *>(dst + i + 8) = make_uint4(o[4], o[5], o[6], o[7]);
+                                }
                             }
                         }
                     }
@@ -389,6 +395,7 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
     p.tiles_m = (int)((M + mt * BM - 1) / (mt * BM));
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.out_i32 = out_i32;
+    p.out_32b_aligned = (reinterpret_cast<uintptr_t>(out) % 32 == 0) ? 1 : 0; // (N is a multiple of 16)
     p.status = &hdr->status;
     const void *kernel = (mt == 2) ? (const void *)prefill_gemm_kernel<2> : (const void *)prefill_gemm_kernel<1>;
     const uint32_t smem_bytes = (mt == 2) ? Cfg<2>::kSmemBytes : Cfg<1>::kSmemBytes;

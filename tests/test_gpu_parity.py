@@ -207,7 +207,7 @@ TC_SHAPES = [(128, 128, 256), (1, 16, 16), (65, 3200, 320), (200, 8640, 528), (3
              (64, 4096, 4096), (129, 144, 4112)]
 
 
-@pytest.mark.parametrize("path", [B.PATH_TCGEN05, B.PATH_TCGEN05_PAIR])
+@pytest.mark.parametrize("path", [B.PATH_TCGEN05, B.PATH_TCGEN05_PAIR, B.PATH_TCGEN05_TS])
 @pytest.mark.parametrize("M,K,N", TC_SHAPES)
 def test_matmul_i32_tcgen05(oracle, M, K, N, path):
     T, Xq, packed = make_operands(oracle, M, K, N, M + 3 * K + N)
