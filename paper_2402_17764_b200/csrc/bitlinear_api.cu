@@ -72,7 +72,8 @@ Layout single_layout(int64_t M, int64_t N, int64_t K)
     L.lists = off;
     off += align_up(kOwnedListsBytes, 256);
     L.xq = off;
-    off += align_up((size_t)M * col_tiles(K) * kTileCols, 256); // room for either layout of the int8 activations
+    // room for either layout of the int8 activations; at least kMinGemmRows rows (see launch_prefill)
+    off += align_up((size_t)(M < kMinGemmRows ? kMinGemmRows : M) * col_tiles(K) * kTileCols, 256);
     L.beta = off;
     off += align_up((size_t)M * 4, 256);
     L.rowsum = off;
@@ -97,11 +98,12 @@ __global__ void rowsum_kernel(const int8_t *__restrict__ Xq, int K, int32_t *__r
     }
 }
 
-// More than 64 tokens always go to the tensor-core GEMM; BITLINEAR_TCGEN05_MIN_M (a measurement aid) lowers the
-// switch-over point.
+// From 17 tokens on a single matmul goes to the tensor-core GEMM: measured on 110080 x 4096, the GEMM takes the
+// same 52 us from 17 to 128 tokens, the weight-streaming kernel 59 us at 16 tokens, 92 us at 32 and 174 us at 64.
+// BITLINEAR_TCGEN05_MIN_M (a measurement aid) moves the switch-over point.
 bool use_tcgen05_for(int64_t M)
 {
-    static const int min_m = env_int("BITLINEAR_TCGEN05_MIN_M", kMaxDecodeM + 1);
+    static const int min_m = env_int("BITLINEAR_TCGEN05_MIN_M", 17);
     return M > kMaxDecodeM || M >= min_m;
 }
 
@@ -129,14 +131,15 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
 }
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
-bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, cudaStream_t stream)
+// x_rows: rows of int8 activations that exist behind e.Xq (>= e.M; the rows past e.M may hold anything).
+bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, int64_t x_rows, cudaStream_t stream)
 {
     WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
     OwnedList *lists = reinterpret_cast<OwnedList *>(ws + lists_offset);
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
                     (path == BITLINEAR_PATH_TCGEN05_TS) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
     if (tc) {
-        static const int ts_tokens = env_int("BITLINEAR_PREFILL_TS_TOKENS", 0); // 192 or 256 (a measurement aid)
+        static const int ts_tokens = env_int("BITLINEAR_PREFILL_TS_TOKENS", 0); // 64, 192 or 256 (a measurement aid)
         if (path == BITLINEAR_PATH_TCGEN05_TS || (path == BITLINEAR_PATH_AUTO && ts_tokens > 0)) {
             cudaError_t err = launch_prefill_ts(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out, e.out_i32,
                                                 ts_tokens > 0 ? ts_tokens : 256, hdr, stream);
@@ -149,8 +152,8 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
                           (path == BITLINEAR_PATH_AUTO && e.M >= pair_min_m && prefill_pair_capacity() > 0);
         cudaError_t err = pair ? launch_prefill_pair(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out,
                                                      e.out_i32, hdr, stream)
-                               : launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out, e.out_i32,
-                                                hdr, stream);
+                               : launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, x_rows, e.K, e.N, e.out,
+                                                e.out_i32, hdr, stream);
         return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
@@ -250,7 +253,7 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     const size_t zero_bytes = use_tcgen05_for(M) ? sizeof(WorkspaceHeader) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, (cudaStream_t)stream);
+    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M, (cudaStream_t)stream);
 }
 
 bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
@@ -285,7 +288,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     }
     rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
     if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], path, ws, L.lists, s);
+    return run_matmul(inl.e[0], path, ws, L.lists, M, s); // (the caller's rows: exactly M of them)
 }
 
 bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)

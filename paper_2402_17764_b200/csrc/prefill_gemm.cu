@@ -348,17 +348,18 @@ EncodeTiledFn encode_tiled_fn()
 } // namespace
 
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
-                           const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
-                           WorkspaceHeader *hdr, cudaStream_t stream)
+                           const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
+                           int out_i32, WorkspaceHeader *hdr, cudaStream_t stream)
 {
+    if (x_rows < M) return cudaErrorInvalidValue;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
     const int KB = (int)((K + BK - 1) / BK);
 
     CUtensorMap tmap_x, tmap_w;
     {
-        // int8 activations [M rows][K bytes]; box 128 bytes x 128 rows; rows/columns past the end read 0
-        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
+        // int8 activations [x_rows rows][K bytes]; box 128 bytes x 128 rows; rows/columns past the end read 0
+        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)x_rows};
         const cuuint64_t strides[1] = {(cuuint64_t)K};
         const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
         const cuuint32_t estr[2] = {1, 1};

@@ -41,7 +41,7 @@ constexpr int BW = 128;         // output features per tile (MMA M, TMEM lanes)
 constexpr int BK = 128;         // int8 elements (= bytes) of K per stage
 constexpr int kACols = BK / 4;  // TMEM columns of one weight k block
 constexpr int kTmemCols = 512;
-constexpr int kMaxStages = 6;
+constexpr int kMaxStages = 12;
 
 constexpr int kProducerWarp = 0;
 constexpr int kMmaWarp = 1;
@@ -56,10 +56,12 @@ template <int NTOK>
 struct Cfg {
     static constexpr int kAccBufs = (2 * NTOK + 4 * kACols <= kTmemCols) ? 2 : 1;
     static constexpr int kRingCols = kTmemCols - kAccBufs * NTOK;
-    static constexpr int kStages = (kRingCols / kACols < kMaxStages) ? kRingCols / kACols : kMaxStages;
+    static constexpr int kSmemStages = (227 * 1024 - 2048) / (NTOK * BK + (int)kPBytes);
+    static constexpr int kTmemStages = (kRingCols / kACols < kMaxStages) ? kRingCols / kACols : kMaxStages;
+    static constexpr int kStages = kTmemStages < kSmemStages ? kTmemStages : kSmemStages;
     static constexpr uint32_t kXBytes = NTOK * BK; // int8 activations
     static constexpr uint32_t kStageBytes = kXBytes + kPBytes;
-    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 512 /*barriers*/;
     static_assert(NTOK % 16 == 0 && NTOK >= 16 && NTOK <= 256, "MMA N");
     static_assert(kXBytes % 1024 == 0, "swizzled tiles need 1024-byte alignment");
     static_assert(kStages >= 2, "ring too short");
@@ -75,7 +77,7 @@ struct Barriers {
     uint32_t tmem_base;
     int abort_flag;
 };
-static_assert(sizeof(Barriers) <= 256, "barrier block");
+static_assert(sizeof(Barriers) <= 512, "barrier block");
 
 struct Params {
     const float *gamma;
@@ -421,6 +423,8 @@ cudaError_t launch_prefill_ts(const void *packed, const float *gamma, const int8
                               const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
                               int tokens_per_tile, WorkspaceHeader *hdr, cudaStream_t stream)
 {
+    if (tokens_per_tile == 64)
+        return launch_ts<64>(packed, gamma, Xq, beta, rowsum, M, K, N, out, out_i32, hdr, stream);
     if (tokens_per_tile == 192)
         return launch_ts<192>(packed, gamma, Xq, beta, rowsum, M, K, N, out, out_i32, hdr, stream);
     return launch_ts<256>(packed, gamma, Xq, beta, rowsum, M, K, N, out, out_i32, hdr, stream);
