@@ -151,7 +151,9 @@ bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma
 /*
  * A list of independent BitLinear forwards executed by one persistent launch (the seven projections of
  * every decoder layer of a decode step, Section 2 "LLaMA-alike Components").  All inputs X must be
- * ready when the call is enqueued: entries do not depend on each other.  Every entry needs M <= 64.
+ * ready when the call is enqueued: entries do not depend on each other.  The entries may have different M;
+ * the largest decides the kernel for all of them: up to 16 tokens the weight-streaming kernel, from 17 on the
+ * tensor-core GEMM walking the CTA tiles of all matmuls in one launch.
  */
 typedef struct {
     const void *packed; /* device */

@@ -339,7 +339,10 @@ bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma
 }
 
 // ---- sequences -------------------------------------------------------------------------------
-// Workspace: [header | all acc32 | descriptor table | per-warp lists | per-entry Xq, beta, rowsum]
+// Workspace: [header | all acc32 | descriptor table | per-warp lists | GEMM table | per-entry Xq, beta, rowsum]
+// A sequence whose largest matmul has 17 tokens or more runs all its matmuls in one launch of the tensor-core
+// GEMM (no int32 scratch, row-major activations with at least kMinGemmRows rows each); otherwise in one launch
+// of the weight-streaming kernel.
 
 struct bitlinear_sequence {
     char *workspace;
@@ -349,27 +352,43 @@ struct bitlinear_sequence {
     size_t zero_bytes;
     const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
     bitlinear::InlineTable inl;
+    const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
+    int gemm_tiles, token_tiles;
 };
 
 namespace {
 struct SeqLayout {
-    size_t acc32, table, lists, data, total;
+    size_t acc32, table, lists, gemm, data, total;
+    bool use_gemm;
 };
+
+inline size_t seq_xq_bytes(int64_t M, int64_t K, bool gemm)
+{
+    const int64_t rows = (gemm && M < kMinGemmRows) ? kMinGemmRows : M;
+    return align_up((size_t)rows * col_tiles(K) * kTileCols, 256);
+}
 
 bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::vector<size_t> *entry_off)
 {
     if (!layers || n <= 0 || n > 65536) return false;
     size_t acc = 0, data = 0;
-    uint64_t tiles = 0;
+    uint64_t tiles = 0, gemm_tiles = 0;
+    int64_t max_M = 0;
+    for (int i = 0; i < n; ++i)
+        if (layers[i].M > max_M) max_M = layers[i].M;
+    const bool gemm = use_tcgen05_for(max_M);
+    S.use_gemm = gemm;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
-        if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1 || d.M > kMaxDecodeM) return false;
-        acc += align_up((size_t)d.M * d.N * 4, 256);
+        if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1) return false;
+        if (!gemm) acc += align_up((size_t)d.M * d.N * 4, 256);
         tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K)); // an upper bound of the work items in either mode
+        gemm_tiles += (uint64_t)((d.M + 127) / 128) * (uint64_t)((d.N + 255) / 256); // the same for the GEMM's CTA tiles
         if (entry_off) entry_off->push_back(data);
-        data += align_up((size_t)d.M * col_tiles(d.K) * kTileCols, 256) + 2 * align_up((size_t)d.M * 4, 256);
+        data += seq_xq_bytes(d.M, d.K, gemm) + 2 * align_up((size_t)d.M * 4, 256);
     }
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
+    if (gemm && gemm_tiles > 0x7FFFFFFFull) return false;
     size_t off = sizeof(WorkspaceHeader);
     S.acc32 = off;
     off += acc;
@@ -377,6 +396,8 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
     off += align_up((size_t)n * sizeof(DecodeEntry), 256);
     S.lists = off;
     off += align_up(kOwnedListsBytes, 256);
+    S.gemm = off;
+    if (gemm) off += align_up((size_t)n * kGemmProblemBytes, 256);
     S.data = off;
     off += data;
     S.total = off;
@@ -417,20 +438,33 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     for (int i = 0; i < n; ++i)
         if ((int)layers[i].M > max_M) max_M = (int)layers[i].M;
     const bool wide = decode_is_wide(max_M); // one kernel serves the whole sequence
+    const bool gemm = S.use_gemm;
+    const int token_tiles = prefill_token_tiles(max_M);
+    std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
+    int gemm_tiles = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         Layout L{};
         L.acc32 = a_off;
         L.xq = S.data + entry_off[(size_t)i];
-        L.beta = L.xq + align_up((size_t)d.M * col_tiles(d.K) * kTileCols, 256);
+        L.beta = L.xq + seq_xq_bytes(d.M, d.K, gemm);
         L.rowsum = L.beta + align_up((size_t)d.M * 4, 256);
-        a_off += align_up((size_t)d.M * d.N * 4, 256);
-        fill_entry(table[(size_t)i], d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
-        table[(size_t)i].xq_tiled = 1;
-        table[(size_t)i].tile_begin = tiles;
-        table[(size_t)i].token_begin = tokens;
-        tiles += decode_items(table[(size_t)i].NB, table[(size_t)i].KB, wide);
+        if (!gemm) a_off += align_up((size_t)d.M * d.N * 4, 256);
+        DecodeEntry &e = table[(size_t)i];
+        fill_entry(e, d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
+        e.xq_tiled = gemm ? 0 : 1;
+        e.tile_begin = tiles;
+        e.token_begin = tokens;
+        tiles += decode_items(e.NB, e.KB, wide);
         tokens += (int)d.M;
+        if (gemm) {
+            int nt = 0;
+            if (prefill_table_entry(gemm_table.data() + (size_t)i * kGemmProblemBytes, e.packed, e.gamma, e.Xq, e.beta,
+                                    e.rowsum, d.M, d.M < kMinGemmRows ? kMinGemmRows : d.M, d.K, d.N, d.Y, token_tiles,
+                                    gemm_tiles, reinterpret_cast<WorkspaceHeader *>(ws), &nt) != cudaSuccess)
+                return BITLINEAR_ERR_CUDA;
+            gemm_tiles += nt;
+        }
     }
     bitlinear_sequence *seq = new (std::nothrow) bitlinear_sequence();
     if (!seq) return BITLINEAR_ERR_ARG;
@@ -440,8 +474,18 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     seq->tiles = tiles;
     seq->tokens = tokens;
     seq->max_M = max_M;
-    seq->zero_bytes = S.table; // header and int32 scratch
+    seq->zero_bytes = gemm ? sizeof(WorkspaceHeader) : S.table; // header and int32 scratch
     seq->dev_table = nullptr;
+    seq->gemm_table = nullptr;
+    seq->gemm_tiles = gemm_tiles;
+    seq->token_tiles = token_tiles;
+    if (gemm) {
+        if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
+            delete seq;
+            return BITLINEAR_ERR_CUDA;
+        }
+        seq->gemm_table = ws + S.gemm;
+    }
     if (n <= kInlineEntries) {
         for (int i = 0; i < n; ++i) seq->inl.e[i] = table[(size_t)i];
     } else {
@@ -464,10 +508,13 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
         launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes, s) !=
             cudaSuccess)
         return BITLINEAR_ERR_CUDA;
-    if (stage != 1 &&
-        launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
-                      reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s) != cudaSuccess)
-        return BITLINEAR_ERR_CUDA;
+    if (stage != 1) {
+        const cudaError_t err =
+            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->token_tiles, s)
+                            : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
+                                            reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s);
+        if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    }
     return BITLINEAR_OK;
 }
 

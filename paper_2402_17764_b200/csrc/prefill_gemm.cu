@@ -27,6 +27,8 @@
 // Roofline: int8 tensor throughput; algorithmic work 2*M*N*K integer operations.
 #include <cuda.h>
 
+#include <cstring>
+
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -81,13 +83,37 @@ struct Params {
     int tiles_m, tiles_n; // CTA tiles: MT * 128 tokens x 256 features
     int out_i32;
     int out_32b_aligned; // rows of the bf16 output start on 32-byte boundaries
+    int tile_begin;      // first CTA tile of this matmul in the launch-wide tile sequence
     int32_t *status;
 };
 
-template <int MT>
+// One matmul of a launch: its two tensor maps and its parameters.  A single matmul travels as a kernel
+// parameter; the matmuls of a sequence stand in a table in device memory (written once, by the host).
+struct alignas(64) GemmProblem {
+    CUtensorMap tmap_x, tmap_w;
+    Params p;
+};
+static_assert(sizeof(GemmProblem) == kGemmProblemBytes, "internal.cuh states the size of a table entry");
+
+// The matmul a tile belongs to.  A CTA's tiles only go up, so the search resumes where it stopped.
+template <bool kTable>
+struct ProblemCursor {
+    const GemmProblem *table;
+    int n, i;
+    __device__ ProblemCursor(const GemmProblem &one, const GemmProblem *t, int n_) : table(kTable ? t : &one), n(n_), i(0) {}
+    __device__ const GemmProblem &seek(int tile)
+    {
+        if (kTable) {
+            while (i + 1 < n && tile >= table[i + 1].p.tile_begin) ++i;
+        }
+        return table[i];
+    }
+};
+
+template <int MT, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
-prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                    const Params p)
+prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems,
+                    int n_tiles)
 {
     constexpr int kStages = Cfg<MT>::kStages, kAccBufs = Cfg<MT>::kAccBufs;
     constexpr uint32_t kStageBytes = Cfg<MT>::kStageBytes;
@@ -124,19 +150,24 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     tc_fence_after_sync();
     const uint32_t tmem_base = bars->tmem_base;
 
-    const int n_tiles = p.tiles_m * p.tiles_n;
-    const int KB = p.KB;
+    int32_t *const status = kTable ? table[0].p.status : one.p.status; // (the same for every matmul of a launch)
 
     if (warp == kProducerWarp) {
         if (lane == 0) {
-            prefetch_tensormap(&tmap_x);
-            prefetch_tensormap(&tmap_w);
+            ProblemCursor<kTable> cur(one, table, n_problems);
+            if (!kTable) {
+                prefetch_tensormap(&one.tmap_x);
+                prefetch_tensormap(&one.tmap_w);
+            }
             griddep_wait(); // the activations are written by the launch before this one
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % p.tiles_m) * (MT * BM);
-                const int n0 = (tile / p.tiles_m) * BN;
+                const GemmProblem &g = cur.seek(tile);
+                const Params &p = g.p;
+                const int local = tile - p.tile_begin, KB = p.KB;
+                const int m0 = (local % p.tiles_m) * (MT * BM);
+                const int n0 = (local / p.tiles_m) * BN;
                 const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // a second token tile past the end is left out
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     const int s = it % kStages;
@@ -149,23 +180,26 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const uint32_t a_dst = base + s * kStageBytes;
                     const uint32_t p_dst = a_dst + MT * kABytes + kBBytes;
                     mbar_arrive_expect_tx(full, halves * kABytes + kPBytes);
-                    tma_load_2d(a_dst, &tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
-                    if (halves == 2) tma_load_2d(a_dst + kABytes, &tmap_x, kb * BK, m0 + BM, full);
-                    tma_load_3d(p_dst, &tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
+                    tma_load_2d(a_dst, &g.tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
+                    if (halves == 2) tma_load_2d(a_dst + kABytes, &g.tmap_x, kb * BK, m0 + BM, full);
+                    tma_load_3d(p_dst, &g.tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
                 }
             }
         }
     } else if (warp == kMmaWarp) {
         constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
+        ProblemCursor<kTable> cur(one, table, n_problems);
         uint32_t it = 0, tile_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+            const Params &p = cur.seek(tile).p;
+            const int KB = p.KB;
             const int buf = tile_it % kAccBufs;
             const uint32_t use = tile_it / kAccBufs;
             if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag)) break;
             tc_fence_after_sync();
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
-            const bool two = MT == 2 && (tile % p.tiles_m) * (MT * BM) + BM < p.M;
+            const bool two = MT == 2 && ((tile - p.tile_begin) % p.tiles_m) * (MT * BM) + BM < p.M;
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int s = it % kStages;
                 const uint32_t parity = (it / kStages) & 1;
@@ -205,9 +239,11 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         const int g = (lane & 4) ? ((q ^ 1) + 4) : q, tq = lane & 3;
         const int slot = 4 * g + tq;
         const int rbi = ew >> 1, kti = ew & 1;
+        ProblemCursor<kTable> cur(one, table, n_problems);
         uint32_t it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            const int KB = cur.seek(tile).p.KB;
             for (int kb = 0; kb < KB; ++kb, ++it) {
                 const int s = it % kStages;
                 const uint32_t parity = (it / kStages) & 1;
@@ -240,11 +276,14 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
     } else {
         // epilogue: warp w may touch TMEM lanes 32*(w % 4) .. +31
         const int q = warp & 3;
+        ProblemCursor<kTable> cur(one, table, n_problems);
         uint32_t tile_it = 0;
-        const float gamma = p.out_i32 ? 0.0f : *p.gamma;
         for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_it) {
-            const int m0 = (tile % p.tiles_m) * (MT * BM);
-            const int n0 = (tile / p.tiles_m) * BN;
+            const Params &p = cur.seek(tile).p;
+            const float gamma = p.out_i32 ? 0.0f : *p.gamma;
+            const int local = tile - p.tile_begin;
+            const int m0 = (local % p.tiles_m) * (MT * BM);
+            const int n0 = (local / p.tiles_m) * BN;
             const int buf = tile_it % kAccBufs;
             const uint32_t parity = (tile_it / kAccBufs) & 1;
             if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), parity, abort_flag)) break;
@@ -311,7 +350,7 @@ prefill_gemm_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
     // common tail: every thread arrives here, also after an expired wait
     if (*abort_flag) {
-        if (threadIdx.x == 0) atomicExch(p.status, (int32_t)BITLINEAR_ERR_TIMEOUT);
+        if (threadIdx.x == 0) atomicExch(status, (int32_t)BITLINEAR_ERR_TIMEOUT);
         // give copies and MMAs that may still be in flight time to land before shared memory and TMEM go away
         const uint64_t t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
@@ -345,25 +384,21 @@ EncodeTiledFn encode_tiled_fn()
     return fn;
 }
 
-} // namespace
-
-cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
-                           const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, WorkspaceHeader *hdr, cudaStream_t stream)
+// Tensor maps and parameters of one matmul, for `mt` token tiles per CTA tile.
+static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
+                                const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
+                                int out_i32, int mt, int tile_begin, int32_t *status)
 {
-    if (x_rows < M) return cudaErrorInvalidValue;
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
-    const int KB = (int)((K + BK - 1) / BK);
-
-    CUtensorMap tmap_x, tmap_w;
+    if (x_rows < M) return cudaErrorInvalidValue;
     {
         // int8 activations [x_rows rows][K bytes]; box 128 bytes x 128 rows; rows/columns past the end read 0
         const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)x_rows};
         const cuuint64_t strides[1] = {(cuuint64_t)K};
         const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
         const cuuint32_t estr[2] = {1, 1};
-        if (encode(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides, box, estr,
+        if (encode(&g.tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
@@ -378,42 +413,55 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
         const cuuint64_t strides[2] = {(cuuint64_t)kTileBytes, tiles_k * kTileBytes};
         const cuuint32_t box[3] = {kTileBytes / 4, (cuuint32_t)(BK / kTileCols), (cuuint32_t)(BN / kTileRows)};
         const cuuint32_t estr[3] = {1, 1, 1};
-        if (encode(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(packed), dims, strides, box, estr,
+        if (encode(&g.tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(packed), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return cudaErrorInvalidValue;
     }
-
-    Params p;
+    Params &p = g.p;
     p.gamma = gamma;
     p.beta = beta;
     p.rowsum = rowsum;
     p.out = out;
     p.M = (int)M;
     p.N = (int)N;
-    p.KB = KB;
-    const int mt = (M > BM) ? 2 : 1; // token tiles per CTA tile
+    p.KB = (int)((K + BK - 1) / BK);
     p.tiles_m = (int)((M + mt * BM - 1) / (mt * BM));
     p.tiles_n = (int)((N + BN - 1) / BN);
     p.out_i32 = out_i32;
     p.out_32b_aligned = (reinterpret_cast<uintptr_t>(out) % 32 == 0) ? 1 : 0; // (N is a multiple of 16)
-    p.status = &hdr->status;
-    const void *kernel = (mt == 2) ? (const void *)prefill_gemm_kernel<2> : (const void *)prefill_gemm_kernel<1>;
-    const uint32_t smem_bytes = (mt == 2) ? Cfg<2>::kSmemBytes : Cfg<1>::kSmemBytes;
+    p.tile_begin = tile_begin;
+    p.status = status;
+    return cudaSuccess;
+}
 
+// Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
+static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int mt,
+                               cudaStream_t stream)
+{
+    const void *kernel = table ? (mt == 2 ? (const void *)prefill_gemm_kernel<2, true> : (const void *)prefill_gemm_kernel<1, true>)
+                               : (mt == 2 ? (const void *)prefill_gemm_kernel<2, false> : (const void *)prefill_gemm_kernel<1, false>);
+    const uint32_t smem_bytes = (mt == 2) ? Cfg<2>::kSmemBytes : Cfg<1>::kSmemBytes;
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)Cfg<1>::kSmemBytes);
         if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(prefill_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+            e = cudaFuncSetAttribute(prefill_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)Cfg<1>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                     (int)Cfg<2>::kSmemBytes);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(prefill_gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                      (int)Cfg<2>::kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    int grid = p.tiles_m * p.tiles_n;
+    if (n_tiles <= 0) return cudaSuccess;
+    int grid = n_tiles;
     if (grid > sm_count()) grid = sm_count();
     // programmatic dependent launch: see the head of this file
     cudaLaunchAttribute attr;
@@ -426,8 +474,42 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
     cfg.stream = stream;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    void *args[] = {(void *)&tmap_x, (void *)&tmap_w, (void *)&p};
+    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles};
     return cudaLaunchKernelExC(&cfg, kernel, args);
+}
+
+} // namespace
+
+int prefill_token_tiles(int64_t max_M) { return max_M > BM ? 2 : 1; }
+
+cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
+                           const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
+                           int out_i32, WorkspaceHeader *hdr, cudaStream_t stream)
+{
+    const int mt = prefill_token_tiles(M);
+    GemmProblem g;
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, mt, 0, &hdr->status);
+    if (e != cudaSuccess) return e;
+    return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, stream);
+}
+
+cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
+                                const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
+                                int token_tiles, int tile_begin, WorkspaceHeader *hdr, int *n_tiles)
+{
+    GemmProblem g;
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, 0, token_tiles, tile_begin,
+                                 &hdr->status);
+    if (e != cudaSuccess) return e;
+    memcpy(slot, &g, sizeof(g));
+    *n_tiles = g.p.tiles_m * g.p.tiles_n;
+    return cudaSuccess;
+}
+
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int token_tiles, cudaStream_t stream)
+{
+    GemmProblem unused{};
+    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, token_tiles, stream);
 }
 
 } // namespace bitlinear

@@ -340,10 +340,18 @@ def test_forward_sequence_matches_single_calls(oracle):
         seq.close()
 
 
-def test_forward_sequence_with_mixed_token_counts(oracle):
-    """Entries of one sequence may have different M; one entry above 8 tokens puts the whole sequence on the
-    kernel in which the warps of a CTA share the activations.  Ragged shapes: N and K not multiples of 64."""
-    specs = [(3, 144, 48), (20, 1536, 1040), (1, 3200, 512), (64, 80, 528), (9, 8640, 16)]
+@pytest.mark.parametrize("specs", [
+    # largest M in 9..16: the weight-streaming kernel in which the warps of a CTA share the activations
+    [(3, 144, 48), (16, 1536, 1040), (1, 3200, 512), (12, 80, 528), (9, 8640, 16)],
+    # largest M in 17..128: every matmul in one launch of the tensor-core GEMM, one token tile per CTA tile
+    [(3, 144, 48), (20, 1536, 1040), (1, 3200, 512), (64, 80, 528), (9, 8640, 16)],
+    # largest M above 128: the same with two token tiles per CTA tile; more entries than travel as kernel parameters
+    [(3, 144, 48), (300, 1536, 1040), (1, 3200, 512), (129, 80, 528), (9, 8640, 16), (256, 272, 272), (40, 144, 4112),
+     (7, 16, 16), (130, 1024, 320), (2, 4096, 256)],
+], ids=["max16", "max64", "max300"])
+def test_forward_sequence_with_mixed_token_counts(oracle, specs):
+    """Entries of one sequence may have different M; the largest one decides which kernel runs the whole sequence.
+    Ragged shapes: N and K not multiples of 64."""
     layers, refs = [], []
     for i, (M, K, N) in enumerate(specs):
         W = S.latent_weights(N, K, 40 + i)
