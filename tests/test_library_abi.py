@@ -69,7 +69,10 @@ def test_argument_errors_are_reported_before_any_device_work(lib):
     assert L.bitlinear_forward_sequence(null, null) == B.ERR_ARG
     L.bitlinear_sequence_destroy(null)  # allowed
     descs = (B.LayerDesc * 1)(B.LayerDesc(fake, fake, fake, fake, 65, 16, 16))
-    assert L.bitlinear_sequence_workspace_bytes(descs, 1) == 0  # M > 64 is not a decode entry
+    assert L.bitlinear_sequence_workspace_bytes(descs, 1) > 0  # any M from 1 to 2^20 is a sequence entry
+    for bad_m in (0, (1 << 20) + 1):
+        descs = (B.LayerDesc * 1)(B.LayerDesc(fake, fake, fake, fake, bad_m, 16, 16))
+        assert L.bitlinear_sequence_workspace_bytes(descs, 1) == 0
 
 
 def test_no_cpu_fallback():
