@@ -353,7 +353,7 @@ struct bitlinear_sequence {
     const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
     bitlinear::InlineTable inl;
     const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
-    int gemm_tiles, token_tiles;
+    int gemm_tiles;
 };
 
 namespace {
@@ -439,7 +439,6 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
         if ((int)layers[i].M > max_M) max_M = (int)layers[i].M;
     const bool wide = decode_is_wide(max_M); // one kernel serves the whole sequence
     const bool gemm = S.use_gemm;
-    const int token_tiles = prefill_token_tiles(max_M);
     std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
     int gemm_tiles = 0;
     for (int i = 0; i < n; ++i) {
@@ -460,7 +459,7 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
         if (gemm) {
             int nt = 0;
             if (prefill_table_entry(gemm_table.data() + (size_t)i * kGemmProblemBytes, e.packed, e.gamma, e.Xq, e.beta,
-                                    e.rowsum, d.M, d.M < kMinGemmRows ? kMinGemmRows : d.M, d.K, d.N, d.Y, token_tiles,
+                                    e.rowsum, d.M, d.M < kMinGemmRows ? kMinGemmRows : d.M, d.K, d.N, d.Y, max_M,
                                     gemm_tiles, reinterpret_cast<WorkspaceHeader *>(ws), &nt) != cudaSuccess)
                 return BITLINEAR_ERR_CUDA;
             gemm_tiles += nt;
@@ -478,7 +477,6 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     seq->dev_table = nullptr;
     seq->gemm_table = nullptr;
     seq->gemm_tiles = gemm_tiles;
-    seq->token_tiles = token_tiles;
     if (gemm) {
         if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
             delete seq;
@@ -510,7 +508,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {
         const cudaError_t err =
-            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->token_tiles, s)
+            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->max_M, s)
                             : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
                                             reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s);
         if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;

@@ -98,13 +98,14 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
 
 // The same kernel over the matmuls of a sequence in ONE launch.  The host fills a table of kGemmProblemBytes-sized
 // entries (tensor maps + parameters) with prefill_table_entry, copies it to device memory (64-byte aligned) once, and
-// launches over all the CTA tiles; token_tiles = prefill_token_tiles(largest M of the sequence) for every entry.
+// launches over all the CTA tiles; max_M = the largest M of the sequence, the same for every entry and the launch
+// (it fixes the tile shape: prefill_token_tiles(max_M) token tiles of 128 tokens per CTA tile).
 constexpr size_t kGemmProblemBytes = 384;
 int prefill_token_tiles(int64_t max_M);
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int token_tiles, int tile_begin, WorkspaceHeader *hdr, int *n_tiles);
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int token_tiles, cudaStream_t stream);
+                                int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles);
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, cudaStream_t stream);
 
 // The same GEMM on pairs of SMs (tcgen05 cta_group::2): 256 tokens x 256 features per pair tile.
 // prefill_pair_capacity: CTA pairs that can be resident at once (0: not available on this device).

@@ -41,7 +41,8 @@ using namespace ptx;
 constexpr int BM = 128;      // tokens per MMA (MMA M, TMEM lanes); a CTA tile has MT of them
 constexpr int BN = 256;      // features per tile (MMA N, TMEM columns per accumulator)
 constexpr int BK = 128;      // int8 elements (= bytes) of K per stage
-constexpr int kMaxStages = 4;
+constexpr int kMaxStages = 12; // ring of TMA stages (activations + packed weights); its depth is chosen at launch
+constexpr int kMaxBSlots = 3;  // ring of expanded weight tiles (its depth: Cfg)
 constexpr int kTmemCols = 512;
 
 constexpr int kProducerWarp = 0;
@@ -55,23 +56,64 @@ constexpr uint32_t kABytes = BM * BK;            // 16 KiB int8 activations per 
 constexpr uint32_t kBBytes = BN * BK;            // 32 KiB expanded weights
 constexpr uint32_t kPBytes = (BN / kTileRows) * (BK / kTileCols) * kTileBytes; //  8 KiB packed weights
 
+// Expanding one k block takes a warp about 700 cycles from the stage's arrival to the hand-over (two waits, 32 KiB
+// of stores that all eight warps push through shared memory at once, a proxy fence of about 300 cycles), whatever
+// the number of warps that share it.  With two token tiles the MMAs of a k block take longer than that.  With one
+// they take 512 cycles, so there the expander warps form two groups that take k blocks in turn (each warp two
+// packed tiles of every other k block), with a third expanded tile so that both groups can be ahead of the MMAs.
 template <int MT>
 struct Cfg {
-    static constexpr int kStages = (MT == 1) ? 4 : 3;
     static constexpr int kAccBufs = (MT == 1) ? 2 : 1; // MT * BN * kAccBufs = all 512 TMEM columns
-    static constexpr uint32_t kStageBytes = MT * kABytes + kBBytes + kPBytes;
-    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
-    static_assert(kSmemBytes <= 232448, "exceeds the 227 KiB shared memory of an SM");
+    static constexpr int kGroups = (MT == 1) ? 2 : 1;  // expander groups
+    static constexpr int kBSlots = (MT == 1) ? 3 : 2;  // expanded weight tiles
 };
 
+// Shared memory: [expanded weight tiles: 2 or 3 x 32 KiB][TMA stages: n x (activations | 8 KiB packed)][barriers].
+// What waits on memory (the TMA stages) and what the expander hands to the tensor core (the expanded tiles)
+// have rings of their own: the expanded tile is four times the packed one, and with one ring the 227 KiB held
+// three or four k blocks in flight, too few to cover the latency of HBM when the weights are streamed once
+// (few tokens).  A stage's activation part is a_rows rows of 128 bytes per token tile: 128, or 64 when no matmul
+// of the launch has more than 64 tokens (the MMA then also reads 64 rows of whatever follows in shared memory,
+// into accumulator rows that are never stored).
+constexpr uint32_t kSmemLimit = 232448; // 227 KiB
+constexpr uint32_t kBarrierBytes = 512;
+__host__ __device__ constexpr uint32_t stage_bytes(int mt, int a_rows) { return (uint32_t)(mt * a_rows * BK) + kPBytes; }
+inline int b_slots(int mt) { return mt == 1 ? Cfg<1>::kBSlots : Cfg<2>::kBSlots; }
+inline int stages_that_fit(int mt, int a_rows)
+{
+    const int n = (int)((kSmemLimit - 1024 /*alignment slack*/ - kBarrierBytes - b_slots(mt) * kBBytes) / stage_bytes(mt, a_rows));
+    return n < kMaxStages ? n : kMaxStages;
+}
+inline uint32_t smem_bytes_for(int mt, int a_rows, int n_stages)
+{
+    return 1024 + b_slots(mt) * kBBytes + (uint32_t)n_stages * stage_bytes(mt, a_rows) + kBarrierBytes;
+}
+
 struct Barriers {
-    uint64_t full[kMaxStages];      // TMA bytes landed (activations + packed weights)
-    uint64_t expanded[kMaxStages];  // int8 weight tile written
-    uint64_t empty[kMaxStages];     // MMAs that read the stage have completed
-    uint64_t acc_full[2];           // accumulator(s) of a tile complete
-    uint64_t acc_empty[2];          // drained by the epilogue
+    uint64_t full[kMaxStages];   // TMA bytes landed (activations + packed weights)
+    uint64_t empty[kMaxStages];  // MMAs that read the stage have completed
+    uint64_t expanded[kMaxBSlots]; // int8 weight tile written
+    uint64_t acc_full[2];        // accumulator(s) of a tile complete
+    uint64_t acc_empty[2];       // drained by the epilogue
     uint32_t tmem_base;
     int abort_flag;
+};
+static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block");
+
+// Position in the ring of TMA stages and in the ring of expanded tiles after `it` k blocks.
+struct RingPos {
+    int s;          // TMA stage
+    uint32_t round; // times the TMA ring has been gone through
+    uint32_t it;    // k blocks so far: expanded-tile slot it % slots, use it / slots
+    __device__ RingPos() : s(0), round(0), it(0) {}
+    __device__ void advance(int n_stages)
+    {
+        ++it;
+        if (++s == n_stages) {
+            s = 0;
+            ++round;
+        }
+    }
 };
 
 struct Params {
@@ -113,26 +155,28 @@ struct ProblemCursor {
 template <int MT, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems,
-                    int n_tiles)
+                    int n_tiles, int a_rows, int n_stages)
 {
-    constexpr int kStages = Cfg<MT>::kStages, kAccBufs = Cfg<MT>::kAccBufs;
-    constexpr uint32_t kStageBytes = Cfg<MT>::kStageBytes;
+    constexpr int kAccBufs = Cfg<MT>::kAccBufs, kBSlots = Cfg<MT>::kBSlots, kGroups = Cfg<MT>::kGroups;
+    const uint32_t kStageBytes = stage_bytes(MT, a_rows), kAHalfBytes = (uint32_t)(a_rows * BK);
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t base = (raw + 1023u) & ~1023u; // swizzled tiles need 1024-byte alignment
     uint8_t *smem = smem_raw + (base - raw);
-    // layout: [stage][A | B | P], then the barrier block
-    Barriers *bars = reinterpret_cast<Barriers *>(smem + kStages * kStageBytes);
+    const uint32_t stages = base + kBSlots * kBBytes; // first TMA stage
+    Barriers *bars = reinterpret_cast<Barriers *>(smem + kBSlots * kBBytes + (uint32_t)n_stages * kStageBytes);
     volatile int *abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kStages; ++s) {
+        for (int s = 0; s < n_stages; ++s) {
             mbar_init(smem_u32(&bars->full[s]), 1);
-            mbar_init(smem_u32(&bars->expanded[s]), kExpanderWarps);
             mbar_init(smem_u32(&bars->empty[s]), 1);
+        }
+        for (int b = 0; b < kBSlots; ++b) {
+            mbar_init(smem_u32(&bars->expanded[b]), kExpanderWarps / kGroups);
         }
         for (int b = 0; b < kAccBufs; ++b) {
             mbar_init(smem_u32(&bars->acc_full[b]), 1);
@@ -160,7 +204,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 prefetch_tensormap(&one.tmap_w);
             }
             griddep_wait(); // the activations are written by the launch before this one
-            uint32_t it = 0;
+            RingPos pos;
             bool ok = true;
             for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
                 const GemmProblem &g = cur.seek(tile);
@@ -169,65 +213,67 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 const int m0 = (local % p.tiles_m) * (MT * BM);
                 const int n0 = (local / p.tiles_m) * BN;
                 const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // a second token tile past the end is left out
-                for (int kb = 0; kb < KB; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t round = it / kStages;
-                    if (round > 0 && !mbar_wait_bounded(smem_u32(&bars->empty[s]), (round - 1) & 1, abort_flag)) {
+                for (int kb = 0; kb < KB; ++kb, pos.advance(n_stages)) {
+                    const int s = pos.s;
+                    if (pos.round > 0 && !mbar_wait_bounded(smem_u32(&bars->empty[s]), (pos.round - 1) & 1, abort_flag)) {
                         ok = false;
                         break;
                     }
                     const uint32_t full = smem_u32(&bars->full[s]);
-                    const uint32_t a_dst = base + s * kStageBytes;
-                    const uint32_t p_dst = a_dst + MT * kABytes + kBBytes;
-                    mbar_arrive_expect_tx(full, halves * kABytes + kPBytes);
+                    const uint32_t a_dst = stages + s * kStageBytes;
+                    const uint32_t p_dst = a_dst + MT * kAHalfBytes;
+                    mbar_arrive_expect_tx(full, halves * kAHalfBytes + kPBytes);
                     tma_load_2d(a_dst, &g.tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
-                    if (halves == 2) tma_load_2d(a_dst + kABytes, &g.tmap_x, kb * BK, m0 + BM, full);
+                    if (halves == 2) tma_load_2d(a_dst + kAHalfBytes, &g.tmap_x, kb * BK, m0 + BM, full);
                     tma_load_3d(p_dst, &g.tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
                 }
             }
         }
     } else if (warp == kMmaWarp) {
-        constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
-        ProblemCursor<kTable> cur(one, table, n_problems);
-        uint32_t it = 0, tile_it = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
-            const Params &p = cur.seek(tile).p;
-            const int KB = p.KB;
-            const int buf = tile_it % kAccBufs;
-            const uint32_t use = tile_it / kAccBufs;
-            if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag)) break;
-            tc_fence_after_sync();
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
-            const bool two = MT == 2 && ((tile - p.tile_begin) % p.tiles_m) * (MT * BM) + BM < p.M;
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % kStages;
-                const uint32_t parity = (it / kStages) & 1;
-                if (!mbar_wait_bounded(smem_u32(&bars->full[s]), parity, abort_flag) ||
-                    !mbar_wait_bounded(smem_u32(&bars->expanded[s]), parity, abort_flag)) {
-                    ok = false;
-                    break;
-                }
+        // ONE thread runs this loop.  What it executes per k block (a wait, the MMAs, a commit: 60 to 90 cycles
+        // each on B200) is serial, and the tensor core idles whenever that takes longer than the MMAs themselves,
+        // so there is one wait and one commit per k block: `expanded` implies `full` (the expander warps waited for
+        // the stage before they arrived), and `empty` also tells the expander that the expanded tile was read.
+        if (lane == 0) {
+            constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
+            ProblemCursor<kTable> cur(one, table, n_problems);
+            RingPos pos;
+            uint32_t tile_it = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+                const Params &p = cur.seek(tile).p;
+                const int KB = p.KB;
+                const int buf = tile_it % kAccBufs;
+                const uint32_t use = tile_it / kAccBufs;
+                if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag)) break;
                 tc_fence_after_sync();
-                if (lane == 0) {
-                    const uint32_t a_addr = base + s * kStageBytes;
-                    const uint32_t b_addr = a_addr + MT * kABytes;
+                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
+                const bool two = MT == 2 && ((tile - p.tile_begin) % p.tiles_m) * (MT * BM) + BM < p.M;
+                for (int kb = 0; kb < KB; ++kb, pos.advance(n_stages)) {
+                    const int s = pos.s, b = (int)(pos.it % kBSlots);
+                    if (!mbar_wait_bounded(smem_u32(&bars->expanded[b]), (pos.it / kBSlots) & 1, abort_flag)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after_sync();
+                    const uint32_t a_addr = stages + s * kStageBytes;
+                    const uint32_t b_addr = base + b * kBBytes;
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 32; ++k4) {
                         const uint64_t b_desc = smem_desc_k_sw128(b_addr + 32 * k4);
                         const uint32_t accumulate = (kb > 0 || k4 > 0) ? 1u : 0u;
                         mma_i8_ss(d_tmem, smem_desc_k_sw128(a_addr + 32 * k4), b_desc, idesc, accumulate);
-                        if (two) mma_i8_ss(d_tmem + BN, smem_desc_k_sw128(a_addr + kABytes + 32 * k4), b_desc, idesc, accumulate);
+                        if (two) mma_i8_ss(d_tmem + BN, smem_desc_k_sw128(a_addr + kAHalfBytes + 32 * k4), b_desc, idesc, accumulate);
                     }
-                    mma_commit(smem_u32(&bars->empty[s])); // stage reusable once these MMAs have read it
+                    mma_commit(smem_u32(&bars->empty[s])); // stage and expanded tile are reusable once these MMAs have read them
                 }
-                __syncwarp();
+                if (ok) mma_commit(smem_u32(&bars->acc_full[buf]));
             }
-            if (ok && lane == 0) mma_commit(smem_u32(&bars->acc_full[buf]));
-            __syncwarp();
         }
     } else if (warp >= kFirstExpanderWarp) {
-        // Expander warp ew owns packed tile (row block ew / 2, column tile ew % 2) of the stage.  The 16 bytes
+        // An expander warp owns packed tile (row block rbi, column tile kti) of the stage: warp ew tile
+        // (ew / 2, ew % 2) of every k block, or, in two groups, warp ew tiles (ew % 4, 0) and (ew % 4, 1) of the k
+        // blocks with it % 2 == ew / 4.  The 16 bytes
         // at slot 4 g + tq of each slab hold the codes of rows 16 f + 8 h + g at columns
         // 16 tq + 8 s + 4 hi + b (slab s, word 2 hi + h, byte b, field f): 16 consecutive columns of a row
         // are words (h, 2 + h) of slab 0 followed by words (h, 2 + h) of slab 1.
@@ -238,39 +284,55 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         const int q = lane >> 3;
         const int g = (lane & 4) ? ((q ^ 1) + 4) : q, tq = lane & 3;
         const int slot = 4 * g + tq;
-        const int rbi = ew >> 1, kti = ew & 1;
+        const int group = (kGroups == 2) ? (ew >> 2) : 0;
+        const int rbi = (kGroups == 2) ? (ew & 3) : (ew >> 1);
         ProblemCursor<kTable> cur(one, table, n_problems);
-        uint32_t it = 0;
+        RingPos pos, reader; // reader: the k block kBSlots steps back, whose MMAs read the expanded tile written next
         bool ok = true;
         for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
             const int KB = cur.seek(tile).p.KB;
-            for (int kb = 0; kb < KB; ++kb, ++it) {
-                const int s = it % kStages;
-                const uint32_t parity = (it / kStages) & 1;
-                if (!mbar_wait_bounded(smem_u32(&bars->full[s]), parity, abort_flag)) {
+            for (int kb = 0; kb < KB; ++kb, pos.advance(n_stages)) {
+                const int s = pos.s, b = (int)(pos.it % kBSlots);
+                const bool mine = kGroups == 1 || (int)(pos.it & 1u) == group;
+                const bool has_reader = pos.it >= (uint32_t)kBSlots;
+                const int rs = reader.s;
+                const uint32_t rround = reader.round;
+                if (has_reader) reader.advance(n_stages);
+                if (!mine) continue;
+                if (!mbar_wait_bounded(smem_u32(&bars->full[s]), pos.round & 1, abort_flag)) {
                     ok = false;
                     break;
                 }
-                uint8_t *stage = smem + s * kStageBytes;
-                const uint4 *packed = reinterpret_cast<const uint4 *>(stage + MT * kABytes + kBBytes) + ew * (kTileBytes / 16);
-                uint8_t *bt = stage + MT * kABytes;
-                const uint4 w0 = packed[slot], w1 = packed[32 + slot];
-                const uint32_t lo[2][2] = {{w0.x, w0.z}, {w0.y, w0.w}}; // [h][hi], slab 0
-                const uint32_t up[2][2] = {{w1.x, w1.z}, {w1.y, w1.w}}; // slab 1
-                const int chunk = (kti * 4 + tq) ^ g; // 16-byte chunk of the 128-byte row, swizzled by row % 8 = g
+                // (the reader's stage is not refilled before this tile is expanded: its `empty` phase is the latest)
+                if (has_reader && !mbar_wait_bounded(smem_u32(&bars->empty[rs]), rround & 1, abort_flag)) {
+                    ok = false;
+                    break;
+                }
+                const uint8_t *stage = smem + kBSlots * kBBytes + s * kStageBytes;
+                uint8_t *bt = smem + b * kBBytes;
 #pragma unroll
-                for (int f = 0; f < 4; ++f) {
-                    const uint32_t mask = 0x03030303u << (2 * f);
+                for (int kk = 0; kk < kGroups; ++kk) { // the packed tiles of this warp
+                    const int kti = (kGroups == 2) ? kk : (ew & 1);
+                    const uint4 *packed =
+                        reinterpret_cast<const uint4 *>(stage + MT * kAHalfBytes) + (rbi * 2 + kti) * (kTileBytes / 16);
+                    const uint4 w0 = packed[slot], w1 = packed[32 + slot];
+                    const uint32_t lo[2][2] = {{w0.x, w0.z}, {w0.y, w0.w}}; // [h][hi], slab 0
+                    const uint32_t up[2][2] = {{w1.x, w1.z}, {w1.y, w1.w}}; // slab 1
+                    const int chunk = (kti * 4 + tq) ^ g; // 16-byte chunk of the 128-byte row, swizzled by row % 8 = g
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const int r = rbi * kTileRows + 16 * f + 8 * h + g;
-                        *reinterpret_cast<uint4 *>(bt + r * 128 + (chunk << 4)) =
-                            make_uint4(lo[h][0] & mask, lo[h][1] & mask, up[h][0] & mask, up[h][1] & mask);
+                    for (int f = 0; f < 4; ++f) {
+                        const uint32_t mask = 0x03030303u << (2 * f);
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const int r = rbi * kTileRows + 16 * f + 8 * h + g;
+                            *reinterpret_cast<uint4 *>(bt + r * 128 + (chunk << 4)) =
+                                make_uint4(lo[h][0] & mask, lo[h][1] & mask, up[h][0] & mask, up[h][1] & mask);
+                        }
                     }
                 }
                 fence_proxy_async_smem(); // generic-proxy writes -> visible to the tensor core
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars->expanded[s]));
+                if (lane == 0) mbar_arrive(smem_u32(&bars->expanded[b]));
             }
         }
     } else {
@@ -387,7 +449,7 @@ EncodeTiledFn encode_tiled_fn()
 // Tensor maps and parameters of one matmul, for `mt` token tiles per CTA tile.
 static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int out_i32, int mt, int tile_begin, int32_t *status)
+                                int out_i32, int mt, int a_rows, int tile_begin, int32_t *status)
 {
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return cudaErrorNotSupported;
@@ -396,7 +458,7 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
         // int8 activations [x_rows rows][K bytes]; box 128 bytes x 128 rows; rows/columns past the end read 0
         const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)x_rows};
         const cuuint64_t strides[1] = {(cuuint64_t)K};
-        const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
+        const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)a_rows};
         const cuuint32_t estr[2] = {1, 1};
         if (encode(&g.tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides, box, estr,
                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -436,28 +498,23 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
 }
 
 // Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
-static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int mt,
+static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int mt, int a_rows,
                                cudaStream_t stream)
 {
     const void *kernel = table ? (mt == 2 ? (const void *)prefill_gemm_kernel<2, true> : (const void *)prefill_gemm_kernel<1, true>)
                                : (mt == 2 ? (const void *)prefill_gemm_kernel<2, false> : (const void *)prefill_gemm_kernel<1, false>);
-    const uint32_t smem_bytes = (mt == 2) ? Cfg<2>::kSmemBytes : Cfg<1>::kSmemBytes;
+    int n_stages = stages_that_fit(mt, a_rows);
+    const uint32_t smem_bytes = smem_bytes_for(mt, a_rows, n_stages);
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_gemm_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)Cfg<1>::kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(prefill_gemm_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)Cfg<1>::kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(prefill_gemm_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)Cfg<2>::kSmemBytes);
-        if (e == cudaSuccess)
-            e = cudaFuncSetAttribute(prefill_gemm_kernel<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                     (int)Cfg<2>::kSmemBytes);
-        if (e != cudaSuccess) return e;
+        const void *all[4] = {(const void *)prefill_gemm_kernel<1, false>, (const void *)prefill_gemm_kernel<1, true>,
+                              (const void *)prefill_gemm_kernel<2, false>, (const void *)prefill_gemm_kernel<2, true>};
+        for (const void *k : all) {
+            cudaError_t e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemLimit);
+            if (e != cudaSuccess) return e;
+        }
         attr_set[dev] = true;
     }
     if (n_tiles <= 0) return cudaSuccess;
@@ -474,42 +531,46 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
     cfg.stream = stream;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles};
+    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles, (void *)&a_rows, (void *)&n_stages};
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
 } // namespace
 
 int prefill_token_tiles(int64_t max_M) { return max_M > BM ? 2 : 1; }
+// rows of activations per token tile in a TMA stage, for the largest M of a launch
+static int prefill_a_rows(int64_t max_M) { return max_M <= 64 ? 64 : BM; }
 
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
                            int out_i32, WorkspaceHeader *hdr, cudaStream_t stream)
 {
-    const int mt = prefill_token_tiles(M);
+    const int mt = prefill_token_tiles(M), a_rows = prefill_a_rows(M);
     GemmProblem g;
-    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, mt, 0, &hdr->status);
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, mt, a_rows, 0,
+                                 &hdr->status);
     if (e != cudaSuccess) return e;
-    return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, stream);
+    return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, a_rows, stream);
 }
 
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int token_tiles, int tile_begin, WorkspaceHeader *hdr, int *n_tiles)
+                                int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles)
 {
     GemmProblem g;
-    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, 0, token_tiles, tile_begin,
-                                 &hdr->status);
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, 0, prefill_token_tiles(max_M),
+                                 prefill_a_rows(max_M), tile_begin, &hdr->status);
     if (e != cudaSuccess) return e;
     memcpy(slot, &g, sizeof(g));
     *n_tiles = g.p.tiles_m * g.p.tiles_n;
     return cudaSuccess;
 }
 
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int token_tiles, cudaStream_t stream)
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, cudaStream_t stream)
 {
     GemmProblem unused{};
-    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, token_tiles, stream);
+    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, prefill_token_tiles(max_M),
+                       prefill_a_rows(max_M), stream);
 }
 
 } // namespace bitlinear
