@@ -1,16 +1,17 @@
-// Kernel (d): ternary x int8 GEMM for many tokens (prefill) on the tcgen05 tensor cores.
+// Kernel (d): ternary x int8 GEMM for 17 tokens and more on the tcgen05 tensor cores.
 //
 // With hundreds of tokens every weight is reused hundreds of times, so the integer matmul
 // (Section 1 / Section 3 "Energy": matrix multiplication dominates) is a dense contraction and
-// belongs on the tensor cores.  Per CTA tile of 128 tokens x 256 output features, per 128-wide
+// belongs on the tensor cores; from 17 to 128 tokens the same kernel streams the weights faster than the
+// warp-level MMAs of the decode kernel can.  Per CTA tile of 128 tokens x 256 output features, per 128-wide
 // k block:
 //   producer warp  : TMA loads the int8 activation tile (128 x 128 B, 128-byte swizzle) and the
 //                    packed 2-bit weight tiles (4 row blocks x 2 column tiles x 1 KiB) into shared memory;
 //   expander warps : turn the 2-bit codes into unsigned bytes with ONE mask per four weights -- the field
 //                    of row 16 f + r stays where it is, so the byte is code * 4^f -- and write them
 //                    K-major with the same 128-byte swizzle the tensor core expects;
-//   MMA warp       : one thread issues four tcgen05.mma kind::i8 (128 x 256 x 32, s8 x u8) per k block
-//                    into a TMEM accumulator; tcgen05.commit releases the stage;
+//   MMA thread     : issues four tcgen05.mma kind::i8 (128 x 256 x 32, s8 x u8) per k block into a TMEM
+//                    accumulator; one tcgen05.commit releases the TMA stage and the expanded tile;
 //   epilogue warps : tcgen05.ld the finished int32 accumulators, undo the 4^f of their output row with an
 //                    exact shift, subtract the token's sum of q (codes are T + 1), scale by
 //                    gamma * beta_t / 127, round to bf16 and store, while the MMA warp fills the second
@@ -19,6 +20,8 @@
 // tile, the costly operand (written once and read once per MMA through shared memory, whose bandwidth bounds
 // this kernel), then feeds two MMAs per k step, and the two accumulators fill the tensor memory, so the
 // epilogue of a tile no longer overlaps the next tile's MMAs.
+// One launch runs one matmul (passed as a kernel parameter) or all the matmuls of a sequence (a table in device
+// memory): the CTAs walk one launch-wide sequence of CTA tiles.
 // The kernel is a programmatic dependent of the activation quantiser: set-up (barriers, tensor memory,
 // descriptor prefetch) runs while the quantiser finishes; the producer waits for it before the first load.
 // All waits are bounded; on expiry the CTA sets the workspace status to BITLINEAR_ERR_TIMEOUT,
