@@ -61,13 +61,19 @@ struct Layout {
 inline int64_t row_blocks(int64_t N) { return (N + kTileRows - 1) / kTileRows; }
 inline int64_t col_tiles(int64_t K) { return (K + kTileCols - 1) / kTileCols; }
 
-// Workspace of one matmul: [header | acc32 (at most 64 tokens) | per-warp lists | Xq | beta | rowsum]
+inline int64_t gemm_k_blocks(int64_t K) { return (K + 127) / 128; }
+
+// Workspace of one matmul: [header | int32 scratch | per-warp lists | Xq | beta | rowsum].  The scratch serves the
+// weight-streaming kernel (sums of row blocks shared by several warps, at most 64 tokens) or the GEMM (tiles cut
+// along K), whichever is larger, so that the layout does not depend on the kernel chosen.
 Layout single_layout(int64_t M, int64_t N, int64_t K)
 {
     Layout L{};
     size_t off = sizeof(WorkspaceHeader);
     L.acc32 = off;
-    off += align_up((size_t)(M < kMaxDecodeM ? M : kMaxDecodeM) * N * 4, 256);
+    const size_t decode_scratch = (size_t)(M < kMaxDecodeM ? M : kMaxDecodeM) * N * 4;
+    const size_t gemm_scratch = M > 0 ? prefill_split_bytes(prefill_tile_count(M, N, M), M) : 0;
+    off += align_up(decode_scratch > gemm_scratch ? decode_scratch : gemm_scratch, 256);
     L.table = off; // end of what is cleared before every call
     L.lists = off;
     off += align_up(kOwnedListsBytes, 256);
@@ -132,7 +138,9 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
 // x_rows: rows of int8 activations that exist behind e.Xq (>= e.M; the rows past e.M may hold anything).
-bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, int64_t x_rows, cudaStream_t stream)
+// split_scratch: zeroed scratch for GEMM tiles cut along K, or null (then none are cut).
+bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, int64_t x_rows, void *split_scratch,
+                            cudaStream_t stream)
 {
     WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
     OwnedList *lists = reinterpret_cast<OwnedList *>(ws + lists_offset);
@@ -153,7 +161,7 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
         cudaError_t err = pair ? launch_prefill_pair(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out,
                                                      e.out_i32, hdr, stream)
                                : launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, x_rows, e.K, e.N, e.out,
-                                                e.out_i32, hdr, stream);
+                                                e.out_i32, hdr, split_scratch, stream);
         return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
@@ -248,12 +256,16 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     char *ws = reinterpret_cast<char *>(workspace);
     InlineTable inl{};
     fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L);
-    inl.e[0].xq_tiled = use_tcgen05_for(M) ? 0 : 1;
-    // quantise the tokens; the same launch clears the header and, for the streaming kernel, its scratch
-    const size_t zero_bytes = use_tcgen05_for(M) ? sizeof(WorkspaceHeader) : L.table;
+    const bool tc = use_tcgen05_for(M);
+    inl.e[0].xq_tiled = tc ? 0 : 1;
+    // quantise the tokens; the same launch clears the header and the scratch of the kernel that follows, if it uses it
+    const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
+    const bool split = clear > 0;
+    const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M, (cudaStream_t)stream);
+    return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M,
+                      split ? ws + L.acc32 : nullptr, (cudaStream_t)stream);
 }
 
 bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
@@ -277,7 +289,12 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                     (path == BITLINEAR_PATH_TCGEN05_TS) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
     InlineTable inl{};
     fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
-    const size_t zero_bytes = tc ? sizeof(WorkspaceHeader) : L.table;
+    // (only the one-SM GEMM with weights in shared memory cuts tiles along K)
+    const size_t clear = (path == BITLINEAR_PATH_TCGEN05 || (path == BITLINEAR_PATH_AUTO && tc))
+                             ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M)
+                             : 0;
+    const bool split = clear > 0;
+    const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, s);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     if (tc) {
@@ -288,7 +305,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     }
     rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
     if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], path, ws, L.lists, M, s); // (the caller's rows: exactly M of them)
+    return run_matmul(inl.e[0], path, ws, L.lists, M, split ? ws + L.acc32 : nullptr, s); // (the caller's rows: exactly M)
 }
 
 bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)
@@ -353,13 +370,15 @@ struct bitlinear_sequence {
     const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
     bitlinear::InlineTable inl;
     const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
-    int gemm_tiles;
+    int gemm_tiles, gemm_min_kb;
+    void *split_scratch;    // inside the workspace; null: no GEMM tile of this sequence is cut along K
 };
 
 namespace {
 struct SeqLayout {
     size_t acc32, table, lists, gemm, data, total;
     bool use_gemm;
+    int min_kb; // fewest k blocks of 128 columns among the matmuls
 };
 
 inline size_t seq_xq_bytes(int64_t M, int64_t K, bool gemm)
@@ -373,6 +392,7 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
     if (!layers || n <= 0 || n > 65536) return false;
     size_t acc = 0, data = 0;
     uint64_t tiles = 0, gemm_tiles = 0;
+    int64_t min_kb = INT32_MAX;
     int64_t max_M = 0;
     for (int i = 0; i < n; ++i)
         if (layers[i].M > max_M) max_M = layers[i].M;
@@ -384,11 +404,18 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
         if (!gemm) acc += align_up((size_t)d.M * d.N * 4, 256);
         tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K)); // an upper bound of the work items in either mode
         gemm_tiles += (uint64_t)((d.M + 127) / 128) * (uint64_t)((d.N + 255) / 256); // the same for the GEMM's CTA tiles
+        if (gemm_k_blocks(d.K) < min_kb) min_kb = gemm_k_blocks(d.K);
         if (entry_off) entry_off->push_back(data);
         data += seq_xq_bytes(d.M, d.K, gemm) + 2 * align_up((size_t)d.M * 4, 256);
     }
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
     if (gemm && gemm_tiles > 0x7FFFFFFFull) return false;
+    if (gemm) { // scratch for tiles cut along K, where the streaming kernel has its int32 scratch
+        uint64_t exact = 0;
+        for (int i = 0; i < n; ++i) exact += (uint64_t)prefill_tile_count(layers[i].M, layers[i].N, max_M);
+        acc = align_up(prefill_split_bytes((int64_t)exact, max_M), 256);
+    }
+    S.min_kb = (int)min_kb;
     size_t off = sizeof(WorkspaceHeader);
     S.acc32 = off;
     off += acc;
@@ -473,10 +500,14 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     seq->tiles = tiles;
     seq->tokens = tokens;
     seq->max_M = max_M;
-    seq->zero_bytes = gemm ? sizeof(WorkspaceHeader) : S.table; // header and int32 scratch
+    const size_t clear = gemm ? prefill_split_clear_bytes(gemm_tiles, S.min_kb, max_M) : 0;
+    const bool split = clear > 0;
+    seq->zero_bytes = gemm ? S.acc32 + align_up(clear, 256) : S.table; // header and the int32 scratch in use
     seq->dev_table = nullptr;
     seq->gemm_table = nullptr;
     seq->gemm_tiles = gemm_tiles;
+    seq->gemm_min_kb = S.min_kb;
+    seq->split_scratch = split ? ws + S.acc32 : nullptr;
     if (gemm) {
         if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
             delete seq;
@@ -508,7 +539,8 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {
         const cudaError_t err =
-            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->max_M, s)
+            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->max_M, seq->gemm_min_kb,
+                                                 seq->split_scratch, s)
                             : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
                                             reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s);
         if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;

@@ -94,7 +94,16 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
 // Xq; the rows past M may hold anything (they only reach accumulator rows that are never stored).
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, WorkspaceHeader *hdr, cudaStream_t stream);
+                           int out_i32, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream);
+
+// Cutting tiles along K.  When the CTA tiles of a launch leave most SMs idle in their last round, the kernel cuts
+// the tiles of that round along K and adds the partial sums up in `split_scratch` (prefill_split_bytes(tiles, max_M)
+// bytes, 256-byte aligned; null: never cut).  prefill_split_clear_bytes tells how many bytes at the start of the
+// scratch must be ZERO when a launch over n_tiles CTA tiles, whose matmuls have at least min_KB k blocks of 128
+// columns, starts: 0 if that launch cuts no tile (the scratch is not touched then).
+int64_t prefill_tile_count(int64_t M, int64_t N, int64_t max_M);
+size_t prefill_split_bytes(int64_t n_tiles, int64_t max_M);
+size_t prefill_split_clear_bytes(int64_t n_tiles, int64_t min_KB, int64_t max_M);
 
 // The same kernel over the matmuls of a sequence in ONE launch.  The host fills a table of kGemmProblemBytes-sized
 // entries (tensor maps + parameters) with prefill_table_entry, copies it to device memory (64-byte aligned) once, and
@@ -105,7 +114,8 @@ int prefill_token_tiles(int64_t max_M);
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
                                 int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles);
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, cudaStream_t stream);
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, int min_KB,
+                                 void *split_scratch, cudaStream_t stream);
 
 // The same GEMM on pairs of SMs (tcgen05 cta_group::2): 256 tokens x 256 features per pair tile.
 // prefill_pair_capacity: CTA pairs that can be resident at once (0: not available on this device).

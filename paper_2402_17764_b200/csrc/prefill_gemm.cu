@@ -30,6 +30,7 @@
 // Roofline: int8 tensor throughput; algorithmic work 2*M*N*K integer operations.
 #include <cuda.h>
 
+#include <cstdlib>
 #include <cstring>
 
 #include "internal.cuh"
@@ -100,8 +101,50 @@ struct Barriers {
     uint64_t acc_empty[2];       // drained by the epilogue
     uint32_t tmem_base;
     int abort_flag;
+    int split_last; // this CTA added the last partial sums of a cut tile
 };
 static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block");
+
+// Work units of a launch.  Units 0 .. full-1 are whole CTA tiles.  When the tiles do not fill the last round of
+// the SMs (fewer than half of them busy), the tiles of that round are cut along K into `slices` units each, so
+// that all SMs work on them: every unit adds its partial sums into an int32 scratch tile (bulk reduce from shared
+// memory, which is idle by then: a cut unit is the last unit of its CTA), and the CTA that adds last (a counter
+// per tile) dequantises the tile from the scratch.  Scratch and counters must be zero at the start of the launch.
+struct SplitPlan {
+    int n_units, full, slices;
+    int32_t *scratch;   // per cut tile: [token tile][lane quarter][chunk of 32 features][lane][32 sums], see split_piece
+    uint32_t *counters; // per cut tile
+};
+constexpr uint32_t kSplitTileBytes = BM * BN * 4; // scratch per token tile of a cut CTA tile
+constexpr int kMaxSplitTiles = 80;                // tiles that can be cut in one launch (half the SMs of the largest part)
+constexpr int kMinSplitKB = 64;                   // k blocks a tile must have for a cut to pay (measured)
+constexpr size_t kSplitCounterBytes = 512;        // counters in front of the scratch tiles
+
+struct Unit {
+    int tile, slice;
+    bool split;
+    __device__ Unit(const SplitPlan &sp, int u)
+    {
+        if (u < sp.full) {
+            tile = u;
+            slice = 0;
+            split = false;
+        } else {
+            const int v = u - sp.full;
+            tile = sp.full + v / sp.slices;
+            slice = v - (v / sp.slices) * sp.slices;
+            split = true;
+        }
+    }
+    // k blocks [kb0, kb1) of the KB of the tile's matmul (slices <= KB: never empty)
+    __device__ int kb0(const SplitPlan &sp, int KB) const { return split ? (int)((long long)slice * KB / sp.slices) : 0; }
+    __device__ int kb1(const SplitPlan &sp, int KB) const { return split ? (int)((long long)(slice + 1) * KB / sp.slices) : KB; }
+};
+
+// Byte offset of 16-byte piece `piece` (of 8) of lane `lane` inside a chunk of 32 lanes x 128 bytes: pieces are
+// swizzled by lane so that the 16-byte shared-memory stores of a warp are free of bank conflicts.  The scratch in
+// global memory has the same layout (it is added to with one bulk reduce per 32 KiB).
+__device__ __forceinline__ uint32_t split_piece(int lane, int piece) { return (uint32_t)(lane * 128 + ((piece ^ (lane & 7)) << 4)); }
 
 // Position in the ring of TMA stages and in the ring of expanded tiles after `it` k blocks.
 struct RingPos {
@@ -158,7 +201,7 @@ struct ProblemCursor {
 template <int MT, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems,
-                    int n_tiles, int a_rows, int n_stages)
+                    const SplitPlan sp, int a_rows, int n_stages)
 {
     constexpr int kAccBufs = Cfg<MT>::kAccBufs, kBSlots = Cfg<MT>::kBSlots, kGroups = Cfg<MT>::kGroups;
     const uint32_t kStageBytes = stage_bytes(MT, a_rows), kAHalfBytes = (uint32_t)(a_rows * BK);
@@ -209,14 +252,17 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             griddep_wait(); // the activations are written by the launch before this one
             RingPos pos;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+            for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x) {
+                const Unit unit(sp, u);
+                const int tile = unit.tile;
                 const GemmProblem &g = cur.seek(tile);
                 const Params &p = g.p;
-                const int local = tile - p.tile_begin, KB = p.KB;
+                const int local = tile - p.tile_begin;
+                const int kb_begin = unit.kb0(sp, p.KB), kb_end = unit.kb1(sp, p.KB);
                 const int m0 = (local % p.tiles_m) * (MT * BM);
                 const int n0 = (local / p.tiles_m) * BN;
                 const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // a second token tile past the end is left out
-                for (int kb = 0; kb < KB; ++kb, pos.advance(n_stages)) {
+                for (int kb = kb_begin; kb < kb_end; ++kb, pos.advance(n_stages)) {
                     const int s = pos.s;
                     if (pos.round > 0 && !mbar_wait_bounded(smem_u32(&bars->empty[s]), (pos.round - 1) & 1, abort_flag)) {
                         ok = false;
@@ -243,16 +289,18 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             RingPos pos;
             uint32_t tile_it = 0;
             bool ok = true;
-            for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++tile_it) {
+            for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x, ++tile_it) {
+                const Unit unit(sp, u);
+                const int tile = unit.tile;
                 const Params &p = cur.seek(tile).p;
-                const int KB = p.KB;
+                const int kb_begin = unit.kb0(sp, p.KB), kb_end = unit.kb1(sp, p.KB);
                 const int buf = tile_it % kAccBufs;
                 const uint32_t use = tile_it / kAccBufs;
                 if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
                 const bool two = MT == 2 && ((tile - p.tile_begin) % p.tiles_m) * (MT * BM) + BM < p.M;
-                for (int kb = 0; kb < KB; ++kb, pos.advance(n_stages)) {
+                for (int kb = kb_begin; kb < kb_end; ++kb, pos.advance(n_stages)) {
                     const int s = pos.s, b = (int)(pos.it % kBSlots);
                     if (!mbar_wait_bounded(smem_u32(&bars->expanded[b]), (pos.it / kBSlots) & 1, abort_flag)) {
                         ok = false;
@@ -264,7 +312,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
 #pragma unroll
                     for (int k4 = 0; k4 < BK / 32; ++k4) {
                         const uint64_t b_desc = smem_desc_k_sw128(b_addr + 32 * k4);
-                        const uint32_t accumulate = (kb > 0 || k4 > 0) ? 1u : 0u;
+                        const uint32_t accumulate = (kb > kb_begin || k4 > 0) ? 1u : 0u;
                         mma_i8_ss(d_tmem, smem_desc_k_sw128(a_addr + 32 * k4), b_desc, idesc, accumulate);
                         if (two) mma_i8_ss(d_tmem + BN, smem_desc_k_sw128(a_addr + kAHalfBytes + 32 * k4), b_desc, idesc, accumulate);
                     }
@@ -292,9 +340,11 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         ProblemCursor<kTable> cur(one, table, n_problems);
         RingPos pos, reader; // reader: the k block kBSlots steps back, whose MMAs read the expanded tile written next
         bool ok = true;
-        for (int tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
-            const int KB = cur.seek(tile).p.KB;
-            for (int kb = 0; kb < KB; ++kb, pos.advance(n_stages)) {
+        for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x) {
+            const Unit unit(sp, u);
+            const int KB = cur.seek(unit.tile).p.KB;
+            const int kb_end = unit.kb1(sp, KB);
+            for (int kb = unit.kb0(sp, KB); kb < kb_end; ++kb, pos.advance(n_stages)) {
                 const int s = pos.s, b = (int)(pos.it % kBSlots);
                 const bool mine = kGroups == 1 || (int)(pos.it & 1u) == group;
                 const bool has_reader = pos.it >= (uint32_t)kBSlots;
@@ -343,7 +393,9 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         const int q = warp & 3;
         ProblemCursor<kTable> cur(one, table, n_problems);
         uint32_t tile_it = 0;
-        for (int tile = blockIdx.x; tile < n_tiles; tile += gridDim.x, ++tile_it) {
+        for (int u = blockIdx.x; u < sp.n_units; u += gridDim.x, ++tile_it) {
+            const Unit unit(sp, u);
+            const int tile = unit.tile;
             const Params &p = cur.seek(tile).p;
             const float gamma = p.out_i32 ? 0.0f : *p.gamma;
             const int local = tile - p.tile_begin;
@@ -351,65 +403,146 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             const int n0 = (local / p.tiles_m) * BN;
             const int buf = tile_it % kAccBufs;
             const uint32_t parity = (tile_it / kAccBufs) & 1;
+            const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // no MMA wrote the accumulator of an absent token tile
             if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), parity, abort_flag)) break;
             tc_fence_after_sync();
-#pragma unroll 1
-            for (int half = 0; half < MT; ++half) {
-            if (half == 1 && m0 + BM >= p.M) break; // no MMA wrote that accumulator
-            const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
-            const int t = m0 + half * BM + 32 * q + lane;
-            const bool row_ok = t < p.M;
-            float scale = 0.0f;
-            int rowsum = 0;
-            if (row_ok) {
-                rowsum = p.rowsum[t];
-                if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), (float)kQb);
-            }
-#pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
-                uint32_t v[32];
-                tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
-                tmem_ld_wait();
+
+            // shift, subtract, scale, round and store the 32 sums `v` of chunk c (features n0 + 32 c ..) of token t
+            auto emit = [&](const uint32_t (&v)[32], int c, int t, int rowsum, float scale) {
                 const int n = n0 + c * 32;
                 // output row n + i carries the factor 4^f, f = ((n + i) % 64) / 16 = 2 (c % 2) + i / 16
                 const int sh_lo = 4 * (c & 1), sh_hi = sh_lo + 2;
                 int a[32];
 #pragma unroll
                 for (int i = 0; i < 32; ++i) a[i] = ((int)v[i] >> (i < 16 ? sh_lo : sh_hi)) - rowsum;
-                if (row_ok) {
-                    if (p.out_i32) {
-                        int32_t *dst = reinterpret_cast<int32_t *>(p.out) + (size_t)t * p.N + n;
+                if (t >= p.M) return;
+                if (p.out_i32) {
+                    int32_t *dst = reinterpret_cast<int32_t *>(p.out) + (size_t)t * p.N + n;
 #pragma unroll
-                        for (int i = 0; i < 32; i += 4)
-                            if (n + i < p.N) *reinterpret_cast<int4 *>(dst + i) = make_int4(a[i], a[i + 1], a[i + 2], a[i + 3]);
-                    } else {
-                        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)t * p.N + n;
+                    for (int i = 0; i < 32; i += 4)
+                        if (n + i < p.N) *reinterpret_cast<int4 *>(dst + i) = make_int4(a[i], a[i + 1], a[i + 2], a[i + 3]);
+                } else {
+                    __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)t * p.N + n;
 #pragma unroll
-                        for (int i = 0; i < 32; i += 16) { // N is a multiple of 16: 16 features are in or out together
-                            if (n + i < p.N) {
-                                uint32_t o[8];
+                    for (int i = 0; i < 32; i += 16) { // N is a multiple of 16: 16 features are in or out together
+                        if (n + i < p.N) {
+                            uint32_t o[8];
 #pragma unroll
-                                for (int h = 0; h < 8; ++h) {
-                                    const float x0 = __fmul_rn((float)a[i + 2 * h], scale);
-                                    const float x1 = __fmul_rn((float)a[i + 2 * h + 1], scale);
-                                    const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
-                                    o[h] = *reinterpret_cast<const uint32_t *>(&pr);
-                                }
-                                if (p.out_32b_aligned) {
-                                    st_global_v8(dst + i, o);
-                                } else {
-                                    *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
-                                    *reinterpret_cast<uint4 *>(dst + i + 8) = make_uint4(o[4], o[5], o[6], o[7]);
-                                }
+                            for (int h = 0; h < 8; ++h) {
+                                const float x0 = __fmul_rn((float)a[i + 2 * h], scale);
+                                const float x1 = __fmul_rn((float)a[i + 2 * h + 1], scale);
+                                const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
+                                o[h] = *reinterpret_cast<const uint32_t *>(&pr);
+                            }
+                            if (p.out_32b_aligned) {
+                                st_global_v8(dst + i, o);
+                            } else {
+                                *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+                                *reinterpret_cast<uint4 *>(dst + i + 8) = make_uint4(o[4], o[5], o[6], o[7]);
                             }
                         }
                     }
                 }
+            };
+            auto token_scale = [&](int t, int &rowsum, float &scale) {
+                rowsum = 0;
+                scale = 0.0f;
+                if (t < p.M) {
+                    rowsum = p.rowsum[t];
+                    if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), (float)kQb);
+                }
+            };
+
+            if (!unit.split) {
+#pragma unroll 1
+                for (int half = 0; half < halves; ++half) {
+                    const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
+                    const int t = m0 + half * BM + 32 * q + lane;
+                    int rowsum;
+                    float scale;
+                    token_scale(t, rowsum, scale);
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        uint32_t v[32];
+                        tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
+                        tmem_ld_wait();
+                        emit(v, c, t, rowsum, scale);
+                    }
+                }
+                tc_fence_before_sync();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                continue;
             }
-            } // token tiles
+
+            // ---- a unit that holds a K slice of its tile: the last unit of this CTA, so every ring is idle and the
+            // shared memory from `base` on (at least 200 KiB) serves as staging: 32 KiB per epilogue warp.
+            const int cut = tile - sp.full; // which cut tile
+            uint8_t *stage_w = smem + q * (BN / 32) * 4096;
+            int32_t *scratch_tile = sp.scratch + (size_t)cut * (MT * kSplitTileBytes / 4);
+#pragma unroll 1
+            for (int half = 0; half < halves; ++half) {
+                const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
+                if (half > 0) { // the bulk reduce of the first token tile must have read the staging area
+                    if (lane == 0) bulk_wait_group_read0();
+                    __syncwarp();
+                }
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int pc = 0; pc < 8; ++pc)
+                        *reinterpret_cast<uint4 *>(stage_w + c * 4096 + split_piece(lane, pc)) =
+                            make_uint4(v[4 * pc], v[4 * pc + 1], v[4 * pc + 2], v[4 * pc + 3]);
+                }
+                fence_proxy_async_smem(); // generic-proxy writes -> visible to the bulk copy engine
+                __syncwarp();
+                if (lane == 0) {
+                    bulk_reduce_add_s32(scratch_tile + (size_t)(half * 4 + q) * (BN / 32) * 1024, smem_u32(stage_w),
+                                        (BN / 32) * 4096);
+                    bulk_commit_group();
+                }
+            }
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+            if (lane == 0) {
+                mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                bulk_wait_group0(); // the sums have been added
+                __threadfence();
+            }
+            named_bar_sync(1, 128); // the four epilogue warps
+            if (warp == 2 && lane == 0) {
+                const uint32_t before = atomicAdd(&sp.counters[cut], 1u);
+                bars->split_last = (before == (uint32_t)sp.slices - 1u) ? 1 : 0;
+                __threadfence();
+            }
+            named_bar_sync(1, 128);
+            if (bars->split_last) { // every slice has been added: dequantise the tile from the scratch
+#pragma unroll 1
+                for (int half = 0; half < halves; ++half) {
+                    const int t = m0 + half * BM + 32 * q + lane;
+                    int rowsum;
+                    float scale;
+                    token_scale(t, rowsum, scale);
+#pragma unroll 1
+                    for (int c = 0; c < BN / 32; ++c) {
+                        const uint8_t *src =
+                            reinterpret_cast<const uint8_t *>(scratch_tile + (size_t)(half * 4 + q) * (BN / 32) * 1024) + c * 4096;
+                        uint32_t v[32];
+#pragma unroll
+                        for (int pc = 0; pc < 8; ++pc) {
+                            const int4 w = __ldcg(reinterpret_cast<const int4 *>(src + split_piece(lane, pc)));
+                            v[4 * pc] = (uint32_t)w.x;
+                            v[4 * pc + 1] = (uint32_t)w.y;
+                            v[4 * pc + 2] = (uint32_t)w.z;
+                            v[4 * pc + 3] = (uint32_t)w.w;
+                        }
+                        emit(v, c, t, rowsum, scale);
+                    }
+                }
+            }
         }
     }
 
@@ -501,8 +634,25 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
 }
 
 // Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
+// How many K slices the tiles of the last, partly filled round of the SMs are cut into (1: none are cut).
+static int split_slices(int n_tiles, int min_KB, int sms)
+{
+    static const int enabled = [] {
+        const char *v = std::getenv("BITLINEAR_PREFILL_SPLIT");
+        return (v && *v) ? std::atoi(v) : 1;
+    }();
+    const int r = n_tiles % sms;
+    if (!enabled || r == 0 || 2 * r > sms || r > kMaxSplitTiles) return 1;
+    int s = sms / r;
+    if (s > min_KB) s = min_KB;
+    // Adding up and dequantising a cut tile costs 15 to 25 us (measured), a tile of KB k blocks takes about
+    // 0.6 us x KB: cut only where several times that is saved.
+    if (min_KB < kMinSplitKB || s < 3) s = 1;
+    return s;
+}
+
 static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int mt, int a_rows,
-                               cudaStream_t stream)
+                               int min_KB, void *split_scratch, cudaStream_t stream)
 {
     const void *kernel = table ? (mt == 2 ? (const void *)prefill_gemm_kernel<2, true> : (const void *)prefill_gemm_kernel<1, true>)
                                : (mt == 2 ? (const void *)prefill_gemm_kernel<2, false> : (const void *)prefill_gemm_kernel<1, false>);
@@ -521,8 +671,15 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
         attr_set[dev] = true;
     }
     if (n_tiles <= 0) return cudaSuccess;
-    int grid = n_tiles;
-    if (grid > sm_count()) grid = sm_count();
+    const int sms = sm_count();
+    SplitPlan sp;
+    sp.slices = split_scratch ? split_slices(n_tiles, min_KB, sms) : 1;
+    sp.full = sp.slices > 1 ? (n_tiles / sms) * sms : n_tiles;
+    sp.n_units = sp.full + (n_tiles - sp.full) * sp.slices;
+    sp.counters = reinterpret_cast<uint32_t *>(split_scratch);
+    sp.scratch = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(split_scratch) + kSplitCounterBytes);
+    int grid = sp.n_units;
+    if (grid > sms) grid = sms;
     // programmatic dependent launch: see the head of this file
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -534,26 +691,46 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
     cfg.stream = stream;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles, (void *)&a_rows, (void *)&n_stages};
+    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&sp, (void *)&a_rows, (void *)&n_stages};
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
 } // namespace
 
 int prefill_token_tiles(int64_t max_M) { return max_M > BM ? 2 : 1; }
+
+int64_t prefill_tile_count(int64_t M, int64_t N, int64_t max_M)
+{
+    const int64_t mt = prefill_token_tiles(max_M);
+    return ((M + mt * BM - 1) / (mt * BM)) * ((N + BN - 1) / BN);
+}
+
+size_t prefill_split_bytes(int64_t n_tiles, int64_t max_M)
+{
+    const int64_t cut = n_tiles < kMaxSplitTiles ? n_tiles : kMaxSplitTiles;
+    return kSplitCounterBytes + (size_t)cut * (size_t)prefill_token_tiles(max_M) * kSplitTileBytes;
+}
+
+size_t prefill_split_clear_bytes(int64_t n_tiles, int64_t min_KB, int64_t max_M)
+{
+    if (n_tiles > 0x7FFFFFFF) return 0;
+    const int sms = sm_count();
+    if (split_slices((int)n_tiles, (int)(min_KB > 0x7FFFFFFF ? 0x7FFFFFFF : min_KB), sms) < 2) return 0;
+    return kSplitCounterBytes + (size_t)(n_tiles % sms) * (size_t)prefill_token_tiles(max_M) * kSplitTileBytes;
+}
 // rows of activations per token tile in a TMA stage, for the largest M of a launch
 static int prefill_a_rows(int64_t max_M) { return max_M <= 64 ? 64 : BM; }
 
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, WorkspaceHeader *hdr, cudaStream_t stream)
+                           int out_i32, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream)
 {
     const int mt = prefill_token_tiles(M), a_rows = prefill_a_rows(M);
     GemmProblem g;
     cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, mt, a_rows, 0,
                                  &hdr->status);
     if (e != cudaSuccess) return e;
-    return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, a_rows, stream);
+    return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, a_rows, g.p.KB, split_scratch, stream);
 }
 
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
@@ -569,11 +746,12 @@ cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gam
     return cudaSuccess;
 }
 
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, cudaStream_t stream)
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, int min_KB,
+                                 void *split_scratch, cudaStream_t stream)
 {
     GemmProblem unused{};
     return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, prefill_token_tiles(max_M),
-                       prefill_a_rows(max_M), stream);
+                       prefill_a_rows(max_M), min_KB, split_scratch, stream);
 }
 
 } // namespace bitlinear

@@ -96,6 +96,29 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
 // Makes generic-proxy shared-memory writes visible to the async proxy (TMA, tcgen05.mma operands).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
+// ---- bulk reduce, named barriers ---------------------------------------------------------------------
+
+// Adds `bytes` of int32 from shared memory to global memory (both 16-byte aligned, bytes a multiple of 16);
+// completion is tracked by the bulk async-group of the issuing thread.
+__device__ __forceinline__ void bulk_reduce_add_s32(void *gptr, uint32_t smem_addr, uint32_t bytes)
+{
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.s32 [%0], [%1], %2;" ::"l"(gptr), "r"(smem_addr),
+                 "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// all bulk groups of this thread have read their shared-memory source
+__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// all bulk groups of this thread are complete
+__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// Barrier `id` (1..15) among `n_threads` threads of the CTA (a hardware barrier without a limit: every one of them
+// must get here).
+__device__ __forceinline__ void named_bar_sync(int id, int n_threads)
+{
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(n_threads) : "memory");
+}
+
 // ---- TMA ------------------------------------------------------------------------------------------
 
 __device__ __forceinline__ void prefetch_tensormap(const CUtensorMap *m)

@@ -204,7 +204,9 @@ def test_matmul_i32_mma_wider_batches(oracle, M, K, N):
 
 
 TC_SHAPES = [(128, 128, 256), (1, 16, 16), (65, 3200, 320), (200, 8640, 528), (300, 1536, 1024), (512, 5120, 256),
-             (64, 4096, 4096), (129, 144, 4112)]
+             (64, 4096, 4096), (129, 144, 4112),
+             # few tiles and a long K: the tiles are cut along K and summed through the int32 scratch
+             (300, 8640, 272), (40, 16384, 1040)]
 
 
 @pytest.mark.parametrize("path", [B.PATH_TCGEN05, B.PATH_TCGEN05_PAIR, B.PATH_TCGEN05_TS])
