@@ -141,6 +141,29 @@ def test_13b_prefill_sampled(timing_oracle, M):
         del W, X, Y, ws, packed
 
 
+def test_13b_prefill_as_one_sequence_sampled(timing_oracle):
+    """Both 13B-shaped matrices at 2048 tokens in ONE launch of the tensor-core GEMM (table of matmuls)."""
+    M = 2048
+    cfg = S.CONFIGS["13b_prefill"]
+    rng = np.random.default_rng(7)
+    layers, meta = build_stack(cfg["layers"], 1, M)
+    seq = B.Sequence(layers)
+    seq.forward()
+    torch.cuda.synchronize()
+    assert B.poll_status(seq.workspace) == 0
+    for (packed, gamma, X, Y, N), (seed, sh) in zip(layers, meta):
+        W = S.latent_weights(sh.N, sh.K, seed, device="cuda").cpu().numpy()
+        tokens = np.sort(rng.choice(M, size=48, replace=False))
+        tokens[0], tokens[-1] = 0, M - 1
+        rows = np.sort(rng.choice(sh.N, size=64, replace=False))
+        rows[0], rows[-1] = 0, sh.N - 1
+        t_idx = torch.as_tensor(tokens, device="cuda")
+        want = expected_samples(timing_oracle, W, torch_bf16_to_bits(X[t_idx]), rows)
+        check_samples(Y[t_idx], want, rows, f"13B prefill sequence {sh.N}x{sh.K} M={M}")
+        assert bool(torch.isfinite(Y.float()).all())
+    seq.close()
+
+
 @pytest.mark.parametrize("M", [1, 16])
 def test_70b_layer_sampled(timing_oracle, M):
     """The seven projections of 70B-shaped layers (8192 hidden, 8 KV heads, FFN 28672) through one sequence;
