@@ -28,6 +28,7 @@
 
 #include "internal.cuh"
 #include "ptx.cuh"
+#include "tma_host.cuh"
 
 namespace bitlinear {
 
@@ -323,25 +324,6 @@ prefill_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 
 // ---- host side ---------------------------------------------------------------------------------
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
-                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn encode_tiled_fn()
-{
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *sym = nullptr;
-        cudaDriverEntryPointQueryResult qres;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
-            qres == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(sym);
-    }
-    return fn;
-}
-
 } // namespace
 
 // Number of CTA pairs that can be resident at once (0: the kernel cannot run here).
@@ -370,36 +352,14 @@ cudaError_t launch_prefill_pair(const void *packed, const float *gamma, const in
                                 const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
                                 WorkspaceHeader *hdr, cudaStream_t stream)
 {
-    EncodeTiledFn encode = encode_tiled_fn();
     const int capacity = prefill_pair_capacity();
-    if (!encode || capacity <= 0) return cudaErrorNotSupported;
+    if (!encode_tiled_fn() || capacity <= 0) return cudaErrorNotSupported;
     const int KB = (int)((K + BK - 1) / BK);
 
+    // activations: box of 128 rows; weights: box of 2 row blocks x 2 column tiles (each CTA expands half a tile)
     CUtensorMap tmap_x, tmap_w;
-    {
-        // int8 activations [M rows][K bytes]; box 128 bytes x 128 rows; rows/columns past the end read 0
-        const cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)M};
-        const cuuint64_t strides[1] = {(cuuint64_t)K};
-        const cuuint32_t box[2] = {(cuuint32_t)BK, (cuuint32_t)BM};
-        const cuuint32_t estr[2] = {1, 1};
-        if (encode(&tmap_x, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<int8_t *>(Xq), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return cudaErrorInvalidValue;
-    }
-    {
-        // packed weights as [NB row blocks][KB column tiles][256 words]; box = 2 row blocks x 2 column tiles
-        const cuuint64_t tiles_k = (cuuint64_t)((K + kTileCols - 1) / kTileCols);
-        const cuuint64_t tiles_n = (cuuint64_t)((N + kTileRows - 1) / kTileRows);
-        const cuuint64_t dims[3] = {kTileBytes / 4, tiles_k, tiles_n};
-        const cuuint64_t strides[2] = {(cuuint64_t)kTileBytes, tiles_k * kTileBytes};
-        const cuuint32_t box[3] = {kTileBytes / 4, (cuuint32_t)(BK / kTileCols), (cuuint32_t)(BNH / kTileRows)};
-        const cuuint32_t estr[3] = {1, 1, 1};
-        if (encode(&tmap_w, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void *>(packed), dims, strides, box, estr,
-                   CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-            return cudaErrorInvalidValue;
-    }
+    if (!encode_activation_map(&tmap_x, Xq, M, K, BM) || !encode_packed_weight_map(&tmap_w, packed, N, K, BNH / kTileRows))
+        return cudaErrorInvalidValue;
 
     Params p;
     p.gamma = gamma;
