@@ -309,6 +309,39 @@ def test_forward_is_deterministic(oracle):
     assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
 
 
+def test_tiles_cut_along_k_are_reusable(oracle):
+    """Few tiles and a long K: the GEMM cuts its tiles along K and sums them through an int32 scratch in the workspace.
+    The scratch is cleared by every call, so the same workspace gives the same (oracle) result twice: as a single
+    matmul, and as a sequence whose matmuls all have a long K (table-driven launch)."""
+    specs = [(48, 8640, 272), (300, 16384, 528)]
+    layers, refs = [], []
+    for i, (M, K, N) in enumerate(specs):
+        W = S.latent_weights(N, K, 60 + i)
+        X = S.activations(M, K, 60 + i, outlier_frac=0.01, outlier_scale=20.0)
+        T_ref, g_ref = oracle.quantize_weights(W.numpy())
+        refs.append(oracle.forward(T_ref, g_ref, torch_bf16_to_bits(X)))
+        packed, gamma = B.quantize_weights(dev(W))
+        Y = torch.zeros((M, N), dtype=torch.bfloat16, device="cuda")
+        layers.append((packed, gamma, dev(X), Y, N))
+    for (packed, gamma, X, Y, N), ref, (M, K, _) in zip(layers, refs, specs):
+        ws = B.alloc_workspace(M, N, K)
+        for _ in range(3):
+            Y.zero_()
+            B.forward(packed, gamma, X, N, Y=Y, workspace=ws)
+            assert B.poll_status(ws) == 0
+            assert np.array_equal(torch_bf16_to_bits(Y), ref)
+    seq = B.Sequence(layers)
+    for _ in range(3):
+        for l in layers:
+            l[3].zero_()
+        seq.forward()
+        torch.cuda.synchronize()
+        assert B.poll_status(seq.workspace) == 0
+        for l, ref in zip(layers, refs):
+            assert np.array_equal(torch_bf16_to_bits(l[3]), ref)
+    seq.close()
+
+
 def test_forward_sequence_matches_single_calls(oracle):
     """A small decoder layer set (7 projections x 2 layers) at M = 1 and M = 5."""
     for M in (1, 5):
