@@ -287,9 +287,18 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         if (lane == 0) {
             constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
             ProblemCursor<kTable> cur(one, table, n_problems);
-            RingPos pos;
             uint32_t tile_it = 0;
             bool ok = true;
+            // The thread's own instructions are on the critical path too, so nothing is recomputed per k block: the
+            // low words of the operand descriptors (address / 16) and the barrier addresses of the ring positions
+            // advance by constants, the high word of the descriptors never changes.
+            const uint32_t desc_hi = (uint32_t)(smem_desc_k_sw128(0) >> 32);
+            auto desc = [&](uint32_t lo) { return ((uint64_t)desc_hi << 32) | lo; };
+            const uint32_t a_lo0 = (uint32_t)smem_desc_k_sw128(stages), a_step = kStageBytes >> 4, a_half = kAHalfBytes >> 4;
+            const uint32_t b_lo0 = (uint32_t)smem_desc_k_sw128(base), b_step = kBBytes >> 4;
+            const uint32_t empty0 = smem_u32(&bars->empty[0]), expanded0 = smem_u32(&bars->expanded[0]);
+            uint32_t s = 0, b = 0, b_parity = 0; // TMA stage; expanded tile and the parity of its use
+            uint32_t a_lo = a_lo0, b_lo = b_lo0, empty_bar = empty0, expanded_bar = expanded0;
             for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x, ++tile_it) {
                 const Unit unit(sp, u);
                 const int tile = unit.tile;
@@ -301,23 +310,38 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
                 const bool two = MT == 2 && ((tile - p.tile_begin) % p.tiles_m) * (MT * BM) + BM < p.M;
-                for (int kb = kb_begin; kb < kb_end; ++kb, pos.advance(n_stages)) {
-                    const int s = pos.s, b = (int)(pos.it % kBSlots);
-                    if (!mbar_wait_bounded(smem_u32(&bars->expanded[b]), (pos.it / kBSlots) & 1, abort_flag)) {
+                uint32_t accumulate = 0;
+                for (int kb = kb_begin; kb < kb_end; ++kb) {
+                    if (!mbar_wait_bounded(expanded_bar, b_parity, abort_flag)) {
                         ok = false;
                         break;
                     }
                     tc_fence_after_sync();
-                    const uint32_t a_addr = stages + s * kStageBytes;
-                    const uint32_t b_addr = base + b * kBBytes;
 #pragma unroll
-                    for (int k4 = 0; k4 < BK / 32; ++k4) {
-                        const uint64_t b_desc = smem_desc_k_sw128(b_addr + 32 * k4);
-                        const uint32_t accumulate = (kb > kb_begin || k4 > 0) ? 1u : 0u;
-                        mma_i8_ss(d_tmem, smem_desc_k_sw128(a_addr + 32 * k4), b_desc, idesc, accumulate);
-                        if (two) mma_i8_ss(d_tmem + BN, smem_desc_k_sw128(a_addr + kAHalfBytes + 32 * k4), b_desc, idesc, accumulate);
+                    for (int k4 = 0; k4 < BK / 32; ++k4) { // 32 bytes of K = 2 descriptor units further
+                        const uint64_t b_desc = desc(b_lo + 2 * k4);
+                        mma_i8_ss(d_tmem, desc(a_lo + 2 * k4), b_desc, idesc, accumulate);
+                        if (two) mma_i8_ss(d_tmem + BN, desc(a_lo + a_half + 2 * k4), b_desc, idesc, accumulate);
+                        accumulate = 1;
                     }
-                    mma_commit(smem_u32(&bars->empty[s])); // stage and expanded tile are reusable once these MMAs have read them
+                    mma_commit(empty_bar); // stage and expanded tile are reusable once these MMAs have read them
+                    if (++s == (uint32_t)n_stages) {
+                        s = 0;
+                        a_lo = a_lo0;
+                        empty_bar = empty0;
+                    } else {
+                        a_lo += a_step;
+                        empty_bar += 8;
+                    }
+                    if (++b == (uint32_t)kBSlots) {
+                        b = 0;
+                        b_lo = b_lo0;
+                        expanded_bar = expanded0;
+                        b_parity ^= 1u;
+                    } else {
+                        b_lo += b_step;
+                        expanded_bar += 8;
+                    }
                 }
                 if (ok) mma_commit(smem_u32(&bars->acc_full[buf]));
             }
