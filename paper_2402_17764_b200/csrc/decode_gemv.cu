@@ -1,4 +1,5 @@
-// Kernel (c): weight-streaming ternary x int8 matmul for M <= 64 tokens (decode).
+// Kernel (c): weight-streaming ternary x int8 matmul for few tokens (decode): the kernels take up to 64 tokens,
+// the library sends them up to 16 (from 17 on the tensor-core GEMM is faster).
 //
 // The cost of decode is moving the weights from HBM once (Section 1: loading weights from DRAM is
 // the expensive part; Section 3: time per output token).  All matrices of a launch form ONE sequence
