@@ -15,7 +15,7 @@
 //   epilogue warps : tcgen05.ld the finished int32 accumulators, undo the 4^f of their output row with an
 //                    exact shift, subtract the token's sum of q (codes are T + 1), scale by
 //                    gamma * beta_t / 127, round to bf16 and store, while the MMA warp fills the second
-//                    TMEM buffer.  |acc| <= 64 * 3 * 127 * K < 2^31 for every K the library accepts.
+//                    TMEM buffer.  |acc| <= 64 * 2 * 127 * K < 2^31 for every K the library accepts.
 // With more than 128 tokens a CTA takes TWO token tiles per feature tile (MT = 2): the expanded weight
 // tile, the costly operand (written once and read once per MMA through shared memory, whose bandwidth bounds
 // this kernel), then feeds two MMAs per k step, and the two accumulators fill the tensor memory, so the
