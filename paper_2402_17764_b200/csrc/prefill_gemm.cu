@@ -78,8 +78,7 @@ struct Cfg {
 // have rings of their own: the expanded tile is four times the packed one, and with one ring the 227 KiB held
 // three or four k blocks in flight, too few to cover the latency of HBM when the weights are streamed once
 // (few tokens).  A stage's activation part is a_rows rows of 128 bytes per token tile: 128, or 64 when no matmul
-// of the launch has more than 64 tokens (the MMA then also reads 64 rows of whatever follows in shared memory,
-// into accumulator rows that are never stored).
+// of the launch has more than 64 tokens (the MMAs then have M = 64).
 constexpr uint32_t kSmemLimit = 232448; // 227 KiB
 constexpr uint32_t kBarrierBytes = 512;
 __host__ __device__ constexpr uint32_t stage_bytes(int mt, int a_rows) { return (uint32_t)(mt * a_rows * BK) + kPBytes; }
@@ -285,7 +284,9 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         // so there is one wait and one commit per k block: `expanded` implies `full` (the expander warps waited for
         // the stage before they arrived), and `empty` also tells the expander that the expanded tile was read.
         if (lane == 0) {
-            constexpr uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
+            // With 64 activation rows per stage the MMA has M = 64: half the operand reads from shared memory.  Its
+            // accumulator rows 16 i .. 16 i + 15 stand in TMEM lanes 32 i .. 32 i + 15.
+            const uint32_t idesc = idesc_i8(a_rows == 64 ? 64 : BM, BN, /*a_signed=*/1, /*b_signed=*/0);
             ProblemCursor<kTable> cur(one, table, n_problems);
             uint32_t tile_it = 0;
             bool ok = true;
@@ -469,6 +470,11 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                     }
                 }
             };
+            // the token whose sums this thread's TMEM lane holds (past M: none)
+            auto token_of_lane = [&](int half) {
+                if (MT == 1 && a_rows == 64) return lane < 16 ? m0 + 16 * q + lane : 0x7FFFFFFF; // M = 64 MMA: see above
+                return m0 + half * BM + 32 * q + lane;
+            };
             auto token_scale = [&](int t, int &rowsum, float &scale) {
                 rowsum = 0;
                 scale = 0.0f;
@@ -482,7 +488,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
 #pragma unroll 1
                 for (int half = 0; half < halves; ++half) {
                     const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
-                    const int t = m0 + half * BM + 32 * q + lane;
+                    const int t = token_of_lane(half);
                     int rowsum;
                     float scale;
                     token_scale(t, rowsum, scale);
@@ -547,7 +553,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             if (bars->split_last) { // every slice has been added: dequantise the tile from the scratch
 #pragma unroll 1
                 for (int half = 0; half < halves; ++half) {
-                    const int t = m0 + half * BM + 32 * q + lane;
+                    const int t = token_of_lane(half);
                     int rowsum;
                     float scale;
                     token_scale(t, rowsum, scale);
