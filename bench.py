@@ -282,12 +282,13 @@ def extras(peaks):
     # 70B-shaped full decode step: 80 layers, 17.1 GB of packed weights resident
     cfg = S.CONFIGS["70b_decode"]
     res = {}
-    for M in cfg["M"]:
+    # (176 tokens: the batch size of the paper's throughput comparison on the 70B model, Table 3; tensor-core GEMM)
+    for M in list(cfg["M"]) + [176]:
         st = Stack(cfg["layers"], cfg["n_layers"], M)
         ms, kern = time_sequence(st, 5, 3)
         gbs = st.algorithmic_bytes / (ms * 1e-3) / 1e9
         res[f"M{M}"] = {"ms_per_step": round(ms, 3), "GB/s": round(gbs, 1), "frac_hbm_measured": round(gbs / hbm, 3),
-                        "packed_bytes": st.algorithmic_bytes}
+                        "TOPS": round(st.int_ops / (ms * 1e-3) / 1e12, 1), "packed_bytes": st.algorithmic_bytes}
         del st
         torch.cuda.empty_cache()
     out["decode_70b_step"] = res

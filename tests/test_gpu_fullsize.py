@@ -164,10 +164,12 @@ def test_13b_prefill_as_one_sequence_sampled(timing_oracle):
     seq.close()
 
 
-@pytest.mark.parametrize("M", [1, 16])
+@pytest.mark.parametrize("M", [1, 16, 176])
 def test_70b_layer_sampled(timing_oracle, M):
     """The seven projections of 70B-shaped layers (8192 hidden, 8 KV heads, FFN 28672) through one sequence;
-    two layers, so that several matrices of each shape follow each other in the tile stream."""
+    two layers, so that several matrices of each shape follow each other in the tile stream.  176 tokens (the batch
+    size of the paper's throughput comparison, Table 3) run on the table-driven tensor-core GEMM, whose last round
+    of tiles is cut along K here."""
     cfg = S.CONFIGS["70b_decode"]
     layers, meta = build_stack(cfg["layers"], 2, M)
     seq = B.Sequence(layers)
