@@ -256,6 +256,74 @@ int oracle_quantize_acts(const uint16_t *X_bf16, int64_t M, int64_t K,
     return ORACLE_OK;
 }
 
+/* ---------- RMSNorm in front of the activation quantiser ----------
+ *
+ * The paper builds its models from "LLaMA-alike components", RMSNorm among them (Section 2, "LLaMA-alike
+ * Components"), and gives no formula for it: what stands in front of a BitLinear is taken here as the textbook
+ * RMSNorm, x_k = h_k / sqrt(mean_k(h_k^2) + eps_n) * g_k, followed by the activation quantiser above.
+ * Because the normalised values decide integers, the arithmetic is fixed (readings, not the paper's):
+ *   N1  the sum of squares is EXACT and order-free: h_k is a bfloat16, so h_k * h_k is exact in fp32, and the
+ *       terms are added in 2^-64 fixed point like the weights' magnitudes (R2); |h_k| must stay below 2^12;
+ *   N2  mean = (float)(sum / K), the division in double; r = 1.0f / sqrtf(mean + eps_n): fp32 add, IEEE square
+ *       root, IEEE divide;
+ *   N3  x_k = (h_k * r) * g_k: two fp32 multiplications in this order, no fused multiply-add;
+ *   N4  the quantiser then works on the fp32 x_k exactly as on bfloat16 inputs (R4, R5, R6).
+ * Parity pins (tests/test_oracle_pins.py): a hand case, agreement of x with a double-precision evaluation of the
+ * formula and with torch's rms_norm, scale invariance for eps_n = 0, reduction to the plain quantiser.
+ */
+int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, float eps_n, int64_t M, int64_t K,
+                                 int8_t *Xq, float *beta, int32_t *rowsum, float *x_out /* may be NULL: [M][K] */)
+{
+    if (!H_bf16 || !gain || !Xq || !beta || !rowsum || M < 0 || K <= 0 || !(eps_n >= 0.0f))
+        return ORACLE_ERR_ARG;
+    int status = ORACLE_OK;
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        unsigned __int128 total = 0; /* N1 */
+        int bad = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            float h = bf16_to_float(H_bf16[t * K + k]);
+            float sq = h * h; /* exact: two 8-bit significands */
+            uint32_t u;
+            memcpy(&u, &sq, sizeof u);
+            if ((u >> 23) >= 151u) { bad = 1; continue; } /* |h| >= 2^12, infinity or NaN */
+            total += fix64_of_magnitude(u);
+        }
+        if (bad) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            status = ORACLE_ERR_RANGE;
+            continue;
+        }
+        uint64_t hi = (uint64_t)(total >> 64), lo = (uint64_t)total;
+        double sum = ((double)hi * 18446744073709551616.0 + (double)lo) * (1.0 / 18446744073709551616.0);
+        float mean = (float)(sum / (double)K);        /* N2 */
+        float r = 1.0f / sqrtf(mean + eps_n);
+        float amax = 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            float x = (bf16_to_float(H_bf16[t * K + k]) * r) * gain[k]; /* N3 */
+            if (x_out) x_out[t * K + k] = x;
+            float a = fabsf(x);
+            if (a > amax) amax = a;
+        }
+        float b = amax > BETA_FLOOR ? amax : BETA_FLOOR; /* R6 */
+        float s = (float)QB / b;
+        int32_t acc = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            float x = (bf16_to_float(H_bf16[t * K + k]) * r) * gain[k];
+            int q = round_clip(x * s, -QB, QB);
+            Xq[t * K + k] = (int8_t)q;
+            acc += q;
+        }
+        beta[t] = b;
+        rowsum[t] = acc;
+    }
+    return status;
+}
+
 /* ---------- integer matrix product: the plain definition ---------- */
 
 /* acc[t][n] = sum_k Xq[t][k] * T[n][k], exact in int32 (|acc| <= 127*K). */

@@ -56,6 +56,7 @@ class Oracle:
         L.oracle_pack_weights.argtypes = [_p, _i64, _i64, _p]
         L.oracle_unpack_weights.argtypes = [_p, _i64, _i64, _p]
         L.oracle_quantize_acts.argtypes = [_p, _i64, _i64, _p, _p, _p]
+        L.oracle_rmsnorm_quantize_acts.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p, _p, _p, _p]
         L.oracle_matmul_i32.argtypes = [_p, _p, _i64, _i64, _i64, _p]
         L.oracle_dequant.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p]
         L.oracle_forward.argtypes = [_p, ctypes.c_float, _p, _i64, _i64, _i64, _p, _p, _p, _p, _p]
@@ -123,6 +124,22 @@ class Oracle:
         rc = self.lib.oracle_quantize_acts(self._ptr(X), M, K, self._ptr(Xq), self._ptr(beta), self._ptr(rs))
         self._check(rc, "quantize_acts")
         return Xq, beta, rs
+
+    def rmsnorm_quantize_acts(self, H_bf16_bits: np.ndarray, gain: np.ndarray, eps_n: float, return_x: bool = False):
+        """RMSNorm (gain, eps_n) followed by the activation quantiser -> (Xq, beta, rowsum[, x float32 [M,K]])."""
+        H = self._c(H_bf16_bits, np.uint16)
+        g = self._c(gain, np.float32)
+        M, K = H.shape
+        assert g.shape == (K,)
+        Xq = np.empty((M, K), np.int8)
+        beta = np.empty(M, np.float32)
+        rs = np.empty(M, np.int32)
+        x = np.empty((M, K), np.float32) if return_x else None
+        rc = self.lib.oracle_rmsnorm_quantize_acts(self._ptr(H), self._ptr(g), ctypes.c_float(float(eps_n)), M, K,
+                                                   self._ptr(Xq), self._ptr(beta), self._ptr(rs),
+                                                   self._ptr(x) if return_x else None)
+        self._check(rc, "rmsnorm_quantize_acts")
+        return (Xq, beta, rs, x) if return_x else (Xq, beta, rs)
 
     def matmul_i32(self, Xq: np.ndarray, T: np.ndarray) -> np.ndarray:
         Xq = self._c(Xq, np.int8)

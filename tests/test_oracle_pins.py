@@ -273,3 +273,73 @@ def test_timing_build_equals_parity_build(oracle):
     T2, g2 = fast.quantize_weights(W)
     assert g == g2 and np.array_equal(T, T2)
     assert np.array_equal(oracle.forward(T, g, xbits), fast.forward(T, g, xbits))
+
+
+# ---------------------------------------------------------------- RMSNorm in front of the quantiser
+
+def _bf16(x):
+    """bfloat16 bit patterns of x, the low 16 bits of each fp32 dropped (any bfloat16 input will do here)."""
+    return (np.ascontiguousarray(x, np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def test_rmsnorm_quantiser_hand_case(oracle):
+    """h = [3, 4, 0, -12], gain 1, eps_n 0: sum of squares 169, mean 42.25, rms 6.5 exactly; x = h / 6.5;
+    beta = 12 / 6.5; x * 127 / beta = h * 127 / 12 = [31.75, 42.33, 0, -127] -> [32, 42, 0, -127]."""
+    q, beta, rs, x = oracle.rmsnorm_quantize_acts(_bf16([[3, 4, 0, -12]]), np.ones(4, np.float32), 0.0, return_x=True)
+    assert q.tolist() == [[32, 42, 0, -127]] and rs.tolist() == [-53]
+    assert abs(float(beta[0]) - 12 / 6.5) < 2e-7 and np.allclose(x[0], np.array([3, 4, 0, -12]) / 6.5, rtol=3e-7, atol=0)
+    # the gain multiplies after the normalisation: gain [2, 1, 1, 0.5] -> x = [6, 4, 0, -6] / 6.5, beta = 6 / 6.5
+    q, beta, rs = oracle.rmsnorm_quantize_acts(_bf16([[3, 4, 0, -12]]), np.array([2, 1, 1, 0.5], np.float32), 0.0)
+    assert q.tolist() == [[127, 85, 0, -127]] and rs.tolist() == [85]  # 4/6*127 = 84.67 -> 85
+    # eps_n enters under the square root: mean 42.25 + 21.75 = 64 -> r = 1/8
+    _, beta, _, x = oracle.rmsnorm_quantize_acts(_bf16([[3, 4, 0, -12]]), np.ones(4, np.float32), 21.75, return_x=True)
+    assert x.tolist() == [[0.375, 0.5, 0.0, -1.5]] and beta.tolist() == [1.5]
+
+
+def test_rmsnorm_matches_double_precision_and_library(oracle):
+    import torch
+    rng = np.random.default_rng(21)
+    M, K, eps_n = 6, 1536, 1e-5
+    h = rng.standard_normal((M, K)).astype(np.float32)
+    h[:, rng.choice(K, 15, replace=False)] *= 20.0
+    g = (1.0 + 0.1 * rng.standard_normal(K)).astype(np.float32)
+    hb = _bf16(h)
+    hf = bits_to_f32(hb).astype(np.float64)
+    q, beta, rs, x = oracle.rmsnorm_quantize_acts(hb, g, eps_n, return_x=True)
+    x64 = hf / np.sqrt((hf * hf).mean(axis=1, keepdims=True) + eps_n) * g.astype(np.float64)
+    assert np.all(np.abs(x - x64) <= 4 * np.spacing(np.abs(x64).astype(np.float32)))      # a few fp32 roundings
+    lib = torch.nn.functional.rms_norm(torch.from_numpy(hf), (K,), torch.from_numpy(g.astype(np.float64)), eps_n).numpy()
+    assert np.allclose(x, lib, rtol=1e-6, atol=1e-9)
+    b64 = np.abs(x64).max(axis=1)
+    assert np.allclose(beta, b64, rtol=1e-6)
+    scaled = x64 * (127.0 / b64)[:, None]
+    clear = np.abs(scaled - np.floor(scaled) - 0.5) > 1e-3   # away from rounding ties, fp32 and fp64 must agree
+    assert clear.mean() > 0.99 and np.array_equal(q[clear], np.rint(scaled)[clear].astype(np.int8))
+    assert np.array_equal(rs, q.astype(np.int32).sum(axis=1)) and np.abs(q).max() == 127
+
+
+def test_rmsnorm_quantiser_invariants(oracle):
+    rng = np.random.default_rng(22)
+    M, K = 5, 320
+    hb = _bf16(rng.standard_normal((M, K)))
+    g = (1.0 + 0.2 * rng.standard_normal(K)).astype(np.float32)
+    q, beta, rs = oracle.rmsnorm_quantize_acts(hb, g, 0.0)
+    # without eps_n the scale of h cancels exactly (powers of two are exact in every step)
+    q2, beta2, rs2 = oracle.rmsnorm_quantize_acts(_bf16(np.ldexp(bits_to_f32(hb), -5)), g, 0.0)
+    assert np.array_equal(q2, q) and np.array_equal(beta2, beta) and np.array_equal(rs2, rs)
+    # a permutation of the features (of h and the gain together) permutes the codes
+    perm = rng.permutation(K)
+    qp, betap, rsp = oracle.rmsnorm_quantize_acts(hb[:, perm], g[perm], 0.0)
+    assert np.array_equal(qp, q[:, perm]) and np.array_equal(betap, beta) and np.array_equal(rsp, rs)
+    # tokens with mean square exactly 1 and gain 1 are not changed by the normalisation: the plain quantiser
+    ones = _bf16(rng.choice([-1.0, 1.0], size=(M, K)))
+    qa, ba, ra = oracle.rmsnorm_quantize_acts(ones, np.ones(K, np.float32), 0.0)
+    qb, bb, rb = oracle.quantize_acts(ones)
+    assert np.array_equal(qa, qb) and np.array_equal(ba, bb) and np.array_equal(ra, rb)
+    # an all-zero token gives zeros (beta at its floor), with or without eps_n
+    for e in (0.0, 1e-5):
+        qz, bz, rz = oracle.rmsnorm_quantize_acts(_bf16(np.zeros((1, K))), g, e)
+        assert not qz.any() and rz[0] == 0
+    # values of 2^12 and more are refused (their squares leave the exact sum's range)
+    with pytest.raises(ValueError):
+        oracle.rmsnorm_quantize_acts(_bf16([[4096.0] + [0.0] * 15]), np.ones(16, np.float32), 0.0)
