@@ -113,6 +113,20 @@ bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K,
                                          int8_t *Xq, float *beta, int32_t *rowsum, void *stream);
 
 /*
+ * RMSNorm followed by the activation quantiser, in one pass over the token.  Section 2, "LLaMA-alike
+ * Components" names RMSNorm among the parts the models are built from and gives no formula; this is the textbook
+ * one, x_k = h_k / sqrt(mean_k(h_k^2) + norm_eps) * gain_k, with the arithmetic fixed so that the int8 codes are
+ * reproducible bit for bit: exact order-free sum of squares, mean = (float)(sum / K) divided in double,
+ * r = 1 / sqrt(mean + norm_eps) in IEEE fp32, x_k = (h_k * r) * gain_k, then quantised as above.
+ *   H        in   bf16 [M, K] row-major; finite, |h| < 4096 (a token that breaks this gets beta = NaN)
+ *   gain     in   fp32 [K], 16-byte aligned
+ *   norm_eps      >= 0
+ *   Xq, beta, rowsum   out, as for bitlinear_quantize_acts
+ */
+bitlinear_status bitlinear_rmsnorm_quantize_acts(const void *H, const float *gain, float norm_eps, int64_t M, int64_t K,
+                                                 int8_t *Xq, float *beta, int32_t *rowsum, void *stream);
+
+/*
  * The BitLinear forward: activation quantisation, ternary x int8 matmul with exact int32 accumulation,
  * dequantisation to bf16 (Section 2; no bias, "removes all biases").
  *   packed, gamma   in   from bitlinear_quantize_weights (gamma stays on the device)
@@ -125,6 +139,14 @@ bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K,
 bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X,
                                    int64_t M, int64_t K, int64_t N, void *Y,
                                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same forward with the RMSNorm of bitlinear_rmsnorm_quantize_acts in front of the activation quantiser (one
+ * launch normalises and quantises; the matmul and its epilogue are unchanged): Y = BitLinear(RMSNorm(H)).
+ */
+bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamma, const void *H, const float *gain,
+                                           float norm_eps, int64_t M, int64_t K, int64_t N, void *Y,
+                                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * The same forward for callers that cannot give it a workspace.  (The paper has no counterpart: this is a

@@ -25,7 +25,9 @@ EXPORTS = [
     "bitlinear_workspace_bytes",
     "bitlinear_quantize_weights",
     "bitlinear_quantize_acts",
+    "bitlinear_rmsnorm_quantize_acts",
     "bitlinear_forward",
+    "bitlinear_forward_rmsnorm",
     "bitlinear_forward_static",
     "bitlinear_sequence_workspace_bytes",
     "bitlinear_sequence_create",
@@ -79,6 +81,8 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_quantize_weights.argtypes = [vp, i64, i64, cf, vp, vp, vp]
     L.bitlinear_quantize_acts.argtypes = [vp, i64, i64, vp, vp, vp, vp]
     L.bitlinear_forward.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
+    L.bitlinear_rmsnorm_quantize_acts.argtypes = [vp, vp, cf, i64, i64, vp, vp, vp, vp]
+    L.bitlinear_forward_rmsnorm.argtypes = [vp, vp, vp, vp, cf, i64, i64, i64, vp, vp, sz, vp]
     L.bitlinear_forward_static.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.bitlinear_sequence_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci]
     L.bitlinear_sequence_workspace_bytes.restype = sz
@@ -150,6 +154,32 @@ def quantize_acts(X: torch.Tensor, stream=None):
     st = load_library().bitlinear_quantize_acts(_ptr(X), M, K, _ptr(Xq), _ptr(beta), _ptr(rowsum), _stream(stream))
     _check(st, "bitlinear_quantize_acts")
     return Xq, beta, rowsum
+
+
+def rmsnorm_quantize_acts(H: torch.Tensor, gain: torch.Tensor, norm_eps: float, stream=None):
+    """bitlinear_rmsnorm_quantize_acts: bf16 [M, K], fp32 gain [K] -> (Xq int8 [M, K], beta fp32 [M], rowsum int32 [M])."""
+    M, K = H.shape
+    Xq = torch.empty((M, K), dtype=torch.int8, device=H.device)
+    beta = torch.empty(max(M, 1), dtype=torch.float32, device=H.device)[:M]
+    rowsum = torch.empty(max(M, 1), dtype=torch.int32, device=H.device)[:M]
+    st = load_library().bitlinear_rmsnorm_quantize_acts(_ptr(H), _ptr(gain), float(norm_eps), M, K, _ptr(Xq), _ptr(beta),
+                                                        _ptr(rowsum), _stream(stream))
+    _check(st, "bitlinear_rmsnorm_quantize_acts")
+    return Xq, beta, rowsum
+
+
+def forward_rmsnorm(packed: torch.Tensor, gamma: torch.Tensor, H: torch.Tensor, gain: torch.Tensor, norm_eps: float, N: int,
+                    Y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """bitlinear_forward_rmsnorm: BitLinear(RMSNorm(H)), bf16 [M, K] -> bf16 [M, N]."""
+    M, K = H.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=H.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, H.device)
+    st = load_library().bitlinear_forward_rmsnorm(_ptr(packed), _ptr(gamma), _ptr(H), _ptr(gain), float(norm_eps), M, K, N,
+                                                  _ptr(Y), _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "bitlinear_forward_rmsnorm")
+    return Y
 
 
 def forward(packed: torch.Tensor, gamma: torch.Tensor, X: torch.Tensor, N: int, Y: torch.Tensor | None = None,

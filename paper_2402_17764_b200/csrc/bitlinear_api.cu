@@ -134,6 +134,8 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.token_begin = 0;
     e.out_i32 = out_i32;
     e.xq_tiled = 0;
+    e.gain = nullptr;
+    e.norm_eps = 0.0f;
 }
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
@@ -220,13 +222,16 @@ bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
-bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K, int8_t *Xq, float *beta,
-                                         int32_t *rowsum, void *stream)
+namespace {
+// gain == null: the plain quantiser
+bitlinear_status quantize_acts_rows(const void *X, const float *gain, float norm_eps, int64_t M, int64_t K, int8_t *Xq,
+                                    float *beta, int32_t *rowsum, void *stream)
 {
     if (M > 0 && (!X || !Xq || !beta || !rowsum)) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, 16, K);
     if (st != BITLINEAR_OK) return st;
     if (!aligned(X, 16) || !aligned(Xq, 16) || !aligned(beta, 4) || !aligned(rowsum, 4)) return BITLINEAR_ERR_ALIGN;
+    if (gain && !aligned(gain, 16)) return BITLINEAR_ERR_ALIGN;
     if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
     if (M == 0) return BITLINEAR_OK;
     InlineTable inl{};
@@ -237,12 +242,52 @@ bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K, in
     e.rowsum = rowsum;
     e.M = (int)M;
     e.K = (int)K;
+    e.gain = gain;
+    e.norm_eps = norm_eps;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, (cudaStream_t)stream);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+} // namespace
+
+bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K, int8_t *Xq, float *beta,
+                                         int32_t *rowsum, void *stream)
+{
+    return quantize_acts_rows(X, nullptr, 0.0f, M, K, Xq, beta, rowsum, stream);
+}
+
+bitlinear_status bitlinear_rmsnorm_quantize_acts(const void *H, const float *gain, float norm_eps, int64_t M, int64_t K,
+                                                 int8_t *Xq, float *beta, int32_t *rowsum, void *stream)
+{
+    if (!gain || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
+    return quantize_acts_rows(H, gain, norm_eps, M, K, Xq, beta, rowsum, stream);
+}
+
+namespace {
+bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const float *gain, float norm_eps,
+                              int64_t M, int64_t K, int64_t N, void *Y, void *workspace, size_t workspace_bytes,
+                              void *stream);
 }
 
 bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
                                    int64_t N, void *Y, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return forward_impl(packed, gamma, X, nullptr, 0.0f, M, K, N, Y, workspace, workspace_bytes, stream);
+}
+
+bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamma, const void *H, const float *gain,
+                                           float norm_eps, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
+                                           size_t workspace_bytes, void *stream)
+{
+    if (!gain || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
+    if (!aligned(gain, 16)) return BITLINEAR_ERR_ALIGN;
+    return forward_impl(packed, gamma, H, gain, norm_eps, M, K, N, Y, workspace, workspace_bytes, stream);
+}
+
+namespace {
+// gain == null: no normalisation in front of the quantiser
+bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const float *gain, float norm_eps,
+                              int64_t M, int64_t K, int64_t N, void *Y, void *workspace, size_t workspace_bytes,
+                              void *stream)
 {
     if (!packed || !gamma || !workspace || (M > 0 && (!X || !Y))) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, N, K);
@@ -258,6 +303,8 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L);
     const bool tc = use_tcgen05_for(M);
     inl.e[0].xq_tiled = tc ? 0 : 1;
+    inl.e[0].gain = gain;
+    inl.e[0].norm_eps = norm_eps;
     // quantise the tokens; the same launch clears the header and the scratch of the kernel that follows, if it uses it
     const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
@@ -267,6 +314,7 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
     return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M,
                       split ? ws + L.acc32 : nullptr, (cudaStream_t)stream);
 }
+} // namespace
 
 bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
                                       int32_t *acc, int path, void *workspace, size_t workspace_bytes, void *stream)

@@ -56,6 +56,8 @@ struct DecodeEntry {
     int token_begin;       // first token of this entry in the batched quantiser's grid
     int out_i32;           // 1: write raw int32 accumulators instead of bf16
     int xq_tiled;          // layout of Xq (the streaming kernel reads tiles, the tensor-core GEMM rows)
+    const float *gain;     // null, or [K] fp32: X is normalised first (RMSNorm with this gain) and then quantised
+    float norm_eps;        // the RMSNorm's epsilon (added to the mean square)
 };
 
 constexpr int kInlineEntries = 4;

@@ -6,39 +6,12 @@
 //      to finish turns it into gamma,
 //   3. ternarise with round-half-to-even and write the interleaved 2-bit tiles.
 // HBM-bound: two reads of the fp32 matrix (8 B per weight) and 0.25 B written per weight.
+#include "exact_sum.cuh"
 #include "internal.cuh"
 
 namespace bitlinear {
 
 namespace {
-
-struct U128 {
-    unsigned long long lo, hi;
-};
-
-__device__ __forceinline__ void add128(U128 &a, unsigned long long lo, unsigned long long hi)
-{
-    a.lo += lo;
-    a.hi += hi + (a.lo < lo ? 1ull : 0ull);
-}
-
-// floor(|v| * 2^64) for an fp32 magnitude given as bits (sign cleared, exponent < 151).
-__device__ __forceinline__ void fix64(uint32_t mag, unsigned long long &lo, unsigned long long &hi)
-{
-    uint32_t e = mag >> 23;
-    uint32_t frac = mag & 0x7FFFFFu;
-    unsigned long long sig = e ? (frac | 0x800000u) : frac;
-    int shift = (int)(e ? e : 1u) - 86; // value = sig * 2^shift
-    if (shift >= 0) {
-        if (shift == 0) { lo = sig; hi = 0; }
-        else if (shift < 64) { lo = sig << shift; hi = sig >> (64 - shift); }
-        else { lo = 0; hi = sig << (shift - 64); }
-    } else {
-        int s = -shift;
-        lo = (s < 24) ? (sig >> s) : 0ull;
-        hi = 0;
-    }
-}
 
 // scratch words (unsigned long long): [0] sum.lo  [1] sum.hi  [2] blocks done  [3] range violation flag
 __global__ void __launch_bounds__(256) absmean_kernel(const float4 *__restrict__ W4, size_t n_vec,

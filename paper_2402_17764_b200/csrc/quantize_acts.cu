@@ -9,6 +9,14 @@
 // ([column tile of 64][token][64 bytes], zero beyond K, for the weight-streaming kernel, which fetches the
 // activations of a run of column tiles with one bulk copy).
 // HBM-bound: 2 B read + 1 B written per element.
+//
+// With a gain vector the token is normalised first (RMSNorm, one of the "LLaMA-alike components" of Section 2):
+// x_k = h_k / sqrt(mean(h^2) + eps) * g_k, then quantised as above.  The normalised values decide integers, so
+// the arithmetic is fixed: the sum of squares is exact and order-free (h is bfloat16, so h * h is exact in fp32;
+// the terms are added in 2^-64 fixed point), mean = (float)(sum / K) with the division in double,
+// r = 1 / sqrt(mean + eps) with IEEE fp32 add, square root and divide, x_k = (h_k * r) * g_k with two fp32
+// multiplications.  |h_k| must be finite and below 2^12; a token that breaks this gets beta = NaN.
+#include "exact_sum.cuh"
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -61,6 +69,8 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
 {
     __shared__ uint32_t s_max[kThreads / 32];
     __shared__ int s_sum[kThreads / 32];
+    __shared__ U128 s_sq[kThreads / 32];
+    __shared__ uint32_t s_bad[kThreads / 32];
 
     // The matmul that follows may be launched early: it streams weights until it needs what this kernel writes.
     ptx::griddep_launch_dependents();
@@ -95,6 +105,131 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
     };
 
     uint4 cache[kCache];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (e.gain) {
+        // ---- RMSNorm, then the quantiser on the fp32 values (see the head of this file)
+        const float4 *gain4 = reinterpret_cast<const float4 *>(e.gain);
+        U128 sq = {0ull, 0ull};
+        uint32_t bad = 0;
+        auto add_squares = [&](const uint4 &v) {
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    const float h = __uint_as_float(half ? (w[i] & 0xFFFF0000u) : (w[i] << 16));
+                    const uint32_t mag = __float_as_uint(__fmul_rn(h, h)); // exact, and never negative
+                    if ((mag >> 23) >= 151u) {
+                        bad = 1;
+                    } else {
+                        unsigned long long lo, hi;
+                        fix64(mag, lo, hi);
+                        add128(sq, lo, hi);
+                    }
+                }
+            }
+        };
+#pragma unroll
+        for (int c = 0; c < kCache; ++c) {
+            const int i = threadIdx.x + c * kThreads;
+            if (i < n_vec) {
+                cache[c] = __ldg(row + i);
+                add_squares(cache[c]);
+            }
+        }
+        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) add_squares(__ldg(row + i));
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const unsigned long long lo = __shfl_xor_sync(0xffffffffu, sq.lo, off);
+            const unsigned long long hi = __shfl_xor_sync(0xffffffffu, sq.hi, off);
+            add128(sq, lo, hi);
+            bad |= __shfl_xor_sync(0xffffffffu, bad, off);
+        }
+        if (lane == 0) {
+            s_sq[warp] = sq;
+            s_bad[warp] = bad;
+        }
+        __syncthreads();
+        U128 tot = {0ull, 0ull};
+        bad = 0;
+#pragma unroll
+        for (int w = 0; w < kThreads / 32; ++w) { // every thread forms the same total
+            add128(tot, s_sq[w].lo, s_sq[w].hi);
+            bad |= s_bad[w];
+        }
+        const float mean = exact_mean(tot, (double)K);
+        const float r = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(mean, e.norm_eps)));
+
+        // the eight normalised values of vector i
+        auto normalised = [&](const uint4 &v, int i, float (&x)[8]) {
+            const float4 g0 = __ldg(gain4 + 2 * i), g1 = __ldg(gain4 + 2 * i + 1);
+            const float g[8] = {g0.x, g0.y, g0.z, g0.w, g1.x, g1.y, g1.z, g1.w};
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                x[2 * j] = __fmul_rn(__fmul_rn(__uint_as_float(w[j] << 16), r), g[2 * j]);
+                x[2 * j + 1] = __fmul_rn(__fmul_rn(__uint_as_float(w[j] & 0xFFFF0000u), r), g[2 * j + 1]);
+            }
+        };
+        uint32_t mx = 0; // |x| as an unsigned integer is monotone in the magnitude
+        auto absmax8 = [&](const uint4 &v, int i) {
+            float x[8];
+            normalised(v, i, x);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mx = max(mx, __float_as_uint(x[j]) & 0x7FFFFFFFu);
+        };
+#pragma unroll
+        for (int c = 0; c < kCache; ++c) {
+            const int i = threadIdx.x + c * kThreads;
+            if (i < n_vec) absmax8(cache[c], i);
+        }
+        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) absmax8(__ldg(row + i), i);
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        if (lane == 0) s_max[warp] = mx;
+        __syncthreads();
+        mx = s_max[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) mx = max(mx, s_max[w]);
+        const float b = fmaxf(__uint_as_float(mx), kBetaFloor);
+        const float s = __fdiv_rn((float)kQb, b);
+
+        int sum = 0;
+        auto quantise8 = [&](const uint4 &v, int i) {
+            float x[8];
+            normalised(v, i, x);
+            int q[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) q[j] = max(-kQb, min(kQb, __float2int_rn(__fmul_rn(x[j], s))));
+            uint2 o;
+            o.x = (uint32_t)(q[0] & 0xFF) | ((uint32_t)(q[1] & 0xFF) << 8) | ((uint32_t)(q[2] & 0xFF) << 16) |
+                  ((uint32_t)(q[3] & 0xFF) << 24);
+            o.y = (uint32_t)(q[4] & 0xFF) | ((uint32_t)(q[5] & 0xFF) << 8) | ((uint32_t)(q[6] & 0xFF) << 16) |
+                  ((uint32_t)(q[7] & 0xFF) << 24);
+            out_at(i) = o;
+            sum += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+        };
+#pragma unroll
+        for (int c = 0; c < kCache; ++c) {
+            const int i = threadIdx.x + c * kThreads;
+            if (i < n_vec) quantise8(cache[c], i);
+        }
+        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) quantise8(__ldg(row + i), i);
+        if (tiled) // the last column tile is filled up with zeros
+            for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += kThreads) out_at(i) = make_uint2(0u, 0u);
+        sum = __reduce_add_sync(0xffffffffu, sum);
+        if (lane == 0) s_sum[warp] = sum;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int total = 0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) total += s_sum[w];
+            e.beta[t] = bad ? __int_as_float(0x7FC00000) : b;
+            e.rowsum[t] = total;
+        }
+        return;
+    }
+
     uint32_t m = 0;
 #pragma unroll
     for (int c = 0; c < kCache; ++c) {
@@ -108,7 +243,6 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
         m = absmax_bits(m, __ldg(row + i));
 
     m = __reduce_max_sync(0xffffffffu, m);
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (lane == 0) s_max[warp] = m;
     __syncthreads();
     m = s_max[0];
