@@ -279,6 +279,27 @@ def extras(peaks):
             del X, Y, ws
     out["prefill_13b_shapes"] = res
 
+    # RMSNorm fused into the activation quantiser (HBM-bound: 2 B read + 1 B written per element; inputs larger
+    # than L2) next to the plain quantiser, and the forward with it at the 13B-shaped up projection
+    res = {}
+    for M, K in [(16384, 8192), (32768, 5120)]:
+        H = S.activations(M, K, 0, device="cuda")
+        gain = torch.ones(K, dtype=torch.float32, device="cuda")
+        Xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        beta = torch.empty(M, dtype=torch.float32, device="cuda")
+        rs = torch.empty(M, dtype=torch.int32, device="cuda")
+        L = B.load_library()
+        stream = torch.cuda.current_stream().cuda_stream
+        ms_n = time_forward_calls(lambda: L.bitlinear_rmsnorm_quantize_acts(H.data_ptr(), gain.data_ptr(), 1e-5, M, K,
+                                                                            Xq.data_ptr(), beta.data_ptr(), rs.data_ptr(), stream), 10)
+        ms_p = time_forward_calls(lambda: L.bitlinear_quantize_acts(H.data_ptr(), M, K, Xq.data_ptr(), beta.data_ptr(),
+                                                                    rs.data_ptr(), stream), 10)
+        res[f"M{M}_K{K}"] = {"rmsnorm_quantiser_ms": round(ms_n, 4), "GB/s": round(3.0 * M * K / ms_n / 1e6, 1),
+                             "frac_hbm_measured": round(3.0 * M * K / ms_n / 1e6 / hbm, 3),
+                             "plain_quantiser_ms": round(ms_p, 4), "plain_GB/s": round(3.0 * M * K / ms_p / 1e6, 1)}
+        del H, Xq
+    out["rmsnorm_quantiser"] = res
+
     # 70B-shaped full decode step: 80 layers, 17.1 GB of packed weights resident
     cfg = S.CONFIGS["70b_decode"]
     res = {}

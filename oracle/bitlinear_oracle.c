@@ -262,10 +262,15 @@ int oracle_quantize_acts(const uint16_t *X_bf16, int64_t M, int64_t K,
  * Components"), and gives no formula for it: what stands in front of a BitLinear is taken here as the textbook
  * RMSNorm, x_k = h_k / sqrt(mean_k(h_k^2) + eps_n) * g_k, followed by the activation quantiser above.
  * Because the normalised values decide integers, the arithmetic is fixed (readings, not the paper's):
- *   N1  the sum of squares is EXACT and order-free: h_k is a bfloat16, so h_k * h_k is exact in fp32, and the
- *       terms are added in 2^-64 fixed point like the weights' magnitudes (R2); |h_k| must stay below 2^12;
- *   N2  mean = (float)(sum / K), the division in double; r = 1.0f / sqrtf(mean + eps_n): fp32 add, IEEE square
- *       root, IEEE divide;
+ *   N1  the sum of squares is EXACT integer arithmetic, hence order-free: with E the exponent field of the
+ *       token's largest |h_k| (a bfloat16: 8-bit exponent field e, 8-bit significand m with its hidden bit; e = 0
+ *       counts as 1 without hidden bit), h_k^2 = m_k^2 * 4^(e_k - 134), and the token's sum is
+ *           S = sum_k floor( m_k^2 * 2^30 / 4^(E - e_k) )        (terms with E - e_k > 23 are 0)
+ *       in units of 4^(E - 134) * 2^-30: every term is below 2^46, so S < 2^63 for K <= 2^17.  What a term loses is
+ *       below 2^-44 of the largest square, far below fp32 resolution, and the sum does not depend on the scale
+ *       of h.  Infinities and NaNs are refused;
+ *   N2  mean = (float)( (double)S / (double)K * 2^(2E - 298) ) (the conversion of S rounds to nearest even, the power
+ *       of two is exact); r = 1.0f / sqrtf(mean + eps_n): fp32 add, IEEE square root, IEEE divide;
  *   N3  x_k = (h_k * r) * g_k: two fp32 multiplications in this order, no fused multiply-add;
  *   N4  the quantiser then works on the fp32 x_k exactly as on bfloat16 inputs (R4, R5, R6).
  * Parity pins (tests/test_oracle_pins.py): a hand case, agreement of x with a double-precision evaluation of the
@@ -281,15 +286,14 @@ int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, floa
 #pragma omp parallel for
 #endif
     for (int64_t t = 0; t < M; ++t) {
-        unsigned __int128 total = 0; /* N1 */
+        /* N1: exponent field of the largest magnitude, then the integer sum */
+        unsigned E = 0;
         int bad = 0;
         for (int64_t k = 0; k < K; ++k) {
-            float h = bf16_to_float(H_bf16[t * K + k]);
-            float sq = h * h; /* exact: two 8-bit significands */
-            uint32_t u;
-            memcpy(&u, &sq, sizeof u);
-            if ((u >> 23) >= 151u) { bad = 1; continue; } /* |h| >= 2^12, infinity or NaN */
-            total += fix64_of_magnitude(u);
+            unsigned e = (H_bf16[t * K + k] >> 7) & 0xFFu;
+            if (e == 255u) bad = 1;
+            if (e < 1u) e = 1u;
+            if (e > E) E = e;
         }
         if (bad) {
 #ifdef _OPENMP
@@ -298,9 +302,16 @@ int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, floa
             status = ORACLE_ERR_RANGE;
             continue;
         }
-        uint64_t hi = (uint64_t)(total >> 64), lo = (uint64_t)total;
-        double sum = ((double)hi * 18446744073709551616.0 + (double)lo) * (1.0 / 18446744073709551616.0);
-        float mean = (float)(sum / (double)K);        /* N2 */
+        uint64_t S = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            unsigned bits = H_bf16[t * K + k];
+            unsigned e = (bits >> 7) & 0xFFu;
+            uint64_t m = bits & 0x7Fu;
+            if (e) m |= 0x80u; else e = 1u;
+            unsigned twice = 2u * (E - e);
+            if (twice <= 46u) S += ((m * m) << 30) >> twice;
+        }
+        float mean = (float)(ldexp((double)S / (double)K, 2 * (int)E - 298)); /* N2 */
         float r = 1.0f / sqrtf(mean + eps_n);
         float amax = 0.0f;
         for (int64_t k = 0; k < K; ++k) {

@@ -1,6 +1,6 @@
 // Order-free exact sums of fp32 magnitudes: each term is floor(|v| * 2^64) as an unsigned 128-bit integer, so the
-// sum does not depend on the order in which threads, warps and blocks add (the weight scale gamma, Eq. 3, and the
-// sum of squares of the RMSNorm in front of the activation quantiser are formed this way).
+// sum does not depend on the order in which threads, warps and blocks add (the weight scale gamma, Eq. 3, is formed
+// this way).
 #pragma once
 
 #include <cstdint>
@@ -33,14 +33,6 @@ __device__ __forceinline__ void fix64(uint32_t mag, unsigned long long &lo, unsi
         lo = (s < 24) ? (sig >> s) : 0ull;
         hi = 0;
     }
-}
-
-// sum * 2^-64 / count, rounded once to fp32 from the double quotient
-__device__ __forceinline__ float exact_mean(const U128 &sum, double count)
-{
-    const double v = __dmul_rn(__dadd_rn(__dmul_rn(__ull2double_rn(sum.hi), 18446744073709551616.0), __ull2double_rn(sum.lo)),
-                               1.0 / 18446744073709551616.0);
-    return __double2float_rn(__ddiv_rn(v, count));
 }
 
 } // namespace bitlinear

@@ -12,11 +12,12 @@
 //
 // With a gain vector the token is normalised first (RMSNorm, one of the "LLaMA-alike components" of Section 2):
 // x_k = h_k / sqrt(mean(h^2) + eps) * g_k, then quantised as above.  The normalised values decide integers, so
-// the arithmetic is fixed: the sum of squares is exact and order-free (h is bfloat16, so h * h is exact in fp32;
-// the terms are added in 2^-64 fixed point), mean = (float)(sum / K) with the division in double,
+// the arithmetic is fixed.  The sum of squares is an exact integer, hence order-free: with E the exponent field of the
+// token's largest |h| (bfloat16: exponent field e, 8-bit significand m with its hidden bit; e = 0 counts as 1 without
+// hidden bit), S = sum_k floor(m_k^2 * 2^30 / 4^(E - e_k)) < 2^63 in 64-bit arithmetic (terms more than 23 binades
+// below the largest add nothing), sum h^2 = S * 2^(2E - 298).  Then mean = (float)((double)S / K * 2^(2E - 298)),
 // r = 1 / sqrt(mean + eps) with IEEE fp32 add, square root and divide, x_k = (h_k * r) * g_k with two fp32
-// multiplications.  |h_k| must be finite and below 2^12; a token that breaks this gets beta = NaN.
-#include "exact_sum.cuh"
+// multiplications.  A token with an infinity or a NaN gets beta = NaN.
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -69,8 +70,7 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
 {
     __shared__ uint32_t s_max[kThreads / 32];
     __shared__ int s_sum[kThreads / 32];
-    __shared__ U128 s_sq[kThreads / 32];
-    __shared__ uint32_t s_bad[kThreads / 32];
+    __shared__ unsigned long long s_sq[kThreads / 32];
 
     // The matmul that follows may be launched early: it streams weights until it needs what this kernel writes.
     ptx::griddep_launch_dependents();
@@ -110,55 +110,59 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
     if (e.gain) {
         // ---- RMSNorm, then the quantiser on the fp32 values (see the head of this file)
         const float4 *gain4 = reinterpret_cast<const float4 *>(e.gain);
-        U128 sq = {0ull, 0ull};
-        uint32_t bad = 0;
+        // largest magnitude of the token: |bf16| as a 15-bit integer is monotone, its upper 8 bits are the exponent
+        uint32_t top = 0;
+#pragma unroll
+        for (int c = 0; c < kCache; ++c) {
+            const int i = threadIdx.x + c * kThreads;
+            if (i < n_vec) {
+                cache[c] = __ldg(row + i);
+                top = absmax_bits(top, cache[c]);
+            }
+        }
+        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) top = absmax_bits(top, __ldg(row + i));
+        top = __reduce_max_sync(0xffffffffu, top);
+        if (lane == 0) s_max[warp] = top;
+        __syncthreads();
+        top = s_max[0];
+#pragma unroll
+        for (int w = 1; w < kThreads / 32; ++w) top = max(top, s_max[w]);
+        __syncthreads(); // s_max is used again below
+        const bool bad = (top >> 7) == 255u; // an infinity or a NaN somewhere in the token
+        const int E = max((int)(top >> 7), 1);
+
+        unsigned long long sq = 0;
         auto add_squares = [&](const uint4 &v) {
             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
-                    const float h = __uint_as_float(half ? (w[i] & 0xFFFF0000u) : (w[i] << 16));
-                    const uint32_t mag = __float_as_uint(__fmul_rn(h, h)); // exact, and never negative
-                    if ((mag >> 23) >= 151u) {
-                        bad = 1;
-                    } else {
-                        unsigned long long lo, hi;
-                        fix64(mag, lo, hi);
-                        add128(sq, lo, hi);
-                    }
+                    const uint32_t bits = half ? (w[i] >> 16) : (w[i] & 0xFFFFu);
+                    int e = (int)((bits >> 7) & 0xFFu);
+                    uint32_t m = bits & 0x7Fu;
+                    if (e) m |= 0x80u; else e = 1;
+                    const int twice = 2 * (E - e);
+                    if (twice <= 46) sq += ((unsigned long long)(m * m) << 30) >> twice;
                 }
             }
         };
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
             const int i = threadIdx.x + c * kThreads;
-            if (i < n_vec) {
-                cache[c] = __ldg(row + i);
-                add_squares(cache[c]);
-            }
+            if (i < n_vec) add_squares(cache[c]);
         }
         for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) add_squares(__ldg(row + i));
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) {
-            const unsigned long long lo = __shfl_xor_sync(0xffffffffu, sq.lo, off);
-            const unsigned long long hi = __shfl_xor_sync(0xffffffffu, sq.hi, off);
-            add128(sq, lo, hi);
-            bad |= __shfl_xor_sync(0xffffffffu, bad, off);
-        }
-        if (lane == 0) {
-            s_sq[warp] = sq;
-            s_bad[warp] = bad;
-        }
+        for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
+        if (lane == 0) s_sq[warp] = sq;
         __syncthreads();
-        U128 tot = {0ull, 0ull};
-        bad = 0;
+        unsigned long long tot = 0;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) { // every thread forms the same total
-            add128(tot, s_sq[w].lo, s_sq[w].hi);
-            bad |= s_bad[w];
-        }
-        const float mean = exact_mean(tot, (double)K);
+        for (int w = 0; w < kThreads / 32; ++w) tot += s_sq[w]; // every thread forms the same total
+        // mean = S / K * 2^(2E - 298): the power of two as a double built from its exponent field
+        const double pow2 = __longlong_as_double((long long)(2 * E - 298 + 1023) << 52);
+        const float mean = __double2float_rn(__dmul_rn(__ddiv_rn(__ull2double_rn(tot), (double)K), pow2));
         const float r = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(mean, e.norm_eps)));
 
         // the eight normalised values of vector i

@@ -50,7 +50,7 @@ def test_rmsnorm_quantiser_bit_exact(M, K, seed, frac, scale, eps_n):
 
 
 def test_rmsnorm_quantiser_special_tokens():
-    """An all-zero token (beta at its floor, codes 0) next to ordinary ones; a token with a value of 4096 is flagged
+    """An all-zero token (beta at its floor, codes 0) next to ordinary ones; a token with an infinity is flagged
     with beta = NaN; unit gain and eps_n = 0 on a token of +-1 leave the plain quantiser's result."""
     K = 320
     H = S.activations(4, K, 9)
@@ -61,7 +61,7 @@ def test_rmsnorm_quantiser_special_tokens():
     assert np.array_equal(Xq.cpu().numpy(), q_ref) and not Xq[1].any()
     assert np.array_equal(beta.cpu().numpy().view(np.uint32), b_ref.view(np.uint32))
     assert np.array_equal(rowsum.cpu().numpy(), s_ref)
-    H[2, 5] = 4096.0
+    H[2, 5] = float("inf")
     _, beta, _ = B.rmsnorm_quantize_acts(H.cuda(), g.cuda(), 1e-5)
     assert bool(torch.isnan(beta[2])) and not bool(torch.isnan(beta[[0, 1, 3]]).any())
     ones = (torch.randint(0, 2, (3, K), generator=torch.Generator().manual_seed(3)) * 2 - 1).to(torch.bfloat16)

@@ -340,6 +340,12 @@ def test_rmsnorm_quantiser_invariants(oracle):
     for e in (0.0, 1e-5):
         qz, bz, rz = oracle.rmsnorm_quantize_acts(_bf16(np.zeros((1, K))), g, e)
         assert not qz.any() and rz[0] == 0
-    # values of 2^12 and more are refused (their squares leave the exact sum's range)
-    with pytest.raises(ValueError):
-        oracle.rmsnorm_quantize_acts(_bf16([[4096.0] + [0.0] * 15]), np.ones(16, np.float32), 0.0)
+    # a huge spread inside a token: what lies more than 23 binades below the largest value adds nothing
+    big = np.zeros((1, 16), np.float32)
+    big[0, 0], big[0, 1] = 2.0 ** 30, 2.0 ** -10
+    qs, bs, _ = oracle.rmsnorm_quantize_acts(_bf16(big), np.ones(16, np.float32), 0.0)
+    assert qs[0, 0] == 127 and not qs[0, 1:].any() and bs[0] == 4.0   # x_0 = 2^30 / sqrt(2^60 / 16) = 4
+    # infinities and NaNs are refused
+    for v in (np.inf, np.nan):
+        with pytest.raises(ValueError):
+            oracle.rmsnorm_quantize_acts(_bf16([[v] + [0.0] * 15]), np.ones(16, np.float32), 0.0)
