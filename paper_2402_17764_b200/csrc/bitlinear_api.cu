@@ -244,7 +244,7 @@ bitlinear_status quantize_acts_rows(const void *X, const float *gain, float norm
     e.K = (int)K;
     e.gain = gain;
     e.norm_eps = norm_eps;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, (cudaStream_t)stream);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, gain != nullptr, (cudaStream_t)stream);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 } // namespace
@@ -309,7 +309,7 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (cudaStream_t)stream);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, gain != nullptr, (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M,
                       split ? ws + L.acc32 : nullptr, (cudaStream_t)stream);
@@ -343,7 +343,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                              : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, s);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, false, s);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     if (tc) {
         inl.e[0].Xq = const_cast<int8_t *>(Xq); // the GEMM reads the caller's rows in place
@@ -582,7 +582,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
     if (!seq || stage < 0 || stage > 2) return BITLINEAR_ERR_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     if (stage != 2 &&
-        launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes, s) !=
+        launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes, false, s) !=
             cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {

@@ -26,7 +26,7 @@ namespace bitlinear {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kCache = 8; // 16-byte vectors kept in registers per thread (8 * 8 * 256 = 16384 elements)
+constexpr int kCache = 4; // 16-byte vectors kept in registers per thread (4 * 8 * 256 = 8192 elements)
 
 __device__ __forceinline__ uint32_t absmax_bits(uint32_t m, const uint4 &v)
 {
@@ -64,7 +64,9 @@ __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
     return q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
 }
 
-__global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
+// kNorm: entries may carry a gain vector (RMSNorm in front); the plain form is compiled without that branch.
+template <bool kNorm>
+__global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
                                                                  const DecodeEntry *__restrict__ table, int n_entries,
                                                                  int total_tokens, uint4 *zero_ptr, size_t zero_vecs)
 {
@@ -107,7 +109,7 @@ __global__ void __launch_bounds__(kThreads) quantize_acts_kernel(const __grid_co
     uint4 cache[kCache];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    if (e.gain) {
+    if (kNorm && e.gain) {
         // ---- RMSNorm, then the quantiser on the fp32 values (see the head of this file)
         const float4 *gain4 = reinterpret_cast<const float4 *>(e.gain);
         // largest magnitude of the token: |bf16| as a 15-bit integer is monotone, its upper 8 bits are the exponent
@@ -307,7 +309,7 @@ cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *t
 }
 
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
-                                 void *zero_ptr, size_t zero_bytes, cudaStream_t stream)
+                                 void *zero_ptr, size_t zero_bytes, bool with_norm, cudaStream_t stream)
 {
     const size_t zero_vecs = zero_bytes / 16;
     int zero_blocks = 0;
@@ -319,8 +321,12 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     }
     const int grid = total_tokens + zero_blocks;
     if (grid == 0) return cudaSuccess;
-    quantize_acts_kernel<<<grid, kThreads, 0, stream>>>(inl, table, n_entries, total_tokens,
-                                                        reinterpret_cast<uint4 *>(zero_ptr), zero_vecs);
+    if (with_norm)
+        quantize_acts_kernel<true><<<grid, kThreads, 0, stream>>>(inl, table, n_entries, total_tokens,
+                                                                  reinterpret_cast<uint4 *>(zero_ptr), zero_vecs);
+    else
+        quantize_acts_kernel<false><<<grid, kThreads, 0, stream>>>(inl, table, n_entries, total_tokens,
+                                                                   reinterpret_cast<uint4 *>(zero_ptr), zero_vecs);
     return cudaGetLastError();
 }
 
