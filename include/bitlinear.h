@@ -117,8 +117,8 @@ bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K,
  * Components" names RMSNorm among the parts the models are built from and gives no formula; this is the textbook
  * one, x_k = h_k / sqrt(mean_k(h_k^2) + norm_eps) * gain_k, with the arithmetic fixed so that the int8 codes are
  * reproducible bit for bit: exact order-free sum of squares, mean = (float)(sum / K) divided in double,
- * r = 1 / sqrt(mean + norm_eps) in IEEE fp32, x_k = (h_k * r) * gain_k, then quantised as above.
- *   H        in   bf16 [M, K] row-major; finite, |h| < 4096 (a token that breaks this gets beta = NaN)
+ * r = 1 / sqrt(max(mean + norm_eps, 2^-126)) in IEEE fp32, x_k = (h_k * r) * gain_k, then quantised as above.
+ *   H        in   bf16 [M, K] row-major; finite (a token with an infinity or a NaN gets beta = NaN)
  *   gain     in   fp32 [K], 16-byte aligned
  *   norm_eps      >= 0
  *   Xq, beta, rowsum   out, as for bitlinear_quantize_acts

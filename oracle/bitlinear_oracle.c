@@ -270,7 +270,9 @@ int oracle_quantize_acts(const uint16_t *X_bf16, int64_t M, int64_t K,
  *       below 2^-44 of the largest square, far below fp32 resolution, and the sum does not depend on the scale
  *       of h.  Infinities and NaNs are refused;
  *   N2  mean = (float)( (double)S / (double)K * 2^(2E - 298) ) (the conversion of S rounds to nearest even, the power
- *       of two is exact); r = 1.0f / sqrtf(mean + eps_n): fp32 add, IEEE square root, IEEE divide;
+ *       of two is exact); r = 1.0f / sqrtf(max(mean + eps_n, 2^-126)): fp32 add, IEEE square root, IEEE divide
+ *       (the floor, the smallest normal fp32, only matters for an all-zero token or one whose mean square
+ *       underflows fp32 with eps_n = 0: r stays finite there);
  *   N3  x_k = (h_k * r) * g_k: two fp32 multiplications in this order, no fused multiply-add;
  *   N4  the quantiser then works on the fp32 x_k exactly as on bfloat16 inputs (R4, R5, R6).
  * Parity pins (tests/test_oracle_pins.py): a hand case, agreement of x with a double-precision evaluation of the
@@ -312,7 +314,9 @@ int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, floa
             if (twice <= 46u) S += ((m * m) << 30) >> twice;
         }
         float mean = (float)(ldexp((double)S / (double)K, 2 * (int)E - 298)); /* N2 */
-        float r = 1.0f / sqrtf(mean + eps_n);
+        float d = mean + eps_n;
+        if (!(d > 1.17549435e-38f)) d = 1.17549435e-38f; /* an all-zero or vanishing token: r stays finite */
+        float r = 1.0f / sqrtf(d);
         float amax = 0.0f;
         for (int64_t k = 0; k < K; ++k) {
             float x = (bf16_to_float(H_bf16[t * K + k]) * r) * gain[k]; /* N3 */

@@ -16,7 +16,7 @@
 // token's largest |h| (bfloat16: exponent field e, 8-bit significand m with its hidden bit; e = 0 counts as 1 without
 // hidden bit), S = sum_k floor(m_k^2 * 2^30 / 4^(E - e_k)) < 2^63 in 64-bit arithmetic (terms more than 23 binades
 // below the largest add nothing), sum h^2 = S * 2^(2E - 298).  Then mean = (float)((double)S / K * 2^(2E - 298)),
-// r = 1 / sqrt(mean + eps) with IEEE fp32 add, square root and divide, x_k = (h_k * r) * g_k with two fp32
+// r = 1 / sqrt(max(mean + eps, 2^-126)) with IEEE fp32 add, square root and divide, x_k = (h_k * r) * g_k with two fp32
 // multiplications.  A token with an infinity or a NaN gets beta = NaN.
 #include "internal.cuh"
 #include "ptx.cuh"
@@ -40,28 +40,32 @@ __device__ __forceinline__ uint32_t absmax_bits(uint32_t m, const uint4 &v)
     return m;
 }
 
-__device__ __forceinline__ int quant1(uint32_t bf16_bits, float s)
+// Four rounded products -> four int8 in one word.  cvt.pack saturates to [-128, 127]; the products never leave
+// [-127, 127] after rounding (|x| <= beta and s = fl(127 / beta), so |x * s| < 127.5), which makes the clip of the
+// definition a no-op for finite inputs.
+__device__ __forceinline__ uint32_t pack4(float a, float b, float c, float d)
 {
-    const float x = __uint_as_float(bf16_bits << 16);
-    int q = __float2int_rn(__fmul_rn(x, s)); // one multiply, round half to even
-    return max(-kQb, min(kQb, q));
+    const int qa = __float2int_rn(a), qb = __float2int_rn(b), qc = __float2int_rn(c), qd = __float2int_rn(d);
+    // cvt.pack d, a, b, c: d = (c << 16) | (sat8(a) << 8) | sat8(b)
+    uint32_t hi, out;
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(hi) : "r"(qd), "r"(qc), "r"(0));
+    asm("cvt.pack.sat.s8.s32.b32 %0, %1, %2, %3;" : "=r"(out) : "r"(qb), "r"(qa), "r"(hi));
+    return out;
 }
 
 // 8 bf16 -> 8 int8 (two 32-bit words), returns the sum of the eight codes
 __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
 {
     const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    int q[8];
+    float p[8];
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-        q[2 * i] = quant1(w[i] & 0xFFFFu, s);
-        q[2 * i + 1] = quant1(w[i] >> 16, s);
+        p[2 * i] = __fmul_rn(__uint_as_float(w[i] << 16), s); // one multiply, then round half to even
+        p[2 * i + 1] = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), s);
     }
-    out.x = (uint32_t)(q[0] & 0xFF) | ((uint32_t)(q[1] & 0xFF) << 8) | ((uint32_t)(q[2] & 0xFF) << 16) |
-            ((uint32_t)(q[3] & 0xFF) << 24);
-    out.y = (uint32_t)(q[4] & 0xFF) | ((uint32_t)(q[5] & 0xFF) << 8) | ((uint32_t)(q[6] & 0xFF) << 16) |
-            ((uint32_t)(q[7] & 0xFF) << 24);
-    return q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+    out.x = pack4(p[0], p[1], p[2], p[3]);
+    out.y = pack4(p[4], p[5], p[6], p[7]);
+    return __dp4a((int)out.x, 0x01010101, __dp4a((int)out.y, 0x01010101, 0));
 }
 
 // kNorm: entries may carry a gain vector (RMSNorm in front); the plain form is compiled without that branch.
@@ -133,20 +137,24 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         const bool bad = (top >> 7) == 255u; // an infinity or a NaN somewhere in the token
         const int E = max((int)(top >> 7), 1);
 
+        // h * 2^(149 - E) has the magnitude m * 2^(e - E + 15) (exact; what underflows belongs to terms that are 0),
+        // its square is m^2 * 4^(e - E) * 2^30 (exact in fp32: 16 significant bits), and the conversion truncates.
+        // 2^(149 - E) is no fp32 when E < 22 (a token of values below 2^-105): then the factor is applied in two steps.
+        const bool one_step = E >= 22;
+        const float up = __uint_as_float((uint32_t)(one_step ? 276 - E : 254 - E) << 23); // 2^(149 - E) or 2^(127 - E)
         unsigned long long sq = 0;
         auto add_squares = [&](const uint4 &v) {
             const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-#pragma unroll
-                for (int half = 0; half < 2; ++half) {
-                    const uint32_t bits = half ? (w[i] >> 16) : (w[i] & 0xFFFFu);
-                    int e = (int)((bits >> 7) & 0xFFu);
-                    uint32_t m = bits & 0x7Fu;
-                    if (e) m |= 0x80u; else e = 1;
-                    const int twice = 2 * (E - e);
-                    if (twice <= 46) sq += ((unsigned long long)(m * m) << 30) >> twice;
+                float a = __fmul_rn(__uint_as_float(w[i] << 16), up);
+                float b = __fmul_rn(__uint_as_float(w[i] & 0xFFFF0000u), up);
+                if (!one_step) { // (the same for the whole CTA)
+                    a = __fmul_rn(a, 4194304.0f); // 2^22
+                    b = __fmul_rn(b, 4194304.0f);
                 }
+                sq += __float2ull_rz(__fmul_rn(a, a));
+                sq += __float2ull_rz(__fmul_rn(b, b));
             }
         };
 #pragma unroll
@@ -165,7 +173,8 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         // mean = S / K * 2^(2E - 298): the power of two as a double built from its exponent field
         const double pow2 = __longlong_as_double((long long)(2 * E - 298 + 1023) << 52);
         const float mean = __double2float_rn(__dmul_rn(__ddiv_rn(__ull2double_rn(tot), (double)K), pow2));
-        const float r = __fdiv_rn(1.0f, __fsqrt_rn(__fadd_rn(mean, e.norm_eps)));
+        // (the floor 2^-126 only matters for an all-zero token or one whose mean square underflows fp32: r stays finite)
+        const float r = __fdiv_rn(1.0f, __fsqrt_rn(fmaxf(__fadd_rn(mean, e.norm_eps), 1.17549435e-38f)));
 
         // the eight normalised values of vector i
         auto normalised = [&](const uint4 &v, int i, float (&x)[8]) {
@@ -204,16 +213,11 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         auto quantise8 = [&](const uint4 &v, int i) {
             float x[8];
             normalised(v, i, x);
-            int q[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) q[j] = max(-kQb, min(kQb, __float2int_rn(__fmul_rn(x[j], s))));
             uint2 o;
-            o.x = (uint32_t)(q[0] & 0xFF) | ((uint32_t)(q[1] & 0xFF) << 8) | ((uint32_t)(q[2] & 0xFF) << 16) |
-                  ((uint32_t)(q[3] & 0xFF) << 24);
-            o.y = (uint32_t)(q[4] & 0xFF) | ((uint32_t)(q[5] & 0xFF) << 8) | ((uint32_t)(q[6] & 0xFF) << 16) |
-                  ((uint32_t)(q[7] & 0xFF) << 24);
+            o.x = pack4(__fmul_rn(x[0], s), __fmul_rn(x[1], s), __fmul_rn(x[2], s), __fmul_rn(x[3], s));
+            o.y = pack4(__fmul_rn(x[4], s), __fmul_rn(x[5], s), __fmul_rn(x[6], s), __fmul_rn(x[7], s));
             out_at(i) = o;
-            sum += q[0] + q[1] + q[2] + q[3] + q[4] + q[5] + q[6] + q[7];
+            sum = __dp4a((int)o.x, 0x01010101, __dp4a((int)o.y, 0x01010101, sum));
         };
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {

@@ -94,6 +94,27 @@ def test_forward_rmsnorm_matches_oracle(M, K, N, seed):
         assert np.array_equal(y, Y_ref), "expected bit-identical bf16 outputs"
 
 
+def test_rmsnorm_quantiser_extreme_scales():
+    """Tokens of very small and very large values, subnormal bfloat16s, and a spread of 40 binades inside a token: the
+    integer sum of squares is relative to the token's own largest exponent, so none of this loses exactness."""
+    K = 1024
+    H = S.activations(6, K, 11).float()
+    H[0] *= 2.0 ** -110          # the largest exponent field is below 22
+    H[1] *= 2.0 ** -125          # mostly subnormal bfloat16 values
+    H[2] *= 2.0 ** 100
+    H[3, 0], H[3, 1] = 2.0 ** 30, 2.0 ** -10
+    H[4] = 0
+    H[4, 7] = 2.0 ** -130        # a single subnormal value
+    H = H.to(torch.bfloat16)
+    g = gain_vector(K, 11)
+    for eps_n in (0.0, 1e-5):
+        q_ref, b_ref, s_ref = timing_oracle().rmsnorm_quantize_acts(torch_bf16_to_bits(H), g.numpy(), eps_n)
+        Xq, beta, rowsum = B.rmsnorm_quantize_acts(H.cuda(), g.cuda(), eps_n)
+        assert np.array_equal(Xq.cpu().numpy(), q_ref)
+        assert np.array_equal(beta.cpu().numpy().view(np.uint32), b_ref.view(np.uint32))
+        assert np.array_equal(rowsum.cpu().numpy(), s_ref)
+
+
 def test_rmsnorm_entry_points_reject_bad_arguments():
     L = B.load_library()
     fake = 0x1000
