@@ -516,6 +516,19 @@ def profile_case(name: str):
         ops = 2 * M * 13824 * 5120
         print(json.dumps({"case": name, "int_ops_per_launch": ops, "forward_ms": round(ms, 4),
                           "TOPS": round(ops / ms / 1e9, 1)}))
+    elif name.startswith("quantiser"):
+        # activation quantiser alone on 16384 x 8192 bf16 (268 MB read, 134 MB written); quantiser:norm = with RMSNorm
+        M, K = 16384, 8192
+        H = S.activations(M, K, 0, device="cuda")
+        gain = torch.ones(K, dtype=torch.float32, device="cuda")
+        norm = name.endswith(":norm")
+        fn = (lambda: B.rmsnorm_quantize_acts(H, gain, 1e-5)) if norm else (lambda: B.quantize_acts(H))
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ms = time_forward_calls(fn, 10)
+        print(json.dumps({"case": name, "bytes_per_launch": 3 * M * K, "ms": round(ms, 4),
+                          "GB/s": round(3.0 * M * K / ms / 1e6, 1)}))
     else:
         raise SystemExit(f"unknown profile case {name}")
 
@@ -527,7 +540,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M] | prefill[:M]) and exit")
+    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | prefill[:M] | quantiser[:norm]) and exit")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)
