@@ -198,6 +198,16 @@ typedef struct bitlinear_sequence bitlinear_sequence;
 bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
                                            size_t workspace_bytes, bitlinear_sequence **out);
 
+/*
+ * The same with an RMSNorm (see bitlinear_rmsnorm_quantize_acts) in front of the quantiser of chosen entries:
+ * `gains` is a HOST array of n DEVICE pointers, gains[i] = the fp32 gain vector [K_i] of entry i (16-byte aligned) or
+ * NULL for an entry that is quantised as it is; norm_eps >= 0 serves all of them.  Workspace as for
+ * bitlinear_sequence_create.
+ */
+bitlinear_status bitlinear_sequence_create_rmsnorm(const bitlinear_layer_desc *layers, const float *const *gains,
+                                                   float norm_eps, int n, void *workspace, size_t workspace_bytes,
+                                                   bitlinear_sequence **out);
+
 /* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch, one persistent matmul
  * launch that starts while the quantiser is still running (programmatic dependent launch) and one very small
  * finishing launch.  Calls on the same sequence must be stream-ordered, not concurrent. */

@@ -31,6 +31,7 @@ EXPORTS = [
     "bitlinear_forward_static",
     "bitlinear_sequence_workspace_bytes",
     "bitlinear_sequence_create",
+    "bitlinear_sequence_create_rmsnorm",
     "bitlinear_forward_sequence",
     "bitlinear_forward_sequence_stage",
     "bitlinear_sequence_destroy",
@@ -87,6 +88,8 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_sequence_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci]
     L.bitlinear_sequence_workspace_bytes.restype = sz
     L.bitlinear_sequence_create.argtypes = [ctypes.POINTER(LayerDesc), ci, vp, sz, ctypes.POINTER(vp)]
+    L.bitlinear_sequence_create_rmsnorm.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(vp), cf, ci, vp, sz,
+                                                    ctypes.POINTER(vp)]
     L.bitlinear_forward_sequence.argtypes = [vp, vp]
     L.bitlinear_forward_sequence_stage.argtypes = [vp, ci, vp]
     L.bitlinear_sequence_destroy.argtypes = [vp]
@@ -237,11 +240,14 @@ class Sequence:
     """bitlinear_sequence_*: a fixed list of independent BitLinear forwards run by one persistent launch.
 
     `layers` is a list of (packed, gamma, X, Y, N) with torch tensors; the object keeps them alive.
+    `gains` (optional): one fp32 gain vector [K] or None per layer; those layers get an RMSNorm with `norm_eps` in front
+    of their activation quantiser (bitlinear_sequence_create_rmsnorm).
     """
 
-    def __init__(self, layers, device="cuda"):
+    def __init__(self, layers, device="cuda", gains=None, norm_eps: float = 1e-5):
         L = load_library()
         self._keep = list(layers)
+        self._gains = list(gains) if gains is not None else None
         n = len(self._keep)
         arr = (LayerDesc * n)()
         for i, (packed, gamma, X, Y, N) in enumerate(self._keep):
@@ -252,7 +258,13 @@ class Sequence:
             raise BitLinearError(ERR_SHAPE, "bitlinear_sequence_workspace_bytes")
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
         handle = ctypes.c_void_p()
-        st = L.bitlinear_sequence_create(arr, n, _ptr(self.workspace), nbytes, ctypes.byref(handle))
+        if self._gains is None:
+            st = L.bitlinear_sequence_create(arr, n, _ptr(self.workspace), nbytes, ctypes.byref(handle))
+        else:
+            assert len(self._gains) == n
+            garr = (ctypes.c_void_p * n)(*[(_ptr(g) if g is not None else None) for g in self._gains])
+            st = L.bitlinear_sequence_create_rmsnorm(arr, garr, float(norm_eps), n, _ptr(self.workspace), nbytes,
+                                                     ctypes.byref(handle))
         _check(st, "bitlinear_sequence_create")
         self._handle = handle
         self.n = n

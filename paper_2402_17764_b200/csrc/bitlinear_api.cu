@@ -419,6 +419,7 @@ struct bitlinear_sequence {
     bitlinear::InlineTable inl;
     const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
     int gemm_tiles, gemm_min_kb;
+    bool with_norm;         // some entry is normalised (RMSNorm) in front of the quantiser
     void *split_scratch;    // inside the workspace; null: no GEMM tile of this sequence is cut along K
 };
 
@@ -487,8 +488,31 @@ size_t bitlinear_sequence_workspace_bytes(const bitlinear_layer_desc *layers, in
     return S.total;
 }
 
+namespace {
+bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains, float norm_eps,
+                                      int n, void *workspace, size_t workspace_bytes, bitlinear_sequence **out);
+}
+
 bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
                                            size_t workspace_bytes, bitlinear_sequence **out)
+{
+    return sequence_create_impl(layers, nullptr, 0.0f, n, workspace, workspace_bytes, out);
+}
+
+bitlinear_status bitlinear_sequence_create_rmsnorm(const bitlinear_layer_desc *layers, const float *const *gains,
+                                                   float norm_eps, int n, void *workspace, size_t workspace_bytes,
+                                                   bitlinear_sequence **out)
+{
+    if (!gains || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
+    for (int i = 0; i < n; ++i)
+        if (gains[i] && !aligned(gains[i], 16)) return BITLINEAR_ERR_ALIGN;
+    return sequence_create_impl(layers, gains, norm_eps, n, workspace, workspace_bytes, out);
+}
+
+namespace {
+// gains == null: no entry is normalised; gains[i] == null: entry i is not
+bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains, float norm_eps,
+                                      int n, void *workspace, size_t workspace_bytes, bitlinear_sequence **out)
 {
     if (!layers || !workspace || !out || n <= 0) return BITLINEAR_ERR_ARG;
     *out = nullptr;
@@ -516,6 +540,7 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     const bool gemm = S.use_gemm;
     std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
     int gemm_tiles = 0;
+    bool with_norm = false;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         Layout L{};
@@ -527,6 +552,9 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
         DecodeEntry &e = table[(size_t)i];
         fill_entry(e, d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
         e.xq_tiled = gemm ? 0 : 1;
+        e.gain = gains ? gains[i] : nullptr;
+        e.norm_eps = norm_eps;
+        with_norm = with_norm || e.gain != nullptr;
         e.tile_begin = tiles;
         e.token_begin = tokens;
         tiles += decode_items(e.NB, e.KB, wide);
@@ -555,6 +583,7 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     seq->gemm_table = nullptr;
     seq->gemm_tiles = gemm_tiles;
     seq->gemm_min_kb = S.min_kb;
+    seq->with_norm = with_norm;
     seq->split_scratch = split ? ws + S.acc32 : nullptr;
     if (gemm) {
         if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -576,13 +605,15 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
     *out = seq;
     return BITLINEAR_OK;
 }
+} // namespace
 
 bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq, int stage, void *stream)
 {
     if (!seq || stage < 0 || stage > 2) return BITLINEAR_ERR_ARG;
     cudaStream_t s = (cudaStream_t)stream;
     if (stage != 2 &&
-        launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes, false, s) !=
+        launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes,
+                             seq->with_norm, s) !=
             cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {

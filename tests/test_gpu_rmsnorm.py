@@ -115,6 +115,41 @@ def test_rmsnorm_quantiser_extreme_scales():
         assert np.array_equal(rowsum.cpu().numpy(), s_ref)
 
 
+@pytest.mark.parametrize("M", [1, 5, 12, 40])
+def test_sequence_with_rmsnorm_gains(M):
+    """A decoder layer's seven projections in one sequence: q, k, v and gate, up read the normalised block input
+    (they carry a gain), o and down are quantised as they are.  On the weight-streaming kernels (1, 5, 12 tokens) and
+    on the table-driven GEMM (40 tokens); twice on one workspace."""
+    orc = timing_oracle()
+    shapes = S.decoder_layer_shapes(256, 704, kv_dim=64)
+    normed = {"q", "k", "v", "gate", "up"}
+    layers, gains, refs = [], [], []
+    for mi, sh in enumerate(shapes):
+        W = S.latent_weights(sh.N, sh.K, 80 + mi)
+        H = S.activations(M, sh.K, 80 + mi, outlier_frac=0.02, outlier_scale=10.0)
+        g = gain_vector(sh.K, 80 + mi) if sh.name in normed else None
+        T_ref, g_ref = orc.quantize_weights(W.numpy(), 1e-5)
+        if g is not None:
+            q_ref, b_ref, _ = orc.rmsnorm_quantize_acts(torch_bf16_to_bits(H), g.numpy(), 1e-6)
+            refs.append(orc.dequant(orc.matmul_i32(q_ref, T_ref), b_ref, g_ref))
+        else:
+            refs.append(orc.forward(T_ref, g_ref, torch_bf16_to_bits(H)))
+        packed, gamma = B.quantize_weights(W.cuda(), 1e-5)
+        layers.append((packed, gamma, H.cuda(), torch.zeros((M, sh.N), dtype=torch.bfloat16, device="cuda"), sh.N))
+        gains.append(g.cuda() if g is not None else None)
+    assert any(g is None for g in gains) and any(g is not None for g in gains)
+    seq = B.Sequence(layers, gains=gains, norm_eps=1e-6)
+    for _ in range(2):
+        for l in layers:
+            l[3].zero_()
+        seq.forward()
+        torch.cuda.synchronize()
+        assert B.poll_status(seq.workspace) == 0
+        for l, ref in zip(layers, refs):
+            assert np.array_equal(torch_bf16_to_bits(l[3]), ref)
+    seq.close()
+
+
 def test_rmsnorm_entry_points_reject_bad_arguments():
     L = B.load_library()
     fake = 0x1000
