@@ -178,3 +178,23 @@ def test_70b_layer_sampled(timing_oracle, M):
     assert B.poll_status(seq.workspace) == 0
     sample_check_layers(timing_oracle, layers, meta, [0, 1, 4, 6, 7 + 2, 7 + 6], M, np.random.default_rng(70 + M), "70B layer")
     seq.close()
+
+
+@pytest.mark.parametrize("N,K,M,iters", [(13824, 5120, 2048, 40), (5120, 13824, 2048, 40), (11008, 4096, 64, 100),
+                                         (4096, 11008, 33, 100), (8640, 3200, 1, 100)])
+def test_repeated_runs_are_identical(N, K, M, iters):
+    """Every kernel hands data between warps through barriers (and, where tiles are cut along K, between CTAs through
+    an int32 scratch): many runs on one workspace must give the first run's bits every time."""
+    W = S.latent_weights(N, K, 1, device="cuda")
+    packed, gamma = B.quantize_weights(W)
+    del W
+    X = S.activations(M, K, 1, device="cuda")
+    ws = B.alloc_workspace(M, N, K)
+    first = B.forward(packed, gamma, X, N, workspace=ws).clone()
+    Y = torch.empty_like(first)
+    differing = 0
+    for _ in range(iters):
+        B.forward(packed, gamma, X, N, Y=Y, workspace=ws)
+        differing += int(not torch.equal(Y.view(torch.int16), first.view(torch.int16)))
+    assert B.poll_status(ws) == 0
+    assert differing == 0
