@@ -57,7 +57,6 @@ constexpr int kFirstExpanderWarp = 6; // 8 warps
 constexpr int kExpanderWarps = 8;
 constexpr int kThreads = (kFirstExpanderWarp + kExpanderWarps) * 32; // 448
 
-constexpr uint32_t kABytes = BM * BK;            // 16 KiB int8 activations per token tile
 constexpr uint32_t kBBytes = BN * BK;            // 32 KiB expanded weights
 constexpr uint32_t kPBytes = (BN / kTileRows) * (BK / kTileCols) * kTileBytes; //  8 KiB packed weights
 
