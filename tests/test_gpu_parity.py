@@ -282,7 +282,9 @@ def test_forward_decode_shapes(oracle, M, K, N, seed):
                                         # them backed by spare workspace rows
                                         (17, 3200, 1040, 5), (31, 144, 4112, 6), (32, 1536, 512, 7), (48, 8640, 272, 8),
                                         # the largest K the library takes (accumulators up to 127 * 131072), smallest N
-                                        (2, 131072, 16, 9), (40, 131072, 32, 10), (200, 131072, 16, 11)])
+                                        (2, 131072, 16, 9), (40, 131072, 32, 10), (200, 131072, 16, 11),
+                                        # the largest M the library takes
+                                        (1 << 20, 16, 16, 12)])
 def test_forward_prefill_shapes(oracle, M, K, N, seed):
     same = run_forward_case(oracle, M, K, N, seed, big=True)
     assert same == 1.0
