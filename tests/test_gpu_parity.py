@@ -271,7 +271,10 @@ def test_forward_first_workload(oracle):
 
 
 @pytest.mark.parametrize("M,K,N,seed", [(1, 3200, 3200, 1), (1, 8640, 3200, 2), (4, 4096, 11008, 3), (16, 11008, 4096, 4),
-                                        (64, 4096, 4096, 5), (1, 16, 16, 6), (7, 144, 48, 7)])
+                                        (64, 4096, 4096, 5), (1, 16, 16, 6), (7, 144, 48, 7),
+                                        # a million output features behind the smallest K (16384 row blocks of one
+                                        # padded column tile), on the streaming kernel and on the GEMM
+                                        (1, 16, 1 << 20, 8), (40, 16, 1 << 18, 9)])
 def test_forward_decode_shapes(oracle, M, K, N, seed):
     same = run_forward_case(oracle, M, K, N, seed, frac=0.005, scale=30.0, big=True)
     assert same == 1.0
