@@ -244,7 +244,7 @@ bitlinear_status quantize_acts_rows(const void *X, const float *gain, float norm
     e.K = (int)K;
     e.gain = gain;
     e.norm_eps = norm_eps;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, gain != nullptr, (cudaStream_t)stream);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, gain != nullptr, (int)K, (cudaStream_t)stream);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 } // namespace
@@ -309,7 +309,7 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, gain != nullptr, (cudaStream_t)stream);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, gain != nullptr, (int)K, (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M,
                       split ? ws + L.acc32 : nullptr, (cudaStream_t)stream);
@@ -343,7 +343,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                              : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, false, s);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, false, (int)K, s);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     if (tc) {
         inl.e[0].Xq = const_cast<int8_t *>(Xq); // the GEMM reads the caller's rows in place
@@ -412,7 +412,7 @@ bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma
 struct bitlinear_sequence {
     char *workspace;
     bitlinear::OwnedList *lists;
-    int n, tokens, max_M;
+    int n, tokens, max_M, max_K;
     uint32_t tiles;
     size_t zero_bytes;
     const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
@@ -576,6 +576,9 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     seq->tiles = tiles;
     seq->tokens = tokens;
     seq->max_M = max_M;
+    seq->max_K = 0;
+    for (int i = 0; i < n; ++i)
+        if ((int)layers[i].K > seq->max_K) seq->max_K = (int)layers[i].K;
     const size_t clear = gemm ? prefill_split_clear_bytes(gemm_tiles, S.min_kb, max_M) : 0;
     const bool split = clear > 0;
     seq->zero_bytes = gemm ? S.acc32 + align_up(clear, 256) : S.table; // header and the int32 scratch in use
@@ -613,7 +616,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
     cudaStream_t s = (cudaStream_t)stream;
     if (stage != 2 &&
         launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes,
-                             seq->with_norm, s) !=
+                             seq->with_norm, seq->max_K, s) !=
             cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {

@@ -77,9 +77,9 @@ cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *t
 
 // Quantises the tokens of every entry (entries with X == nullptr are skipped) and zeroes
 // `zero_bytes` bytes at `zero_ptr` (control words and split-K scratch) in the same launch.  with_norm: some entry
-// carries a gain vector (RMSNorm in front of the quantiser).
+// carries a gain vector (RMSNorm in front of the quantiser).  max_K: the longest token among the entries.
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
-                                 void *zero_ptr, size_t zero_bytes, bool with_norm, cudaStream_t stream);
+                                 void *zero_ptr, size_t zero_bytes, bool with_norm, int max_K, cudaStream_t stream);
 
 // The weight-streaming matmul has two kernels: up to 8 tokens every warp streams tiles on its own; from 9
 // tokens the eight warps of a CTA share the activations and the CTA walks group tiles (8 row blocks x 1

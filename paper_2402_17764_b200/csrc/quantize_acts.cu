@@ -69,14 +69,17 @@ __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
 }
 
 // kNorm: entries may carry a gain vector (RMSNorm in front); the plain form is compiled without that branch.
-template <bool kNorm>
-__global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
+// NT threads per token (64, 128, 192 or 256): what a CTA does besides touching its elements (finding its entry,
+// three block-wide reductions) is a fixed cost per thread, so short tokens take fewer threads with kCache vectors
+// each.  Tokens of more than 8192 elements re-read their tail, which hits L2.
+template <bool kNorm, int NT>
+__global__ void __launch_bounds__(NT, (kNorm ? 768 : 1024) / NT) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
                                                                  const DecodeEntry *__restrict__ table, int n_entries,
                                                                  int total_tokens, uint4 *zero_ptr, size_t zero_vecs)
 {
-    __shared__ uint32_t s_max[kThreads / 32];
-    __shared__ int s_sum[kThreads / 32];
-    __shared__ unsigned long long s_sq[kThreads / 32];
+    __shared__ uint32_t s_max[NT / 32];
+    __shared__ int s_sum[NT / 32];
+    __shared__ unsigned long long s_sq[NT / 32];
 
     // The matmul that follows may be launched early: it streams weights until it needs what this kernel writes.
     ptx::griddep_launch_dependents();
@@ -84,8 +87,8 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
     if ((int)blockIdx.x >= total_tokens) {
         // trailing blocks clear control words and split-K scratch for the matmul that follows
         const size_t n_zero_blocks = gridDim.x - total_tokens;
-        for (size_t i = (size_t)(blockIdx.x - total_tokens) * kThreads + threadIdx.x; i < zero_vecs;
-             i += n_zero_blocks * kThreads)
+        for (size_t i = (size_t)(blockIdx.x - total_tokens) * NT + threadIdx.x; i < zero_vecs;
+             i += n_zero_blocks * NT)
             zero_ptr[i] = make_uint4(0u, 0u, 0u, 0u);
         return;
     }
@@ -120,19 +123,19 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         uint32_t top = 0;
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
-            const int i = threadIdx.x + c * kThreads;
+            const int i = threadIdx.x + c * NT;
             if (i < n_vec) {
                 cache[c] = __ldg(row + i);
                 top = absmax_bits(top, cache[c]);
             }
         }
-        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) top = absmax_bits(top, __ldg(row + i));
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) top = absmax_bits(top, __ldg(row + i));
         top = __reduce_max_sync(0xffffffffu, top);
         if (lane == 0) s_max[warp] = top;
         __syncthreads();
         top = s_max[0];
 #pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) top = max(top, s_max[w]);
+        for (int w = 1; w < NT / 32; ++w) top = max(top, s_max[w]);
         __syncthreads(); // s_max is used again below
         const bool bad = (top >> 7) == 255u; // an infinity or a NaN somewhere in the token
         const int E = max((int)(top >> 7), 1);
@@ -159,17 +162,17 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         };
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
-            const int i = threadIdx.x + c * kThreads;
+            const int i = threadIdx.x + c * NT;
             if (i < n_vec) add_squares(cache[c]);
         }
-        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) add_squares(__ldg(row + i));
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) add_squares(__ldg(row + i));
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) sq += __shfl_xor_sync(0xffffffffu, sq, off);
         if (lane == 0) s_sq[warp] = sq;
         __syncthreads();
         unsigned long long tot = 0;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) tot += s_sq[w]; // every thread forms the same total
+        for (int w = 0; w < NT / 32; ++w) tot += s_sq[w]; // every thread forms the same total
         // mean = S / K * 2^(2E - 298): the power of two as a double built from its exponent field
         const double pow2 = __longlong_as_double((long long)(2 * E - 298 + 1023) << 52);
         const float mean = __double2float_rn(__dmul_rn(__ddiv_rn(__ull2double_rn(tot), (double)K), pow2));
@@ -196,16 +199,16 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         };
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
-            const int i = threadIdx.x + c * kThreads;
+            const int i = threadIdx.x + c * NT;
             if (i < n_vec) absmax8(cache[c], i);
         }
-        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) absmax8(__ldg(row + i), i);
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) absmax8(__ldg(row + i), i);
         mx = __reduce_max_sync(0xffffffffu, mx);
         if (lane == 0) s_max[warp] = mx;
         __syncthreads();
         mx = s_max[0];
 #pragma unroll
-        for (int w = 1; w < kThreads / 32; ++w) mx = max(mx, s_max[w]);
+        for (int w = 1; w < NT / 32; ++w) mx = max(mx, s_max[w]);
         const float b = fmaxf(__uint_as_float(mx), kBetaFloor);
         const float s = __fdiv_rn((float)kQb, b);
 
@@ -221,19 +224,19 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
         };
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
-            const int i = threadIdx.x + c * kThreads;
+            const int i = threadIdx.x + c * NT;
             if (i < n_vec) quantise8(cache[c], i);
         }
-        for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) quantise8(__ldg(row + i), i);
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) quantise8(__ldg(row + i), i);
         if (tiled) // the last column tile is filled up with zeros
-            for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += kThreads) out_at(i) = make_uint2(0u, 0u);
+            for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += NT) out_at(i) = make_uint2(0u, 0u);
         sum = __reduce_add_sync(0xffffffffu, sum);
         if (lane == 0) s_sum[warp] = sum;
         __syncthreads();
         if (threadIdx.x == 0) {
             int total = 0;
 #pragma unroll
-            for (int w = 0; w < kThreads / 32; ++w) total += s_sum[w];
+            for (int w = 0; w < NT / 32; ++w) total += s_sum[w];
             e.beta[t] = bad ? __int_as_float(0x7FC00000) : b;
             e.rowsum[t] = total;
         }
@@ -243,13 +246,13 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
     uint32_t m = 0;
 #pragma unroll
     for (int c = 0; c < kCache; ++c) {
-        const int i = threadIdx.x + c * kThreads;
+        const int i = threadIdx.x + c * NT;
         if (i < n_vec) {
             cache[c] = __ldg(row + i);
             m = absmax_bits(m, cache[c]);
         }
     }
-    for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads)
+    for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT)
         m = absmax_bits(m, __ldg(row + i));
 
     m = __reduce_max_sync(0xffffffffu, m);
@@ -257,7 +260,7 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
     __syncthreads();
     m = s_max[0];
 #pragma unroll
-    for (int w = 1; w < kThreads / 32; ++w) m = max(m, s_max[w]);
+    for (int w = 1; w < NT / 32; ++w) m = max(m, s_max[w]);
 
     const float amax = __uint_as_float(m << 16);
     const float b = fmaxf(amax, kBetaFloor);
@@ -266,27 +269,27 @@ __global__ void __launch_bounds__(kThreads, kNorm ? 3 : 4) quantize_acts_kernel(
     int sum = 0;
 #pragma unroll
     for (int c = 0; c < kCache; ++c) {
-        const int i = threadIdx.x + c * kThreads;
+        const int i = threadIdx.x + c * NT;
         if (i < n_vec) {
             uint2 o;
             sum += quant8(cache[c], s, o);
             out_at(i) = o;
         }
     }
-    for (int i = threadIdx.x + kCache * kThreads; i < n_vec; i += kThreads) {
+    for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
         uint2 o;
         sum += quant8(__ldg(row + i), s, o);
         out_at(i) = o;
     }
     if (tiled) // the last column tile is filled up with zeros
-        for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += kThreads) out_at(i) = make_uint2(0u, 0u);
+        for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += NT) out_at(i) = make_uint2(0u, 0u);
     sum = __reduce_add_sync(0xffffffffu, sum);
     if (lane == 0) s_sum[warp] = sum;
     __syncthreads();
     if (threadIdx.x == 0) {
         int tot = 0;
 #pragma unroll
-        for (int w = 0; w < kThreads / 32; ++w) tot += s_sum[w];
+        for (int w = 0; w < NT / 32; ++w) tot += s_sum[w];
         e.beta[t] = b;
         e.rowsum[t] = tot;
     }
@@ -313,24 +316,44 @@ cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *t
 }
 
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
-                                 void *zero_ptr, size_t zero_bytes, bool with_norm, cudaStream_t stream)
+                                 void *zero_ptr, size_t zero_bytes, bool with_norm, int max_K, cudaStream_t stream)
 {
+    // threads per token: the smallest count whose register caches hold the longest token
+    const int n_vec = max_K >> 3;
+    // (longer tokens re-read their tail, which hits L2: CTAs of 512 and 1024 threads measured slower)
+    static const int counts[4] = {64, 128, 192, 256};
+    int nt = 256;
+    for (int c : counts)
+        if (n_vec <= c * kCache) {
+            nt = c;
+            break;
+        }
     const size_t zero_vecs = zero_bytes / 16;
     int zero_blocks = 0;
     if (zero_vecs > 0) {
-        zero_blocks = (int)((zero_vecs + kThreads * 4 - 1) / (kThreads * 4));
-        const int cap = sm_count() * 4;
+        zero_blocks = (int)((zero_vecs + (size_t)nt * 4 - 1) / ((size_t)nt * 4));
+        const int cap = sm_count() * 1024 / nt;
         if (zero_blocks > cap) zero_blocks = cap;
         if (zero_blocks < 1) zero_blocks = 1;
     }
     const int grid = total_tokens + zero_blocks;
     if (grid == 0) return cudaSuccess;
-    if (with_norm)
-        quantize_acts_kernel<true><<<grid, kThreads, 0, stream>>>(inl, table, n_entries, total_tokens,
-                                                                  reinterpret_cast<uint4 *>(zero_ptr), zero_vecs);
-    else
-        quantize_acts_kernel<false><<<grid, kThreads, 0, stream>>>(inl, table, n_entries, total_tokens,
-                                                                   reinterpret_cast<uint4 *>(zero_ptr), zero_vecs);
+    uint4 *zp = reinterpret_cast<uint4 *>(zero_ptr);
+#define BITLINEAR_LAUNCH_QUANTISER(NORM, NT_) \
+    quantize_acts_kernel<NORM, NT_><<<grid, NT_, 0, stream>>>(inl, table, n_entries, total_tokens, zp, zero_vecs)
+#define BITLINEAR_LAUNCH_BOTH(NT_) \
+    do { \
+        if (with_norm) BITLINEAR_LAUNCH_QUANTISER(true, NT_); \
+        else BITLINEAR_LAUNCH_QUANTISER(false, NT_); \
+    } while (0)
+    switch (nt) {
+    case 64: BITLINEAR_LAUNCH_BOTH(64); break;
+    case 128: BITLINEAR_LAUNCH_BOTH(128); break;
+    case 192: BITLINEAR_LAUNCH_BOTH(192); break;
+    default: BITLINEAR_LAUNCH_BOTH(256); break;
+    }
+#undef BITLINEAR_LAUNCH_BOTH
+#undef BITLINEAR_LAUNCH_QUANTISER
     return cudaGetLastError();
 }
 
