@@ -158,15 +158,25 @@ __device__ __forceinline__ float token_scale(const DecodeEntry &e, int token)
     return __fdiv_rn(__fmul_rn(*e.gamma, e.beta[token]), (float)kQb); // (gamma * beta_t) / Qb
 }
 
-// End of a row block.  `each(fn)` calls fn(token, row, partial row sum) for every output this lane holds.
-// If all KB column tiles went into the sums they are final; otherwise they are added to the int32 scratch.
+// What the epilogue needs of a token, fetched once per token and lane: the stores of a lane's outputs may alias
+// these loads as far as the compiler knows, so asking per output would reload (and divide) every time.
+struct TokenTerms {
+    int rowsum;
+    float scale;
+};
+
+// End of a row block.  `each(begin, fn)` calls begin(token) once for every token this lane holds outputs of and then
+// fn(terms, token, row, partial row sum) for each of them.  If all KB column tiles went into the sums they are final;
+// otherwise they are added to the int32 scratch.
 template <class Each>
 __device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete, Each each)
 {
     if (complete)
-        each([&](int token, int row, int v) { store_result(e, token, row, v, e.rowsum[token], token_scale(e, token)); });
+        each([&](int token) { return TokenTerms{e.rowsum[token], token_scale(e, token)}; },
+             [&](const TokenTerms &tt, int token, int row, int v) { store_result(e, token, row, v, tt.rowsum, tt.scale); });
     else
-        each([&](int token, int row, int v) { atomicAdd(&e.acc32[(size_t)token * e.N + row], v); });
+        each([&](int) { return TokenTerms{0, 0.0f}; },
+             [&](const TokenTerms &, int token, int row, int v) { atomicAdd(&e.acc32[(size_t)token * e.N + row], v); });
 }
 
 // Finishing launch: dequantises the row blocks on one list from the scratch and leaves the scratch clean for
@@ -268,8 +278,8 @@ __device__ __forceinline__ void mma_slab(int (&acc)[4][4], const uint4 &w, uint3
 
 // Un-mixes the four scaled accumulators of every (row, token) this lane holds and hands the row sums to fn.
 // C fragment of field f: c0 (row 16f + g, token 2tq), c1 (same row, 2tq + 1), c2 (row 16f + 8 + g, 2tq), c3.
-template <int NT, class Fn>
-__device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, int N, int row0, int tq, Fn fn)
+template <int NT, class Begin, class Fn>
+__device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, int N, int row0, int tq, Begin begin, Fn fn)
 {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -277,6 +287,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, i
         for (int tb = 0; tb < 2; ++tb) {
             const int token = 8 * nt + 2 * tq + tb;
             if (token >= M) continue;
+            const auto terms = begin(token);
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int c = 2 * h + tb;
@@ -287,7 +298,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, i
 #pragma unroll
                 for (int f = 0; f < 4; ++f) {
                     const int r = row0 + 16 * f + 8 * h;
-                    if (r < N) fn(token, r, S[f]);
+                    if (r < N) fn(terms, token, r, S[f]);
                 }
             }
         }
@@ -559,7 +570,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             if (lane == 0) owned[n_owned] = make_uint2((uint32_t)(e - tab), (uint32_t)rb);
             ++n_owned; // cannot exceed kMaxOwned: see next_piece
         }
-        finish_block(*e, complete, [&](auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, fn); });
+        finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, begin, fn); });
 
         // next row block, or next matrix
         if (kt == KB) {
@@ -809,7 +820,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
                     ++n_owned;
                 }
             }
-            finish_block(*e, complete, [&](auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, fn); });
+            finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, begin, fn); });
         }
     }
     }();
