@@ -339,6 +339,97 @@ int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, floa
     return status;
 }
 
+/* ---------- SwiGLU in front of the activation quantiser ----------
+ *
+ * SwiGLU is another of the paper's "LLaMA-alike components" (Section 2), again without a formula: the input of the
+ * down projection is taken here as the textbook h_k = silu(g_k) * u_k, silu(g) = g * sigmoid(g) = g / (1 + e^-g), of
+ * the gate and up projections' outputs g and u (bfloat16, as BitLinear writes them), followed by the activation
+ * quantiser above.  The values decide integers, so the arithmetic is fixed in fp32 (readings, not the paper's):
+ *   G1  e^t for t = -g by range reduction and a Taylor polynomial, every step one IEEE fp32 operation:
+ *           z = t * log2(e)         (log2(e) as fp32),           n = z rounded to the nearest integer, ties to even,
+ *           r = fma(n, -ln2_hi, t), r = fma(n, -ln2_lo, r)       (ln 2 = ln2_hi + ln2_lo, ln2_hi with 9 trailing zero bits),
+ *           p = 1 + r + r^2/2 + ... + r^7/5040                   (Horner's scheme, seven fused multiply-adds from the top),
+ *           e^t = p * 2^n                                        (exact: t is kept within [-87, 87], so 2^n and the
+ *                                                                 product are normal numbers);
+ *   G2  sigmoid(g) = 1 / (1 + e^-g): one fp32 addition and one IEEE division; for g > 87 it is 1, for g < -87 it
+ *       is 0 (the true value is within 2^-125 of that);
+ *   G3  h_k = (g_k * sigmoid(g_k)) * u_k: two fp32 multiplications in this order;
+ *   G4  the quantiser then works on the fp32 h_k exactly as on bfloat16 inputs (R4, R5, R6).  Infinities and NaNs in
+ *       g or u, and a product h_k that overflows fp32, are refused.
+ * Parity pins (tests/test_oracle_pins.py): agreement of h with a double-precision evaluation of the definition and
+ * with torch's silu, hand cases (g = 0, the saturated ends), reduction to the plain quantiser for saturated gates,
+ * odd symmetry in u.
+ */
+static float sigmoid_f32(float g)
+{
+    float t = -g;
+    if (t > 87.0f) return 0.0f;
+    if (t < -87.0f) return 1.0f;
+    float z = t * 1.44269502162933349609375f;                 /* log2(e) rounded to fp32 */
+    float n = rintf(z);                                       /* default rounding mode: ties to even */
+    float r = fmaf(n, -0.693145751953125f, t);                /* ln2_hi */
+    r = fmaf(n, -1.42860676533018704503775e-06f, r);          /* ln2_lo = fp32(ln 2 - ln2_hi) */
+    float p = fmaf(r, 1.0f / 5040.0f, 1.0f / 720.0f);
+    p = fmaf(p, r, 1.0f / 120.0f);
+    p = fmaf(p, r, 1.0f / 24.0f);
+    p = fmaf(p, r, 1.0f / 6.0f);
+    p = fmaf(p, r, 0.5f);
+    p = fmaf(p, r, 1.0f);
+    p = fmaf(p, r, 1.0f);
+    float e = ldexpf(p, (int)n);
+    return 1.0f / (1.0f + e);
+}
+
+int oracle_swiglu_quantize_acts(const uint16_t *G_bf16, const uint16_t *U_bf16, int64_t M, int64_t K,
+                                int8_t *Xq, float *beta, int32_t *rowsum, float *h_out /* may be NULL: [M][K] */)
+{
+    if (!G_bf16 || !U_bf16 || !Xq || !beta || !rowsum || M < 0 || K <= 0)
+        return ORACLE_ERR_ARG;
+    int status = ORACLE_OK;
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        float amax = 0.0f;
+        int bad = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            float g = bf16_to_float(G_bf16[t * K + k]), u = bf16_to_float(U_bf16[t * K + k]);
+            if (!isfinite(g) || !isfinite(u)) {
+                bad = 1;
+                break;
+            }
+            float h = (g * sigmoid_f32(g)) * u; /* G3 */
+            if (!isfinite(h)) {
+                bad = 1;
+                break;
+            }
+            if (h_out) h_out[t * K + k] = h;
+            float a = fabsf(h);
+            if (a > amax) amax = a;
+        }
+        if (bad) {
+#ifdef _OPENMP
+#pragma omp critical
+#endif
+            status = ORACLE_ERR_RANGE;
+            continue;
+        }
+        float b = amax > BETA_FLOOR ? amax : BETA_FLOOR; /* R6 */
+        float s = (float)QB / b;
+        int32_t acc = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            float g = bf16_to_float(G_bf16[t * K + k]), u = bf16_to_float(U_bf16[t * K + k]);
+            float h = (g * sigmoid_f32(g)) * u;
+            int q = round_clip(h * s, -QB, QB);
+            Xq[t * K + k] = (int8_t)q;
+            acc += q;
+        }
+        beta[t] = b;
+        rowsum[t] = acc;
+    }
+    return status;
+}
+
 /* ---------- integer matrix product: the plain definition ---------- */
 
 /* acc[t][n] = sum_k Xq[t][k] * T[n][k], exact in int32 (|acc| <= 127*K). */

@@ -57,6 +57,7 @@ class Oracle:
         L.oracle_unpack_weights.argtypes = [_p, _i64, _i64, _p]
         L.oracle_quantize_acts.argtypes = [_p, _i64, _i64, _p, _p, _p]
         L.oracle_rmsnorm_quantize_acts.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p, _p, _p, _p]
+        L.oracle_swiglu_quantize_acts.argtypes = [_p, _p, _i64, _i64, _p, _p, _p, _p]
         L.oracle_matmul_i32.argtypes = [_p, _p, _i64, _i64, _i64, _p]
         L.oracle_dequant.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p]
         L.oracle_forward.argtypes = [_p, ctypes.c_float, _p, _i64, _i64, _i64, _p, _p, _p, _p, _p]
@@ -140,6 +141,21 @@ class Oracle:
                                                    self._ptr(x) if return_x else None)
         self._check(rc, "rmsnorm_quantize_acts")
         return (Xq, beta, rs, x) if return_x else (Xq, beta, rs)
+
+    def swiglu_quantize_acts(self, G_bf16_bits: np.ndarray, U_bf16_bits: np.ndarray, return_h: bool = False):
+        """h = silu(g) * u in fp32 followed by the activation quantiser -> (Xq, beta, rowsum[, h float32 [M,K]])."""
+        G = self._c(G_bf16_bits, np.uint16)
+        U = self._c(U_bf16_bits, np.uint16)
+        M, K = G.shape
+        assert U.shape == (M, K)
+        Xq = np.empty((M, K), np.int8)
+        beta = np.empty(M, np.float32)
+        rs = np.empty(M, np.int32)
+        h = np.empty((M, K), np.float32) if return_h else None
+        rc = self.lib.oracle_swiglu_quantize_acts(self._ptr(G), self._ptr(U), M, K, self._ptr(Xq), self._ptr(beta),
+                                                  self._ptr(rs), self._ptr(h) if return_h else None)
+        self._check(rc, "swiglu_quantize_acts")
+        return (Xq, beta, rs, h) if return_h else (Xq, beta, rs)
 
     def matmul_i32(self, Xq: np.ndarray, T: np.ndarray) -> np.ndarray:
         Xq = self._c(Xq, np.int8)

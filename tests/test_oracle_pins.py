@@ -349,3 +349,74 @@ def test_rmsnorm_quantiser_invariants(oracle):
     for v in (np.inf, np.nan):
         with pytest.raises(ValueError):
             oracle.rmsnorm_quantize_acts(_bf16([[v] + [0.0] * 15]), np.ones(16, np.float32), 0.0)
+
+
+# ---- SwiGLU in front of the activation quantiser ----
+
+def test_swiglu_quantiser_hand_cases(oracle):
+    """g = 0: silu = 0.  Saturated gates: silu(g) = g for g > 87 and 0 for g < -87.  g = 1: 1 / (1 + 1/e)."""
+    g = _bf16([[0.0, 128.0, -128.0, 1.0, -1.0, 96.0, 0.0, 0.0]])
+    u = _bf16([[5.0, 0.5, 3.0, 2.0, 2.0, -1.0, 0.0, 0.0]])
+    q, beta, rs, h = oracle.swiglu_quantize_acts(g, u, return_h=True)
+    assert h[0, 0] == 0.0 and h[0, 1] == 64.0 and h[0, 2] == 0.0 and h[0, 5] == -96.0
+    s1 = 1.0 / (1.0 + math.exp(-1.0))
+    assert abs(float(h[0, 3]) - 2.0 * s1) < 3e-7 and abs(float(h[0, 4]) + 2.0 * (1.0 - s1)) < 3e-7
+    assert beta.tolist() == [96.0]
+    # 64 * 127 / 96 = 84.67, 2 * 0.7311 * 127 / 96 = 1.934, -2 * 0.2689 * 127 / 96 = -0.7115
+    assert q.tolist() == [[0, 85, 0, 2, -1, -127, 0, 0]] and rs.tolist() == [-41]
+
+
+def test_swiglu_matches_double_precision_and_library(oracle):
+    import torch
+    rng = np.random.default_rng(31)
+    M, K = 6, 2048
+    g = (2.5 * rng.standard_normal((M, K))).astype(np.float32)
+    g[0, :64] = np.linspace(-87.0, 87.0, 64)          # the whole range of the exponential
+    g[1, :64] = np.linspace(-20.0, 20.0, 64)
+    u = rng.standard_normal((M, K)).astype(np.float32)
+    gb, ub = _bf16(g), _bf16(u)
+    g64, u64 = bits_to_f32(gb).astype(np.float64), bits_to_f32(ub).astype(np.float64)
+    q, beta, rs, h = oracle.swiglu_quantize_acts(gb, ub, return_h=True)
+    h64 = g64 / (1.0 + np.exp(-g64)) * u64
+    # polynomial (below 1 ulp), the addition, the division and two products: a few fp32 roundings
+    assert np.all(np.abs(h - h64) <= 6 * np.spacing(np.abs(h64).astype(np.float32)))
+    lib = (torch.nn.functional.silu(torch.from_numpy(g64)) * torch.from_numpy(u64)).numpy()
+    assert np.allclose(h, lib, rtol=1e-6, atol=1e-30)
+    b64 = np.abs(h64).max(axis=1)
+    assert np.allclose(beta, b64, rtol=1e-6)
+    scaled = h64 * (127.0 / b64)[:, None]
+    clear = np.abs(scaled - np.floor(scaled) - 0.5) > 1e-3   # away from rounding ties, fp32 and fp64 must agree
+    assert clear.mean() > 0.99 and np.array_equal(q[clear], np.rint(scaled)[clear].astype(np.int8))
+    assert np.array_equal(rs, q.astype(np.int32).sum(axis=1)) and np.abs(q).max() == 127
+
+
+def test_swiglu_quantiser_invariants(oracle):
+    rng = np.random.default_rng(32)
+    M, K = 5, 320
+    ub = _bf16(rng.standard_normal((M, K)))
+    # a saturated gate 2^7 multiplies u by a power of two, which the quantiser does not see: the plain quantiser of u
+    gate = _bf16(np.full((M, K), 128.0))
+    q, beta, rs = oracle.swiglu_quantize_acts(gate, ub)
+    qp, bp, rp = oracle.quantize_acts(ub)
+    assert np.array_equal(q, qp) and np.array_equal(beta, 128.0 * bp) and np.array_equal(rs, rp)
+    # odd in u; a permutation of the features permutes the codes
+    gb = _bf16(3.0 * rng.standard_normal((M, K)))
+    q, beta, rs = oracle.swiglu_quantize_acts(gb, ub)
+    qn, bn, rn = oracle.swiglu_quantize_acts(gb, ub ^ np.uint16(0x8000))
+    assert np.array_equal(qn, -q) and np.array_equal(bn, beta) and np.array_equal(rn, -rs)
+    perm = rng.permutation(K)
+    qq, bq, rq = oracle.swiglu_quantize_acts(gb[:, perm], ub[:, perm])
+    assert np.array_equal(qq, q[:, perm]) and np.array_equal(bq, beta) and np.array_equal(rq, rs)
+    # silu(g) - silu(-g) = g: the two halves of the sigmoid add up to one
+    _, _, _, hp = oracle.swiglu_quantize_acts(gb, _bf16(np.ones((M, K))), return_h=True)
+    _, _, _, hm = oracle.swiglu_quantize_acts(gb ^ np.uint16(0x8000), _bf16(np.ones((M, K))), return_h=True)
+    gf = bits_to_f32(gb)
+    assert np.all(np.abs((hp - hm) - gf) <= 4 * np.spacing(np.abs(gf)))
+    # zero gates or zero ups give zeros (beta at its floor)
+    for a, b in ((np.zeros((1, K)), rng.standard_normal((1, K))), (rng.standard_normal((1, K)), np.zeros((1, K)))):
+        qz, bz, rz = oracle.swiglu_quantize_acts(_bf16(a), _bf16(b))
+        assert not qz.any() and rz[0] == 0 and bz[0] == np.float32(1e-5)
+    # infinities, NaNs and products beyond fp32 are refused
+    for gv, uv in ((np.inf, 1.0), (1.0, np.nan), (-np.inf, 1.0), (2.0 ** 100, 2.0 ** 100)):
+        with pytest.raises(ValueError):
+            oracle.swiglu_quantize_acts(_bf16([[gv] + [0.0] * 15]), _bf16([[uv] + [1.0] * 15]))
