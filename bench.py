@@ -300,6 +300,24 @@ def extras(peaks):
         del H, Xq
     out["rmsnorm_quantiser"] = res
 
+    # SwiGLU fused into the activation quantiser of the down projection (2 x 2 B read + 1 B written per element; the
+    # product silu(gate) * up is never written), at the feed-forward widths of the 7B- and 13B-shaped layers
+    res = {}
+    for M, K in [(8192, 11008), (8192, 13824)]:
+        gate = S.activations(M, K, 0, device="cuda")
+        up = S.activations(M, K, 1, device="cuda")
+        Xq = torch.empty((M, K), dtype=torch.int8, device="cuda")
+        beta = torch.empty(M, dtype=torch.float32, device="cuda")
+        rs = torch.empty(M, dtype=torch.int32, device="cuda")
+        L = B.load_library()
+        stream = torch.cuda.current_stream().cuda_stream
+        ms_s = time_forward_calls(lambda: L.bitlinear_swiglu_quantize_acts(gate.data_ptr(), up.data_ptr(), M, K, Xq.data_ptr(),
+                                                                           beta.data_ptr(), rs.data_ptr(), stream), 10)
+        res[f"M{M}_K{K}"] = {"swiglu_quantiser_ms": round(ms_s, 4), "GB/s": round(5.0 * M * K / ms_s / 1e6, 1),
+                             "frac_hbm_measured": round(5.0 * M * K / ms_s / 1e6 / hbm, 3)}
+        del gate, up, Xq
+    out["swiglu_quantiser"] = res
+
     # the headline step with the RMSNorm fused into the quantiser of q, k, v, gate and up (130 of the 182 matrices)
     cfg = S.CONFIGS[WORKLOAD]
     st = Stack(cfg["layers"], cfg["n_layers"], 1)
@@ -533,18 +551,22 @@ def profile_case(name: str):
         print(json.dumps({"case": name, "int_ops_per_launch": ops, "forward_ms": round(ms, 4),
                           "TOPS": round(ops / ms / 1e9, 1)}))
     elif name.startswith("quantiser"):
-        # activation quantiser alone on 16384 x 8192 bf16 (268 MB read, 134 MB written); quantiser:norm = with RMSNorm
-        M, K = 16384, 8192
+        # activation quantiser alone on 16384 x 8192 bf16 (268 MB read, 134 MB written); quantiser:norm = with RMSNorm;
+        # quantiser:swiglu = with SwiGLU on 8192 x 11008 gate and up inputs (361 MB read, 90 MB written)
+        norm, swiglu = name.endswith(":norm"), name.endswith(":swiglu")
+        M, K = (8192, 11008) if swiglu else (16384, 8192)
         H = S.activations(M, K, 0, device="cuda")
         gain = torch.ones(K, dtype=torch.float32, device="cuda")
-        norm = name.endswith(":norm")
-        fn = (lambda: B.rmsnorm_quantize_acts(H, gain, 1e-5)) if norm else (lambda: B.quantize_acts(H))
+        up = S.activations(M, K, 1, device="cuda") if swiglu else None
+        fn = ((lambda: B.swiglu_quantize_acts(H, up)) if swiglu else
+              (lambda: B.rmsnorm_quantize_acts(H, gain, 1e-5)) if norm else (lambda: B.quantize_acts(H)))
         for _ in range(3):
             fn()
         torch.cuda.synchronize()
         ms = time_forward_calls(fn, 10)
-        print(json.dumps({"case": name, "bytes_per_launch": 3 * M * K, "ms": round(ms, 4),
-                          "GB/s": round(3.0 * M * K / ms / 1e6, 1)}))
+        per_element = 5 if swiglu else 3
+        print(json.dumps({"case": name, "bytes_per_launch": per_element * M * K, "ms": round(ms, 4),
+                          "GB/s": round(float(per_element) * M * K / ms / 1e6, 1)}))
     else:
         raise SystemExit(f"unknown profile case {name}")
 
@@ -556,7 +578,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | prefill[:M] | quantiser[:norm]) and exit")
+    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | prefill[:M] | quantiser[:norm|:swiglu]) and exit")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)

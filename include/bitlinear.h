@@ -127,6 +127,22 @@ bitlinear_status bitlinear_rmsnorm_quantize_acts(const void *H, const float *gai
                                                  int8_t *Xq, float *beta, int32_t *rowsum, void *stream);
 
 /*
+ * SwiGLU followed by the activation quantiser, in one pass over the token: what stands in front of the down
+ * projection.  Section 2, "LLaMA-alike Components" names SwiGLU and gives no formula; this is the textbook one,
+ * h_k = silu(gate_k) * up_k with silu(g) = g / (1 + e^-g), on the bf16 outputs of the gate and up projections, with
+ * the arithmetic fixed in fp32 so that the int8 codes are reproducible bit for bit: e^-g by range reduction
+ * (n = round(-g * log2 e), r = -g - n * ln 2 with ln 2 in two parts and fused multiply-adds), the Taylor polynomial of
+ * degree 7 in Horner's scheme and an exact scaling by 2^n; sigmoid = 1 / (1 + e^-g) with one addition and one IEEE
+ * division (0 below g = -87, 1 above 87); h_k = (gate_k * sigmoid) * up_k; then quantised as above.  The product h
+ * is never written to memory.
+ *   gate, up  in   bf16 [M, K] row-major, 16-byte aligned; finite, with finite products (a token with an infinity
+ *                  or a NaN, or whose h overflows fp32, gets beta = NaN)
+ *   Xq, beta, rowsum   out, as for bitlinear_quantize_acts
+ */
+bitlinear_status bitlinear_swiglu_quantize_acts(const void *gate, const void *up, int64_t M, int64_t K,
+                                                int8_t *Xq, float *beta, int32_t *rowsum, void *stream);
+
+/*
  * The BitLinear forward: activation quantisation, ternary x int8 matmul with exact int32 accumulation,
  * dequantisation to bf16 (Section 2; no bias, "removes all biases").
  *   packed, gamma   in   from bitlinear_quantize_weights (gamma stays on the device)
@@ -147,6 +163,15 @@ bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const
 bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamma, const void *H, const float *gain,
                                            float norm_eps, int64_t M, int64_t K, int64_t N, void *Y,
                                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * The same forward with the SwiGLU of bitlinear_swiglu_quantize_acts in front of the activation quantiser (one
+ * launch forms silu(gate) * up and quantises it; the matmul and its epilogue are unchanged):
+ * Y = BitLinear(silu(gate) * up), the down projection of a feed-forward block.  gate, up: bf16 [M, K].
+ */
+bitlinear_status bitlinear_forward_swiglu(const void *packed, const float *gamma, const void *gate, const void *up,
+                                          int64_t M, int64_t K, int64_t N, void *Y,
+                                          void *workspace, size_t workspace_bytes, void *stream);
 
 /*
  * The same forward for callers that cannot give it a workspace.  (The paper has no counterpart: this is a
@@ -207,6 +232,16 @@ bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, i
 bitlinear_status bitlinear_sequence_create_rmsnorm(const bitlinear_layer_desc *layers, const float *const *gains,
                                                    float norm_eps, int n, void *workspace, size_t workspace_bytes,
                                                    bitlinear_sequence **out);
+
+/*
+ * The same with, besides, a SwiGLU (see bitlinear_swiglu_quantize_acts) in front of the quantiser of chosen entries:
+ * `ups` is a HOST array of n DEVICE pointers, ups[i] = the bf16 up input [M_i, K_i] of entry i (16-byte aligned), whose
+ * X then is the gate, or NULL for an entry without SwiGLU.  `gains` as above, or NULL when no entry is normalised; an
+ * entry takes at most one of the two (else BITLINEAR_ERR_ARG).
+ */
+bitlinear_status bitlinear_sequence_create_swiglu(const bitlinear_layer_desc *layers, const float *const *gains,
+                                                  const void *const *ups, float norm_eps, int n, void *workspace,
+                                                  size_t workspace_bytes, bitlinear_sequence **out);
 
 /* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch, one persistent matmul
  * launch that starts while the quantiser is still running (programmatic dependent launch) and one very small

@@ -26,12 +26,15 @@ EXPORTS = [
     "bitlinear_quantize_weights",
     "bitlinear_quantize_acts",
     "bitlinear_rmsnorm_quantize_acts",
+    "bitlinear_swiglu_quantize_acts",
     "bitlinear_forward",
     "bitlinear_forward_rmsnorm",
+    "bitlinear_forward_swiglu",
     "bitlinear_forward_static",
     "bitlinear_sequence_workspace_bytes",
     "bitlinear_sequence_create",
     "bitlinear_sequence_create_rmsnorm",
+    "bitlinear_sequence_create_swiglu",
     "bitlinear_forward_sequence",
     "bitlinear_forward_sequence_stage",
     "bitlinear_sequence_destroy",
@@ -84,12 +87,16 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_forward.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
     L.bitlinear_rmsnorm_quantize_acts.argtypes = [vp, vp, cf, i64, i64, vp, vp, vp, vp]
     L.bitlinear_forward_rmsnorm.argtypes = [vp, vp, vp, vp, cf, i64, i64, i64, vp, vp, sz, vp]
+    L.bitlinear_swiglu_quantize_acts.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
+    L.bitlinear_forward_swiglu.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
     L.bitlinear_forward_static.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.bitlinear_sequence_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci]
     L.bitlinear_sequence_workspace_bytes.restype = sz
     L.bitlinear_sequence_create.argtypes = [ctypes.POINTER(LayerDesc), ci, vp, sz, ctypes.POINTER(vp)]
     L.bitlinear_sequence_create_rmsnorm.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(vp), cf, ci, vp, sz,
                                                     ctypes.POINTER(vp)]
+    L.bitlinear_sequence_create_swiglu.argtypes = [ctypes.POINTER(LayerDesc), ctypes.POINTER(vp), ctypes.POINTER(vp), cf,
+                                                   ci, vp, sz, ctypes.POINTER(vp)]
     L.bitlinear_forward_sequence.argtypes = [vp, vp]
     L.bitlinear_forward_sequence_stage.argtypes = [vp, ci, vp]
     L.bitlinear_sequence_destroy.argtypes = [vp]
@@ -185,6 +192,34 @@ def forward_rmsnorm(packed: torch.Tensor, gamma: torch.Tensor, H: torch.Tensor, 
     return Y
 
 
+def swiglu_quantize_acts(gate: torch.Tensor, up: torch.Tensor, stream=None):
+    """bitlinear_swiglu_quantize_acts: bf16 gate, up [M, K] -> (Xq int8 [M, K], beta fp32 [M], rowsum int32 [M])."""
+    M, K = gate.shape
+    assert up.shape == gate.shape
+    Xq = torch.empty((M, K), dtype=torch.int8, device=gate.device)
+    beta = torch.empty(max(M, 1), dtype=torch.float32, device=gate.device)[:M]
+    rowsum = torch.empty(max(M, 1), dtype=torch.int32, device=gate.device)[:M]
+    st = load_library().bitlinear_swiglu_quantize_acts(_ptr(gate), _ptr(up), M, K, _ptr(Xq), _ptr(beta), _ptr(rowsum),
+                                                       _stream(stream))
+    _check(st, "bitlinear_swiglu_quantize_acts")
+    return Xq, beta, rowsum
+
+
+def forward_swiglu(packed: torch.Tensor, gamma: torch.Tensor, gate: torch.Tensor, up: torch.Tensor, N: int,
+                   Y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """bitlinear_forward_swiglu: BitLinear(silu(gate) * up), bf16 [M, K] x 2 -> bf16 [M, N]."""
+    M, K = gate.shape
+    assert up.shape == gate.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=gate.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, gate.device)
+    st = load_library().bitlinear_forward_swiglu(_ptr(packed), _ptr(gamma), _ptr(gate), _ptr(up), M, K, N, _ptr(Y),
+                                                 _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "bitlinear_forward_swiglu")
+    return Y
+
+
 def forward(packed: torch.Tensor, gamma: torch.Tensor, X: torch.Tensor, N: int, Y: torch.Tensor | None = None,
             workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
     """bitlinear_forward: bf16 [M, K] -> bf16 [M, N]."""
@@ -242,12 +277,15 @@ class Sequence:
     `layers` is a list of (packed, gamma, X, Y, N) with torch tensors; the object keeps them alive.
     `gains` (optional): one fp32 gain vector [K] or None per layer; those layers get an RMSNorm with `norm_eps` in front
     of their activation quantiser (bitlinear_sequence_create_rmsnorm).
+    `ups` (optional): one bf16 tensor [M, K] or None per layer; those layers quantise silu(X) * up
+    (bitlinear_sequence_create_swiglu).
     """
 
-    def __init__(self, layers, device="cuda", gains=None, norm_eps: float = 1e-5):
+    def __init__(self, layers, device="cuda", gains=None, norm_eps: float = 1e-5, ups=None):
         L = load_library()
         self._keep = list(layers)
         self._gains = list(gains) if gains is not None else None
+        self._ups = list(ups) if ups is not None else None
         n = len(self._keep)
         arr = (LayerDesc * n)()
         for i, (packed, gamma, X, Y, N) in enumerate(self._keep):
@@ -258,7 +296,15 @@ class Sequence:
             raise BitLinearError(ERR_SHAPE, "bitlinear_sequence_workspace_bytes")
         self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=device)
         handle = ctypes.c_void_p()
-        if self._gains is None:
+        def pointers(tensors):
+            assert len(tensors) == n
+            return (ctypes.c_void_p * n)(*[(_ptr(x) if x is not None else None) for x in tensors])
+
+        if self._ups is not None:
+            st = L.bitlinear_sequence_create_swiglu(arr, pointers(self._gains) if self._gains is not None else None,
+                                                    pointers(self._ups), float(norm_eps), n, _ptr(self.workspace), nbytes,
+                                                    ctypes.byref(handle))
+        elif self._gains is None:
             st = L.bitlinear_sequence_create(arr, n, _ptr(self.workspace), nbytes, ctypes.byref(handle))
         else:
             assert len(self._gains) == n

@@ -136,6 +136,7 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.xq_tiled = 0;
     e.gain = nullptr;
     e.norm_eps = 0.0f;
+    e.up = nullptr;
 }
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
@@ -223,15 +224,16 @@ bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K
 }
 
 namespace {
-// gain == null: the plain quantiser
-bitlinear_status quantize_acts_rows(const void *X, const float *gain, float norm_eps, int64_t M, int64_t K, int8_t *Xq,
-                                    float *beta, int32_t *rowsum, void *stream)
+// gain == null and up == null: the plain quantiser; gain: RMSNorm in front; up: SwiGLU in front (X is the gate)
+bitlinear_status quantize_acts_rows(const void *X, const void *up, const float *gain, float norm_eps, int64_t M, int64_t K,
+                                    int8_t *Xq, float *beta, int32_t *rowsum, void *stream)
 {
     if (M > 0 && (!X || !Xq || !beta || !rowsum)) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, 16, K);
     if (st != BITLINEAR_OK) return st;
     if (!aligned(X, 16) || !aligned(Xq, 16) || !aligned(beta, 4) || !aligned(rowsum, 4)) return BITLINEAR_ERR_ALIGN;
     if (gain && !aligned(gain, 16)) return BITLINEAR_ERR_ALIGN;
+    if (up && !aligned(up, 16)) return BITLINEAR_ERR_ALIGN;
     if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
     if (M == 0) return BITLINEAR_OK;
     InlineTable inl{};
@@ -244,7 +246,9 @@ bitlinear_status quantize_acts_rows(const void *X, const float *gain, float norm
     e.K = (int)K;
     e.gain = gain;
     e.norm_eps = norm_eps;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, gain != nullptr, (int)K, (cudaStream_t)stream);
+    e.up = reinterpret_cast<const __nv_bfloat16 *>(up);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, (gain ? 1 : 0) | (up ? 2 : 0), (int)K,
+                                           (cudaStream_t)stream);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 } // namespace
@@ -252,26 +256,33 @@ bitlinear_status quantize_acts_rows(const void *X, const float *gain, float norm
 bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K, int8_t *Xq, float *beta,
                                          int32_t *rowsum, void *stream)
 {
-    return quantize_acts_rows(X, nullptr, 0.0f, M, K, Xq, beta, rowsum, stream);
+    return quantize_acts_rows(X, nullptr, nullptr, 0.0f, M, K, Xq, beta, rowsum, stream);
 }
 
 bitlinear_status bitlinear_rmsnorm_quantize_acts(const void *H, const float *gain, float norm_eps, int64_t M, int64_t K,
                                                  int8_t *Xq, float *beta, int32_t *rowsum, void *stream)
 {
     if (!gain || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
-    return quantize_acts_rows(H, gain, norm_eps, M, K, Xq, beta, rowsum, stream);
+    return quantize_acts_rows(H, nullptr, gain, norm_eps, M, K, Xq, beta, rowsum, stream);
+}
+
+bitlinear_status bitlinear_swiglu_quantize_acts(const void *gate, const void *up, int64_t M, int64_t K, int8_t *Xq,
+                                                float *beta, int32_t *rowsum, void *stream)
+{
+    if (M > 0 && !up) return BITLINEAR_ERR_ARG;
+    return quantize_acts_rows(gate, up, nullptr, 0.0f, M, K, Xq, beta, rowsum, stream);
 }
 
 namespace {
-bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const float *gain, float norm_eps,
-                              int64_t M, int64_t K, int64_t N, void *Y, void *workspace, size_t workspace_bytes,
-                              void *stream);
+bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const void *up, const float *gain,
+                              float norm_eps, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
+                              size_t workspace_bytes, void *stream);
 }
 
 bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
                                    int64_t N, void *Y, void *workspace, size_t workspace_bytes, void *stream)
 {
-    return forward_impl(packed, gamma, X, nullptr, 0.0f, M, K, N, Y, workspace, workspace_bytes, stream);
+    return forward_impl(packed, gamma, X, nullptr, nullptr, 0.0f, M, K, N, Y, workspace, workspace_bytes, stream);
 }
 
 bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamma, const void *H, const float *gain,
@@ -280,14 +291,23 @@ bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamm
 {
     if (!gain || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
     if (!aligned(gain, 16)) return BITLINEAR_ERR_ALIGN;
-    return forward_impl(packed, gamma, H, gain, norm_eps, M, K, N, Y, workspace, workspace_bytes, stream);
+    return forward_impl(packed, gamma, H, nullptr, gain, norm_eps, M, K, N, Y, workspace, workspace_bytes, stream);
+}
+
+bitlinear_status bitlinear_forward_swiglu(const void *packed, const float *gamma, const void *gate, const void *up,
+                                          int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
+                                          size_t workspace_bytes, void *stream)
+{
+    if (M > 0 && !up) return BITLINEAR_ERR_ARG;
+    if (!aligned(up, 16)) return BITLINEAR_ERR_ALIGN;
+    return forward_impl(packed, gamma, gate, up, nullptr, 0.0f, M, K, N, Y, workspace, workspace_bytes, stream);
 }
 
 namespace {
-// gain == null: no normalisation in front of the quantiser
-bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const float *gain, float norm_eps,
-                              int64_t M, int64_t K, int64_t N, void *Y, void *workspace, size_t workspace_bytes,
-                              void *stream)
+// gain == null: no normalisation in front of the quantiser; up != null: X is the gate of a SwiGLU in front of it
+bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const void *up, const float *gain,
+                              float norm_eps, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
+                              size_t workspace_bytes, void *stream)
 {
     if (!packed || !gamma || !workspace || (M > 0 && (!X || !Y))) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, N, K);
@@ -305,11 +325,13 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     inl.e[0].xq_tiled = tc ? 0 : 1;
     inl.e[0].gain = gain;
     inl.e[0].norm_eps = norm_eps;
+    inl.e[0].up = reinterpret_cast<const __nv_bfloat16 *>(up);
     // quantise the tokens; the same launch clears the header and the scratch of the kernel that follows, if it uses it
     const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
-    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, gain != nullptr, (int)K, (cudaStream_t)stream);
+    cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (gain ? 1 : 0) | (up ? 2 : 0), (int)K,
+                                           (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M,
                       split ? ws + L.acc32 : nullptr, (cudaStream_t)stream);
@@ -419,7 +441,7 @@ struct bitlinear_sequence {
     bitlinear::InlineTable inl;
     const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
     int gemm_tiles, gemm_min_kb;
-    bool with_norm;         // some entry is normalised (RMSNorm) in front of the quantiser
+    int fronts;             // bit 0: some entry has an RMSNorm in front of the quantiser, bit 1: some entry a SwiGLU
     void *split_scratch;    // inside the workspace; null: no GEMM tile of this sequence is cut along K
 };
 
@@ -489,14 +511,15 @@ size_t bitlinear_sequence_workspace_bytes(const bitlinear_layer_desc *layers, in
 }
 
 namespace {
-bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains, float norm_eps,
-                                      int n, void *workspace, size_t workspace_bytes, bitlinear_sequence **out);
+bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains,
+                                      const void *const *ups, float norm_eps, int n, void *workspace,
+                                      size_t workspace_bytes, bitlinear_sequence **out);
 }
 
 bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
                                            size_t workspace_bytes, bitlinear_sequence **out)
 {
-    return sequence_create_impl(layers, nullptr, 0.0f, n, workspace, workspace_bytes, out);
+    return sequence_create_impl(layers, nullptr, nullptr, 0.0f, n, workspace, workspace_bytes, out);
 }
 
 bitlinear_status bitlinear_sequence_create_rmsnorm(const bitlinear_layer_desc *layers, const float *const *gains,
@@ -506,13 +529,26 @@ bitlinear_status bitlinear_sequence_create_rmsnorm(const bitlinear_layer_desc *l
     if (!gains || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
     for (int i = 0; i < n; ++i)
         if (gains[i] && !aligned(gains[i], 16)) return BITLINEAR_ERR_ALIGN;
-    return sequence_create_impl(layers, gains, norm_eps, n, workspace, workspace_bytes, out);
+    return sequence_create_impl(layers, gains, nullptr, norm_eps, n, workspace, workspace_bytes, out);
+}
+
+bitlinear_status bitlinear_sequence_create_swiglu(const bitlinear_layer_desc *layers, const float *const *gains,
+                                                  const void *const *ups, float norm_eps, int n, void *workspace,
+                                                  size_t workspace_bytes, bitlinear_sequence **out)
+{
+    if (!ups || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
+    for (int i = 0; i < n; ++i) {
+        if (gains && gains[i] && ups[i]) return BITLINEAR_ERR_ARG; // one front per entry
+        if ((gains && gains[i] && !aligned(gains[i], 16)) || (ups[i] && !aligned(ups[i], 16))) return BITLINEAR_ERR_ALIGN;
+    }
+    return sequence_create_impl(layers, gains, ups, norm_eps, n, workspace, workspace_bytes, out);
 }
 
 namespace {
-// gains == null: no entry is normalised; gains[i] == null: entry i is not
-bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains, float norm_eps,
-                                      int n, void *workspace, size_t workspace_bytes, bitlinear_sequence **out)
+// gains == null: no entry is normalised; gains[i] == null: entry i is not; ups likewise (SwiGLU in front)
+bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains,
+                                      const void *const *ups, float norm_eps, int n, void *workspace,
+                                      size_t workspace_bytes, bitlinear_sequence **out)
 {
     if (!layers || !workspace || !out || n <= 0) return BITLINEAR_ERR_ARG;
     *out = nullptr;
@@ -540,7 +576,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     const bool gemm = S.use_gemm;
     std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
     int gemm_tiles = 0;
-    bool with_norm = false;
+    int fronts = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         Layout L{};
@@ -554,7 +590,8 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
         e.xq_tiled = gemm ? 0 : 1;
         e.gain = gains ? gains[i] : nullptr;
         e.norm_eps = norm_eps;
-        with_norm = with_norm || e.gain != nullptr;
+        e.up = reinterpret_cast<const __nv_bfloat16 *>(ups ? ups[i] : nullptr);
+        fronts |= (e.gain ? 1 : 0) | (e.up ? 2 : 0);
         e.tile_begin = tiles;
         e.token_begin = tokens;
         tiles += decode_items(e.NB, e.KB, wide);
@@ -586,7 +623,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     seq->gemm_table = nullptr;
     seq->gemm_tiles = gemm_tiles;
     seq->gemm_min_kb = S.min_kb;
-    seq->with_norm = with_norm;
+    seq->fronts = fronts;
     seq->split_scratch = split ? ws + S.acc32 : nullptr;
     if (gemm) {
         if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -616,7 +653,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
     cudaStream_t s = (cudaStream_t)stream;
     if (stage != 2 &&
         launch_quantize_acts(seq->inl, seq->dev_table, seq->n, seq->tokens, seq->workspace, seq->zero_bytes,
-                             seq->with_norm, seq->max_K, s) !=
+                             seq->fronts, seq->max_K, s) !=
             cudaSuccess)
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {

@@ -58,6 +58,7 @@ struct DecodeEntry {
     int xq_tiled;          // layout of Xq (the streaming kernel reads tiles, the tensor-core GEMM rows)
     const float *gain;     // null, or [K] fp32: X is normalised first (RMSNorm with this gain) and then quantised
     float norm_eps;        // the RMSNorm's epsilon (added to the mean square)
+    const __nv_bfloat16 *up; // null, or bf16 [M, K]: the quantiser's input is silu(X) * up (SwiGLU; X holds the gate)
 };
 
 constexpr int kInlineEntries = 4;
@@ -76,10 +77,10 @@ cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, c
 cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *tiled, cudaStream_t stream);
 
 // Quantises the tokens of every entry (entries with X == nullptr are skipped) and zeroes
-// `zero_bytes` bytes at `zero_ptr` (control words and split-K scratch) in the same launch.  with_norm: some entry
-// carries a gain vector (RMSNorm in front of the quantiser).  max_K: the longest token among the entries.
+// `zero_bytes` bytes at `zero_ptr` (control words and split-K scratch) in the same launch.  fronts: bit 0, some
+// entry carries a gain vector (RMSNorm in front of the quantiser); bit 1, some entry a second input (SwiGLU).  max_K: the longest token among the entries.
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
-                                 void *zero_ptr, size_t zero_bytes, bool with_norm, int max_K, cudaStream_t stream);
+                                 void *zero_ptr, size_t zero_bytes, int fronts, int max_K, cudaStream_t stream);
 
 // The weight-streaming matmul has two kernels: up to 8 tokens every warp streams tiles on its own; from 9
 // tokens the eight warps of a CTA share the activations and the CTA walks group tiles (8 row blocks x 1

@@ -18,6 +18,13 @@
 // below the largest add nothing), sum h^2 = S * 2^(2E - 298).  Then mean = (float)((double)S / K * 2^(2E - 298)),
 // r = 1 / sqrt(max(mean + eps, 2^-126)) with IEEE fp32 add, square root and divide, x_k = (h_k * r) * g_k with two fp32
 // multiplications.  A token with an infinity or a NaN gets beta = NaN.
+//
+// With a second input the token is h_k = silu(gate_k) * up_k (SwiGLU, another of those components: the input of the
+// down projection), then quantised as above; the arithmetic is fixed again.  e^-g: z = -g * log2(e), n = z rounded to
+// the nearest integer (ties to even), r = fma(n, -ln2_hi, -g), r = fma(n, -ln2_lo, r), p = the Taylor polynomial of
+// degree 7 in r by Horner's scheme (seven fused multiply-adds), e^-g = p * 2^n (exact); sigmoid = 1 / (1 + e^-g) with
+// one addition and one IEEE reciprocal, taken as 0 below g = -87 and as 1 above 87; h = (g * sigmoid) * u with two
+// multiplications.  A token with an infinity or a NaN in either input, or with a product beyond fp32, gets beta = NaN.
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -53,6 +60,40 @@ __device__ __forceinline__ uint32_t pack4(float a, float b, float c, float d)
     return out;
 }
 
+// sigmoid(g) in the fixed fp32 steps stated at the head of this file
+__device__ __forceinline__ float sigmoid_steps(float g)
+{
+    const float t = -g;
+    const float tc = fminf(fmaxf(t, -87.0f), 87.0f); // (outside, the result is replaced below)
+    const float z = __fmul_rn(tc, 1.44269502162933349609375f); // log2(e)
+    const float n = rintf(z);
+    float r = __fmaf_rn(n, -0.693145751953125f, tc);             // ln2_hi: exact product
+    r = __fmaf_rn(n, -1.42860676533018704503775e-06f, r);        // ln2_lo
+    float p = __fmaf_rn(r, 1.0f / 5040.0f, 1.0f / 720.0f);
+    p = __fmaf_rn(p, r, 1.0f / 120.0f);
+    p = __fmaf_rn(p, r, 1.0f / 24.0f);
+    p = __fmaf_rn(p, r, 1.0f / 6.0f);
+    p = __fmaf_rn(p, r, 0.5f);
+    p = __fmaf_rn(p, r, 1.0f);
+    p = __fmaf_rn(p, r, 1.0f);
+    const float e = __fmul_rn(p, __int_as_float(((int)n + 127) << 23)); // |n| <= 126: 2^n is a normal number
+    const float sg = __frcp_rn(__fadd_rn(1.0f, e));                      // correctly rounded: the same as 1 / (1 + e)
+    return t > 87.0f ? 0.0f : (t < -87.0f ? 1.0f : sg);
+}
+
+// h = silu(gate) * up of eight elements
+__device__ __forceinline__ void swiglu8(const uint4 &gv, const uint4 &uv, float (&h)[8])
+{
+    const uint32_t gw[4] = {gv.x, gv.y, gv.z, gv.w}, uw[4] = {uv.x, uv.y, uv.z, uv.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        const float g0 = __uint_as_float(gw[j] << 16), g1 = __uint_as_float(gw[j] & 0xFFFF0000u);
+        const float u0 = __uint_as_float(uw[j] << 16), u1 = __uint_as_float(uw[j] & 0xFFFF0000u);
+        h[2 * j] = __fmul_rn(__fmul_rn(g0, sigmoid_steps(g0)), u0);
+        h[2 * j + 1] = __fmul_rn(__fmul_rn(g1, sigmoid_steps(g1)), u1);
+    }
+}
+
 // 8 bf16 -> 8 int8 (two 32-bit words), returns the sum of the eight codes
 __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
 {
@@ -68,12 +109,14 @@ __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
     return __dp4a((int)out.x, 0x01010101, __dp4a((int)out.y, 0x01010101, 0));
 }
 
-// kNorm: entries may carry a gain vector (RMSNorm in front); the plain form is compiled without that branch.
+// kFronts: bit 0, entries may carry a gain vector (RMSNorm in front); bit 1, a second input (SwiGLU in front).  Each
+// form is compiled with the branches it needs only, and with the registers they need (a thread keeps 16-byte vectors
+// of the token, or, for SwiGLU, the products themselves, in registers between the passes).
 // NT threads per token (64, 128, 192 or 256): what a CTA does besides touching its elements (finding its entry,
 // three block-wide reductions) is a fixed cost per thread, so short tokens take fewer threads with kCache vectors
 // each.  Tokens of more than 8192 elements re-read their tail, which hits L2.
-template <bool kNorm, int NT>
-__global__ void __launch_bounds__(NT, (kNorm ? 768 : 1024) / NT) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
+template <int kFronts, int NT>
+__global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
                                                                  const DecodeEntry *__restrict__ table, int n_entries,
                                                                  int total_tokens, uint4 *zero_ptr, size_t zero_vecs)
 {
@@ -116,7 +159,7 @@ __global__ void __launch_bounds__(NT, (kNorm ? 768 : 1024) / NT) quantize_acts_k
     uint4 cache[kCache];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
-    if (kNorm && e.gain) {
+    if ((kFronts & 1) && e.gain) {
         // ---- RMSNorm, then the quantiser on the fp32 values (see the head of this file)
         const float4 *gain4 = reinterpret_cast<const float4 *>(e.gain);
         // largest magnitude of the token: |bf16| as a 15-bit integer is monotone, its upper 8 bits are the exponent
@@ -243,6 +286,73 @@ __global__ void __launch_bounds__(NT, (kNorm ? 768 : 1024) / NT) quantize_acts_k
         return;
     }
 
+    if ((kFronts & 2) && e.up) {
+        // ---- SwiGLU, then the quantiser on the fp32 values (see the head of this file).  The values of the first
+        // 8 * kCache * NT elements stay in registers; longer tokens form the rest a second time.
+        const uint4 *urow = reinterpret_cast<const uint4 *>(e.up + (size_t)t * K);
+        float hc[kCache][8];
+        uint32_t raw = 0; // largest |gate|, |up| as 15-bit integers: tells infinities and NaNs
+        uint32_t mx = 0;  // largest |h| as an unsigned integer
+        auto form = [&](int i, float (&h)[8]) {
+            const uint4 gv = __ldg(row + i), uv = __ldg(urow + i);
+            raw = absmax_bits(absmax_bits(raw, gv), uv);
+            swiglu8(gv, uv, h);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) mx = max(mx, __float_as_uint(h[j]) & 0x7FFFFFFFu);
+        };
+#pragma unroll
+        for (int c = 0; c < kCache; ++c) {
+            const int i = threadIdx.x + c * NT;
+            if (i < n_vec) form(i, hc[c]);
+        }
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
+            float h[8];
+            form(i, h);
+        }
+        if ((raw >> 7) == 255u) mx = 0x7FC00000u;
+        mx = __reduce_max_sync(0xffffffffu, mx);
+        if (lane == 0) s_max[warp] = mx;
+        __syncthreads();
+        mx = s_max[0];
+#pragma unroll
+        for (int w = 1; w < NT / 32; ++w) mx = max(mx, s_max[w]);
+        const bool bad = mx >= 0x7F800000u; // an infinity or a NaN in an input, or a product beyond fp32
+        const float b = fmaxf(__uint_as_float(mx), kBetaFloor);
+        const float s = __fdiv_rn((float)kQb, b);
+
+        int sum = 0;
+        auto quantise8 = [&](const float (&h)[8], int i) {
+            uint2 o;
+            o.x = pack4(__fmul_rn(h[0], s), __fmul_rn(h[1], s), __fmul_rn(h[2], s), __fmul_rn(h[3], s));
+            o.y = pack4(__fmul_rn(h[4], s), __fmul_rn(h[5], s), __fmul_rn(h[6], s), __fmul_rn(h[7], s));
+            out_at(i) = o;
+            sum = __dp4a((int)o.x, 0x01010101, __dp4a((int)o.y, 0x01010101, sum));
+        };
+#pragma unroll
+        for (int c = 0; c < kCache; ++c) {
+            const int i = threadIdx.x + c * NT;
+            if (i < n_vec) quantise8(hc[c], i);
+        }
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
+            float h[8];
+            swiglu8(__ldg(row + i), __ldg(urow + i), h);
+            quantise8(h, i);
+        }
+        if (tiled) // the last column tile is filled up with zeros
+            for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += NT) out_at(i) = make_uint2(0u, 0u);
+        sum = __reduce_add_sync(0xffffffffu, sum);
+        if (lane == 0) s_sum[warp] = sum;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int total = 0;
+#pragma unroll
+            for (int w = 0; w < NT / 32; ++w) total += s_sum[w];
+            e.beta[t] = bad ? __int_as_float(0x7FC00000) : b;
+            e.rowsum[t] = total;
+        }
+        return;
+    }
+
     uint32_t m = 0;
 #pragma unroll
     for (int c = 0; c < kCache; ++c) {
@@ -316,7 +426,7 @@ cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *t
 }
 
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
-                                 void *zero_ptr, size_t zero_bytes, bool with_norm, int max_K, cudaStream_t stream)
+                                 void *zero_ptr, size_t zero_bytes, int fronts, int max_K, cudaStream_t stream)
 {
     // threads per token: the smallest count whose register caches hold the longest token
     const int n_vec = max_K >> 3;
@@ -339,12 +449,16 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     const int grid = total_tokens + zero_blocks;
     if (grid == 0) return cudaSuccess;
     uint4 *zp = reinterpret_cast<uint4 *>(zero_ptr);
-#define BITLINEAR_LAUNCH_QUANTISER(NORM, NT_) \
-    quantize_acts_kernel<NORM, NT_><<<grid, NT_, 0, stream>>>(inl, table, n_entries, total_tokens, zp, zero_vecs)
+#define BITLINEAR_LAUNCH_QUANTISER(FRONTS, NT_) \
+    quantize_acts_kernel<FRONTS, NT_><<<grid, NT_, 0, stream>>>(inl, table, n_entries, total_tokens, zp, zero_vecs)
 #define BITLINEAR_LAUNCH_BOTH(NT_) \
     do { \
-        if (with_norm) BITLINEAR_LAUNCH_QUANTISER(true, NT_); \
-        else BITLINEAR_LAUNCH_QUANTISER(false, NT_); \
+        switch (fronts & 3) { \
+        case 0: BITLINEAR_LAUNCH_QUANTISER(0, NT_); break; \
+        case 1: BITLINEAR_LAUNCH_QUANTISER(1, NT_); break; \
+        case 2: BITLINEAR_LAUNCH_QUANTISER(2, NT_); break; \
+        default: BITLINEAR_LAUNCH_QUANTISER(3, NT_); break; \
+        } \
     } while (0)
     switch (nt) {
     case 64: BITLINEAR_LAUNCH_BOTH(64); break;
