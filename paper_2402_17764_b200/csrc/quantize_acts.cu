@@ -64,9 +64,12 @@ __device__ __forceinline__ uint32_t pack4(float a, float b, float c, float d)
 __device__ __forceinline__ float sigmoid_steps(float g)
 {
     const float t = -g;
-    const float tc = fminf(fmaxf(t, -87.0f), 87.0f); // (outside, the result is replaced below)
+    const float tc = fminf(fmaxf(t, -87.0f), 87.0f); // (beyond 87 the result is replaced below)
     const float z = __fmul_rn(tc, 1.44269502162933349609375f); // log2(e)
-    const float n = rintf(z);
+    // |z| < 2^22: adding 1.5 * 2^23 rounds z to the nearest integer, ties to even, and leaves it in the low bits
+    const float shifted = __fadd_rn(z, 12582912.0f);
+    const float n = __fadd_rn(shifted, -12582912.0f);
+    const int ni = __float_as_int(shifted) - 0x4B400000;
     float r = __fmaf_rn(n, -0.693145751953125f, tc);             // ln2_hi: exact product
     r = __fmaf_rn(n, -1.42860676533018704503775e-06f, r);        // ln2_lo
     float p = __fmaf_rn(r, 1.0f / 5040.0f, 1.0f / 720.0f);
@@ -76,9 +79,11 @@ __device__ __forceinline__ float sigmoid_steps(float g)
     p = __fmaf_rn(p, r, 0.5f);
     p = __fmaf_rn(p, r, 1.0f);
     p = __fmaf_rn(p, r, 1.0f);
-    const float e = __fmul_rn(p, __int_as_float(((int)n + 127) << 23)); // |n| <= 126: 2^n is a normal number
-    const float sg = __frcp_rn(__fadd_rn(1.0f, e));                      // correctly rounded: the same as 1 / (1 + e)
-    return t > 87.0f ? 0.0f : (t < -87.0f ? 1.0f : sg);
+    // p * 2^n by adding n to the exponent field: p lies in [0.7, 1.42] and e^t >= e^-87 is a normal number
+    const float e = __int_as_float(__float_as_int(p) + ni * 8388608);
+    const float sg = __frcp_rn(__fadd_rn(1.0f, e)); // correctly rounded: the same as 1 / (1 + e)
+    // (for g > 87 the steps give e^-87 < 2^-125, 1 + e = 1 and so exactly 1 by themselves)
+    return t > 87.0f ? 0.0f : sg;
 }
 
 // h = silu(gate) * up of eight elements
@@ -291,12 +296,11 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
         // 8 * kCache * NT elements stay in registers; longer tokens form the rest a second time.
         const uint4 *urow = reinterpret_cast<const uint4 *>(e.up + (size_t)t * K);
         float hc[kCache][8];
-        uint32_t raw = 0; // largest |gate|, |up| as 15-bit integers: tells infinities and NaNs
-        uint32_t mx = 0;  // largest |h| as an unsigned integer
+        // largest |h| as an unsigned integer.  An infinity or a NaN in either input makes h an infinity or a NaN (a
+        // gate of -inf: -inf * 0), and their bit patterns are the largest.
+        uint32_t mx = 0;
         auto form = [&](int i, float (&h)[8]) {
-            const uint4 gv = __ldg(row + i), uv = __ldg(urow + i);
-            raw = absmax_bits(absmax_bits(raw, gv), uv);
-            swiglu8(gv, uv, h);
+            swiglu8(__ldg(row + i), __ldg(urow + i), h);
 #pragma unroll
             for (int j = 0; j < 8; ++j) mx = max(mx, __float_as_uint(h[j]) & 0x7FFFFFFFu);
         };
@@ -309,7 +313,6 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
             float h[8];
             form(i, h);
         }
-        if ((raw >> 7) == 255u) mx = 0x7FC00000u;
         mx = __reduce_max_sync(0xffffffffu, mx);
         if (lane == 0) s_max[warp] = mx;
         __syncthreads();
@@ -431,10 +434,11 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     // threads per token: the smallest count whose register caches hold the longest token
     const int n_vec = max_K >> 3;
     // (longer tokens re-read their tail, which hits L2: CTAs of 512 and 1024 threads measured slower)
-    static const int counts[4] = {64, 128, 192, 256};
-    int nt = 256;
+    // (with SwiGLU in front a token beyond the caches costs its exponentials a second time: 384 threads there)
+    static const int counts[5] = {64, 128, 192, 256, 384};
+    int nt = (fronts & 2) ? 384 : 256;
     for (int c : counts)
-        if (n_vec <= c * kCache) {
+        if (n_vec <= c * kCache && c <= nt) {
             nt = c;
             break;
         }
@@ -464,6 +468,10 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     case 64: BITLINEAR_LAUNCH_BOTH(64); break;
     case 128: BITLINEAR_LAUNCH_BOTH(128); break;
     case 192: BITLINEAR_LAUNCH_BOTH(192); break;
+    case 384:
+        if (fronts & 1) BITLINEAR_LAUNCH_QUANTISER(3, 384);
+        else BITLINEAR_LAUNCH_QUANTISER(2, 384);
+        break;
     default: BITLINEAR_LAUNCH_BOTH(256); break;
     }
 #undef BITLINEAR_LAUNCH_BOTH
