@@ -468,6 +468,63 @@ int oracle_dequant(const int32_t *acc, const float *beta, float gamma, int64_t M
     return ORACLE_OK;
 }
 
+/* ---------- activations of fewer bits ----------
+ *
+ * The paper's outlook (Section 4, on long sequences) expects the activations to go from 8 bits to 4 bits or fewer.
+ * The same forward with b-bit activations, 2 <= b <= 8 (readings, not the paper's):
+ *   B1  Q_b = 2^(b-1) - 1 (b = 8: the 127 of R4; b = 4: 7), symmetric, no zero point;
+ *   B2  beta, the one divide s = Q_b / beta per token, one multiply per element, round half to even and the clip
+ *       to [-Q_b, Q_b] as in R5, R6; the codes are still delivered one per byte;
+ *   B3  dequantisation by (gamma * beta_t) / Q_b, as in R7, R8.
+ * Parity pins (tests/test_oracle_pins.py): a hand case with ties, equality with the 8-bit functions for b = 8, the
+ * value set, the error bound |x - q * beta / Q_b| <= beta / (2 Q_b), the double-precision product.
+ */
+int oracle_quantize_acts_bits(const uint16_t *X_bf16, int64_t M, int64_t K, int bits,
+                              int8_t *Xq, float *beta, int32_t *rowsum)
+{
+    if (!X_bf16 || !Xq || !beta || !rowsum || M < 0 || K <= 0 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    const int qb = (1 << (bits - 1)) - 1; /* B1 */
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        float amax = 0.0f;
+        for (int64_t k = 0; k < K; ++k) {
+            float a = fabsf(bf16_to_float(X_bf16[t * K + k]));
+            if (a > amax) amax = a;
+        }
+        float b = amax > BETA_FLOOR ? amax : BETA_FLOOR;
+        float s = (float)qb / b; /* B2 */
+        int32_t sum = 0;
+        for (int64_t k = 0; k < K; ++k) {
+            int q = round_clip(bf16_to_float(X_bf16[t * K + k]) * s, -qb, qb);
+            Xq[t * K + k] = (int8_t)q;
+            sum += q;
+        }
+        beta[t] = b;
+        rowsum[t] = sum;
+    }
+    return ORACLE_OK;
+}
+
+int oracle_dequant_bits(const int32_t *acc, const float *beta, float gamma, int64_t M, int64_t N, int bits,
+                        uint16_t *Y_bf16)
+{
+    if (!acc || !beta || !Y_bf16 || M < 0 || N <= 0 || bits < 2 || bits > 8)
+        return ORACLE_ERR_ARG;
+    const int qb = (1 << (bits - 1)) - 1;
+#ifdef _OPENMP
+#pragma omp parallel for
+#endif
+    for (int64_t t = 0; t < M; ++t) {
+        float scale = (gamma * beta[t]) / (float)qb; /* B3 */
+        for (int64_t n = 0; n < N; ++n)
+            Y_bf16[t * N + n] = float_to_bf16_rne((float)acc[t * N + n] * scale);
+    }
+    return ORACLE_OK;
+}
+
 /* ---------- the whole forward for an already ternarised weight matrix ---------- */
 
 /*

@@ -58,6 +58,8 @@ class Oracle:
         L.oracle_quantize_acts.argtypes = [_p, _i64, _i64, _p, _p, _p]
         L.oracle_rmsnorm_quantize_acts.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p, _p, _p, _p]
         L.oracle_swiglu_quantize_acts.argtypes = [_p, _p, _i64, _i64, _p, _p, _p, _p]
+        L.oracle_quantize_acts_bits.argtypes = [_p, _i64, _i64, ctypes.c_int, _p, _p, _p]
+        L.oracle_dequant_bits.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, ctypes.c_int, _p]
         L.oracle_matmul_i32.argtypes = [_p, _p, _i64, _i64, _i64, _p]
         L.oracle_dequant.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p]
         L.oracle_forward.argtypes = [_p, ctypes.c_float, _p, _i64, _i64, _i64, _p, _p, _p, _p, _p]
@@ -125,6 +127,27 @@ class Oracle:
         rc = self.lib.oracle_quantize_acts(self._ptr(X), M, K, self._ptr(Xq), self._ptr(beta), self._ptr(rs))
         self._check(rc, "quantize_acts")
         return Xq, beta, rs
+
+    def quantize_acts_bits(self, X_bf16_bits: np.ndarray, bits: int):
+        """The activation quantiser with Q_b = 2^(bits-1) - 1 -> (Xq int8 [M,K], beta float32 [M], rowsum int32 [M])."""
+        X = self._c(X_bf16_bits, np.uint16)
+        M, K = X.shape
+        Xq = np.empty((M, K), np.int8)
+        beta = np.empty(M, np.float32)
+        rs = np.empty(M, np.int32)
+        rc = self.lib.oracle_quantize_acts_bits(self._ptr(X), M, K, int(bits), self._ptr(Xq), self._ptr(beta), self._ptr(rs))
+        self._check(rc, "quantize_acts_bits")
+        return Xq, beta, rs
+
+    def dequant_bits(self, acc: np.ndarray, beta: np.ndarray, gamma, bits: int) -> np.ndarray:
+        acc = self._c(acc, np.int32)
+        beta = self._c(beta, np.float32)
+        M, N = acc.shape
+        Y = np.empty((M, N), np.uint16)
+        rc = self.lib.oracle_dequant_bits(self._ptr(acc), self._ptr(beta), ctypes.c_float(float(gamma)), M, N, int(bits),
+                                          self._ptr(Y))
+        self._check(rc, "dequant_bits")
+        return Y
 
     def rmsnorm_quantize_acts(self, H_bf16_bits: np.ndarray, gain: np.ndarray, eps_n: float, return_x: bool = False):
         """RMSNorm (gain, eps_n) followed by the activation quantiser -> (Xq, beta, rowsum[, x float32 [M,K]])."""

@@ -420,3 +420,54 @@ def test_swiglu_quantiser_invariants(oracle):
     for gv, uv in ((np.inf, 1.0), (1.0, np.nan), (-np.inf, 1.0), (2.0 ** 100, 2.0 ** 100)):
         with pytest.raises(ValueError):
             oracle.swiglu_quantize_acts(_bf16([[gv] + [0.0] * 15]), _bf16([[uv] + [1.0] * 15]))
+
+
+# ---- activations of fewer bits ----
+
+def test_low_bit_activations_hand_case(oracle):
+    """b = 4: Q_b = 7.  A token with absmax 7 has s = 1: codes are the values rounded half to even."""
+    x = _bf16([[7.0, 2.5, 3.5, -1.5, 0.5, -0.5, 6.5, -7.0, 0.25, 1.0, 0, 0, 0, 0, 0, 0]])
+    q, beta, rs = oracle.quantize_acts_bits(x, 4)
+    assert q.tolist() == [[7, 2, 4, -2, 0, 0, 6, -7, 0, 1, 0, 0, 0, 0, 0, 0]] and beta.tolist() == [7.0] and rs.tolist() == [11]
+    # absmax 4: s = 1.75; 1 -> 1.75 -> 2, -2 -> -3.5 -> -4 (tie to even), 0.5 -> 0.875 -> 1, 0.25 -> 0.4375 -> 0
+    q, beta, _ = oracle.quantize_acts_bits(_bf16([[1.0, -2.0, 0.5, 4.0, 0.25] + [0.0] * 11]), 4)
+    assert q[0, :5].tolist() == [2, -4, 1, 7, 0] and beta.tolist() == [4.0]
+    # b = 2: Q_b = 1, a sign with a dead zone below half the absmax
+    q, _, _ = oracle.quantize_acts_bits(_bf16([[1.0, -0.75, 0.5, 0.25, -1.0] + [0.0] * 11]), 2)
+    assert q[0, :5].tolist() == [1, -1, 0, 0, -1]
+    # dequantisation: 14 * (0.5 * 2) / 7 = 2
+    y = oracle.dequant_bits(np.array([[14, -7, 1]], np.int32), np.array([2.0], np.float32), 0.5, 4)
+    assert bits_to_f32(y).tolist() == [[2.0, -1.0, float(bits_to_f32(_bf16([1.0 / 7.0]))[0])]]
+    for bad in (1, 9):
+        with pytest.raises(ValueError):
+            oracle.quantize_acts_bits(x, bad)
+
+
+def test_low_bit_activations_properties(oracle):
+    rng = np.random.default_rng(41)
+    M, K, N = 7, 640, 48
+    xb = _bf16(rng.standard_normal((M, K)))
+    xf = bits_to_f32(xb).astype(np.float64)
+    # b = 8 is the quantiser of Section 2
+    for a, b in zip(oracle.quantize_acts_bits(xb, 8), oracle.quantize_acts(xb)):
+        assert np.array_equal(a, b)
+    acc = rng.integers(-5000, 5000, (M, N)).astype(np.int32)
+    beta8 = oracle.quantize_acts(xb)[1]
+    assert np.array_equal(oracle.dequant_bits(acc, beta8, 0.02, 8), oracle.dequant(acc, beta8, 0.02))
+    for bits in (2, 3, 4, 6):
+        qb = 2 ** (bits - 1) - 1
+        q, beta, rs = oracle.quantize_acts_bits(xb, bits)
+        assert np.abs(q).max() == qb and np.array_equal(rs, q.astype(np.int32).sum(axis=1))
+        assert np.array_equal(beta, np.abs(xf).max(axis=1).astype(np.float32))
+        # each value is reproduced to within half a step
+        err = np.abs(xf - q * (beta.astype(np.float64) / qb)[:, None])
+        assert np.all(err <= (beta.astype(np.float64) / (2 * qb))[:, None] * (1 + 1e-6))
+        # codes equal the double-precision ones away from ties
+        scaled = xf * (qb / beta.astype(np.float64))[:, None]
+        clear = np.abs(scaled - np.floor(scaled) - 0.5) > 1e-4
+        assert clear.mean() > 0.99 and np.array_equal(q[clear], np.rint(scaled)[clear].astype(np.int8))
+        # the forward is the double-precision product of the dequantised operands
+        T = rng.integers(-1, 2, (N, K)).astype(np.int8)
+        y = bits_to_f32(oracle.dequant_bits(oracle.matmul_i32(q, T), beta, 0.02, bits)).astype(np.float64)
+        want = (q.astype(np.float64) * (beta.astype(np.float64) / qb)[:, None]) @ (T.astype(np.float64) * 0.02).T
+        assert np.allclose(y, want, rtol=2.0 ** -8, atol=1e-9)
