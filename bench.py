@@ -382,6 +382,21 @@ def extras(peaks):
         del gate, up, Xq
     out["swiglu_quantiser"] = res
 
+    # the forward with 4-bit activations (Q_b = 7) beside the 8-bit one: the same kernels, another scale
+    res = {}
+    for (N, K, M) in [(11008, 4096, 1), (13824, 5120, 2048)]:
+        W = S.latent_weights(N, K, 0, device="cuda")
+        packed, gamma = B.quantize_weights(W)
+        del W
+        X = S.activations(M, K, 0, device="cuda")
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+        ws = B.alloc_workspace(M, N, K)
+        ms4 = time_forward_calls(lambda: B.forward_act_bits(packed, gamma, X, N, 4, Y=Y, workspace=ws), 50)
+        ms8 = time_forward_calls(lambda: B.forward(packed, gamma, X, N, Y=Y, workspace=ws), 50)
+        res[f"{N}x{K}_M{M}"] = {"forward_4bit_ms": round(ms4, 4), "forward_8bit_ms": round(ms8, 4)}
+        del X, Y, ws, packed
+    out["act_bits_4"] = res
+
     # the headline step with the RMSNorm fused into the quantiser of q, k, v, gate and up (130 of the 182 matrices)
     cfg = S.CONFIGS[WORKLOAD]
     st = Stack(cfg["layers"], cfg["n_layers"], 1)

@@ -174,6 +174,20 @@ bitlinear_status bitlinear_forward_swiglu(const void *packed, const float *gamma
                                           void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The same quantiser and the same forward with activations of fewer bits.  The paper's outlook (Section 4, on long
+ * sequences) expects activations to go from 8 bits to 4 bits or fewer; here Q_b = 2^(act_bits - 1) - 1 (7 for 4 bits,
+ * 127 for 8) replaces the 127 of Section 2 in the quantiser (s = Q_b / beta, clip to [-Q_b, Q_b]) and in the
+ * dequantisation ((gamma * beta_t) / Q_b); everything else, the kernels included, is the forward above.  The codes
+ * are still delivered one per byte (Xq int8 [M, K]): this variant changes the arithmetic, not the storage.
+ *   act_bits   2 .. 8 (else BITLINEAR_ERR_ARG); 8 gives bitlinear_quantize_acts / bitlinear_forward exactly
+ */
+bitlinear_status bitlinear_quantize_acts_bits(const void *X, int64_t M, int64_t K, int act_bits,
+                                              int8_t *Xq, float *beta, int32_t *rowsum, void *stream);
+bitlinear_status bitlinear_forward_act_bits(const void *packed, const float *gamma, const void *X,
+                                            int64_t M, int64_t K, int64_t N, int act_bits, void *Y,
+                                            void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The same forward for callers that cannot give it a workspace.  (The paper has no counterpart: this is a
  * convenience of the library.)  Some code that wants to run a BitLinear layer is not allowed to allocate
  * device memory at the point of the call -- a plug-in that runs inside another framework's memory pool, a

@@ -27,7 +27,9 @@ EXPORTS = [
     "bitlinear_quantize_acts",
     "bitlinear_rmsnorm_quantize_acts",
     "bitlinear_swiglu_quantize_acts",
+    "bitlinear_quantize_acts_bits",
     "bitlinear_forward",
+    "bitlinear_forward_act_bits",
     "bitlinear_forward_rmsnorm",
     "bitlinear_forward_swiglu",
     "bitlinear_forward_static",
@@ -89,6 +91,8 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_forward_rmsnorm.argtypes = [vp, vp, vp, vp, cf, i64, i64, i64, vp, vp, sz, vp]
     L.bitlinear_swiglu_quantize_acts.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp]
     L.bitlinear_forward_swiglu.argtypes = [vp, vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
+    L.bitlinear_quantize_acts_bits.argtypes = [vp, i64, i64, ci, vp, vp, vp, vp]
+    L.bitlinear_forward_act_bits.argtypes = [vp, vp, vp, i64, i64, i64, ci, vp, vp, sz, vp]
     L.bitlinear_forward_static.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp]
     L.bitlinear_sequence_workspace_bytes.argtypes = [ctypes.POINTER(LayerDesc), ci]
     L.bitlinear_sequence_workspace_bytes.restype = sz
@@ -189,6 +193,32 @@ def forward_rmsnorm(packed: torch.Tensor, gamma: torch.Tensor, H: torch.Tensor, 
     st = load_library().bitlinear_forward_rmsnorm(_ptr(packed), _ptr(gamma), _ptr(H), _ptr(gain), float(norm_eps), M, K, N,
                                                   _ptr(Y), _ptr(workspace), workspace.numel(), _stream(stream))
     _check(st, "bitlinear_forward_rmsnorm")
+    return Y
+
+
+def quantize_acts_bits(X: torch.Tensor, act_bits: int, stream=None):
+    """bitlinear_quantize_acts_bits: bf16 [M, K] -> (Xq int8 [M, K] with |q| <= 2^(act_bits-1) - 1, beta, rowsum)."""
+    M, K = X.shape
+    Xq = torch.empty((M, K), dtype=torch.int8, device=X.device)
+    beta = torch.empty(max(M, 1), dtype=torch.float32, device=X.device)[:M]
+    rowsum = torch.empty(max(M, 1), dtype=torch.int32, device=X.device)[:M]
+    st = load_library().bitlinear_quantize_acts_bits(_ptr(X), M, K, int(act_bits), _ptr(Xq), _ptr(beta), _ptr(rowsum),
+                                                     _stream(stream))
+    _check(st, "bitlinear_quantize_acts_bits")
+    return Xq, beta, rowsum
+
+
+def forward_act_bits(packed: torch.Tensor, gamma: torch.Tensor, X: torch.Tensor, N: int, act_bits: int,
+                     Y: torch.Tensor | None = None, workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """bitlinear_forward_act_bits: the forward with act_bits-bit activations, bf16 [M, K] -> bf16 [M, N]."""
+    M, K = X.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, X.device)
+    st = load_library().bitlinear_forward_act_bits(_ptr(packed), _ptr(gamma), _ptr(X), M, K, N, int(act_bits), _ptr(Y),
+                                                   _ptr(workspace), workspace.numel(), _stream(stream))
+    _check(st, "bitlinear_forward_act_bits")
     return Y
 
 

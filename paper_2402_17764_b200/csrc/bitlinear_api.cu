@@ -137,6 +137,7 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.gain = nullptr;
     e.norm_eps = 0.0f;
     e.up = nullptr;
+    e.qb = (float)kQb;
 }
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
@@ -160,11 +161,11 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
         // B200 (1.15 against 2.2 POP/s), so it is not chosen unless asked for.
         static const int pair_min_m = env_int("BITLINEAR_PREFILL_PAIR_MIN_M", 1 << 30);
         const bool pair = (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
-                          (path == BITLINEAR_PATH_AUTO && e.M >= pair_min_m && prefill_pair_capacity() > 0);
+                          (path == BITLINEAR_PATH_AUTO && e.M >= pair_min_m && e.qb == (float)kQb && prefill_pair_capacity() > 0);
         cudaError_t err = pair ? launch_prefill_pair(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out,
                                                      e.out_i32, hdr, stream)
                                : launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, x_rows, e.K, e.N, e.out,
-                                                e.out_i32, hdr, split_scratch, stream);
+                                                e.out_i32, e.qb, hdr, split_scratch, stream);
         return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
@@ -225,9 +226,11 @@ bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K
 
 namespace {
 // gain == null and up == null: the plain quantiser; gain: RMSNorm in front; up: SwiGLU in front (X is the gate)
-bitlinear_status quantize_acts_rows(const void *X, const void *up, const float *gain, float norm_eps, int64_t M, int64_t K,
-                                    int8_t *Xq, float *beta, int32_t *rowsum, void *stream)
+// act_bits: 8 (Section 2), or fewer
+bitlinear_status quantize_acts_rows(const void *X, const void *up, const float *gain, float norm_eps, int act_bits,
+                                    int64_t M, int64_t K, int8_t *Xq, float *beta, int32_t *rowsum, void *stream)
 {
+    if (act_bits < 2 || act_bits > 8) return BITLINEAR_ERR_ARG;
     if (M > 0 && (!X || !Xq || !beta || !rowsum)) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, 16, K);
     if (st != BITLINEAR_OK) return st;
@@ -247,6 +250,7 @@ bitlinear_status quantize_acts_rows(const void *X, const void *up, const float *
     e.gain = gain;
     e.norm_eps = norm_eps;
     e.up = reinterpret_cast<const __nv_bfloat16 *>(up);
+    e.qb = (float)((1 << (act_bits - 1)) - 1);
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, nullptr, 0, (gain ? 1 : 0) | (up ? 2 : 0), (int)K,
                                            (cudaStream_t)stream);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
@@ -256,33 +260,39 @@ bitlinear_status quantize_acts_rows(const void *X, const void *up, const float *
 bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K, int8_t *Xq, float *beta,
                                          int32_t *rowsum, void *stream)
 {
-    return quantize_acts_rows(X, nullptr, nullptr, 0.0f, M, K, Xq, beta, rowsum, stream);
+    return quantize_acts_rows(X, nullptr, nullptr, 0.0f, 8, M, K, Xq, beta, rowsum, stream);
+}
+
+bitlinear_status bitlinear_quantize_acts_bits(const void *X, int64_t M, int64_t K, int act_bits, int8_t *Xq, float *beta,
+                                              int32_t *rowsum, void *stream)
+{
+    return quantize_acts_rows(X, nullptr, nullptr, 0.0f, act_bits, M, K, Xq, beta, rowsum, stream);
 }
 
 bitlinear_status bitlinear_rmsnorm_quantize_acts(const void *H, const float *gain, float norm_eps, int64_t M, int64_t K,
                                                  int8_t *Xq, float *beta, int32_t *rowsum, void *stream)
 {
     if (!gain || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
-    return quantize_acts_rows(H, nullptr, gain, norm_eps, M, K, Xq, beta, rowsum, stream);
+    return quantize_acts_rows(H, nullptr, gain, norm_eps, 8, M, K, Xq, beta, rowsum, stream);
 }
 
 bitlinear_status bitlinear_swiglu_quantize_acts(const void *gate, const void *up, int64_t M, int64_t K, int8_t *Xq,
                                                 float *beta, int32_t *rowsum, void *stream)
 {
     if (M > 0 && !up) return BITLINEAR_ERR_ARG;
-    return quantize_acts_rows(gate, up, nullptr, 0.0f, M, K, Xq, beta, rowsum, stream);
+    return quantize_acts_rows(gate, up, nullptr, 0.0f, 8, M, K, Xq, beta, rowsum, stream);
 }
 
 namespace {
 bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const void *up, const float *gain,
-                              float norm_eps, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
+                              float norm_eps, int act_bits, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
                               size_t workspace_bytes, void *stream);
 }
 
 bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
                                    int64_t N, void *Y, void *workspace, size_t workspace_bytes, void *stream)
 {
-    return forward_impl(packed, gamma, X, nullptr, nullptr, 0.0f, M, K, N, Y, workspace, workspace_bytes, stream);
+    return forward_impl(packed, gamma, X, nullptr, nullptr, 0.0f, 8, M, K, N, Y, workspace, workspace_bytes, stream);
 }
 
 bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamma, const void *H, const float *gain,
@@ -291,7 +301,7 @@ bitlinear_status bitlinear_forward_rmsnorm(const void *packed, const float *gamm
 {
     if (!gain || !(norm_eps >= 0.0f)) return BITLINEAR_ERR_ARG;
     if (!aligned(gain, 16)) return BITLINEAR_ERR_ALIGN;
-    return forward_impl(packed, gamma, H, nullptr, gain, norm_eps, M, K, N, Y, workspace, workspace_bytes, stream);
+    return forward_impl(packed, gamma, H, nullptr, gain, norm_eps, 8, M, K, N, Y, workspace, workspace_bytes, stream);
 }
 
 bitlinear_status bitlinear_forward_swiglu(const void *packed, const float *gamma, const void *gate, const void *up,
@@ -300,15 +310,23 @@ bitlinear_status bitlinear_forward_swiglu(const void *packed, const float *gamma
 {
     if (M > 0 && !up) return BITLINEAR_ERR_ARG;
     if (!aligned(up, 16)) return BITLINEAR_ERR_ALIGN;
-    return forward_impl(packed, gamma, gate, up, nullptr, 0.0f, M, K, N, Y, workspace, workspace_bytes, stream);
+    return forward_impl(packed, gamma, gate, up, nullptr, 0.0f, 8, M, K, N, Y, workspace, workspace_bytes, stream);
+}
+
+bitlinear_status bitlinear_forward_act_bits(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
+                                            int64_t N, int act_bits, void *Y, void *workspace, size_t workspace_bytes,
+                                            void *stream)
+{
+    return forward_impl(packed, gamma, X, nullptr, nullptr, 0.0f, act_bits, M, K, N, Y, workspace, workspace_bytes, stream);
 }
 
 namespace {
 // gain == null: no normalisation in front of the quantiser; up != null: X is the gate of a SwiGLU in front of it
 bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const void *up, const float *gain,
-                              float norm_eps, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
+                              float norm_eps, int act_bits, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
                               size_t workspace_bytes, void *stream)
 {
+    if (act_bits < 2 || act_bits > 8) return BITLINEAR_ERR_ARG;
     if (!packed || !gamma || !workspace || (M > 0 && (!X || !Y))) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, N, K);
     if (st != BITLINEAR_OK) return st;
@@ -326,6 +344,7 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     inl.e[0].gain = gain;
     inl.e[0].norm_eps = norm_eps;
     inl.e[0].up = reinterpret_cast<const __nv_bfloat16 *>(up);
+    inl.e[0].qb = (float)((1 << (act_bits - 1)) - 1);
     // quantise the tokens; the same launch clears the header and the scratch of the kernel that follows, if it uses it
     const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
@@ -599,7 +618,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
         if (gemm) {
             int nt = 0;
             if (prefill_table_entry(gemm_table.data() + (size_t)i * kGemmProblemBytes, e.packed, e.gamma, e.Xq, e.beta,
-                                    e.rowsum, d.M, d.M < kMinGemmRows ? kMinGemmRows : d.M, d.K, d.N, d.Y, max_M,
+                                    e.rowsum, d.M, d.M < kMinGemmRows ? kMinGemmRows : d.M, d.K, d.N, d.Y, e.qb, max_M,
                                     gemm_tiles, reinterpret_cast<WorkspaceHeader *>(ws), &nt) != cudaSuccess)
                 return BITLINEAR_ERR_CUDA;
             gemm_tiles += nt;

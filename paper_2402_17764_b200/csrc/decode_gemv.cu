@@ -155,7 +155,7 @@ __device__ __forceinline__ void store_result(const DecodeEntry &e, int token, in
 __device__ __forceinline__ float token_scale(const DecodeEntry &e, int token)
 {
     if (e.out_i32) return 0.0f;
-    return __fdiv_rn(__fmul_rn(*e.gamma, e.beta[token]), (float)kQb); // (gamma * beta_t) / Qb
+    return __fdiv_rn(__fmul_rn(*e.gamma, e.beta[token]), e.qb); // (gamma * beta_t) / Qb
 }
 
 // What the epilogue needs of a token, fetched once per token and lane: the stores of a lane's outputs may alias

@@ -58,6 +58,7 @@ struct DecodeEntry {
     int xq_tiled;          // layout of Xq (the streaming kernel reads tiles, the tensor-core GEMM rows)
     const float *gain;     // null, or [K] fp32: X is normalised first (RMSNorm with this gain) and then quantised
     float norm_eps;        // the RMSNorm's epsilon (added to the mean square)
+    float qb;              // largest activation code: 127 (Section 2), or 2^(b-1) - 1 for b-bit activations
     const __nv_bfloat16 *up; // null, or bf16 [M, K]: the quantiser's input is silu(X) * up (SwiGLU; X holds the gate)
 };
 
@@ -94,11 +95,11 @@ inline uint32_t decode_items(int NB, int KB, bool wide) { return (uint32_t)(wide
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
                           int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream);
 
-// Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) or raw int32.  x_rows >= M rows of K bytes exist behind
+// Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) (by gamma * beta_t / qb) or raw int32.  x_rows >= M rows of K bytes exist behind
 // Xq; the rows past M may hold anything (they only reach accumulator rows that are never stored).
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream);
+                           int out_i32, float qb, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream);
 
 // Cutting tiles along K.  When the CTA tiles of a launch leave most SMs idle in their last round, the kernel cuts
 // the tiles of that round along K and adds the partial sums up in `split_scratch` (prefill_split_bytes(tiles, max_M)
@@ -117,7 +118,7 @@ constexpr size_t kGemmProblemBytes = 384;
 int prefill_token_tiles(int64_t max_M);
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles);
+                                float qb, int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles);
 cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, int min_KB,
                                  void *split_scratch, cudaStream_t stream);
 

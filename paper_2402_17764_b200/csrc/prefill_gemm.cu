@@ -171,6 +171,7 @@ struct Params {
     int out_i32;
     int out_32b_aligned; // rows of the bf16 output start on 32-byte boundaries
     int tile_begin;      // first CTA tile of this matmul in the launch-wide tile sequence
+    float qb;            // largest activation code (127, or less for activations of fewer bits)
     int32_t *status;
 };
 
@@ -479,7 +480,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 scale = 0.0f;
                 if (t < p.M) {
                     rowsum = p.rowsum[t];
-                    if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), (float)kQb);
+                    if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), p.qb);
                 }
             };
 
@@ -596,7 +597,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
 // Tensor maps and parameters of one matmul, for `mt` token tiles per CTA tile.
 static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int out_i32, int mt, int a_rows, int tile_begin, int32_t *status)
+                                int out_i32, float qb, int mt, int a_rows, int tile_begin, int32_t *status)
 {
     if (!encode_tiled_fn()) return cudaErrorNotSupported;
     if (x_rows < M) return cudaErrorInvalidValue;
@@ -617,6 +618,7 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
     p.out_i32 = out_i32;
     p.out_32b_aligned = (reinterpret_cast<uintptr_t>(out) % 32 == 0) ? 1 : 0; // (N is a multiple of 16)
     p.tile_begin = tile_begin;
+    p.qb = qb;
     p.status = status;
     return cudaSuccess;
 }
@@ -711,11 +713,11 @@ static int prefill_a_rows(int64_t max_M) { return max_M <= 64 ? 64 : BM; }
 
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream)
+                           int out_i32, float qb, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream)
 {
     const int mt = prefill_token_tiles(M), a_rows = prefill_a_rows(M);
     GemmProblem g;
-    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, mt, a_rows, 0,
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, qb, mt, a_rows, 0,
                                  &hdr->status);
     if (e != cudaSuccess) return e;
     return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, a_rows, g.p.KB, split_scratch, stream);
@@ -723,10 +725,10 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
 
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles)
+                                float qb, int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles)
 {
     GemmProblem g;
-    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, 0, prefill_token_tiles(max_M),
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, 0, qb, prefill_token_tiles(max_M),
                                  prefill_a_rows(max_M), tile_begin, &hdr->status);
     if (e != cudaSuccess) return e;
     memcpy(slot, &g, sizeof(g));

@@ -1,5 +1,6 @@
 // Kernel (b): per-token absmax quantisation of bf16 activations to int8
-// (Section 2, paragraph after Eq. 3: scaled to [-Qb, Qb] per token, Qb = 127, no zero point).
+// (Section 2, paragraph after Eq. 3: scaled to [-Qb, Qb] per token, Qb = 127, no zero point; Qb = 2^(b-1) - 1 for
+// the b-bit activations the paper's outlook names, with the codes still one per byte).
 //
 // One CTA per token.  The token is read once with 16-byte loads and kept in registers
 // (up to kCache vectors per thread; longer rows re-read the tail, which hits L2), the absmax
@@ -258,7 +259,7 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
 #pragma unroll
         for (int w = 1; w < NT / 32; ++w) mx = max(mx, s_max[w]);
         const float b = fmaxf(__uint_as_float(mx), kBetaFloor);
-        const float s = __fdiv_rn((float)kQb, b);
+        const float s = __fdiv_rn(e.qb, b);
 
         int sum = 0;
         auto quantise8 = [&](const uint4 &v, int i) {
@@ -321,7 +322,7 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
         for (int w = 1; w < NT / 32; ++w) mx = max(mx, s_max[w]);
         const bool bad = mx >= 0x7F800000u; // an infinity or a NaN in an input, or a product beyond fp32
         const float b = fmaxf(__uint_as_float(mx), kBetaFloor);
-        const float s = __fdiv_rn((float)kQb, b);
+        const float s = __fdiv_rn(e.qb, b);
 
         int sum = 0;
         auto quantise8 = [&](const float (&h)[8], int i) {
@@ -377,7 +378,7 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
 
     const float amax = __uint_as_float(m << 16);
     const float b = fmaxf(amax, kBetaFloor);
-    const float s = __fdiv_rn((float)kQb, b); // one IEEE divide per token
+    const float s = __fdiv_rn(e.qb, b); // one IEEE divide per token
 
     int sum = 0;
 #pragma unroll
