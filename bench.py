@@ -411,6 +411,21 @@ def extras(peaks):
     out["3b_decode_step_with_rmsnorm"] = {"ms_per_step": round(ms, 4), "GB/s": round(st.algorithmic_bytes / ms / 1e6, 1),
                                           "normalised_matrices": sum(g is not None for g in gains)}
     seq.close()
+
+    # the same step (without the RMSNorm) replayed from a CUDA graph that holds ten steps
+    seq = B.Sequence(st.layers)
+    seq.forward()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(10):
+            seq.forward()
+    ms = time_forward_calls(graph.replay, 30, warmup=3) / 10
+    assert B.poll_status(seq.workspace) == 0
+    out["3b_decode_step_cuda_graph"] = {"ms_per_step": round(ms, 4), "GB/s": round(st.algorithmic_bytes / ms / 1e6, 1),
+                                        "steps_per_graph": 10}
+    del graph
+    seq.close()
     del st, seq
 
     # 70B-shaped full decode step: 80 layers, 17.1 GB of packed weights resident

@@ -259,7 +259,8 @@ bitlinear_status bitlinear_sequence_create_swiglu(const bitlinear_layer_desc *la
 
 /* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch, one persistent matmul
  * launch that starts while the quantiser is still running (programmatic dependent launch) and one very small
- * finishing launch.  Calls on the same sequence must be stream-ordered, not concurrent. */
+ * finishing launch.  Calls on the same sequence must be stream-ordered, not concurrent.  Once a sequence has run once
+ * on the device (the first run sets kernel attributes), later calls may be captured into a CUDA graph. */
 bitlinear_status bitlinear_forward_sequence(const bitlinear_sequence *seq, void *stream);
 
 /* The same in two halves, so that a caller can put its own events between them:
