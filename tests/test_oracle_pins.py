@@ -273,6 +273,20 @@ def test_timing_build_equals_parity_build(oracle):
     T2, g2 = fast.quantize_weights(W)
     assert g == g2 and np.array_equal(T, T2)
     assert np.array_equal(oracle.forward(T, g, xbits), fast.forward(T, g, xbits))
+    # the fronts of the quantiser and the b-bit variant: the GPU tests compare against the timing build
+    gain = (1.0 + 0.1 * rng.standard_normal(K)).astype(np.float32)
+    ubits = R.f32_to_bf16_bits_rne(rng.standard_normal((M, K)).astype(np.float32))
+    gbits = R.f32_to_bf16_bits_rne((3.0 * rng.standard_normal((M, K))).astype(np.float32))
+    for a, b in zip(oracle.rmsnorm_quantize_acts(xbits, gain, 1e-5, return_x=True),
+                    fast.rmsnorm_quantize_acts(xbits, gain, 1e-5, return_x=True)):
+        assert np.array_equal(a, b)
+    for a, b in zip(oracle.swiglu_quantize_acts(gbits, ubits, return_h=True), fast.swiglu_quantize_acts(gbits, ubits, return_h=True)):
+        assert np.array_equal(a, b)
+    for a, b in zip(oracle.quantize_acts_bits(xbits, 4), fast.quantize_acts_bits(xbits, 4)):
+        assert np.array_equal(a, b)
+    acc = oracle.matmul_i32(oracle.quantize_acts_bits(xbits, 4)[0], T)
+    beta = oracle.quantize_acts_bits(xbits, 4)[1]
+    assert np.array_equal(oracle.dequant_bits(acc, beta, g, 4), fast.dequant_bits(acc, beta, g, 4))
 
 
 # ---------------------------------------------------------------- RMSNorm in front of the quantiser
