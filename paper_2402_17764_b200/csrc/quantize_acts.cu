@@ -35,6 +35,7 @@ namespace {
 
 constexpr int kThreads = 256;
 constexpr int kCache = 4; // 16-byte vectors kept in registers per thread (4 * 8 * 256 = 8192 elements)
+constexpr int kSwigluSmemBytes = 56 * 1024; // SwiGLU products of one token in shared memory: 14336 elements
 
 __device__ __forceinline__ uint32_t absmax_bits(uint32_t m, const uint4 &v)
 {
@@ -122,10 +123,12 @@ __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
 // three block-wide reductions) is a fixed cost per thread, so short tokens take fewer threads with kCache vectors
 // each.  Tokens of more than 8192 elements re-read their tail, which hits L2.
 template <int kFronts, int NT>
-__global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
+__global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
                                                                  const DecodeEntry *__restrict__ table, int n_entries,
-                                                                 int total_tokens, uint4 *zero_ptr, size_t zero_vecs)
+                                                                 int total_tokens, uint4 *zero_ptr, size_t zero_vecs,
+                                                                 int h_cap_vecs)
 {
+    extern __shared__ float4 h_smem[]; // SwiGLU: the products of the first h_cap_vecs vectors of the token
     __shared__ uint32_t s_max[NT / 32];
     __shared__ int s_sum[NT / 32];
     __shared__ unsigned long long s_sq[NT / 32];
@@ -293,10 +296,12 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
     }
 
     if ((kFronts & 2) && e.up) {
-        // ---- SwiGLU, then the quantiser on the fp32 values (see the head of this file).  The values of the first
-        // 8 * kCache * NT elements stay in registers; longer tokens form the rest a second time.
+        // ---- SwiGLU, then the quantiser on the fp32 values (see the head of this file).  The products wait in shared
+        // memory between the two passes (32 registers per thread for them left too few warps resident to cover the
+        // dependent arithmetic); each thread reads back what it wrote itself.  The two halves of a vector stand
+        // h_cap_vecs apart, so that the 16-byte accesses of a warp are consecutive.  A token longer than the buffer
+        // forms the rest a second time.
         const uint4 *urow = reinterpret_cast<const uint4 *>(e.up + (size_t)t * K);
-        float hc[kCache][8];
         // largest |h| as an unsigned integer.  An infinity or a NaN in either input makes h an infinity or a NaN (a
         // gate of -inf: -inf * 0), and their bit patterns are the largest.
         uint32_t mx = 0;
@@ -305,14 +310,13 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
 #pragma unroll
             for (int j = 0; j < 8; ++j) mx = max(mx, __float_as_uint(h[j]) & 0x7FFFFFFFu);
         };
-#pragma unroll
-        for (int c = 0; c < kCache; ++c) {
-            const int i = threadIdx.x + c * NT;
-            if (i < n_vec) form(i, hc[c]);
-        }
-        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
+        for (int i = threadIdx.x; i < n_vec; i += NT) {
             float h[8];
             form(i, h);
+            if (i < h_cap_vecs) {
+                h_smem[i] = make_float4(h[0], h[1], h[2], h[3]);
+                h_smem[h_cap_vecs + i] = make_float4(h[4], h[5], h[6], h[7]);
+            }
         }
         mx = __reduce_max_sync(0xffffffffu, mx);
         if (lane == 0) s_max[warp] = mx;
@@ -332,14 +336,15 @@ __global__ void __launch_bounds__(NT, (kFronts ? 768 : 1024) / NT) quantize_acts
             out_at(i) = o;
             sum = __dp4a((int)o.x, 0x01010101, __dp4a((int)o.y, 0x01010101, sum));
         };
-#pragma unroll
-        for (int c = 0; c < kCache; ++c) {
-            const int i = threadIdx.x + c * NT;
-            if (i < n_vec) quantise8(hc[c], i);
-        }
-        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
+        for (int i = threadIdx.x; i < n_vec; i += NT) {
             float h[8];
-            swiglu8(__ldg(row + i), __ldg(urow + i), h);
+            if (i < h_cap_vecs) {
+                const float4 a = h_smem[i], c = h_smem[h_cap_vecs + i];
+                h[0] = a.x, h[1] = a.y, h[2] = a.z, h[3] = a.w;
+                h[4] = c.x, h[5] = c.y, h[6] = c.z, h[7] = c.w;
+            } else {
+                swiglu8(__ldg(row + i), __ldg(urow + i), h);
+            }
             quantise8(h, i);
         }
         if (tiled) // the last column tile is filled up with zeros
@@ -435,14 +440,20 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     // threads per token: the smallest count whose register caches hold the longest token
     const int n_vec = max_K >> 3;
     // (longer tokens re-read their tail, which hits L2: CTAs of 512 and 1024 threads measured slower)
-    // (with SwiGLU in front a token beyond the caches costs its exponentials a second time: 384 threads there)
-    static const int counts[5] = {64, 128, 192, 256, 384};
-    int nt = (fronts & 2) ? 384 : 256;
+    static const int counts[4] = {64, 128, 192, 256};
+    int nt = 256;
     for (int c : counts)
-        if (n_vec <= c * kCache && c <= nt) {
+        if (n_vec <= c * kCache) {
             nt = c;
             break;
         }
+    // SwiGLU: room in shared memory for the products of a token (at most kSwigluSmemBytes: four CTAs per SM)
+    int h_cap_vecs = 0;
+    size_t dyn_smem = 0;
+    if (fronts & 2) {
+        h_cap_vecs = n_vec < kSwigluSmemBytes / 32 ? n_vec : kSwigluSmemBytes / 32;
+        dyn_smem = (size_t)h_cap_vecs * 32;
+    }
     const size_t zero_vecs = zero_bytes / 16;
     int zero_blocks = 0;
     if (zero_vecs > 0) {
@@ -455,7 +466,21 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     if (grid == 0) return cudaSuccess;
     uint4 *zp = reinterpret_cast<uint4 *>(zero_ptr);
 #define BITLINEAR_LAUNCH_QUANTISER(FRONTS, NT_) \
-    quantize_acts_kernel<FRONTS, NT_><<<grid, NT_, 0, stream>>>(inl, table, n_entries, total_tokens, zp, zero_vecs)
+    do { \
+        if (FRONTS & 2) { \
+            static bool attr_set[64] = {false}; \
+            int dev = 0; \
+            cudaGetDevice(&dev); \
+            if (dev >= 0 && dev < 64 && !attr_set[dev]) { \
+                cudaError_t e = cudaFuncSetAttribute(quantize_acts_kernel<FRONTS, NT_>, \
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, kSwigluSmemBytes); \
+                if (e != cudaSuccess) return e; \
+                attr_set[dev] = true; \
+            } \
+        } \
+        quantize_acts_kernel<FRONTS, NT_><<<grid, NT_, dyn_smem, stream>>>(inl, table, n_entries, total_tokens, zp, \
+                                                                            zero_vecs, h_cap_vecs); \
+    } while (0)
 #define BITLINEAR_LAUNCH_BOTH(NT_) \
     do { \
         switch (fronts & 3) { \
@@ -469,10 +494,6 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     case 64: BITLINEAR_LAUNCH_BOTH(64); break;
     case 128: BITLINEAR_LAUNCH_BOTH(128); break;
     case 192: BITLINEAR_LAUNCH_BOTH(192); break;
-    case 384:
-        if (fronts & 1) BITLINEAR_LAUNCH_QUANTISER(3, 384);
-        else BITLINEAR_LAUNCH_QUANTISER(2, 384);
-        break;
     default: BITLINEAR_LAUNCH_BOTH(256); break;
     }
 #undef BITLINEAR_LAUNCH_BOTH
