@@ -839,6 +839,9 @@ __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constan
                                                             const OwnedList *__restrict__ lists, uint32_t n_lists)
 {
     const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // The quantiser of a step that follows may become resident at once; it waits for this grid to end before it
+    // touches anything, and the matmul behind it streams weights (never written) until that quantiser has ended.
+    ptx::griddep_launch_dependents();
     ptx::griddep_wait(); // the lists and the scratch are written by the launch before this one
     if (w >= n_lists) return;
     const int n = (int)__ldcg(&lists[w].n);

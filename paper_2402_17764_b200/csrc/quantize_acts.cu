@@ -26,6 +26,8 @@
 // degree 7 in r by Horner's scheme (seven fused multiply-adds), e^-g = p * 2^n (exact); sigmoid = 1 / (1 + e^-g) with
 // one addition and one IEEE reciprocal, taken as 0 below g = -87 and as 1 above 87; h = (g * sigmoid) * u with two
 // multiplications.  A token with an infinity or a NaN in either input, or with a product beyond fp32, gets beta = NaN.
+#include <cstdlib>
+
 #include "internal.cuh"
 #include "ptx.cuh"
 
@@ -135,6 +137,9 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
 
     // The matmul that follows may be launched early: it streams weights until it needs what this kernel writes.
     ptx::griddep_launch_dependents();
+    // This kernel itself may have been launched before the kernel in front of it has ended (the finishing launch of
+    // the step before, which lets its dependents in at once): what it reads and overwrites may still be in use.
+    ptx::griddep_wait();
 
     if ((int)blockIdx.x >= total_tokens) {
         // trailing blocks clear control words and split-K scratch for the matmul that follows
@@ -465,6 +470,21 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     const int grid = total_tokens + zero_blocks;
     if (grid == 0) return cudaSuccess;
     uint4 *zp = reinterpret_cast<uint4 *>(zero_ptr);
+    // A programmatic dependent of whatever stands in front of it on the stream: behind the finishing launch of a
+    // step before, the CTAs are resident and waiting when that launch ends (BITLINEAR_QUANTISER_EARLY_LAUNCH=0: off).
+    static const bool early = [] {
+        const char *v = std::getenv("BITLINEAR_QUANTISER_EARLY_LAUNCH");
+        return !(v && *v == '0');
+    }();
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.dynamicSmemBytes = dyn_smem;
+    cfg.stream = stream;
+    cfg.attrs = &attr;
+    cfg.numAttrs = early ? 1 : 0;
 #define BITLINEAR_LAUNCH_QUANTISER(FRONTS, NT_) \
     do { \
         if (FRONTS & 2) { \
@@ -478,8 +498,10 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
                 attr_set[dev] = true; \
             } \
         } \
-        quantize_acts_kernel<FRONTS, NT_><<<grid, NT_, dyn_smem, stream>>>(inl, table, n_entries, total_tokens, zp, \
-                                                                            zero_vecs, h_cap_vecs); \
+        cfg.blockDim = dim3(NT_); \
+        cudaError_t le = cudaLaunchKernelEx(&cfg, quantize_acts_kernel<FRONTS, NT_>, inl, table, n_entries, total_tokens, \
+                                            zp, zero_vecs, h_cap_vecs); \
+        if (le != cudaSuccess) return le; \
     } while (0)
 #define BITLINEAR_LAUNCH_BOTH(NT_) \
     do { \

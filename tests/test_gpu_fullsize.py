@@ -198,3 +198,45 @@ def test_repeated_runs_are_identical(N, K, M, iters):
         differing += int(not torch.equal(Y.view(torch.int16), first.view(torch.int16)))
     assert B.poll_status(ws) == 0
     assert differing == 0
+
+
+@pytest.mark.parametrize("M", [1, 12])
+def test_back_to_back_steps_without_synchronisation(M):
+    """Steps enqueued one behind the other: the quantiser of a step is a programmatic dependent of the finishing launch
+    of the step before and the matmul behind it starts streaming weights early.  300 steps with nothing between them
+    must leave the first step's bits, and steps with changing inputs (a device copy in front of each, a snapshot behind
+    it, no host synchronisation) must each give what the same step gives alone."""
+    cfg = S.CONFIGS["3b_decode"]
+    layers, _ = build_stack(cfg["layers"], 2, M)
+    seq = B.Sequence(layers)
+    seq.forward()
+    torch.cuda.synchronize()
+    first = [l[3].clone() for l in layers]
+    for _ in range(300):
+        seq.forward()
+    torch.cuda.synchronize()
+    assert B.poll_status(seq.workspace) == 0
+    for l, want in zip(layers, first):
+        assert torch.equal(l[3].view(torch.int16), want.view(torch.int16))
+    # changing inputs: three input sets in turn
+    inputs = [[S.activations(M, l[2].shape[1], 500 + 16 * v + i, device="cuda") for i, l in enumerate(layers)] for v in range(3)]
+    alone = []
+    for v in range(3):
+        for l, x in zip(layers, inputs[v]):
+            l[2].copy_(x)
+        seq.forward()
+        torch.cuda.synchronize()
+        alone.append([l[3].clone() for l in layers])
+    snaps = []
+    for step in range(12):
+        v = step % 3
+        for l, x in zip(layers, inputs[v]):
+            l[2].copy_(x)
+        seq.forward()
+        snaps.append((v, [l[3].clone() for l in layers]))
+    torch.cuda.synchronize()
+    assert B.poll_status(seq.workspace) == 0
+    for v, ys in snaps:
+        for y, want in zip(ys, alone[v]):
+            assert torch.equal(y.view(torch.int16), want.view(torch.int16))
+    seq.close()
