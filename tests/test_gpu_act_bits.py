@@ -77,3 +77,21 @@ def test_entry_points_reject_bad_arguments():
         assert L.bitlinear_quantize_acts_bits(fake, 1, 16, bits, fake, fake, fake, None) == B.ERR_ARG
         assert L.bitlinear_forward_act_bits(fake, fake, fake, 1, 16, 16, bits, fake, fake, 1 << 20, None) == B.ERR_ARG
     assert L.bitlinear_quantize_acts_bits(fake, 1, 24, 4, fake, fake, fake, None) == B.ERR_SHAPE
+
+
+def test_empty_input_and_guard_rows():
+    X = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    Xq, beta, rowsum = B.quantize_acts_bits(X, 4)
+    assert Xq.shape == (0, 64) and beta.numel() == 0 and rowsum.numel() == 0
+    # a forward at 5 tokens writes its 5 rows of Y and nothing around them
+    W = S.latent_weights(48, 80, 2)
+    packed, gamma = B.quantize_weights(W.cuda(), 1e-5)
+    guard = torch.full((7, 48), -3.0, dtype=torch.bfloat16, device="cuda")
+    x = S.activations(5, 80, 2)
+    orc = timing_oracle()
+    T_ref, g_ref = orc.quantize_weights(W.numpy(), 1e-5)
+    q_ref, b_ref, _ = orc.quantize_acts_bits(torch_bf16_to_bits(x), 4)
+    want = orc.dequant_bits(orc.matmul_i32(q_ref, T_ref), b_ref, g_ref, 4)
+    got = B.forward_act_bits(packed, gamma, x.cuda(), 48, 4, Y=guard[1:6])
+    assert np.array_equal(torch_bf16_to_bits(got), want)
+    assert bool((guard[0] == -3.0).all()) and bool((guard[6] == -3.0).all())

@@ -179,3 +179,24 @@ def test_swiglu_entry_points_reject_bad_arguments():
     out = ctypes.c_void_p()
     assert L.bitlinear_sequence_create_swiglu(descs, both, both, 1e-5, 1, fake, 1 << 20, ctypes.byref(out)) == B.ERR_ARG
     assert L.bitlinear_sequence_create_swiglu(descs, None, None, 1e-5, 1, fake, 1 << 20, ctypes.byref(out)) == B.ERR_ARG
+
+
+def test_swiglu_empty_and_smallest_inputs():
+    """No tokens: nothing is launched and nothing is touched; one token of 16 features: the smallest shape."""
+    gate = torch.empty((0, 64), dtype=torch.bfloat16, device="cuda")
+    Xq, beta, rowsum = B.swiglu_quantize_acts(gate, gate.clone())
+    assert Xq.shape == (0, 64) and beta.numel() == 0 and rowsum.numel() == 0
+    W = S.latent_weights(16, 16, 1)
+    packed, gamma = B.quantize_weights(W.cuda(), 1e-5)
+    ws = B.alloc_workspace(1, 16, 16)
+    guard = torch.full((3, 16), 7.0, dtype=torch.bfloat16, device="cuda")
+    Y = B.forward_swiglu(packed, gamma, gate[:, :16].contiguous(), gate[:, :16].contiguous(), 16, Y=guard[1:1], workspace=ws)
+    assert Y.shape == (0, 16) and bool((guard == 7.0).all())
+    g1, u1 = gate_and_up(1, 16, 3)
+    orc = timing_oracle()
+    T_ref, g_ref = orc.quantize_weights(W.numpy(), 1e-5)
+    q_ref, b_ref, _ = orc.swiglu_quantize_acts(torch_bf16_to_bits(g1), torch_bf16_to_bits(u1))
+    want = orc.dequant(orc.matmul_i32(q_ref, T_ref), b_ref, g_ref)
+    got = B.forward_swiglu(packed, gamma, g1.cuda(), u1.cuda(), 16, Y=guard[1:2], workspace=ws)
+    assert np.array_equal(torch_bf16_to_bits(got), want)
+    assert bool((guard[0] == 7.0).all()) and bool((guard[2] == 7.0).all())  # the rows around the output are untouched
