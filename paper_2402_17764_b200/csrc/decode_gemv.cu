@@ -183,7 +183,9 @@ __device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete
 // the next launch.  owned[i] = (entry index, row block).  Up to four row blocks are
 // handled at a time with all loads of one kind issued together, so that the pass costs two memory round
 // trips rather than two per row block.
-__device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, const uint2 *owned, int n_owned, int lane)
+// `word` is the lane's 32-bit word of the warp's 128-byte list (one load for the count and all items: every round
+// trip of this launch is on the critical path of the step): word 0 the count, words 2 i + 2 and 2 i + 3 item i.
+__device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint32_t word, int n_owned, int lane)
 {
     constexpr int kBatch = 4;
     for (int b0 = 0; b0 < n_owned; b0 += kBatch) {
@@ -192,7 +194,8 @@ __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, cons
         int r0[kBatch], N[kBatch];
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
-            const uint2 o = __ldcg(&owned[min(b0 + b, n_owned - 1)]); // slots past the end repeat the last one and store nothing
+            const int item = min(b0 + b, n_owned - 1); // slots past the end repeat the last one and store nothing
+            const uint2 o = make_uint2(__shfl_sync(0xffffffffu, word, 2 * item + 2), __shfl_sync(0xffffffffu, word, 2 * item + 3));
             e[b] = tab + o.x;
             r0[b] = (int)o.y * kTileRows + lane;
         }
@@ -844,9 +847,11 @@ __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constan
     ptx::griddep_launch_dependents();
     ptx::griddep_wait(); // the lists and the scratch are written by the launch before this one
     if (w >= n_lists) return;
-    const int n = (int)__ldcg(&lists[w].n);
+    const int lane = threadIdx.x & 31;
+    const uint32_t word = __ldcg(reinterpret_cast<const uint32_t *>(&lists[w]) + lane);
+    const int n = (int)__shfl_sync(0xffffffffu, word, 0);
     if (n == 0) return;
-    finish_owned_blocks(table ? table : inl.e, lists[w].item, n, threadIdx.x & 31);
+    finish_owned_blocks(table ? table : inl.e, word, n, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
