@@ -89,6 +89,8 @@ struct Ring {
 constexpr uint32_t kStaticPercent = BITLINEAR_DECODE_STATIC_PERCENT; // share of the tiles split statically
 constexpr uint32_t kPiecesPerWarp = BITLINEAR_DECODE_PIECES_PER_WARP; // dynamic pieces per warp, on average
 constexpr uint32_t kMinPieceTiles = 16;
+constexpr size_t kStagedTableBytes = 24 * 1024; // see decode_finish_kernel
+static_assert(sizeof(DecodeEntry) % 16 == 0, "the table is staged with 16-byte copies");
 
 __device__ __forceinline__ void mma_u8s8(int (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                          uint32_t b0, uint32_t b1)
@@ -837,14 +839,25 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
 }
 
 // The finishing launch: warp w takes the list of warp w of the kernel above.
+// staged_entries > 0: the CTA copies that many entries of the table (all of them) into its shared memory while the
+// matmul is still running, which takes the table's round trip to L2 off the chain list -> entry -> sums -> stores.
 __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constant__ InlineTable inl,
                                                             const DecodeEntry *__restrict__ table,
-                                                            const OwnedList *__restrict__ lists, uint32_t n_lists)
+                                                            const OwnedList *__restrict__ lists, uint32_t n_lists,
+                                                            int staged_entries)
 {
+    extern __shared__ uint4 staged_table[];
     const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
     // The quantiser of a step that follows may become resident at once; it waits for this grid to end before it
     // touches anything, and the matmul behind it streams weights (never written) until that quantiser has ended.
     ptx::griddep_launch_dependents();
+    if (staged_entries > 0) { // (the table is written once, when the sequence is created)
+        const int n_vec = staged_entries * (int)(sizeof(DecodeEntry) / 16);
+        const uint4 *src = reinterpret_cast<const uint4 *>(table);
+        for (int i = threadIdx.x; i < n_vec; i += blockDim.x) staged_table[i] = __ldg(src + i);
+        __syncthreads();
+        table = reinterpret_cast<const DecodeEntry *>(staged_table);
+    }
     ptx::griddep_wait(); // the lists and the scratch are written by the launch before this one
     if (w >= n_lists) return;
     const int lane = threadIdx.x & 31;
@@ -956,8 +969,11 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
     cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT>, grid, block, Ring<NT>::kSmem, args, early, stream);
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists};
-    return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
+    // a table that fits beside the matmul's ring (one CTA of each per SM) is staged in the finishing CTAs' shared memory
+    int staged = (table && (size_t)n_entries * sizeof(DecodeEntry) <= kStagedTableBytes) ? n_entries : 0;
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged};
+    return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256),
+                            (size_t)staged * sizeof(DecodeEntry), fargs, early, stream);
 }
 
 template <int NT>
@@ -979,7 +995,8 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
     cudaError_t err = launch_dependent((const void *)decode_wide_kernel<NT>, grid, block, WideRing<NT>::kSmem, args, early, stream);
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists};
+    int staged = 0; // (this kernel's rings leave no room beside them)
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged};
     return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
 }
 
