@@ -137,11 +137,24 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
 
     // The matmul that follows may be launched early: it streams weights until it needs what this kernel writes.
     ptx::griddep_launch_dependents();
+
+    // The descriptors are written once, before the first launch (or travel as a kernel parameter), so finding this
+    // CTA's token in them (a chain of dependent loads) and fetching its descriptor need not wait for anything.
+    const bool clearing = (int)blockIdx.x >= total_tokens;
+    const DecodeEntry *tab = table ? table : inl.e;
+    // entry that owns this token: the last one whose token_begin <= blockIdx.x
+    int lo = 0, hi = clearing ? 0 : n_entries - 1;
+    while (lo < hi) {
+        int mid = (lo + hi + 1) >> 1;
+        if (tab[mid].token_begin <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
+    }
+    const DecodeEntry e = tab[lo]; // a copy: the fields in use are loaded here
+
     // This kernel itself may have been launched before the kernel in front of it has ended (the finishing launch of
     // the step before, which lets its dependents in at once): what it reads and overwrites may still be in use.
     ptx::griddep_wait();
 
-    if ((int)blockIdx.x >= total_tokens) {
+    if (clearing) {
         // trailing blocks clear control words and split-K scratch for the matmul that follows
         const size_t n_zero_blocks = gridDim.x - total_tokens;
         for (size_t i = (size_t)(blockIdx.x - total_tokens) * NT + threadIdx.x; i < zero_vecs;
@@ -150,14 +163,6 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
         return;
     }
 
-    const DecodeEntry *tab = table ? table : inl.e;
-    // entry that owns this token: the last one whose token_begin <= blockIdx.x
-    int lo = 0, hi = n_entries - 1;
-    while (lo < hi) {
-        int mid = (lo + hi + 1) >> 1;
-        if (tab[mid].token_begin <= (int)blockIdx.x) lo = mid; else hi = mid - 1;
-    }
-    const DecodeEntry &e = tab[lo];
     const int t = blockIdx.x - e.token_begin;
     const int K = e.K;
     const int n_vec = K >> 3;
