@@ -50,7 +50,9 @@ enum {
     BITLINEAR_ERR_ARCH = -5,      /* current device is not sm_100 */
     BITLINEAR_ERR_CUDA = -6,      /* a CUDA runtime or driver call failed */
     BITLINEAR_ERR_TIMEOUT = -7,   /* a bounded device-side wait expired (device status) */
-    BITLINEAR_ERR_RANGE = -8      /* a weight was non-finite or >= 2^24 in magnitude (reported as gamma = NaN) */
+    BITLINEAR_ERR_RANGE = -8,     /* a weight was non-finite or >= 2^24 in magnitude (reported on the device, as
+                                     gamma = NaN; no call returns this code) */
+    BITLINEAR_ERR_BADCODE = -9    /* bitlinear_validate_packed found the 2-bit code 3, which no weight has */
 };
 
 /* Matmul code paths selectable through the test hook bitlinear_matmul_i32. */
@@ -58,9 +60,7 @@ enum {
     BITLINEAR_PATH_AUTO = 0,
     BITLINEAR_PATH_DP4A = 1,   /* scalar dp4a, M <= 8 */
     BITLINEAR_PATH_MMA = 2,    /* warp-level integer MMA on register-unpacked weights, M <= 64 */
-    BITLINEAR_PATH_TCGEN05 = 3,     /* TMA + tcgen05 int8 tensor-core GEMM with TMEM accumulators, any M */
-    BITLINEAR_PATH_TCGEN05_PAIR = 4, /* the same GEMM on pairs of SMs (tcgen05 cta_group::2), any M */
-    BITLINEAR_PATH_TCGEN05_TS = 5    /* the same GEMM with the expanded weights in tensor memory, any M */
+    BITLINEAR_PATH_TCGEN05 = 3 /* TMA + tcgen05 int8 tensor-core GEMM with TMEM accumulators, any M */
 };
 
 /* Human-readable name of a status code; never NULL. (host) */
@@ -116,8 +116,11 @@ bitlinear_status bitlinear_quantize_acts(const void *X, int64_t M, int64_t K,
  * RMSNorm followed by the activation quantiser, in one pass over the token.  Section 2, "LLaMA-alike
  * Components" names RMSNorm among the parts the models are built from and gives no formula; this is the textbook
  * one, x_k = h_k / sqrt(mean_k(h_k^2) + norm_eps) * gain_k, with the arithmetic fixed so that the int8 codes are
- * reproducible bit for bit: exact order-free sum of squares, mean = (float)(sum / K) divided in double,
- * r = 1 / sqrt(max(mean + norm_eps, 2^-126)) in IEEE fp32, x_k = (h_k * r) * gain_k, then quantised as above.
+ * reproducible bit for bit: the sum of squares is an integer sum, hence order-free, in which every square is cut off
+ * (truncated) 30 bits below the unit of the token's largest square -- with E the exponent field of the largest |h_k|,
+ * the terms are floor(h_k^2 * 2^(298 - 2E)), which loses less than 2^-44 of the largest square per term --
+ * mean = (float)(sum / K) divided in double, r = 1 / sqrt(max(mean + norm_eps, 2^-126)) in IEEE fp32,
+ * x_k = (h_k * r) * gain_k, then quantised as above.
  *   H        in   bf16 [M, K] row-major; finite (a token with an infinity or a NaN gets beta = NaN)
  *   gain     in   fp32 [K], 16-byte aligned
  *   norm_eps      >= 0
@@ -281,6 +284,25 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                                       int32_t *acc, int path, void *workspace, size_t workspace_bytes,
                                       void *stream);
 bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream);
+
+/*
+ * Checks a packed weight buffer (Section 3, "Memory and Latency": 2-bit storage; a weight is -1, 0 or 1, so the
+ * fourth code never occurs): counts the 2-bit fields that hold 3 into *bad_fields (DEVICE, one int32), synchronises
+ * `stream` and returns BITLINEAR_ERR_BADCODE if there are any, BITLINEAR_OK otherwise.  A buffer that passes is safe
+ * for every kernel; one that does not (a corrupted or foreign file) would give wrong sums, never a fault.
+ */
+bitlinear_status bitlinear_validate_packed(const void *packed, int64_t N, int64_t K, int32_t *bad_fields, void *stream);
+
+/*
+ * Test hook for the bounded waits (no counterpart in the paper).  Every device-side wait of the matmul kernels gives
+ * up after a limit (2 s), sets the workspace's status word to BITLINEAR_ERR_TIMEOUT and lets the kernel return.  This
+ * call arms the NEXT matmul launch of the process (one launch only; the quantiser launch in front of it does not
+ * count): its waits give up after limit_us microseconds (0: the default), and, if skip_arrive is non-zero, one
+ * producer thread of its first CTA leaves out one barrier arrival, so that a wait really runs out.  The launch then
+ * ends with BITLINEAR_ERR_TIMEOUT in the status word and unspecified outputs; the workspace is usable again at once.
+ * Nothing faults or hangs.  (host)
+ */
+void bitlinear_test_expire_next_wait(uint32_t limit_us, int skip_arrive);
 
 /* Synchronises `stream`, then copies the workspace's status word to *device_status (host pointer):
  * BITLINEAR_OK or BITLINEAR_ERR_TIMEOUT.  The return value reports the success of the read itself. */

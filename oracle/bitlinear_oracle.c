@@ -278,6 +278,42 @@ int oracle_quantize_acts(const uint16_t *X_bf16, int64_t M, int64_t K,
  * Parity pins (tests/test_oracle_pins.py): a hand case, agreement of x with a double-precision evaluation of the
  * formula and with torch's rms_norm, scale invariance for eps_n = 0, reduction to the plain quantiser.
  */
+/* N1, N2 for one token of K bfloat16 values: *mean = the fp32 mean square.  Returns 0, or 1 if the token holds an
+ * infinity or a NaN. */
+static int token_mean_square(const uint16_t *h, int64_t K, float *mean)
+{
+    /* N1: exponent field of the largest magnitude, then the integer sum */
+    unsigned E = 0;
+    for (int64_t k = 0; k < K; ++k) {
+        unsigned e = (h[k] >> 7) & 0xFFu;
+        if (e == 255u) return 1;
+        if (e < 1u) e = 1u;
+        if (e > E) E = e;
+    }
+    uint64_t S = 0;
+    for (int64_t k = 0; k < K; ++k) {
+        unsigned bits = h[k];
+        unsigned e = (bits >> 7) & 0xFFu;
+        uint64_t m = bits & 0x7Fu;
+        if (e) m |= 0x80u; else e = 1u;
+        unsigned twice = 2u * (E - e);
+        if (twice <= 46u) S += ((m * m) << 30) >> twice;
+    }
+    *mean = (float)(ldexp((double)S / (double)K, 2 * (int)E - 298)); /* N2 */
+    return 0;
+}
+
+/* The mean square alone, per token (for the pins: compared with the exactly rounded mean of the exact squares). */
+int oracle_rmsnorm_mean_square(const uint16_t *H_bf16, int64_t M, int64_t K, float *mean)
+{
+    if (!H_bf16 || !mean || M < 0 || K <= 0)
+        return ORACLE_ERR_ARG;
+    for (int64_t t = 0; t < M; ++t)
+        if (token_mean_square(H_bf16 + t * K, K, &mean[t]))
+            return ORACLE_ERR_RANGE;
+    return ORACLE_OK;
+}
+
 int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, float eps_n, int64_t M, int64_t K,
                                  int8_t *Xq, float *beta, int32_t *rowsum, float *x_out /* may be NULL: [M][K] */)
 {
@@ -288,32 +324,14 @@ int oracle_rmsnorm_quantize_acts(const uint16_t *H_bf16, const float *gain, floa
 #pragma omp parallel for
 #endif
     for (int64_t t = 0; t < M; ++t) {
-        /* N1: exponent field of the largest magnitude, then the integer sum */
-        unsigned E = 0;
-        int bad = 0;
-        for (int64_t k = 0; k < K; ++k) {
-            unsigned e = (H_bf16[t * K + k] >> 7) & 0xFFu;
-            if (e == 255u) bad = 1;
-            if (e < 1u) e = 1u;
-            if (e > E) E = e;
-        }
-        if (bad) {
+        float mean;
+        if (token_mean_square(H_bf16 + t * K, K, &mean)) {
 #ifdef _OPENMP
 #pragma omp critical
 #endif
             status = ORACLE_ERR_RANGE;
             continue;
         }
-        uint64_t S = 0;
-        for (int64_t k = 0; k < K; ++k) {
-            unsigned bits = H_bf16[t * K + k];
-            unsigned e = (bits >> 7) & 0xFFu;
-            uint64_t m = bits & 0x7Fu;
-            if (e) m |= 0x80u; else e = 1u;
-            unsigned twice = 2u * (E - e);
-            if (twice <= 46u) S += ((m * m) << 30) >> twice;
-        }
-        float mean = (float)(ldexp((double)S / (double)K, 2 * (int)E - 298)); /* N2 */
         float d = mean + eps_n;
         if (!(d > 1.17549435e-38f)) d = 1.17549435e-38f; /* an all-zero or vanishing token: r stays finite */
         float r = 1.0f / sqrtf(d);

@@ -57,6 +57,7 @@ class Oracle:
         L.oracle_unpack_weights.argtypes = [_p, _i64, _i64, _p]
         L.oracle_quantize_acts.argtypes = [_p, _i64, _i64, _p, _p, _p]
         L.oracle_rmsnorm_quantize_acts.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p, _p, _p, _p]
+        L.oracle_rmsnorm_mean_square.argtypes = [_p, _i64, _i64, _p]
         L.oracle_swiglu_quantize_acts.argtypes = [_p, _p, _i64, _i64, _p, _p, _p, _p]
         L.oracle_quantize_acts_bits.argtypes = [_p, _i64, _i64, ctypes.c_int, _p, _p, _p]
         L.oracle_dequant_bits.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, ctypes.c_int, _p]
@@ -164,6 +165,14 @@ class Oracle:
                                                    self._ptr(x) if return_x else None)
         self._check(rc, "rmsnorm_quantize_acts")
         return (Xq, beta, rs, x) if return_x else (Xq, beta, rs)
+
+    def rmsnorm_mean_square(self, H_bf16_bits: np.ndarray) -> np.ndarray:
+        """The fp32 mean square of every token as the RMSNorm front forms it -> float32 [M]."""
+        H = self._c(H_bf16_bits, np.uint16)
+        M, K = H.shape
+        mean = np.empty(M, np.float32)
+        self._check(self.lib.oracle_rmsnorm_mean_square(self._ptr(H), M, K, self._ptr(mean)), "rmsnorm_mean_square")
+        return mean
 
     def swiglu_quantize_acts(self, G_bf16_bits: np.ndarray, U_bf16_bits: np.ndarray, return_h: bool = False):
         """h = silu(g) * u in fp32 followed by the activation quantiser -> (Xq, beta, rowsum[, h float32 [M,K]])."""

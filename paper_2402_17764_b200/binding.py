@@ -16,8 +16,8 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libbitlinear_b200.so"
 
 OK = 0
-ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE = range(-1, -9, -1)
-PATH_AUTO, PATH_DP4A, PATH_MMA, PATH_TCGEN05, PATH_TCGEN05_PAIR, PATH_TCGEN05_TS = 0, 1, 2, 3, 4, 5
+ERR_ARG, ERR_SHAPE, ERR_ALIGN, ERR_WORKSPACE, ERR_ARCH, ERR_CUDA, ERR_TIMEOUT, ERR_RANGE, ERR_BADCODE = range(-1, -10, -1)
+PATH_AUTO, PATH_DP4A, PATH_MMA, PATH_TCGEN05 = 0, 1, 2, 3
 
 EXPORTS = [
     "bitlinear_status_string",
@@ -42,6 +42,8 @@ EXPORTS = [
     "bitlinear_sequence_destroy",
     "bitlinear_matmul_i32",
     "bitlinear_unpack_weights",
+    "bitlinear_validate_packed",
+    "bitlinear_test_expire_next_wait",
     "bitlinear_poll_status",
 ]
 
@@ -108,6 +110,9 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_matmul_i32.argtypes = [vp, vp, i64, i64, i64, vp, ci, vp, sz, vp]
     L.bitlinear_unpack_weights.argtypes = [vp, i64, i64, vp, vp]
     L.bitlinear_poll_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
+    L.bitlinear_validate_packed.argtypes = [vp, i64, i64, vp, vp]
+    L.bitlinear_test_expire_next_wait.argtypes = [ctypes.c_uint32, ci]
+    L.bitlinear_test_expire_next_wait.restype = None
     _lib = L
     return L
 
@@ -292,6 +297,20 @@ def unpack_weights(packed: torch.Tensor, N: int, K: int, stream=None) -> torch.T
     st = load_library().bitlinear_unpack_weights(_ptr(packed), N, K, _ptr(T), _stream(stream))
     _check(st, "bitlinear_unpack_weights")
     return T
+
+
+def validate_packed(packed: torch.Tensor, N: int, K: int, stream=None) -> int:
+    """bitlinear_validate_packed: -> number of 2-bit fields that hold the unused code 3 (0: the buffer is sound)."""
+    bad = torch.empty(1, dtype=torch.int32, device=packed.device)
+    st = load_library().bitlinear_validate_packed(_ptr(packed), N, K, _ptr(bad), _stream(stream))
+    if st not in (OK, ERR_BADCODE):
+        _check(st, "bitlinear_validate_packed")
+    return int(bad.item())
+
+
+def test_expire_next_wait(limit_us: int, skip_arrive: bool):
+    """bitlinear_test_expire_next_wait (test hook): arms the next matmul launch; see include/bitlinear.h."""
+    load_library().bitlinear_test_expire_next_wait(int(limit_us), 1 if skip_arrive else 0)
 
 
 def poll_status(workspace: torch.Tensor, stream=None) -> int:

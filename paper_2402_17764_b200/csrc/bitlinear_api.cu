@@ -1,13 +1,28 @@
 // C ABI of the BitLinear library: argument validation, workspace layout, dispatch.
 // No arithmetic of the method lives here; every step runs in the kernels.
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
 
 #include "internal.cuh"
+#include "ptx.cuh"
 
 namespace bitlinear {
+
+// The wait hooks of the next matmul launch, packed into one word so that setting and taking them are single atomic
+// operations: bits 0..30 the limit in microseconds (0: the default), bit 31 the skipped arrival.
+static std::atomic<uint32_t> g_next_wait_hooks{0};
+
+WaitHooks take_wait_hooks()
+{
+    const uint32_t v = g_next_wait_hooks.exchange(0u);
+    WaitHooks h;
+    h.limit_us = (v & 0x7FFFFFFFu) ? (v & 0x7FFFFFFFu) : ptx::kWaitLimitUs;
+    h.skip_arrive = v >> 31;
+    return h;
+}
 
 int sm_count()
 {
@@ -47,11 +62,18 @@ bitlinear_status check_shape(int64_t M, int64_t N, int64_t K)
     return BITLINEAR_OK;
 }
 
+// Measurement aid, compiled in only with -DBITLINEAR_TUNING (the library as built by build.py reads no environment
+// variable).
 int env_int(const char *name, int fallback)
 {
+#ifdef BITLINEAR_TUNING
     const char *v = std::getenv(name);
     if (!v || !*v) return fallback;
     return std::atoi(v);
+#else
+    (void)name;
+    return fallback;
+#endif
 }
 
 struct Layout {
@@ -106,7 +128,7 @@ __global__ void rowsum_kernel(const int8_t *__restrict__ Xq, int K, int32_t *__r
 
 // From 17 tokens on a single matmul goes to the tensor-core GEMM: measured on 110080 x 4096, the GEMM takes the
 // same 52 us from 17 to 128 tokens, the weight-streaming kernel 59 us at 16 tokens, 92 us at 32 and 174 us at 64.
-// BITLINEAR_TCGEN05_MIN_M (a measurement aid) moves the switch-over point.
+// (In a -DBITLINEAR_TUNING build BITLINEAR_TCGEN05_MIN_M moves the switch-over point.)
 bool use_tcgen05_for(int64_t M)
 {
     static const int min_m = env_int("BITLINEAR_TCGEN05_MIN_M", 17);
@@ -148,24 +170,10 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
 {
     WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
     OwnedList *lists = reinterpret_cast<OwnedList *>(ws + lists_offset);
-    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
-                    (path == BITLINEAR_PATH_TCGEN05_TS) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
+    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
     if (tc) {
-        static const int ts_tokens = env_int("BITLINEAR_PREFILL_TS_TOKENS", 0); // 64, 192 or 256 (a measurement aid)
-        if (path == BITLINEAR_PATH_TCGEN05_TS || (path == BITLINEAR_PATH_AUTO && ts_tokens > 0)) {
-            cudaError_t err = launch_prefill_ts(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out, e.out_i32,
-                                                ts_tokens > 0 ? ts_tokens : 256, hdr, stream);
-            return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
-        }
-        // The two-SM form of the GEMM is correct (the tests run it) but measured slower than the one-SM form on
-        // B200 (1.15 against 2.2 POP/s), so it is not chosen unless asked for.
-        static const int pair_min_m = env_int("BITLINEAR_PREFILL_PAIR_MIN_M", 1 << 30);
-        const bool pair = (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
-                          (path == BITLINEAR_PATH_AUTO && e.M >= pair_min_m && e.qb == (float)kQb && prefill_pair_capacity() > 0);
-        cudaError_t err = pair ? launch_prefill_pair(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, e.K, e.N, e.out,
-                                                     e.out_i32, hdr, stream)
-                               : launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, x_rows, e.K, e.N, e.out,
-                                                e.out_i32, e.qb, hdr, split_scratch, stream);
+        cudaError_t err = launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, x_rows, e.K, e.N, e.out, e.out_i32,
+                                         e.qb, hdr, split_scratch, stream);
         return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
     }
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
@@ -196,6 +204,7 @@ const char *bitlinear_status_string(bitlinear_status s)
     case BITLINEAR_ERR_CUDA: return "CUDA call failed";
     case BITLINEAR_ERR_TIMEOUT: return "device-side wait timed out";
     case BITLINEAR_ERR_RANGE: return "weight out of range";
+    case BITLINEAR_ERR_BADCODE: return "packed weights hold the unused 2-bit code";
     default: return "unknown status";
     }
 }
@@ -361,7 +370,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                                       int32_t *acc, int path, void *workspace, size_t workspace_bytes, void *stream)
 {
     if (!packed || !workspace || (M > 0 && (!Xq || !acc))) return BITLINEAR_ERR_ARG;
-    if (path < BITLINEAR_PATH_AUTO || path > BITLINEAR_PATH_TCGEN05_TS) return BITLINEAR_ERR_ARG;
+    if (path < BITLINEAR_PATH_AUTO || path > BITLINEAR_PATH_TCGEN05) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, N, K);
     if (st != BITLINEAR_OK) return st;
     if (path == BITLINEAR_PATH_DP4A && M > 8) return BITLINEAR_ERR_SHAPE;
@@ -374,14 +383,10 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     if (M == 0) return BITLINEAR_OK;
     char *ws = reinterpret_cast<char *>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
-    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_TCGEN05_PAIR) ||
-                    (path == BITLINEAR_PATH_TCGEN05_TS) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
+    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
     InlineTable inl{};
     fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
-    // (only the one-SM GEMM with weights in shared memory cuts tiles along K)
-    const size_t clear = (path == BITLINEAR_PATH_TCGEN05 || (path == BITLINEAR_PATH_AUTO && tc))
-                             ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M)
-                             : 0;
+    const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, false, (int)K, s);
@@ -408,6 +413,27 @@ bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
 }
 
+bitlinear_status bitlinear_validate_packed(const void *packed, int64_t N, int64_t K, int32_t *bad_fields, void *stream)
+{
+    if (!packed || !bad_fields) return BITLINEAR_ERR_ARG;
+    bitlinear_status st = check_shape(0, N, K);
+    if (st != BITLINEAR_OK) return st;
+    if (!aligned(packed, 16) || !aligned(bad_fields, 4)) return BITLINEAR_ERR_ALIGN;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (launch_count_bad_codes(packed, bitlinear_packed_bytes(N, K), bad_fields, s) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    int32_t n = 0;
+    if (cudaMemcpy(&n, bad_fields, sizeof n, cudaMemcpyDeviceToHost) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    return n == 0 ? BITLINEAR_OK : BITLINEAR_ERR_BADCODE;
+}
+
+void bitlinear_test_expire_next_wait(uint32_t limit_us, int skip_arrive)
+{
+    if (limit_us > 0x7FFFFFFFu) limit_us = 0x7FFFFFFFu;
+    g_next_wait_hooks.store(limit_us | (skip_arrive ? 0x80000000u : 0u));
+}
+
 bitlinear_status bitlinear_poll_status(const void *workspace, void *stream, int *device_status)
 {
     if (!workspace || !device_status) return BITLINEAR_ERR_ARG;
@@ -431,17 +457,23 @@ bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma
     bitlinear_status st = check_shape(M, N, K);
     if (st != BITLINEAR_OK) return st;
     if (single_layout(M, N, K).total > kStaticWorkspaceBytes) return BITLINEAR_ERR_WORKSPACE;
-    // device address of the scratch, looked up once per device while that device is current
-    static void *address[64] = {nullptr};
+    // the checks bitlinear_forward would make, before the device is asked for anything
+    if (!packed || !gamma || (M > 0 && (!X || !Y))) return BITLINEAR_ERR_ARG;
+    if (!aligned(packed, 16) || !aligned(X, 16) || !aligned(Y, 16) || !aligned(gamma, 4)) return BITLINEAR_ERR_ALIGN;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    // device address of the scratch, looked up once per device while that device is current (two host threads that
+    // get here together both look it up and store the same value)
+    static std::atomic<void *> address[64];
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return BITLINEAR_ERR_CUDA;
-    if (!address[dev]) {
+    if (!address[dev].load(std::memory_order_acquire)) {
         void *p = nullptr;
         if (cudaGetSymbolAddress(&p, g_static_workspace) != cudaSuccess || !p) return BITLINEAR_ERR_CUDA;
-        address[dev] = p;
+        address[dev].store(p, std::memory_order_release);
     }
     // bitlinear_forward clears the part of the workspace that has to start at zero on every call
-    return bitlinear_forward(packed, gamma, X, M, K, N, Y, address[dev], kStaticWorkspaceBytes, stream);
+    return bitlinear_forward(packed, gamma, X, M, K, N, Y, address[dev].load(std::memory_order_acquire),
+                             kStaticWorkspaceBytes, stream);
 }
 
 // ---- sequences -------------------------------------------------------------------------------
@@ -481,7 +513,7 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
 {
     if (!layers || n <= 0 || n > 65536) return false;
     size_t acc = 0, data = 0;
-    uint64_t tiles = 0, gemm_tiles = 0;
+    uint64_t tiles = 0, gemm_tiles = 0, tokens = 0;
     int64_t min_kb = INT32_MAX;
     int64_t max_M = 0;
     for (int i = 0; i < n; ++i)
@@ -491,6 +523,7 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
         if (check_shape(d.M, d.N, d.K) != BITLINEAR_OK || d.M < 1) return false;
+        tokens += (uint64_t)d.M;
         if (!gemm) acc += align_up((size_t)d.M * d.N * 4, 256);
         tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K)); // an upper bound of the work items in either mode
         gemm_tiles += (uint64_t)((d.M + 127) / 128) * (uint64_t)((d.N + 255) / 256); // the same for the GEMM's CTA tiles
@@ -499,6 +532,7 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
         data += seq_xq_bytes(d.M, d.K, gemm) + 2 * align_up((size_t)d.M * 4, 256);
     }
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
+    if (tokens > 0x3FFFFFFFull) return false; // tokens (plus the clearing CTAs) index the quantiser's grid with an int
     if (gemm && gemm_tiles > 0x7FFFFFFFull) return false;
     if (gemm) { // scratch for tiles cut along K, where the streaming kernel has its int32 scratch
         uint64_t exact = 0;

@@ -313,7 +313,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, i
 template <int NT>
 __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
-    uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr, OwnedList *lists)
+    uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr, OwnedList *lists, const WaitHooks hooks)
 {
     extern __shared__ __align__(128) uint8_t dsmem[];
     ptx::griddep_launch_dependents(); // the finishing launch may become resident; it waits for this grid to end
@@ -485,7 +485,9 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 #pragma unroll
         for (int i = 0; i < kStages; ++i) {
             if (i < n_held) {
-                ptx::mbar_arrive_expect_tx(bars + 8 * i, held_bytes[i]);
+                // (test device: the first warp of the launch leaves out the arrival that announces its first chunk's
+                // activation bytes; the copy itself is issued and lands, the phase never completes)
+                if (!(hooks.skip_arrive && w == 0 && i == 0)) ptx::mbar_arrive_expect_tx(bars + 8 * i, held_bytes[i]);
                 bulk_copy_g2s(ring + i * R::kSlotBytes + R::kWeightBytes, held_x[i], held_bytes[i], bars + 8 * i);
             }
         }
@@ -530,7 +532,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             const int n = min(min(kChunkTiles, KB - kt), left);
             const uint32_t s = consumed % kStages;
             const uint32_t slot = ring + s * R::kSlotBytes;
-            if (!ptx::mbar_wait_bounded(bars + 8 * s, (consumed / kStages) & 1u, abort_flag)) { alive = false; break; }
+            if (!ptx::mbar_wait_bounded(bars + 8 * s, (consumed / kStages) & 1u, abort_flag, hooks.limit_us)) { alive = false; break; }
             // (n is the same for all lanes: mma.sync needs the whole warp)
             if (n == kChunkTiles) {
 #pragma unroll
@@ -624,7 +626,7 @@ struct WideRing {
 template <int NT>
 __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
-    uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists)
+    uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists, const WaitHooks hooks)
 {
     extern __shared__ __align__(128) uint8_t dsmem[];
     ptx::griddep_launch_dependents();
@@ -722,7 +724,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
             const uint32_t s = issued % kDepth;
             if (warp == 0 && issued >= (uint32_t)kDepth) {
                 // the slot's previous contents must have been consumed by all eight warps
-                if (!ptx::mbar_wait_bounded(xempty + 8 * s, (issued / kDepth - 1) & 1u, abort_flag)) {
+                if (!ptx::mbar_wait_bounded(xempty + 8 * s, (issued / kDepth - 1) & 1u, abort_flag, hooks.limit_us)) {
                     alive = false;
                     break;
                 }
@@ -760,7 +762,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
 #pragma unroll
         for (int i = 0; i < kDepth; ++i) {
             if (i < n_held) {
-                ptx::mbar_arrive_expect_tx(xfull + 8 * i, held_bytes[i]);
+                // (test device: the first CTA leaves out the arrival that announces its first activation chunk)
+                if (!(hooks.skip_arrive && blockIdx.x == 0 && i == 0)) ptx::mbar_arrive_expect_tx(xfull + 8 * i, held_bytes[i]);
                 bulk_copy_g2s(xring + i * R::kXSlotBytes, held_x[i], held_bytes[i], xfull + 8 * i);
             }
         }
@@ -788,8 +791,8 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
             ended = c.ends_group;
             const uint32_t s = consumed % kDepth;
             const uint32_t parity = (consumed / kDepth) & 1u;
-            if (!ptx::mbar_wait_bounded(xfull + 8 * s, parity, abort_flag) ||
-                (active && !ptx::mbar_wait_bounded(wbars + 8 * s, parity, abort_flag))) {
+            if (!ptx::mbar_wait_bounded(xfull + 8 * s, parity, abort_flag, hooks.limit_us) ||
+                (active && !ptx::mbar_wait_bounded(wbars + 8 * s, parity, abort_flag, hooks.limit_us))) {
                 alive = false;
                 break;
             }
@@ -923,13 +926,20 @@ __global__ void __launch_bounds__(kWarps * 32) decode_dp4a_kernel(const __grid_c
 
 } // namespace
 
-// Measurement aid: a positive integer in the environment overrides a tuning constant.
+// Measurement aid, compiled in only with -DBITLINEAR_TUNING (the library as built by build.py reads no environment
+// variable): a positive integer in the environment overrides a tuning constant.
 static uint32_t tuning_from_env(const char *name, uint32_t fallback, uint32_t max_value)
 {
+#ifdef BITLINEAR_TUNING
     const char *v = std::getenv(name);
     if (!v || !*v) return fallback;
     const long x = std::atol(v);
     return (x >= 1 && x <= (long)max_value) ? (uint32_t)x : fallback;
+#else
+    (void)name;
+    (void)max_value;
+    return fallback;
+#endif
 }
 
 // Launches `kernel` as a programmatic dependent of the launch before it in the stream (it may start early and
@@ -955,6 +965,7 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
                               uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr,
                               OwnedList *lists, cudaStream_t stream)
 {
+    WaitHooks hooks = take_wait_hooks();
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -965,7 +976,7 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
     }
     static const bool early = tuning_from_env("BITLINEAR_DECODE_EARLY_LAUNCH", 1, 2) == 1; // 2 = off
     void *args[] = {(void *)&inl, (void *)&table, (void *)&n_entries, (void *)&total_tiles, (void *)&share,
-                    (void *)&dyn, (void *)&hdr, (void *)&lists};
+                    (void *)&dyn, (void *)&hdr, (void *)&lists, (void *)&hooks};
     cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT>, grid, block, Ring<NT>::kSmem, args, early, stream);
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
@@ -981,6 +992,7 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
                                uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists,
                                cudaStream_t stream)
 {
+    WaitHooks hooks = take_wait_hooks();
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -991,7 +1003,7 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
     }
     static const bool early = tuning_from_env("BITLINEAR_DECODE_EARLY_LAUNCH", 1, 2) == 1; // 2 = off
     void *args[] = {(void *)&inl, (void *)&table, (void *)&n_entries, (void *)&total_items, (void *)&share,
-                    (void *)&hdr, (void *)&lists};
+                    (void *)&hdr, (void *)&lists, (void *)&hooks};
     cudaError_t err = launch_dependent((const void *)decode_wide_kernel<NT>, grid, block, WideRing<NT>::kSmem, args, early, stream);
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
@@ -1039,6 +1051,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     uint32_t share = total_tiles / n_warps, dyn = 0;
     if (share >= 4 * kMinPieceTiles && static_percent < 100) {
         share = (uint32_t)((uint64_t)total_tiles * static_percent / 100 / n_warps);
+        if (share == 0) share = 1; // (a warp without a share never draws a piece)
         const uint32_t rest = total_tiles - share * n_warps;
         dyn = rest / (n_warps * pieces_per_warp);
         if (dyn < kMinPieceTiles) dyn = kMinPieceTiles;

@@ -74,6 +74,8 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
                                     cudaStream_t stream);
 cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream);
+// *bad (device) = number of 2-bit fields among the `bytes` bytes of a packed buffer that hold the unused code 3.
+cudaError_t launch_count_bad_codes(const void *packed, size_t bytes, int32_t *bad, cudaStream_t stream);
 // Copies row-major int8 activations [M, K] into the tiled layout [KB][M][64] (columns >= K become 0).
 cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *tiled, cudaStream_t stream);
 
@@ -122,18 +124,16 @@ cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gam
 cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, int min_KB,
                                  void *split_scratch, cudaStream_t stream);
 
-// The same GEMM on pairs of SMs (tcgen05 cta_group::2): 256 tokens x 256 features per pair tile.
-// prefill_pair_capacity: CTA pairs that can be resident at once (0: not available on this device).
-cudaError_t launch_prefill_pair(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
-                                const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
-                                WorkspaceHeader *hdr, cudaStream_t stream);
-int prefill_pair_capacity();
-
-// The same GEMM with the expanded weights in tensor memory: 128 features x tokens_per_tile (192 or 256)
-// tokens per CTA tile.
-cudaError_t launch_prefill_ts(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
-                              const int32_t *rowsum, int64_t M, int64_t K, int64_t N, void *out, int out_i32,
-                              int tokens_per_tile, WorkspaceHeader *hdr, cudaStream_t stream);
+// What a matmul launch is told about its bounded device-side waits.  limit_us: how long a wait may last (2 s unless
+// a test shortened it).  skip_arrive != 0 is a test device: ONE producer thread of the launch (in CTA 0) leaves out ONE
+// barrier arrival, so that the wait behind it runs out and the kernel's way out of an expired wait can be checked;
+// everything else, every copy included, is issued as usual.
+struct WaitHooks {
+    uint32_t limit_us;
+    uint32_t skip_arrive;
+};
+// The hooks for the next matmul launch: the defaults, or what bitlinear_test_expire_next_wait set (used up by this call).
+WaitHooks take_wait_hooks();
 
 int sm_count();
 

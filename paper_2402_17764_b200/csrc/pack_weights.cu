@@ -135,7 +135,34 @@ __global__ void __launch_bounds__(256) unpack_kernel(const uint8_t *__restrict__
     }
 }
 
+// Counts the 2-bit fields of a packed buffer that hold 3, the code no weight has (over the whole buffer, padding
+// included: every field there is 1).  A field is 3 exactly where both of its bits are set.
+__global__ void __launch_bounds__(256) count_bad_codes_kernel(const uint4 *__restrict__ packed, size_t n_vec,
+                                                              int32_t *__restrict__ bad)
+{
+    int found = 0;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n_vec; i += (size_t)gridDim.x * blockDim.x) {
+        const uint4 v = __ldg(packed + i);
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) found += __popc(w[j] & (w[j] >> 1) & 0x55555555u);
+    }
+    found = __reduce_add_sync(0xffffffffu, found);
+    if ((threadIdx.x & 31) == 0 && found) atomicAdd(bad, found);
+}
+
 } // namespace
+
+cudaError_t launch_count_bad_codes(const void *packed, size_t bytes, int32_t *bad, cudaStream_t stream)
+{
+    cudaError_t err = cudaMemsetAsync(bad, 0, sizeof(int32_t), stream);
+    if (err != cudaSuccess) return err;
+    const size_t n_vec = bytes / 16;
+    size_t blocks = (n_vec + 255) / 256;
+    if (blocks > (size_t)sm_count() * 8) blocks = (size_t)sm_count() * 8;
+    count_bad_codes_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint4 *>(packed), n_vec, bad);
+    return cudaGetLastError();
+}
 
 cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
                                     cudaStream_t stream)

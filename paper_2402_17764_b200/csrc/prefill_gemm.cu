@@ -98,6 +98,7 @@ struct Barriers {
     uint64_t expanded[kMaxBSlots]; // int8 weight tile written
     uint64_t acc_full[2];        // accumulator(s) of a tile complete
     uint64_t acc_empty[2];       // drained by the epilogue
+    uint64_t epilogue_met;       // rendezvous of the four epilogue warps (tiles cut along K)
     uint32_t tmem_base;
     int abort_flag;
     int split_last; // this CTA added the last partial sums of a cut tile
@@ -201,7 +202,7 @@ struct ProblemCursor {
 template <int MT, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems,
-                    const SplitPlan sp, int a_rows, int n_stages)
+                    const SplitPlan sp, int a_rows, int n_stages, const WaitHooks hooks)
 {
     constexpr int kAccBufs = Cfg<MT>::kAccBufs, kBSlots = Cfg<MT>::kBSlots, kGroups = Cfg<MT>::kGroups;
     const uint32_t kStageBytes = stage_bytes(MT, a_rows), kAHalfBytes = (uint32_t)(a_rows * BK);
@@ -228,6 +229,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             mbar_init(smem_u32(&bars->acc_full[b]), 1);
             mbar_init(smem_u32(&bars->acc_empty[b]), 4);
         }
+        mbar_init(smem_u32(&bars->epilogue_met), 4);
         bars->abort_flag = 0;
         fence_mbar_init();
     }
@@ -264,14 +266,17 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // a second token tile past the end is left out
                 for (int kb = kb_begin; kb < kb_end; ++kb, pos.advance(n_stages)) {
                     const int s = pos.s;
-                    if (pos.round > 0 && !mbar_wait_bounded(smem_u32(&bars->empty[s]), (pos.round - 1) & 1, abort_flag)) {
+                    if (pos.round > 0 && !mbar_wait_bounded(smem_u32(&bars->empty[s]), (pos.round - 1) & 1, abort_flag, hooks.limit_us)) {
                         ok = false;
                         break;
                     }
                     const uint32_t full = smem_u32(&bars->full[s]);
                     const uint32_t a_dst = stages + s * kStageBytes;
                     const uint32_t p_dst = a_dst + MT * kAHalfBytes;
-                    mbar_arrive_expect_tx(full, halves * kAHalfBytes + kPBytes);
+                    // (test device: the first CTA leaves out the arrival that announces its first stage's bytes; the
+                    // loads are issued and land, the phase never completes)
+                    if (!(hooks.skip_arrive && blockIdx.x == 0 && pos.it == 0))
+                        mbar_arrive_expect_tx(full, halves * kAHalfBytes + kPBytes);
                     tma_load_2d(a_dst, &g.tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
                     if (halves == 2) tma_load_2d(a_dst + kAHalfBytes, &g.tmap_x, kb * BK, m0 + BM, full);
                     tma_load_3d(p_dst, &g.tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
@@ -307,13 +312,13 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 const int kb_begin = unit.kb0(sp, p.KB), kb_end = unit.kb1(sp, p.KB);
                 const int buf = tile_it % kAccBufs;
                 const uint32_t use = tile_it / kAccBufs;
-                if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag)) break;
+                if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag, hooks.limit_us)) break;
                 tc_fence_after_sync();
                 const uint32_t d_tmem = tmem_base + (uint32_t)(buf * MT * BN);
                 const bool two = MT == 2 && ((tile - p.tile_begin) % p.tiles_m) * (MT * BM) + BM < p.M;
                 uint32_t accumulate = 0;
                 for (int kb = kb_begin; kb < kb_end; ++kb) {
-                    if (!mbar_wait_bounded(expanded_bar, b_parity, abort_flag)) {
+                    if (!mbar_wait_bounded(expanded_bar, b_parity, abort_flag, hooks.limit_us)) {
                         ok = false;
                         break;
                     }
@@ -378,12 +383,12 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 const uint32_t rround = reader.round;
                 if (has_reader) reader.advance(n_stages);
                 if (!mine) continue;
-                if (!mbar_wait_bounded(smem_u32(&bars->full[s]), pos.round & 1, abort_flag)) {
+                if (!mbar_wait_bounded(smem_u32(&bars->full[s]), pos.round & 1, abort_flag, hooks.limit_us)) {
                     ok = false;
                     break;
                 }
                 // (the reader's stage is not refilled before this tile is expanded: its `empty` phase is the latest)
-                if (has_reader && !mbar_wait_bounded(smem_u32(&bars->empty[rs]), rround & 1, abort_flag)) {
+                if (has_reader && !mbar_wait_bounded(smem_u32(&bars->empty[rs]), rround & 1, abort_flag, hooks.limit_us)) {
                     ok = false;
                     break;
                 }
@@ -430,7 +435,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             const int buf = tile_it % kAccBufs;
             const uint32_t parity = (tile_it / kAccBufs) & 1;
             const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // no MMA wrote the accumulator of an absent token tile
-            if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), parity, abort_flag)) break;
+            if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), parity, abort_flag, hooks.limit_us)) break;
             tc_fence_after_sync();
 
             // shift, subtract, scale, round and store the 32 sums `v` of chunk c (features n0 + 32 c ..) of token t
@@ -543,13 +548,19 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 bulk_wait_group0(); // the sums have been added
                 __threadfence();
             }
-            named_bar_sync(1, 128); // the four epilogue warps
+            // The four epilogue warps meet twice (a cut unit is its CTA's last, so the barrier's phases are 0 and 1).
+            // The rendezvous is a bounded wait like every other: a warp that left through an expired wait never
+            // arrives, and the others then give up too instead of waiting for it for ever.
+            if (lane == 0) mbar_arrive(smem_u32(&bars->epilogue_met));
+            if (!mbar_wait_bounded(smem_u32(&bars->epilogue_met), 0, abort_flag, hooks.limit_us)) break;
             if (warp == 2 && lane == 0) {
                 const uint32_t before = atomicAdd(&sp.counters[cut], 1u);
                 bars->split_last = (before == (uint32_t)sp.slices - 1u) ? 1 : 0;
                 __threadfence();
             }
-            named_bar_sync(1, 128);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars->epilogue_met));
+            if (!mbar_wait_bounded(smem_u32(&bars->epilogue_met), 1, abort_flag, hooks.limit_us)) break;
             if (bars->split_last) { // every slice has been added: dequantise the tile from the scratch
 #pragma unroll 1
                 for (int half = 0; half < halves; ++half) {
@@ -627,10 +638,14 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
 // How many K slices the tiles of the last, partly filled round of the SMs are cut into (1: none are cut).
 static int split_slices(int n_tiles, int min_KB, int sms)
 {
+#ifdef BITLINEAR_TUNING // measurement aid, not compiled into the library as build.py builds it
     static const int enabled = [] {
         const char *v = std::getenv("BITLINEAR_PREFILL_SPLIT");
         return (v && *v) ? std::atoi(v) : 1;
     }();
+#else
+    constexpr int enabled = 1;
+#endif
     const int r = n_tiles % sms;
     if (!enabled || r == 0 || 2 * r > sms || r > kMaxSplitTiles) return 1;
     int s = sms / r;
@@ -681,7 +696,8 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
     cfg.stream = stream;
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
-    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&sp, (void *)&a_rows, (void *)&n_stages};
+    WaitHooks hooks = take_wait_hooks();
+    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&sp, (void *)&a_rows, (void *)&n_stages, (void *)&hooks};
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 

@@ -1,9 +1,9 @@
 """GPU parity at the full sizes of the benchmark's workloads, in the launch configuration bench.py times.
 
 The oracle cannot finish a whole 3B- or 70B-shaped step in seconds, so outputs are SAMPLED: for chosen
-matrices the oracle ternarises the full latent matrix (Eq. 1-3), quantises the token (Section 2), and the
-sampled outputs are recomputed one by one as exact int32 dot products and dequantised with the same fp32
-formula; they must match the GPU's bf16 bits.  On top of that come properties that hold at any size:
+matrices the oracle ternarises the full latent matrix (Eq. 1-3), quantises the token (Section 2), and computes
+the sampled outputs with its own int32 matmul and its own dequantisation on the sampled rows of the ternary
+matrix; they must match the GPU's bf16 bits.  On top of that come properties that hold at any size:
 every stored 2-bit code is 0, 1 or 2, and every output is finite.
 """
 import numpy as np
@@ -29,20 +29,14 @@ def timing_oracle():
     return load_oracle("timing")
 
 
-def f32_to_bf16_bits_rne(x):
-    u = np.asarray(x, np.float32).view(np.uint32).astype(np.uint64)
-    return (((u + 0x7FFF + ((u >> 16) & 1)) >> 16) & 0xFFFF).astype(np.uint16)
-
-
 def expected_samples(orc, W, X_bits, rows, eps=1e-5):
-    """Oracle values of Y[t, n] for all tokens t and the sampled rows n: (bf16 bits [M, len(rows)])."""
+    """Oracle values of Y[t, n] for all tokens t and the sampled rows n: (bf16 bits [M, len(rows)]).
+    Every step is the oracle's: Eq. 1-3 on the whole latent matrix, the activation quantiser, the int32 matmul on the
+    sampled rows of the ternary matrix, the dequantisation."""
     T, gamma = orc.quantize_weights(W, eps)
     q, beta, _ = orc.quantize_acts(X_bits)
-    acc = q.astype(np.int64) @ T[rows].astype(np.int64).T          # exact
-    assert np.abs(acc).max() < 2 ** 24
-    scale = (np.float32(gamma) * beta.astype(np.float32)) / np.float32(127)
-    y = acc.astype(np.float32) * scale[:, None]
-    return f32_to_bf16_bits_rne(y)
+    acc = orc.matmul_i32(q, np.ascontiguousarray(T[rows]))
+    return orc.dequant(acc, beta, gamma)
 
 
 def check_samples(Y, want_bits, rows, what):

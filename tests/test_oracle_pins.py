@@ -485,3 +485,106 @@ def test_low_bit_activations_properties(oracle):
         y = bits_to_f32(oracle.dequant_bits(oracle.matmul_i32(q, T), beta, 0.02, bits)).astype(np.float64)
         want = (q.astype(np.float64) * (beta.astype(np.float64) / qb)[:, None]) @ (T.astype(np.float64) * 0.02).T
         assert np.allclose(y, want, rtol=2.0 ** -8, atol=1e-9)
+
+
+# ---- the all-zero matrix (0 / 0 in Eq. 1 when eps = 0) ----
+
+def test_all_zero_matrix_quantises_to_zeros(oracle):
+    """W = 0 and eps = 0: gamma = 0 and Eq. 1 divides 0 by 0.  Reading: every weight stays 0, so every stored field
+    holds code 1 (byte 0b01010101) and the forward gives zeros; with eps > 0 the quotient is an ordinary 0."""
+    W = np.zeros((16, 32), np.float32)
+    for eps in (0.0, 1e-5):
+        T, g = oracle.quantize_weights(W, eps)
+        assert g == 0.0 and not T.any()
+        assert np.all(oracle.pack_weights(T) == 0x55)
+        assert np.array_equal(R.quantize_weights(W, eps)[0], T)
+    xbits = f32_to_bf16_bits(np.arange(-16, 16, dtype=np.float32).reshape(1, 32))
+    assert not oracle.forward(oracle.quantize_weights(W, 0.0)[0], 0.0, xbits).any()
+    # a single non-zero weight among zeros is the only one that survives: gamma = 1/512, W/gamma = 512 -> clip 1
+    W[3, 7] = -1.0
+    T, g = oracle.quantize_weights(W, 0.0)
+    assert g == np.float32(1.0 / 512.0) and T[3, 7] == -1 and np.abs(T).sum() == 1
+
+
+# ---- second statements of the fronts and of the b-bit variant (exact rational arithmetic, one rounding per step) ----
+
+def test_f32_of_fraction_is_round_to_nearest_even():
+    from fractions import Fraction as F
+    one = F(1)
+    ulp = F(1, 2 ** 23)
+    assert R.f32_of_fraction(one + ulp / 2) == np.float32(1.0)                  # tie -> even (1.0)
+    assert R.f32_of_fraction(one + 3 * ulp / 2) == np.float32(1.0 + 2.0 ** -22)  # tie -> even (upwards)
+    assert R.f32_of_fraction(one + ulp / 2 + F(1, 2 ** 80)) == np.float32(1.0 + 2.0 ** -23)
+    assert R.f32_of_fraction(F(1, 3)) == np.float32(1.0 / 3.0) and R.f32_of_fraction(F(-1, 10)) == np.float32(-0.1)
+    assert R.f32_of_fraction(F(1, 2 ** 149)) == np.float32(2.0 ** -149)          # smallest subnormal
+    assert R.f32_of_fraction(F(1, 2 ** 150)) == 0.0 and R.f32_of_fraction(F(3, 2 ** 150)) == np.float32(2.0 ** -148)
+    assert R.f32_of_fraction(F(2 ** 24 + 1)) == np.float32(2.0 ** 24) and np.isinf(R.f32_of_fraction(F(2) ** 128))
+    rng = np.random.default_rng(5)
+    for a, b in rng.standard_normal((200, 2)).astype(np.float32):               # numpy's IEEE operations agree
+        assert R._mul(a, b) == a * b and R._add(a, b) == a + b and R._div(a, b) == a / b
+        assert R._sqrt(abs(a)) == np.sqrt(np.float32(abs(a)))
+
+
+def _token_mix(rng, M, K):
+    """Tokens of several kinds: Gaussian, Gaussian with outlier channels, tiny and huge scales, a spread of many
+    binades inside the token, subnormal magnitudes, a token of zeros with one value."""
+    h = rng.standard_normal((M, K)).astype(np.float32)
+    kind = np.arange(M) % 6
+    h[kind == 1, : max(1, K // 64)] *= 30.0
+    h[kind == 2] *= np.float32(2.0 ** -60)
+    h[kind == 3] *= np.float32(2.0 ** 50)
+    spread = np.ldexp(np.float32(1.0), rng.integers(-20, 21, size=(M, K)).astype(np.int32)).astype(np.float32)
+    h[kind == 4] *= spread[kind == 4]
+    h[kind == 5] *= np.float32(2.0 ** -120)
+    return _bf16(h)
+
+
+def test_rmsnorm_mean_square_is_the_exactly_rounded_mean_of_exact_squares(oracle):
+    """The C oracle sums integers in which every square is cut off 30 bits below the largest one and divides in
+    double.  The definition is the exact mean of the exact squares, rounded once.  On 1200 tokens of mixed kinds the two
+    are the same fp32 number (they can differ only if the exact mean lies within a relative 2^-27 of a rounding
+    boundary)."""
+    rng = np.random.default_rng(77)
+    checked = 0
+    for K in (16, 48, 320, 1536):
+        hb = _token_mix(rng, 300, K)
+        got = oracle.rmsnorm_mean_square(hb)
+        want = R.rmsnorm_mean_square(hb)
+        assert np.array_equal(got.view(np.uint32), want.view(np.uint32)), f"K={K}: {(got != want).sum()} tokens differ"
+        checked += len(got)
+    assert checked >= 1000
+    # powers of two: mean square of [2^a, 0, 0, 0] is 4^a / 4 exactly, over the whole exponent range of a bfloat16 square
+    for a in (-60, -31, 0, 17, 60):
+        hb = _bf16(np.array([[np.ldexp(1.0, a)] + [0.0] * 3], np.float32))
+        assert float(oracle.rmsnorm_mean_square(hb)[0]) == np.ldexp(1.0, 2 * a - 2)
+
+
+def test_c_oracle_equals_python_restatement_of_the_fronts(oracle):
+    rng = np.random.default_rng(78)
+    # RMSNorm: x, beta, codes and row sums bit for bit
+    M, K = 24, 80
+    hb = _token_mix(rng, M, K)
+    gain = (1.0 + 0.2 * rng.standard_normal(K)).astype(np.float32)
+    for eps_n in (0.0, 1e-5):
+        q, beta, rs, x = oracle.rmsnorm_quantize_acts(hb, gain, eps_n, return_x=True)
+        q2, beta2, rs2, x2 = R.rmsnorm_quantize_acts(hb, gain, eps_n)
+        assert np.array_equal(x.view(np.uint32), x2.view(np.uint32))
+        assert np.array_equal(q, q2) and np.array_equal(beta, beta2) and np.array_equal(rs, rs2)
+    # SwiGLU: gates over the whole range of the exponential, the saturated ends included
+    M, K = 6, 96
+    g = (4.0 * rng.standard_normal((M, K))).astype(np.float32)
+    g[0] = np.linspace(-90.0, 90.0, K)
+    g[1] = np.linspace(-1.0, 1.0, K)
+    gb, ub = _bf16(g), _bf16(rng.standard_normal((M, K)))
+    q, beta, rs, h = oracle.swiglu_quantize_acts(gb, ub, return_h=True)
+    q2, beta2, rs2, h2 = R.swiglu_quantize_acts(gb, ub)
+    assert np.array_equal(h.view(np.uint32), h2.view(np.uint32))
+    assert np.array_equal(q, q2) and np.array_equal(beta, beta2) and np.array_equal(rs, rs2)
+    # activations of fewer bits
+    xb = _bf16(rng.standard_normal((5, 144)) * (1 + 19 * (rng.random(144) < 0.05)))
+    acc = rng.integers(-20000, 20000, (5, 32)).astype(np.int32)
+    for bits in (2, 3, 4, 5, 8):
+        q, beta, rs = oracle.quantize_acts_bits(xb, bits)
+        q2, beta2, rs2 = R.quantize_acts_bits(xb, bits)
+        assert np.array_equal(q, q2) and np.array_equal(beta, beta2) and np.array_equal(rs, rs2)
+        assert np.array_equal(oracle.dequant_bits(acc, beta, 0.0173, bits), R.dequant_bits(acc, beta, 0.0173, bits))
