@@ -294,11 +294,22 @@ bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t
 bitlinear_status bitlinear_validate_packed(const void *packed, int64_t N, int64_t K, int32_t *bad_fields, void *stream);
 
 /*
+ * Measurement aid (no counterpart in the paper; Section 3, "Energy" is why the prefill matmul is rated against the
+ * int8 tensor throughput): what the int8 tensor cores sustain when nothing but MMAs is issued.  One CTA per SM places
+ * one 128 x 128-byte and one 256 x 128-byte operand tile of pseudo-random bytes in shared memory once and issues
+ * iters x 4 tcgen05.mma kind::i8 of 128 x 256 x 32 on them (1 <= iters <= 2^20; about 0.27 us per iteration).  The
+ * caller times the launch; *int_ops (HOST) receives the integer operations it performs, 2 per multiply-add.
+ * *status (DEVICE, one int32, set it to 0 first) receives BITLINEAR_ERR_TIMEOUT if the launch's one bounded wait expires.
+ */
+bitlinear_status bitlinear_probe_int8_peak(int iters, int32_t *status, int64_t *int_ops, void *stream);
+
+/*
  * Test hook for the bounded waits (no counterpart in the paper).  Every device-side wait of the matmul kernels gives
  * up after a limit (2 s), sets the workspace's status word to BITLINEAR_ERR_TIMEOUT and lets the kernel return.  This
  * call arms the NEXT matmul launch of the process (one launch only; the quantiser launch in front of it does not
  * count): its waits give up after limit_us microseconds (0: the default), and, if skip_arrive is non-zero, one
- * producer thread of its first CTA leaves out one barrier arrival, so that a wait really runs out.  The launch then
+ * producer thread of its first CTA leaves out one barrier arrival (and the copy it announces), so that a wait really
+ * runs out.  The launch then
  * ends with BITLINEAR_ERR_TIMEOUT in the status word and unspecified outputs; the workspace is usable again at once.
  * Nothing faults or hangs.  (host)
  */

@@ -43,6 +43,7 @@ EXPORTS = [
     "bitlinear_matmul_i32",
     "bitlinear_unpack_weights",
     "bitlinear_validate_packed",
+    "bitlinear_probe_int8_peak",
     "bitlinear_test_expire_next_wait",
     "bitlinear_poll_status",
 ]
@@ -111,6 +112,7 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_unpack_weights.argtypes = [vp, i64, i64, vp, vp]
     L.bitlinear_poll_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
     L.bitlinear_validate_packed.argtypes = [vp, i64, i64, vp, vp]
+    L.bitlinear_probe_int8_peak.argtypes = [ci, vp, ctypes.POINTER(i64), vp]
     L.bitlinear_test_expire_next_wait.argtypes = [ctypes.c_uint32, ci]
     L.bitlinear_test_expire_next_wait.restype = None
     _lib = L
@@ -306,6 +308,14 @@ def validate_packed(packed: torch.Tensor, N: int, K: int, stream=None) -> int:
     if st not in (OK, ERR_BADCODE):
         _check(st, "bitlinear_validate_packed")
     return int(bad.item())
+
+
+def probe_int8_peak(iters: int, status: torch.Tensor, stream=None) -> int:
+    """bitlinear_probe_int8_peak (measurement aid): enqueues the MMA issue loop; -> integer operations of the launch."""
+    ops = ctypes.c_int64(0)
+    st = load_library().bitlinear_probe_int8_peak(int(iters), _ptr(status), ctypes.byref(ops), _stream(stream))
+    _check(st, "bitlinear_probe_int8_peak")
+    return int(ops.value)
 
 
 def test_expire_next_wait(limit_us: int, skip_arrive: bool):

@@ -428,6 +428,17 @@ bitlinear_status bitlinear_validate_packed(const void *packed, int64_t N, int64_
     return n == 0 ? BITLINEAR_OK : BITLINEAR_ERR_BADCODE;
 }
 
+bitlinear_status bitlinear_probe_int8_peak(int iters, int32_t *status, int64_t *int_ops, void *stream)
+{
+    if (!status || !int_ops || iters < 1 || iters > (1 << 20)) return BITLINEAR_ERR_ARG;
+    if (!aligned(status, 4)) return BITLINEAR_ERR_ALIGN;
+    if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
+    int ctas = 0;
+    if (launch_int8_issue_probe(iters, status, &ctas, (cudaStream_t)stream) != cudaSuccess) return BITLINEAR_ERR_CUDA;
+    *int_ops = (int64_t)ctas * iters * 4 * (2ll * 128 * 256 * 32);
+    return BITLINEAR_OK;
+}
+
 void bitlinear_test_expire_next_wait(uint32_t limit_us, int skip_arrive)
 {
     if (limit_us > 0x7FFFFFFFu) limit_us = 0x7FFFFFFFu;

@@ -486,8 +486,9 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         for (int i = 0; i < kStages; ++i) {
             if (i < n_held) {
                 // (test device: the first warp of the launch leaves out the arrival that announces its first chunk's
-                // activation bytes; the copy itself is issued and lands, the phase never completes)
-                if (!(hooks.skip_arrive && w == 0 && i == 0)) ptx::mbar_arrive_expect_tx(bars + 8 * i, held_bytes[i]);
+                // activation bytes, and the copy it announces with it: the phase never completes)
+                if (hooks.skip_arrive && w == 0 && i == 0) continue;
+                ptx::mbar_arrive_expect_tx(bars + 8 * i, held_bytes[i]);
                 bulk_copy_g2s(ring + i * R::kSlotBytes + R::kWeightBytes, held_x[i], held_bytes[i], bars + 8 * i);
             }
         }
@@ -762,8 +763,10 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
 #pragma unroll
         for (int i = 0; i < kDepth; ++i) {
             if (i < n_held) {
-                // (test device: the first CTA leaves out the arrival that announces its first activation chunk)
-                if (!(hooks.skip_arrive && blockIdx.x == 0 && i == 0)) ptx::mbar_arrive_expect_tx(xfull + 8 * i, held_bytes[i]);
+                // (test device: the first CTA leaves out the arrival that announces its first activation chunk, and
+                // the copy it announces with it)
+                if (hooks.skip_arrive && blockIdx.x == 0 && i == 0) continue;
+                ptx::mbar_arrive_expect_tx(xfull + 8 * i, held_bytes[i]);
                 bulk_copy_g2s(xring + i * R::kXSlotBytes, held_x[i], held_bytes[i], xfull + 8 * i);
             }
         }

@@ -126,14 +126,18 @@ cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int6
 
 // What a matmul launch is told about its bounded device-side waits.  limit_us: how long a wait may last (2 s unless
 // a test shortened it).  skip_arrive != 0 is a test device: ONE producer thread of the launch (in CTA 0) leaves out ONE
-// barrier arrival, so that the wait behind it runs out and the kernel's way out of an expired wait can be checked;
-// everything else, every copy included, is issued as usual.
+// barrier arrival and the copy that arrival announces, so that the wait behind it runs out and the kernel's way out
+// of an expired wait can be checked; everything else is issued as usual.
 struct WaitHooks {
     uint32_t limit_us;
     uint32_t skip_arrive;
 };
 // The hooks for the next matmul launch: the defaults, or what bitlinear_test_expire_next_wait set (used up by this call).
 WaitHooks take_wait_hooks();
+
+// Measurement aid: one CTA per SM issues `iters` x 4 tcgen05.mma kind::i8 (128 x 256 x 32) on operands that stay in
+// shared memory.  *ctas (host) = CTAs launched; *status (device) receives BITLINEAR_ERR_TIMEOUT if the final wait expires.
+cudaError_t launch_int8_issue_probe(int iters, int32_t *status, int *ctas, cudaStream_t stream);
 
 int sm_count();
 

@@ -273,10 +273,10 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                     const uint32_t full = smem_u32(&bars->full[s]);
                     const uint32_t a_dst = stages + s * kStageBytes;
                     const uint32_t p_dst = a_dst + MT * kAHalfBytes;
-                    // (test device: the first CTA leaves out the arrival that announces its first stage's bytes; the
-                    // loads are issued and land, the phase never completes)
-                    if (!(hooks.skip_arrive && blockIdx.x == 0 && pos.it == 0))
-                        mbar_arrive_expect_tx(full, halves * kAHalfBytes + kPBytes);
+                    // (test device: the first CTA leaves out the arrival that announces its first stage's bytes, and
+                    // the loads it announces with it, so that nothing is in flight for a phase that never completes)
+                    if (hooks.skip_arrive && blockIdx.x == 0 && pos.it == 0) continue;
+                    mbar_arrive_expect_tx(full, halves * kAHalfBytes + kPBytes);
                     tma_load_2d(a_dst, &g.tmap_x, kb * BK, m0, full);       // x = byte column (multiple of 128)
                     if (halves == 2) tma_load_2d(a_dst + kAHalfBytes, &g.tmap_x, kb * BK, m0 + BM, full);
                     tma_load_3d(p_dst, &g.tmap_w, 0, kb * (BK / kTileCols), n0 / kTileRows, full); // x = 0: whole tiles
@@ -588,15 +588,18 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         }
     }
 
-    // common tail: every thread arrives here, also after an expired wait
-    if (*abort_flag) {
+    // common tail: every thread arrives here, also after an expired wait.  The flag is looked at AFTER the barrier:
+    // a thread whose role ended early (the producer of a short matmul, the idle lanes of the one-thread roles) gets
+    // here long before a wait of another role can expire.
+    tc_fence_before_sync();
+    __syncthreads();
+    if (*abort_flag) { // (the same for every thread now)
         if (threadIdx.x == 0) atomicExch(status, (int32_t)BITLINEAR_ERR_TIMEOUT);
         // give copies and MMAs that may still be in flight time to land before shared memory and TMEM go away
         const uint64_t t0 = globaltimer_ns();
         while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+        __syncthreads();
     }
-    tc_fence_before_sync();
-    __syncthreads();
     if (warp == kMmaWarp) {
         tc_fence_after_sync();
         tmem_dealloc(tmem_base, kTmemCols);

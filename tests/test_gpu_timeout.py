@@ -4,7 +4,7 @@ Every wait of the matmul kernels is bounded: when its limit passes, the waiting 
 every role leaves its loop, the kernel writes BITLINEAR_ERR_TIMEOUT into the workspace's status word, gives copies in
 flight time to land, releases tensor memory and RETURNS.  The test hook bitlinear_test_expire_next_wait shortens the
 limit of the next matmul launch to two milliseconds and makes one producer thread of its first CTA leave out one
-barrier arrival (every copy is still issued and lands), on a problem of one CTA.  Checked: the call returns, the
+barrier arrival together with the copy it announces (nothing is left in flight), on a problem of one CTA.  Checked: the call returns, the
 status word says timeout, and the SAME workspace gives the oracle's bits on the next, ordinary call.
 """
 import numpy as np
