@@ -560,6 +560,17 @@ int oracle_forward(const int8_t *T, float gamma, const uint16_t *X_bf16,
     return oracle_dequant(acc, beta, gamma, M, N, Y_bf16);
 }
 
+/* Timing aid (no arithmetic): how many threads the outer loops of the timing build use from now on. */
+void oracle_set_num_threads(int n)
+{
+#ifdef _OPENMP
+    extern void omp_set_num_threads(int);
+    if (n >= 1) omp_set_num_threads(n);
+#else
+    (void)n;
+#endif
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP

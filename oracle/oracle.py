@@ -65,6 +65,8 @@ class Oracle:
         L.oracle_dequant.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p]
         L.oracle_forward.argtypes = [_p, ctypes.c_float, _p, _i64, _i64, _i64, _p, _p, _p, _p, _p]
         L.oracle_num_threads.restype = ctypes.c_int
+        L.oracle_set_num_threads.argtypes = [ctypes.c_int]
+        L.oracle_set_num_threads.restype = None
 
     @staticmethod
     def _c(a: np.ndarray, dtype) -> np.ndarray:
@@ -81,6 +83,10 @@ class Oracle:
 
     def num_threads(self) -> int:
         return int(self.lib.oracle_num_threads())
+
+    def set_num_threads(self, n: int) -> None:
+        """Timing build only: threads used by the outer loops from now on (no effect on results)."""
+        self.lib.oracle_set_num_threads(int(n))
 
     def absmean(self, W: np.ndarray) -> np.float32:
         W = self._c(W, np.float32)

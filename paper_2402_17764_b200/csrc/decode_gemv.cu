@@ -183,17 +183,18 @@ __device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete
 
 // Finishing launch: dequantises the row blocks on one list from the scratch and leaves the scratch clean for
 // the next launch.  owned[i] = (entry index, row block).  Up to four row blocks are
-// handled at a time with all loads of one kind issued together, so that the pass costs two memory round
-// trips rather than two per row block.
+// handled at a time, and up to four tokens of each, with all loads of one kind issued together, so that the pass
+// costs two memory round trips per batch and token group rather than two per row block and token.
 // `word` is the lane's 32-bit word of the warp's 128-byte list (one load for the count and all items: every round
 // trip of this launch is on the critical path of the step): word 0 the count, words 2 i + 2 and 2 i + 3 item i.
+template <int TG> // tokens handled together: 1 (single-token steps), or 4
 __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint32_t word, int n_owned, int lane)
 {
     constexpr int kBatch = 4;
     for (int b0 = 0; b0 < n_owned; b0 += kBatch) {
         const DecodeEntry *e[kBatch];
         int32_t *acc[kBatch];
-        int r0[kBatch], N[kBatch];
+        int r0[kBatch], N[kBatch], M[kBatch], max_M = 0;
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             const int item = min(b0 + b, n_owned - 1); // slots past the end repeat the last one and store nothing
@@ -205,55 +206,37 @@ __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint
         for (int b = 0; b < kBatch; ++b) {
             acc[b] = e[b]->acc32;
             N[b] = (b0 + b < n_owned) ? e[b]->N : 0;
+            M[b] = e[b]->M;
+            if (N[b] > 0) max_M = max(max_M, M[b]);
         }
-        // token 0 of every row block of the batch
-        int v[kBatch][kTileRows / 32], rowsum[kBatch];
-        float scale[kBatch];
+        // TG tokens of every row block of the batch at a time: all loads first, then all stores
+        for (int t0 = 0; t0 < max_M; t0 += TG) {
+            int v[kBatch][TG][kTileRows / 32], rowsum[kBatch][TG];
+            float scale[kBatch][TG];
 #pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
+            for (int b = 0; b < kBatch; ++b) {
 #pragma unroll
-            for (int h = 0; h < kTileRows / 32; ++h) v[b][h] = (r0[b] + 32 * h < N[b]) ? __ldcg(acc[b] + r0[b] + 32 * h) : 0;
-            rowsum[b] = e[b]->rowsum[0];
-            scale[b] = token_scale(*e[b], 0);
-        }
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-#pragma unroll
-            for (int h = 0; h < kTileRows / 32; ++h) {
-                const int r = r0[b] + 32 * h;
-                if (r < N[b]) {
-                    __stcg(acc[b] + r, 0);
-                    store_result(*e[b], 0, r, v[b][h], rowsum[b], scale[b]);
-                }
-            }
-        }
-        // further tokens, eight at a time with their loads issued together
-#pragma unroll
-        for (int b = 0; b < kBatch; ++b) {
-            if (N[b] == 0) continue;
-            const int M = e[b]->M;
-            for (int t0 = 1; t0 < M; t0 += 8) {
-                int tv[8][kTileRows / 32], rs[8];
-                float sc[8];
-#pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const int t = min(t0 + i, M - 1); // slots past the last token repeat it and store nothing
+                for (int i = 0; i < TG; ++i) {
+                    const int t = min(t0 + i, M[b] - 1); // slots past the last token repeat it and store nothing
 #pragma unroll
                     for (int h = 0; h < kTileRows / 32; ++h)
-                        tv[i][h] = (r0[b] + 32 * h < N[b]) ? __ldcg(acc[b] + (size_t)t * N[b] + r0[b] + 32 * h) : 0;
-                    rs[i] = e[b]->rowsum[t];
-                    sc[i] = token_scale(*e[b], t);
+                        v[b][i][h] = (r0[b] + 32 * h < N[b]) ? __ldcg(acc[b] + (size_t)t * N[b] + r0[b] + 32 * h) : 0;
+                    rowsum[b][i] = e[b]->rowsum[t];
+                    scale[b][i] = token_scale(*e[b], t);
                 }
+            }
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
+            for (int b = 0; b < kBatch; ++b) {
+#pragma unroll
+                for (int i = 0; i < TG; ++i) {
                     const int t = t0 + i;
-                    if (t >= M) break;
+                    if (t >= M[b]) continue;
 #pragma unroll
                     for (int h = 0; h < kTileRows / 32; ++h) {
                         const int r = r0[b] + 32 * h;
                         if (r < N[b]) {
                             __stcg(acc[b] + (size_t)t * N[b] + r, 0);
-                            store_result(*e[b], t, r, tv[i][h], rs[i], sc[i]);
+                            store_result(*e[b], t, r, v[b][i][h], rowsum[b][i], scale[b][i]);
                         }
                     }
                 }
@@ -850,7 +833,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
 __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constant__ InlineTable inl,
                                                             const DecodeEntry *__restrict__ table,
                                                             const OwnedList *__restrict__ lists, uint32_t n_lists,
-                                                            int staged_entries)
+                                                            int staged_entries, int single_token)
 {
     extern __shared__ uint4 staged_table[];
     const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -870,7 +853,10 @@ __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constan
     const uint32_t word = __ldcg(reinterpret_cast<const uint32_t *>(&lists[w]) + lane);
     const int n = (int)__shfl_sync(0xffffffffu, word, 0);
     if (n == 0) return;
-    finish_owned_blocks(table ? table : inl.e, word, n, lane);
+    if (single_token)
+        finish_owned_blocks<1>(table ? table : inl.e, word, n, lane);
+    else
+        finish_owned_blocks<4>(table ? table : inl.e, word, n, lane);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -965,10 +951,11 @@ static cudaError_t launch_dependent(const void *kernel, dim3 grid, dim3 block, s
 
 template <int NT>
 static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, const DecodeEntry *table, int n_entries,
-                              uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr,
+                              uint32_t total_tiles, uint32_t share, uint32_t dyn, int max_M, WorkspaceHeader *hdr,
                               OwnedList *lists, cudaStream_t stream)
 {
     WaitHooks hooks = take_wait_hooks();
+    int single_token = max_M == 1 ? 1 : 0;
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -985,7 +972,7 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
     uint32_t n_lists = grid.x * kWarps;
     // a table that fits beside the matmul's ring (one CTA of each per SM) is staged in the finishing CTAs' shared memory
     int staged = (table && (size_t)n_entries * sizeof(DecodeEntry) <= kStagedTableBytes) ? n_entries : 0;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged};
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token};
     return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256),
                             (size_t)staged * sizeof(DecodeEntry), fargs, early, stream);
 }
@@ -1011,7 +998,8 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
     int staged = 0; // (this kernel's rings leave no room beside them)
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged};
+    int single_token = 0;
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token};
     return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
 }
 
@@ -1061,7 +1049,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     } else {
         share = (total_tiles + n_warps - 1) / n_warps; // all static: the last warps may get less, or nothing
     }
-    return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, share, dyn, hdr, lists, stream);
+    return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
 }
 
 } // namespace bitlinear
