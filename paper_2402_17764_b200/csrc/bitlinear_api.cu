@@ -86,15 +86,15 @@ inline int64_t col_tiles(int64_t K) { return (K + kTileCols - 1) / kTileCols; }
 inline int64_t gemm_k_blocks(int64_t K) { return (K + 127) / 128; }
 
 // Workspace of one matmul: [header | int32 scratch | per-warp lists | Xq | beta | rowsum].  The scratch serves the
-// weight-streaming kernel (sums of row blocks shared by several warps, at most 64 tokens) or the GEMM (tiles cut
-// along K), whichever is larger, so that the layout does not depend on the kernel chosen.
+// weight-streaming kernel (sums of row blocks shared by several warps, at most 64 tokens) or the GEMM (flags and a slot
+// of partial sums per CTA when it deals k-block shares), whichever is larger, so that the layout does not depend on the kernel chosen.
 Layout single_layout(int64_t M, int64_t N, int64_t K)
 {
     Layout L{};
     size_t off = sizeof(WorkspaceHeader);
     L.acc32 = off;
     const size_t decode_scratch = (size_t)(M < kMaxDecodeM ? M : kMaxDecodeM) * N * 4;
-    const size_t gemm_scratch = M > 0 ? prefill_split_bytes(prefill_tile_count(M, N, M), M) : 0;
+    const size_t gemm_scratch = M > 0 ? prefill_scratch_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M), M) : 0;
     off += align_up(decode_scratch > gemm_scratch ? decode_scratch : gemm_scratch, 256);
     L.table = off; // end of what is cleared before every call
     L.lists = off;
@@ -164,7 +164,7 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
 
 // Runs the matmul + epilogue of one entry whose activations are already quantised.
 // x_rows: rows of int8 activations that exist behind e.Xq (>= e.M; the rows past e.M may hold anything).
-// split_scratch: zeroed scratch for GEMM tiles cut along K, or null (then none are cut).
+// split_scratch: the GEMM's scratch with its flags zeroed, or null (then it deals whole tiles only).
 bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, int64_t x_rows, void *split_scratch,
                             cudaStream_t stream)
 {
@@ -355,7 +355,7 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     inl.e[0].up = reinterpret_cast<const __nv_bfloat16 *>(up);
     inl.e[0].qb = (float)((1 << (act_bits - 1)) - 1);
     // quantise the tokens; the same launch clears the header and the scratch of the kernel that follows, if it uses it
-    const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
+    const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M)) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (gain ? 1 : 0) | (up ? 2 : 0), (int)K,
@@ -386,7 +386,7 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
     InlineTable inl{};
     fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
-    const size_t clear = tc ? prefill_split_clear_bytes(prefill_tile_count(M, N, M), gemm_k_blocks(K), M) : 0;
+    const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M)) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, false, (int)K, s);
@@ -502,16 +502,17 @@ struct bitlinear_sequence {
     const bitlinear::DecodeEntry *dev_table; // inside the workspace, or null when the table is inline
     bitlinear::InlineTable inl;
     const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
-    int gemm_tiles, gemm_min_kb;
+    int gemm_tiles;
+    int64_t gemm_total_kb;
     int fronts;             // bit 0: some entry has an RMSNorm in front of the quantiser, bit 1: some entry a SwiGLU
-    void *split_scratch;    // inside the workspace; null: no GEMM tile of this sequence is cut along K
+    void *split_scratch;    // inside the workspace; null: the GEMM deals this sequence's tiles whole
 };
 
 namespace {
 struct SeqLayout {
     size_t acc32, table, lists, gemm, data, total;
     bool use_gemm;
-    int min_kb; // fewest k blocks of 128 columns among the matmuls
+    int64_t gemm_tiles, gemm_total_kb; // CTA tiles and k blocks (tiles x k blocks each) of all matmuls on the GEMM
 };
 
 inline size_t seq_xq_bytes(int64_t M, int64_t K, bool gemm)
@@ -525,7 +526,6 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
     if (!layers || n <= 0 || n > 65536) return false;
     size_t acc = 0, data = 0;
     uint64_t tiles = 0, gemm_tiles = 0, tokens = 0;
-    int64_t min_kb = INT32_MAX;
     int64_t max_M = 0;
     for (int i = 0; i < n; ++i)
         if (layers[i].M > max_M) max_M = layers[i].M;
@@ -538,19 +538,20 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
         if (!gemm) acc += align_up((size_t)d.M * d.N * 4, 256);
         tiles += (uint64_t)(row_blocks(d.N) * col_tiles(d.K)); // an upper bound of the work items in either mode
         gemm_tiles += (uint64_t)((d.M + 127) / 128) * (uint64_t)((d.N + 255) / 256); // the same for the GEMM's CTA tiles
-        if (gemm_k_blocks(d.K) < min_kb) min_kb = gemm_k_blocks(d.K);
         if (entry_off) entry_off->push_back(data);
         data += seq_xq_bytes(d.M, d.K, gemm) + 2 * align_up((size_t)d.M * 4, 256);
     }
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
     if (tokens > 0x3FFFFFFFull) return false; // tokens (plus the clearing CTAs) index the quantiser's grid with an int
     if (gemm && gemm_tiles > 0x7FFFFFFFull) return false;
-    if (gemm) { // scratch for tiles cut along K, where the streaming kernel has its int32 scratch
-        uint64_t exact = 0;
-        for (int i = 0; i < n; ++i) exact += (uint64_t)prefill_tile_count(layers[i].M, layers[i].N, max_M);
-        acc = align_up(prefill_split_bytes((int64_t)exact, max_M), 256);
+    S.gemm_tiles = S.gemm_total_kb = 0;
+    if (gemm) { // the GEMM's scratch, where the streaming kernel has its int32 scratch
+        for (int i = 0; i < n; ++i) {
+            S.gemm_tiles += prefill_tile_count(layers[i].M, layers[i].N, max_M);
+            S.gemm_total_kb += prefill_kb_count(layers[i].M, layers[i].N, layers[i].K, max_M);
+        }
+        acc = align_up(prefill_scratch_bytes(S.gemm_tiles, S.gemm_total_kb, max_M), 256);
     }
-    S.min_kb = (int)min_kb;
     size_t off = sizeof(WorkspaceHeader);
     S.acc32 = off;
     off += acc;
@@ -640,6 +641,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     const bool gemm = S.use_gemm;
     std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
     int gemm_tiles = 0;
+    int64_t gemm_kb = 0;
     int fronts = 0;
     for (int i = 0; i < n; ++i) {
         const bitlinear_layer_desc &d = layers[i];
@@ -664,9 +666,10 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
             int nt = 0;
             if (prefill_table_entry(gemm_table.data() + (size_t)i * kGemmProblemBytes, e.packed, e.gamma, e.Xq, e.beta,
                                     e.rowsum, d.M, d.M < kMinGemmRows ? kMinGemmRows : d.M, d.K, d.N, d.Y, e.qb, max_M,
-                                    gemm_tiles, reinterpret_cast<WorkspaceHeader *>(ws), &nt) != cudaSuccess)
+                                    gemm_tiles, gemm_kb, reinterpret_cast<WorkspaceHeader *>(ws), &nt) != cudaSuccess)
                 return BITLINEAR_ERR_CUDA;
             gemm_tiles += nt;
+            gemm_kb += (int64_t)nt * gemm_k_blocks(d.K);
         }
     }
     bitlinear_sequence *seq = new (std::nothrow) bitlinear_sequence();
@@ -680,13 +683,13 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     seq->max_K = 0;
     for (int i = 0; i < n; ++i)
         if ((int)layers[i].K > seq->max_K) seq->max_K = (int)layers[i].K;
-    const size_t clear = gemm ? prefill_split_clear_bytes(gemm_tiles, S.min_kb, max_M) : 0;
+    const size_t clear = gemm ? prefill_scratch_clear_bytes(gemm_tiles, gemm_kb) : 0;
     const bool split = clear > 0;
     seq->zero_bytes = gemm ? S.acc32 + align_up(clear, 256) : S.table; // header and the int32 scratch in use
     seq->dev_table = nullptr;
     seq->gemm_table = nullptr;
     seq->gemm_tiles = gemm_tiles;
-    seq->gemm_min_kb = S.min_kb;
+    seq->gemm_total_kb = gemm_kb;
     seq->fronts = fronts;
     seq->split_scratch = split ? ws + S.acc32 : nullptr;
     if (gemm) {
@@ -722,7 +725,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {
         const cudaError_t err =
-            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->max_M, seq->gemm_min_kb,
+            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->gemm_total_kb, seq->max_M,
                                                  seq->split_scratch, s)
                             : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
                                             reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s);

@@ -108,12 +108,7 @@ __device__ __forceinline__ int dp4a_u8s8(uint32_t a, uint32_t b, int c)
     return d;
 }
 
-__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
-{
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
+using ptx::bulk_copy_g2s;
 
 __device__ __forceinline__ uint4 lds128(uint32_t addr)
 {

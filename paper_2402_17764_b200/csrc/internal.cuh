@@ -99,30 +99,34 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
 
 // Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) (by gamma * beta_t / qb) or raw int32.  x_rows >= M rows of K bytes exist behind
 // Xq; the rows past M may hold anything (they only reach accumulator rows that are never stored).
+// scratch: prefill_scratch_bytes(...) bytes (256-byte aligned) whose first prefill_scratch_clear_bytes(...) bytes are
+// ZERO when the launch starts, or null (then the launch deals whole tiles only).
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, float qb, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream);
+                           int out_i32, float qb, WorkspaceHeader *hdr, void *scratch, cudaStream_t stream);
 
-// Cutting tiles along K.  When the CTA tiles of a launch leave most SMs idle in their last round, the kernel cuts
-// the tiles of that round along K and adds the partial sums up in `split_scratch` (prefill_split_bytes(tiles, max_M)
-// bytes, 256-byte aligned; null: never cut).  prefill_split_clear_bytes tells how many bytes at the start of the
-// scratch must be ZERO when a launch over n_tiles CTA tiles, whose matmuls have at least min_KB k blocks of 128
-// columns, starts: 0 if that launch cuts no tile (the scratch is not touched then).
+// Dealing k-block shares.  When the CTA tiles of a launch would leave a good part of the SMs idle in their last round,
+// the kernel gives every CTA an equal share of the k blocks of all tiles instead; shares begin and end inside tiles, and
+// partial sums travel through a scratch slot per CTA.  prefill_scratch_bytes: bytes of scratch a launch over n_tiles CTA
+// tiles with total_kb k blocks of 128 columns in all needs (0: it deals whole tiles); prefill_scratch_clear_bytes: how
+// many bytes at the start of that scratch must be zero when the launch starts.
 int64_t prefill_tile_count(int64_t M, int64_t N, int64_t max_M);
-size_t prefill_split_bytes(int64_t n_tiles, int64_t max_M);
-size_t prefill_split_clear_bytes(int64_t n_tiles, int64_t min_KB, int64_t max_M);
+int64_t prefill_kb_count(int64_t M, int64_t N, int64_t K, int64_t max_M); // tiles x k blocks of one matmul
+size_t prefill_scratch_bytes(int64_t n_tiles, int64_t total_kb, int64_t max_M);
+size_t prefill_scratch_clear_bytes(int64_t n_tiles, int64_t total_kb);
 
 // The same kernel over the matmuls of a sequence in ONE launch.  The host fills a table of kGemmProblemBytes-sized
 // entries (tensor maps + parameters) with prefill_table_entry, copies it to device memory (64-byte aligned) once, and
 // launches over all the CTA tiles; max_M = the largest M of the sequence, the same for every entry and the launch
-// (it fixes the tile shape: prefill_token_tiles(max_M) token tiles of 128 tokens per CTA tile).
+// (it fixes the tile shape: prefill_token_tiles(max_M) token tiles of 128 tokens per CTA tile).  tile_begin, kb_begin:
+// the CTA tiles and the k blocks (tiles x k blocks each) of the entries in front of this one.
 constexpr size_t kGemmProblemBytes = 384;
 int prefill_token_tiles(int64_t max_M);
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                float qb, int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles);
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, int min_KB,
-                                 void *split_scratch, cudaStream_t stream);
+                                float qb, int64_t max_M, int tile_begin, int64_t kb_begin, WorkspaceHeader *hdr, int *n_tiles);
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t total_kb, int64_t max_M, void *scratch,
+                                 cudaStream_t stream);
 
 // What a matmul launch is told about its bounded device-side waits.  limit_us: how long a wait may last (2 s unless
 // a test shortened it).  skip_arrive != 0 is a test device: ONE producer thread of the launch (in CTA 0) leaves out ONE

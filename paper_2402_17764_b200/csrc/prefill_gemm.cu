@@ -21,7 +21,10 @@
 // this kernel), then feeds two MMAs per k step, and the two accumulators fill the tensor memory, so the
 // epilogue of a tile no longer overlaps the next tile's MMAs.
 // One launch runs one matmul (passed as a kernel parameter) or all the matmuls of a sequence (a table in device
-// memory): the CTAs walk one launch-wide sequence of CTA tiles.
+// memory): the CTAs walk one launch-wide sequence of CTA tiles.  When whole tiles would leave many SMs idle in the
+// last round (160 tiles on 148 SMs), the launch instead gives every CTA an equal, contiguous share of the sequence of
+// K BLOCKS of all tiles: a CTA's share then begins and ends inside tiles, the tile it begins in is finished by the CTA
+// in front of it, and partial sums travel through a scratch slot per CTA (see Schedule below).
 // The kernel is a programmatic dependent of the activation quantiser: set-up (barriers, tensor memory,
 // descriptor prefetch) runs while the quantiser finishes; the producer waits for it before the first load.
 // All waits are bounded; on expiry the CTA sets the workspace status to BITLINEAR_ERR_TIMEOUT,
@@ -49,6 +52,7 @@ constexpr int BK = 128;      // int8 elements (= bytes) of K per stage
 constexpr int kMaxStages = 12; // ring of TMA stages (activations + packed weights); its depth is chosen at launch
 constexpr int kMaxBSlots = 3;  // ring of expanded weight tiles (its depth: Cfg)
 constexpr int kTmemCols = 512;
+constexpr int kFetchBufs = 6;  // see Schedule below
 
 constexpr int kProducerWarp = 0;
 constexpr int kMmaWarp = 1;
@@ -98,53 +102,51 @@ struct Barriers {
     uint64_t expanded[kMaxBSlots]; // int8 weight tile written
     uint64_t acc_full[2];        // accumulator(s) of a tile complete
     uint64_t acc_empty[2];       // drained by the epilogue
-    uint64_t epilogue_met;       // rendezvous of the four epilogue warps (tiles cut along K)
+    uint64_t epilogue_met;       // rendezvous of the four epilogue warps (after a contribution)
+    uint64_t fetched[4][kFetchBufs]; // finisher: a piece of a contribution has landed in an epilogue warp's buffer
     uint32_t tmem_base;
     int abort_flag;
-    int split_last; // this CTA added the last partial sums of a cut tile
 };
 static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block");
 
-// Work units of a launch.  Units 0 .. full-1 are whole CTA tiles.  When the tiles do not fill the last round of
-// the SMs (fewer than half of them busy), the tiles of that round are cut along K into `slices` units each, so
-// that all SMs work on them: every unit adds its partial sums into an int32 scratch tile (bulk reduce from shared
-// memory, which is idle by then: a cut unit is the last unit of its CTA), and the CTA that adds last (a counter
-// per tile) dequantises the tile from the scratch.  Scratch and counters must be zero at the start of the launch.
-struct SplitPlan {
-    int n_units, full, slices;
-    int32_t *scratch;   // per cut tile: [token tile][lane quarter][chunk of 32 features][lane][32 sums], see split_piece
-    uint32_t *counters; // per cut tile
+// How the work of a launch is dealt to its CTAs.
+//   whole tiles : CTA b takes CTA tiles b, b + grid, b + 2 grid, ...
+//   k-block shares (stream_k): the k blocks of all tiles form one sequence of total_kb items, and CTA b takes the
+//     contiguous range [b * total_kb / grid, (b + 1) * total_kb / grid), which it cuts at tile borders into units.  A
+//     unit that covers its whole tile is an ordinary tile.  A unit that begins inside its tile (it can only be the
+//     CTA's first) is a CONTRIBUTION: the CTA writes its int32 partial sums to its own scratch slot with plain stores
+//     and then sets its flag.  A unit that begins with the tile but ends inside it (it can only be the CTA's last) makes
+//     the CTA the tile's FINISHER: the rest of the tile belongs to the first units of the CTAs behind it (b + 1 .. the
+//     CTA that holds the tile's last k block), which were those CTAs' first work and are long done; the finisher waits
+//     for their flags (a bounded wait), adds their slots to its own sums and dequantises.  No CTA ever waits for work
+//     that itself waits, flags must be zero when the launch starts, slots need no clearing.
+struct Schedule {
+    int stream_k;
+    int n_tiles;
+    long long total_kb;
+    uint32_t *flags; // one word per CTA
+    int32_t *slots;  // per CTA: [token tile][lane quarter][chunk of 32 features][lane][32 sums]
 };
-constexpr uint32_t kSplitTileBytes = BM * BN * 4; // scratch per token tile of a cut CTA tile
-constexpr int kMaxSplitTiles = 80;                // tiles that can be cut in one launch (half the SMs of the largest part)
-constexpr int kMinSplitKB = 64;                   // k blocks a tile must have for a cut to pay (measured)
-constexpr size_t kSplitCounterBytes = 512;        // counters in front of the scratch tiles
-
-struct Unit {
-    int tile, slice;
-    bool split;
-    __device__ Unit(const SplitPlan &sp, int u)
-    {
-        if (u < sp.full) {
-            tile = u;
-            slice = 0;
-            split = false;
-        } else {
-            const int v = u - sp.full;
-            tile = sp.full + v / sp.slices;
-            slice = v - (v / sp.slices) * sp.slices;
-            split = true;
-        }
-    }
-    // k blocks [kb0, kb1) of the KB of the tile's matmul (slices <= KB: never empty)
-    __device__ int kb0(const SplitPlan &sp, int KB) const { return split ? (int)((long long)slice * KB / sp.slices) : 0; }
-    __device__ int kb1(const SplitPlan &sp, int KB) const { return split ? (int)((long long)(slice + 1) * KB / sp.slices) : KB; }
-};
+constexpr uint32_t kSlotTileBytes = BM * BN * 4; // partial sums of one token tile of a CTA tile
+constexpr size_t kFlagBytes = 1024;              // flags in front of the slots (one word per CTA)
+// The finisher fetches contributions with bulk copies into shared memory (its rings are idle by then: a finisher unit
+// is its CTA's last), kFetchBufs pieces of kFetchBytes in flight per epilogue warp: reading them with plain loads would
+// be one round trip to L2 after the other (measured: 1.2 us each, 16 per contribution).
+constexpr uint32_t kFetchChunks = 2;                    // chunks of 32 features per piece
+constexpr uint32_t kFetchBytes = kFetchChunks * 4096;   // 8 KiB
+static_assert(4 * kFetchBufs * kFetchBytes <= 3 * 64 * 1024, "the fetch buffers lie inside the idle rings");
 
 // Byte offset of 16-byte piece `piece` (of 8) of lane `lane` inside a chunk of 32 lanes x 128 bytes: pieces are
-// swizzled by lane so that the 16-byte shared-memory stores of a warp are free of bank conflicts.  The scratch in
-// global memory has the same layout (it is added to with one bulk reduce per 32 KiB).
-__device__ __forceinline__ uint32_t split_piece(int lane, int piece) { return (uint32_t)(lane * 128 + ((piece ^ (lane & 7)) << 4)); }
+// swizzled by lane so that 16-byte shared-memory loads of a warp are free of bank conflicts.  The slots in global memory
+// have this layout (they reach shared memory by bulk copies, as they are).
+__device__ __forceinline__ uint32_t slot_piece(int lane, int piece) { return (uint32_t)(lane * 128 + ((piece ^ (lane & 7)) << 4)); }
+
+enum UnitKind { kWholeTile = 0, kContribution = 1, kFinisher = 2 };
+
+struct Unit {
+    int tile, kb0, kb1, kind;
+    int last_contributor; // finisher: the contributions are the first units of CTAs blockIdx.x + 1 .. last_contributor
+};
 
 // Position in the ring of TMA stages and in the ring of expanded tiles after `it` k blocks.
 struct RingPos {
@@ -172,6 +174,7 @@ struct Params {
     int out_i32;
     int out_32b_aligned; // rows of the bf16 output start on 32-byte boundaries
     int tile_begin;      // first CTA tile of this matmul in the launch-wide tile sequence
+    long long kb_begin;  // first k block of this matmul in the launch-wide sequence of k blocks (all tiles)
     float qb;            // largest activation code (127, or less for activations of fewer bits)
     int32_t *status;
 };
@@ -184,7 +187,8 @@ struct alignas(64) GemmProblem {
 };
 static_assert(sizeof(GemmProblem) == kGemmProblemBytes, "internal.cuh states the size of a table entry");
 
-// The matmul a tile belongs to.  A CTA's tiles only go up, so the search resumes where it stopped.
+// The matmul a tile, or a k block of the launch-wide sequence, belongs to.  A CTA's work only goes up, so the search
+// resumes where it stopped.
 template <bool kTable>
 struct ProblemCursor {
     const GemmProblem *table;
@@ -197,12 +201,72 @@ struct ProblemCursor {
         }
         return table[i];
     }
+    __device__ const GemmProblem &seek_kb(long long pos)
+    {
+        if (kTable) {
+            while (i + 1 < n && pos >= table[i + 1].p.kb_begin) ++i;
+        }
+        return table[i];
+    }
+};
+
+// Steps through the units of this CTA.  Every role of the CTA runs its own walker; all of them see the same units.
+template <bool kTable>
+struct UnitWalker {
+    const Schedule &sc;
+    ProblemCursor<kTable> cur;
+    int next_tile;        // whole tiles
+    long long pos, end;   // k-block shares
+    __device__ UnitWalker(const Schedule &sc_, const GemmProblem &one, const GemmProblem *t, int n)
+        : sc(sc_), cur(one, t, n), next_tile((int)blockIdx.x), pos(0), end(0)
+    {
+        if (sc.stream_k) {
+            pos = (long long)blockIdx.x * sc.total_kb / (long long)gridDim.x;
+            end = (long long)(blockIdx.x + 1) * sc.total_kb / (long long)gridDim.x;
+        }
+    }
+    // the next unit and its matmul; false: none is left
+    __device__ bool next(Unit &u, const GemmProblem *&g)
+    {
+        if (!sc.stream_k) {
+            if (next_tile >= sc.n_tiles) return false;
+            g = &cur.seek(next_tile);
+            u.tile = next_tile;
+            u.kb0 = 0;
+            u.kb1 = g->p.KB;
+            u.kind = kWholeTile;
+            u.last_contributor = 0;
+            next_tile += (int)gridDim.x;
+            return true;
+        }
+        if (pos >= end) return false;
+        g = &cur.seek_kb(pos);
+        const int KB = g->p.KB;
+        const long long local = pos - g->p.kb_begin;
+        const int tile_local = (int)(local / KB);
+        u.tile = g->p.tile_begin + tile_local;
+        u.kb0 = (int)(local - (long long)tile_local * KB);
+        const long long tile_start = pos - u.kb0, tile_end = tile_start + KB;
+        u.kb1 = (int)((end < tile_end ? end : tile_end) - tile_start);
+        u.last_contributor = 0;
+        if (u.kb0 > 0) {
+            u.kind = kContribution;
+        } else if (u.kb1 < KB) {
+            u.kind = kFinisher;
+            // the CTA whose range holds the tile's last k block: the largest c with c * total_kb / grid <= tile_end - 1
+            u.last_contributor = (int)((tile_end * (long long)gridDim.x - 1) / sc.total_kb);
+        } else {
+            u.kind = kWholeTile;
+        }
+        pos = tile_start + u.kb1;
+        return true;
+    }
 };
 
 template <int MT, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems,
-                    const SplitPlan sp, int a_rows, int n_stages, const WaitHooks hooks)
+                    const Schedule sc, int a_rows, int n_stages, const WaitHooks hooks)
 {
     constexpr int kAccBufs = Cfg<MT>::kAccBufs, kBSlots = Cfg<MT>::kBSlots, kGroups = Cfg<MT>::kGroups;
     const uint32_t kStageBytes = stage_bytes(MT, a_rows), kAHalfBytes = (uint32_t)(a_rows * BK);
@@ -230,6 +294,8 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             mbar_init(smem_u32(&bars->acc_empty[b]), 4);
         }
         mbar_init(smem_u32(&bars->epilogue_met), 4);
+        for (int w = 0; w < 4; ++w)
+            for (int b = 0; b < kFetchBufs; ++b) mbar_init(smem_u32(&bars->fetched[w][b]), 1);
         bars->abort_flag = 0;
         fence_mbar_init();
     }
@@ -246,7 +312,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
 
     if (warp == kProducerWarp) {
         if (lane == 0) {
-            ProblemCursor<kTable> cur(one, table, n_problems);
+            UnitWalker<kTable> walk(sc, one, table, n_problems);
             if (!kTable) {
                 prefetch_tensormap(&one.tmap_x);
                 prefetch_tensormap(&one.tmap_w);
@@ -254,17 +320,16 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             griddep_wait(); // the activations are written by the launch before this one
             RingPos pos;
             bool ok = true;
-            for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x) {
-                const Unit unit(sp, u);
-                const int tile = unit.tile;
-                const GemmProblem &g = cur.seek(tile);
+            Unit unit;
+            const GemmProblem *gp;
+            while (ok && walk.next(unit, gp)) {
+                const GemmProblem &g = *gp;
                 const Params &p = g.p;
-                const int local = tile - p.tile_begin;
-                const int kb_begin = unit.kb0(sp, p.KB), kb_end = unit.kb1(sp, p.KB);
+                const int local = unit.tile - p.tile_begin;
                 const int m0 = (local % p.tiles_m) * (MT * BM);
                 const int n0 = (local / p.tiles_m) * BN;
                 const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1; // a second token tile past the end is left out
-                for (int kb = kb_begin; kb < kb_end; ++kb, pos.advance(n_stages)) {
+                for (int kb = unit.kb0; kb < unit.kb1; ++kb, pos.advance(n_stages)) {
                     const int s = pos.s;
                     if (pos.round > 0 && !mbar_wait_bounded(smem_u32(&bars->empty[s]), (pos.round - 1) & 1, abort_flag, hooks.limit_us)) {
                         ok = false;
@@ -292,7 +357,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             // With 64 activation rows per stage the MMA has M = 64: half the operand reads from shared memory.  Its
             // accumulator rows 16 i .. 16 i + 15 stand in TMEM lanes 32 i .. 32 i + 15.
             const uint32_t idesc = idesc_i8(a_rows == 64 ? 64 : BM, BN, /*a_signed=*/1, /*b_signed=*/0);
-            ProblemCursor<kTable> cur(one, table, n_problems);
+            UnitWalker<kTable> walk(sc, one, table, n_problems);
             uint32_t tile_it = 0;
             bool ok = true;
             // The thread's own instructions are on the critical path too, so nothing is recomputed per k block: the
@@ -305,11 +370,12 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             const uint32_t empty0 = smem_u32(&bars->empty[0]), expanded0 = smem_u32(&bars->expanded[0]);
             uint32_t s = 0, b = 0, b_parity = 0; // TMA stage; expanded tile and the parity of its use
             uint32_t a_lo = a_lo0, b_lo = b_lo0, empty_bar = empty0, expanded_bar = expanded0;
-            for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x, ++tile_it) {
-                const Unit unit(sp, u);
+            Unit unit;
+            const GemmProblem *gp;
+            for (; ok && walk.next(unit, gp); ++tile_it) {
                 const int tile = unit.tile;
-                const Params &p = cur.seek(tile).p;
-                const int kb_begin = unit.kb0(sp, p.KB), kb_end = unit.kb1(sp, p.KB);
+                const Params &p = gp->p;
+                const int kb_begin = unit.kb0, kb_end = unit.kb1;
                 const int buf = tile_it % kAccBufs;
                 const uint32_t use = tile_it / kAccBufs;
                 if (use > 0 && !mbar_wait_bounded(smem_u32(&bars->acc_empty[buf]), (use - 1) & 1, abort_flag, hooks.limit_us)) break;
@@ -368,14 +434,14 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         const int slot = 4 * g + tq;
         const int group = (kGroups == 2) ? (ew >> 2) : 0;
         const int rbi = (kGroups == 2) ? (ew & 3) : (ew >> 1);
-        ProblemCursor<kTable> cur(one, table, n_problems);
+        UnitWalker<kTable> walk(sc, one, table, n_problems);
         RingPos pos, reader; // reader: the k block kBSlots steps back, whose MMAs read the expanded tile written next
         bool ok = true;
-        for (int u = blockIdx.x; u < sp.n_units && ok; u += gridDim.x) {
-            const Unit unit(sp, u);
-            const int KB = cur.seek(unit.tile).p.KB;
-            const int kb_end = unit.kb1(sp, KB);
-            for (int kb = unit.kb0(sp, KB); kb < kb_end; ++kb, pos.advance(n_stages)) {
+        Unit unit;
+        const GemmProblem *gp;
+        while (ok && walk.next(unit, gp)) {
+            const int kb_end = unit.kb1;
+            for (int kb = unit.kb0; kb < kb_end; ++kb, pos.advance(n_stages)) {
                 const int s = pos.s, b = (int)(pos.it % kBSlots);
                 const bool mine = kGroups == 1 || (int)(pos.it & 1u) == group;
                 const bool has_reader = pos.it >= (uint32_t)kBSlots;
@@ -422,12 +488,13 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
     } else {
         // epilogue: warp w may touch TMEM lanes 32*(w % 4) .. +31
         const int q = warp & 3;
-        ProblemCursor<kTable> cur(one, table, n_problems);
+        UnitWalker<kTable> walk(sc, one, table, n_problems);
         uint32_t tile_it = 0;
-        for (int u = blockIdx.x; u < sp.n_units; u += gridDim.x, ++tile_it) {
-            const Unit unit(sp, u);
+        Unit unit;
+        const GemmProblem *gp;
+        for (; walk.next(unit, gp); ++tile_it) {
             const int tile = unit.tile;
-            const Params &p = cur.seek(tile).p;
+            const Params &p = gp->p;
             const float gamma = p.out_i32 ? 0.0f : *p.gamma;
             const int local = tile - p.tile_begin;
             const int m0 = (local % p.tiles_m) * (MT * BM);
@@ -488,103 +555,119 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                     if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), p.qb);
                 }
             };
+            // the 4 KiB that hold this warp's 32 x 32 sums of chunk c of token tile `half` in the slot of CTA `cta` (the
+            // chunks of a warp follow each other)
+            auto slot_chunk = [&](int cta, int half, int c) {
+                return reinterpret_cast<uint8_t *>(sc.slots) + (size_t)cta * (MT * kSlotTileBytes) +
+                       (size_t)((half * 4 + q) * (BN / 32) + c) * 4096;
+            };
 
-            if (!unit.split) {
+            if (unit.kind == kContribution) {
+                // partial sums of a tile that another CTA finishes: to this CTA's slot as they are, then the flag
 #pragma unroll 1
                 for (int half = 0; half < halves; ++half) {
                     const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
-                    const int t = token_of_lane(half);
-                    int rowsum;
-                    float scale;
-                    token_scale(t, rowsum, scale);
 #pragma unroll 1
                     for (int c = 0; c < BN / 32; ++c) {
                         uint32_t v[32];
                         tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
                         tmem_ld_wait();
-                        emit(v, c, t, rowsum, scale);
+                        uint8_t *dst = slot_chunk((int)blockIdx.x, half, c);
+#pragma unroll
+                        for (int pc = 0; pc < 8; ++pc)
+                            *reinterpret_cast<uint4 *>(dst + slot_piece(lane, pc)) =
+                                make_uint4(v[4 * pc], v[4 * pc + 1], v[4 * pc + 2], v[4 * pc + 3]);
                     }
                 }
                 tc_fence_before_sync();
+                __threadfence(); // this thread's stores are visible to the whole GPU before the flag can be
                 __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                    mbar_arrive(smem_u32(&bars->epilogue_met));
+                }
+                // the four epilogue warps meet (a contribution is the CTA's first unit: phase 0 of this barrier), then
+                // one thread raises the flag
+                if (!mbar_wait_bounded(smem_u32(&bars->epilogue_met), 0, abort_flag, hooks.limit_us)) break;
+                if (warp == 2 && lane == 0) st_release_gpu(sc.flags + blockIdx.x, 1u);
                 continue;
             }
 
-            // ---- a unit that holds a K slice of its tile: the last unit of this CTA, so every ring is idle and the
-            // shared memory from `base` on (at least 200 KiB) serves as staging: 32 KiB per epilogue warp.
-            const int cut = tile - sp.full; // which cut tile
-            uint8_t *stage_w = smem + q * (BN / 32) * 4096;
-            int32_t *scratch_tile = sp.scratch + (size_t)cut * (MT * kSplitTileBytes / 4);
-#pragma unroll 1
-            for (int half = 0; half < halves; ++half) {
-                const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
-                if (half > 0) { // the bulk reduce of the first token tile must have read the staging area
-                    if (lane == 0) bulk_wait_group_read0();
-                    __syncwarp();
+            // The other parts of a finisher's tile are in the slots of the CTAs behind this one, once their flags are up.
+            // They are fetched piece by piece (kFetchChunks chunks of one contribution) into this warp's buffers, in
+            // the order in which they are added: token tile, chunk pair, contribution.
+            const int n_contrib = unit.kind == kFinisher ? unit.last_contributor - (int)blockIdx.x : 0;
+            const int n_jobs = n_contrib * halves * (BN / 32 / (int)kFetchChunks);
+            uint8_t *fetch_base = smem + q * (kFetchBufs * kFetchBytes);
+            int issued = 0, taken = 0;
+            auto issue_fetches = [&]() { // lane 0 only
+                while (issued < n_jobs && issued - taken < kFetchBufs) {
+                    const int j = issued % n_contrib, pair = (issued / n_contrib) % (BN / 32 / (int)kFetchChunks),
+                              half = issued / (n_contrib * (BN / 32 / (int)kFetchChunks));
+                    const int b = issued % kFetchBufs;
+                    const uint32_t bar = smem_u32(&bars->fetched[q][b]);
+                    mbar_arrive_expect_tx(bar, kFetchBytes);
+                    bulk_copy_g2s(smem_u32(fetch_base + b * kFetchBytes),
+                                  slot_chunk((int)blockIdx.x + 1 + j, half, pair * (int)kFetchChunks), kFetchBytes, bar);
+                    ++issued;
                 }
-#pragma unroll 1
-                for (int c = 0; c < BN / 32; ++c) {
-                    uint32_t v[32];
-                    tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
-                    tmem_ld_wait();
-#pragma unroll
-                    for (int pc = 0; pc < 8; ++pc)
-                        *reinterpret_cast<uint4 *>(stage_w + c * 4096 + split_piece(lane, pc)) =
-                            make_uint4(v[4 * pc], v[4 * pc + 1], v[4 * pc + 2], v[4 * pc + 3]);
-                }
-                fence_proxy_async_smem(); // generic-proxy writes -> visible to the bulk copy engine
+            };
+            if (n_contrib > 0) {
+                bool ok = true;
+                for (int cta = (int)blockIdx.x + 1; cta <= unit.last_contributor && ok; ++cta)
+                    ok = flag_wait_bounded(sc.flags + cta, abort_flag, hooks.limit_us);
+                if (!ok) break;
+                fence_proxy_async_smem(); // (the buffers were last touched through the generic proxy or by the tensor core)
                 __syncwarp();
-                if (lane == 0) {
-                    bulk_reduce_add_s32(scratch_tile + (size_t)(half * 4 + q) * (BN / 32) * 1024, smem_u32(stage_w),
-                                        (BN / 32) * 4096);
-                    bulk_commit_group();
+                if (lane == 0) issue_fetches();
+            }
+            bool alive = true;
+#pragma unroll 1
+            for (int half = 0; half < halves && alive; ++half) {
+                const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
+                const int t = token_of_lane(half);
+                int rowsum;
+                float scale;
+                token_scale(t, rowsum, scale);
+#pragma unroll 1
+                for (int c0 = 0; c0 < BN / 32 && alive; c0 += (int)kFetchChunks) {
+                    uint32_t v[kFetchChunks][32];
+#pragma unroll
+                    for (int cc = 0; cc < (int)kFetchChunks; ++cc)
+                        tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)((c0 + cc) * 32), v[cc]);
+                    tmem_ld_wait();
+                    for (int j = 0; j < n_contrib; ++j) {
+                        const int b = taken % kFetchBufs;
+                        if (!mbar_wait_bounded(smem_u32(&bars->fetched[q][b]), (uint32_t)(taken / kFetchBufs) & 1u, abort_flag,
+                                               hooks.limit_us)) {
+                            alive = false;
+                            break;
+                        }
+                        const uint8_t *src = fetch_base + b * kFetchBytes;
+#pragma unroll
+                        for (int cc = 0; cc < (int)kFetchChunks; ++cc) {
+#pragma unroll
+                            for (int pc = 0; pc < 8; ++pc) {
+                                const uint4 w = *reinterpret_cast<const uint4 *>(src + cc * 4096 + slot_piece(lane, pc));
+                                v[cc][4 * pc] += w.x;
+                                v[cc][4 * pc + 1] += w.y;
+                                v[cc][4 * pc + 2] += w.z;
+                                v[cc][4 * pc + 3] += w.w;
+                            }
+                        }
+                        __syncwarp(); // every lane has read the buffer before lane 0 refills it
+                        ++taken;
+                        if (lane == 0) issue_fetches();
+                    }
+                    if (!alive) break;
+#pragma unroll
+                    for (int cc = 0; cc < (int)kFetchChunks; ++cc) emit(v[cc], c0 + cc, t, rowsum, scale);
                 }
             }
+            if (!alive) break;
             tc_fence_before_sync();
             __syncwarp();
-            if (lane == 0) {
-                mbar_arrive(smem_u32(&bars->acc_empty[buf]));
-                bulk_wait_group0(); // the sums have been added
-                __threadfence();
-            }
-            // The four epilogue warps meet twice (a cut unit is its CTA's last, so the barrier's phases are 0 and 1).
-            // The rendezvous is a bounded wait like every other: a warp that left through an expired wait never
-            // arrives, and the others then give up too instead of waiting for it for ever.
-            if (lane == 0) mbar_arrive(smem_u32(&bars->epilogue_met));
-            if (!mbar_wait_bounded(smem_u32(&bars->epilogue_met), 0, abort_flag, hooks.limit_us)) break;
-            if (warp == 2 && lane == 0) {
-                const uint32_t before = atomicAdd(&sp.counters[cut], 1u);
-                bars->split_last = (before == (uint32_t)sp.slices - 1u) ? 1 : 0;
-                __threadfence();
-            }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&bars->epilogue_met));
-            if (!mbar_wait_bounded(smem_u32(&bars->epilogue_met), 1, abort_flag, hooks.limit_us)) break;
-            if (bars->split_last) { // every slice has been added: dequantise the tile from the scratch
-#pragma unroll 1
-                for (int half = 0; half < halves; ++half) {
-                    const int t = token_of_lane(half);
-                    int rowsum;
-                    float scale;
-                    token_scale(t, rowsum, scale);
-#pragma unroll 1
-                    for (int c = 0; c < BN / 32; ++c) {
-                        const uint8_t *src =
-                            reinterpret_cast<const uint8_t *>(scratch_tile + (size_t)(half * 4 + q) * (BN / 32) * 1024) + c * 4096;
-                        uint32_t v[32];
-#pragma unroll
-                        for (int pc = 0; pc < 8; ++pc) {
-                            const int4 w = __ldcg(reinterpret_cast<const int4 *>(src + split_piece(lane, pc)));
-                            v[4 * pc] = (uint32_t)w.x;
-                            v[4 * pc + 1] = (uint32_t)w.y;
-                            v[4 * pc + 2] = (uint32_t)w.z;
-                            v[4 * pc + 3] = (uint32_t)w.w;
-                        }
-                        emit(v, c, t, rowsum, scale);
-                    }
-                }
-            }
+            if (lane == 0) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
         }
     }
 
@@ -611,7 +694,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
 // Tensor maps and parameters of one matmul, for `mt` token tiles per CTA tile.
 static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                int out_i32, float qb, int mt, int a_rows, int tile_begin, int32_t *status)
+                                int out_i32, float qb, int mt, int a_rows, int tile_begin, long long kb_begin, int32_t *status)
 {
     if (!encode_tiled_fn()) return cudaErrorNotSupported;
     if (x_rows < M) return cudaErrorInvalidValue;
@@ -632,35 +715,37 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
     p.out_i32 = out_i32;
     p.out_32b_aligned = (reinterpret_cast<uintptr_t>(out) % 32 == 0) ? 1 : 0; // (N is a multiple of 16)
     p.tile_begin = tile_begin;
+    p.kb_begin = kb_begin;
     p.qb = qb;
     p.status = status;
     return cudaSuccess;
 }
 
-// Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
-// How many K slices the tiles of the last, partly filled round of the SMs are cut into (1: none are cut).
-static int split_slices(int n_tiles, int min_KB, int sms)
+// Whether a launch over n_tiles CTA tiles with total_kb k blocks in all deals k-block shares instead of whole tiles.
+// Shares cost every CTA one contribution (a pass over its accumulators into its slot, about 5 us) and one wait at the
+// end, so they are chosen only where whole tiles would leave a good part of the last round idle: the idle k blocks of
+// that round, spread over all SMs, must come to at least kMinIdleKb (about 8 us) per SM, and a share must have at
+// least kMinShareKb k blocks.
+constexpr long long kMinIdleKb = 12, kMinShareKb = 16;
+static bool deals_shares(long long n_tiles, long long total_kb, int sms)
 {
 #ifdef BITLINEAR_TUNING // measurement aid, not compiled into the library as build.py builds it
     static const int enabled = [] {
         const char *v = std::getenv("BITLINEAR_PREFILL_SPLIT");
         return (v && *v) ? std::atoi(v) : 1;
     }();
-#else
-    constexpr int enabled = 1;
+    if (!enabled) return false;
 #endif
-    const int r = n_tiles % sms;
-    if (!enabled || r == 0 || 2 * r > sms || r > kMaxSplitTiles) return 1;
-    int s = sms / r;
-    if (s > min_KB) s = min_KB;
-    // Adding up and dequantising a cut tile costs 15 to 25 us (measured), a tile of KB k blocks takes about
-    // 0.6 us x KB: cut only where several times that is saved.
-    if (min_KB < kMinSplitKB || s < 3) s = 1;
-    return s;
+    if (n_tiles <= 0 || total_kb < kMinShareKb * sms) return false;
+    const long long r = n_tiles % sms;
+    if (r == 0) return false;
+    const long long idle_kb = (sms - r) * (total_kb / n_tiles) / sms;
+    return idle_kb >= kMinIdleKb;
 }
 
-static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int mt, int a_rows,
-                               int min_KB, void *split_scratch, cudaStream_t stream)
+// Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
+static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, long long total_kb, int mt,
+                               int a_rows, void *scratch, cudaStream_t stream)
 {
     const void *kernel = table ? (mt == 2 ? (const void *)prefill_gemm_kernel<2, true> : (const void *)prefill_gemm_kernel<1, true>)
                                : (mt == 2 ? (const void *)prefill_gemm_kernel<2, false> : (const void *)prefill_gemm_kernel<1, false>);
@@ -680,14 +765,13 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
     }
     if (n_tiles <= 0) return cudaSuccess;
     const int sms = sm_count();
-    SplitPlan sp;
-    sp.slices = split_scratch ? split_slices(n_tiles, min_KB, sms) : 1;
-    sp.full = sp.slices > 1 ? (n_tiles / sms) * sms : n_tiles;
-    sp.n_units = sp.full + (n_tiles - sp.full) * sp.slices;
-    sp.counters = reinterpret_cast<uint32_t *>(split_scratch);
-    sp.scratch = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(split_scratch) + kSplitCounterBytes);
-    int grid = sp.n_units;
-    if (grid > sms) grid = sms;
+    Schedule sc;
+    sc.stream_k = (scratch && deals_shares(n_tiles, total_kb, sms)) ? 1 : 0;
+    sc.n_tiles = n_tiles;
+    sc.total_kb = total_kb;
+    sc.flags = reinterpret_cast<uint32_t *>(scratch);
+    sc.slots = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(scratch) + kFlagBytes);
+    int grid = sc.stream_k ? sms : (n_tiles < sms ? n_tiles : sms);
     // programmatic dependent launch: see the head of this file
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -700,7 +784,7 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     WaitHooks hooks = take_wait_hooks();
-    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&sp, (void *)&a_rows, (void *)&n_stages, (void *)&hooks};
+    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&sc, (void *)&a_rows, (void *)&n_stages, (void *)&hooks};
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
@@ -714,53 +798,56 @@ int64_t prefill_tile_count(int64_t M, int64_t N, int64_t max_M)
     return ((M + mt * BM - 1) / (mt * BM)) * ((N + BN - 1) / BN);
 }
 
-size_t prefill_split_bytes(int64_t n_tiles, int64_t max_M)
+int64_t prefill_kb_count(int64_t M, int64_t N, int64_t K, int64_t max_M) { return prefill_tile_count(M, N, max_M) * ((K + BK - 1) / BK); }
+
+size_t prefill_scratch_bytes(int64_t n_tiles, int64_t total_kb, int64_t max_M)
 {
-    const int64_t cut = n_tiles < kMaxSplitTiles ? n_tiles : kMaxSplitTiles;
-    return kSplitCounterBytes + (size_t)cut * (size_t)prefill_token_tiles(max_M) * kSplitTileBytes;
+    static_assert(kFlagBytes >= 4 * 148, "one flag per CTA");
+    const int sms = sm_count();
+    if (!deals_shares(n_tiles, total_kb, sms)) return 0;
+    return kFlagBytes + (size_t)sms * (size_t)prefill_token_tiles(max_M) * kSlotTileBytes;
 }
 
-size_t prefill_split_clear_bytes(int64_t n_tiles, int64_t min_KB, int64_t max_M)
+size_t prefill_scratch_clear_bytes(int64_t n_tiles, int64_t total_kb)
 {
-    if (n_tiles > 0x7FFFFFFF) return 0;
-    const int sms = sm_count();
-    if (split_slices((int)n_tiles, (int)(min_KB > 0x7FFFFFFF ? 0x7FFFFFFF : min_KB), sms) < 2) return 0;
-    return kSplitCounterBytes + (size_t)(n_tiles % sms) * (size_t)prefill_token_tiles(max_M) * kSplitTileBytes;
+    return deals_shares(n_tiles, total_kb, sm_count()) ? kFlagBytes : 0;
 }
+
 // rows of activations per token tile in a TMA stage, for the largest M of a launch
 static int prefill_a_rows(int64_t max_M) { return max_M <= 64 ? 64 : BM; }
 
 cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                            const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                           int out_i32, float qb, WorkspaceHeader *hdr, void *split_scratch, cudaStream_t stream)
+                           int out_i32, float qb, WorkspaceHeader *hdr, void *scratch, cudaStream_t stream)
 {
     const int mt = prefill_token_tiles(M), a_rows = prefill_a_rows(M);
     GemmProblem g;
-    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, qb, mt, a_rows, 0,
+    cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, out_i32, qb, mt, a_rows, 0, 0,
                                  &hdr->status);
     if (e != cudaSuccess) return e;
-    return launch_gemm(g, nullptr, 1, g.p.tiles_m * g.p.tiles_n, mt, a_rows, g.p.KB, split_scratch, stream);
+    const int n_tiles = g.p.tiles_m * g.p.tiles_n;
+    return launch_gemm(g, nullptr, 1, n_tiles, (long long)n_tiles * g.p.KB, mt, a_rows, scratch, stream);
 }
 
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
-                                float qb, int64_t max_M, int tile_begin, WorkspaceHeader *hdr, int *n_tiles)
+                                float qb, int64_t max_M, int tile_begin, int64_t kb_begin, WorkspaceHeader *hdr, int *n_tiles)
 {
     GemmProblem g;
     cudaError_t e = fill_problem(g, packed, gamma, Xq, beta, rowsum, M, x_rows, K, N, out, 0, qb, prefill_token_tiles(max_M),
-                                 prefill_a_rows(max_M), tile_begin, &hdr->status);
+                                 prefill_a_rows(max_M), tile_begin, kb_begin, &hdr->status);
     if (e != cudaSuccess) return e;
     memcpy(slot, &g, sizeof(g));
     *n_tiles = g.p.tiles_m * g.p.tiles_n;
     return cudaSuccess;
 }
 
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t max_M, int min_KB,
-                                 void *split_scratch, cudaStream_t stream)
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t total_kb, int64_t max_M, void *scratch,
+                                 cudaStream_t stream)
 {
     GemmProblem unused{};
-    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, prefill_token_tiles(max_M),
-                       prefill_a_rows(max_M), min_KB, split_scratch, stream);
+    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, total_kb,
+                       prefill_token_tiles(max_M), prefill_a_rows(max_M), scratch, stream);
 }
 
 } // namespace bitlinear

@@ -94,26 +94,49 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     }
 }
 
+// ---- flags in global memory ---------------------------------------------------------------------------
+
+__device__ __forceinline__ void st_release_gpu(uint32_t *p, uint32_t v)
+{
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+// Waits until *flag is non-zero (an acquire load by every calling thread, so that what the writer stored before its
+// release is visible to each of them).  Returns false if the CTA's abort flag is up or the limit expired (then raises
+// the flag itself).
+__device__ __forceinline__ bool flag_wait_bounded(const uint32_t *flag, volatile int *abort_flag, uint32_t limit_us)
+{
+    if (ld_acquire_gpu(flag) != 0u) return true;
+    const uint64_t t0 = globaltimer_ns();
+    const uint64_t limit_ns = (uint64_t)limit_us * 1000ull;
+    for (uint32_t spin = 1;; ++spin) {
+        if (ld_acquire_gpu(flag) != 0u) return true;
+        if ((spin & 0x3Fu) == 0u) {
+            if (*abort_flag) return false;
+            if (globaltimer_ns() - t0 > limit_ns) {
+                *abort_flag = 1;
+                return false;
+            }
+        }
+        __nanosleep(64);
+    }
+}
+
 // ---- proxy fences ---------------------------------------------------------------------------------
 
 // Makes generic-proxy shared-memory writes visible to the async proxy (TMA, tcgen05.mma operands).
 __device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// ---- bulk reduce ---------------------------------------------------------------------
+// ---- bulk copies ------------------------------------------------------------------------------------
 
-// Adds `bytes` of int32 from shared memory to global memory (both 16-byte aligned, bytes a multiple of 16);
-// completion is tracked by the bulk async-group of the issuing thread.
-__device__ __forceinline__ void bulk_reduce_add_s32(void *gptr, uint32_t smem_addr, uint32_t bytes)
+// Untiled bulk copy global -> this CTA's shared memory (both addresses 16-byte aligned, bytes a multiple of 16);
+// completion is counted in bytes on `bar`.
+__device__ __forceinline__ void bulk_copy_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
 {
-    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.s32 [%0], [%1], %2;" ::"l"(gptr), "r"(smem_addr),
-                 "r"(bytes)
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
-__device__ __forceinline__ void bulk_commit_group() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-// all bulk groups of this thread have read their shared-memory source
-__device__ __forceinline__ void bulk_wait_group_read0() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-// all bulk groups of this thread are complete
-__device__ __forceinline__ void bulk_wait_group0() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
 // ---- TMA ------------------------------------------------------------------------------------------
 

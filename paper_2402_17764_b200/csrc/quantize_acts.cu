@@ -36,7 +36,8 @@ namespace bitlinear {
 namespace {
 
 constexpr int kThreads = 256;
-constexpr int kCache = 4; // 16-byte vectors kept in registers per thread (4 * 8 * 256 = 8192 elements)
+constexpr int kCacheShort = 4; // 16-byte vectors kept in registers per thread (4 * 8 * 256 = 8192 elements)
+constexpr int kCacheLong = 8;  // the same for tokens of 8193 to 16384 elements (plain quantiser only)
 constexpr int kSwigluSmemBytes = 56 * 1024; // SwiGLU products of one token in shared memory: 14336 elements
 
 __device__ __forceinline__ uint32_t absmax_bits(uint32_t m, const uint4 &v)
@@ -123,8 +124,8 @@ __device__ __forceinline__ int quant8(const uint4 &v, float s, uint2 &out)
 // of the token, or, for SwiGLU, the products themselves, in registers between the passes).
 // NT threads per token (64, 128, 192 or 256): what a CTA does besides touching its elements (finding its entry,
 // three block-wide reductions) is a fixed cost per thread, so short tokens take fewer threads with kCache vectors
-// each.  Tokens of more than 8192 elements re-read their tail, which hits L2.
-template <int kFronts, int NT>
+// each.  Tokens of more than 8 * kCache * NT elements re-read their tail, which hits L2.
+template <int kFronts, int NT, int kCache>
 __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantize_acts_kernel(const __grid_constant__ InlineTable inl,
                                                                  const DecodeEntry *__restrict__ table, int n_entries,
                                                                  int total_tokens, uint4 *zero_ptr, size_t zero_vecs,
@@ -381,8 +382,13 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
             m = absmax_bits(m, cache[c]);
         }
     }
-    for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT)
-        m = absmax_bits(m, __ldg(row + i));
+    for (int i = threadIdx.x + kCache * NT; i < n_vec; i += 4 * NT) { // four loads in flight
+        uint4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = (i + j * NT < n_vec) ? __ldg(row + i + j * NT) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) m = absmax_bits(m, v[j]);
+    }
 
     m = __reduce_max_sync(0xffffffffu, m);
     if (lane == 0) s_max[warp] = m;
@@ -405,10 +411,18 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
             out_at(i) = o;
         }
     }
-    for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
-        uint2 o;
-        sum += quant8(__ldg(row + i), s, o);
-        out_at(i) = o;
+    for (int i = threadIdx.x + kCache * NT; i < n_vec; i += 4 * NT) {
+        uint4 v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) v[j] = (i + j * NT < n_vec) ? __ldg(row + i + j * NT) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            if (i + j * NT < n_vec) {
+                uint2 o;
+                sum += quant8(v[j], s, o);
+                out_at(i + j * NT) = o;
+            }
+        }
     }
     if (tiled) // the last column tile is filled up with zeros
         for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += NT) out_at(i) = make_uint2(0u, 0u);
@@ -453,7 +467,7 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
     static const int counts[4] = {64, 128, 192, 256};
     int nt = 256;
     for (int c : counts)
-        if (n_vec <= c * kCache) {
+        if (n_vec <= c * kCacheShort) {
             nt = c;
             break;
         }
@@ -497,15 +511,15 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
             int dev = 0; \
             cudaGetDevice(&dev); \
             if (dev >= 0 && dev < 64 && !attr_set[dev]) { \
-                cudaError_t e = cudaFuncSetAttribute(quantize_acts_kernel<FRONTS, NT_>, \
+                cudaError_t e = cudaFuncSetAttribute(quantize_acts_kernel<FRONTS, NT_, kCacheShort>, \
                                                      cudaFuncAttributeMaxDynamicSharedMemorySize, kSwigluSmemBytes); \
                 if (e != cudaSuccess) return e; \
                 attr_set[dev] = true; \
             } \
         } \
         cfg.blockDim = dim3(NT_); \
-        cudaError_t le = cudaLaunchKernelEx(&cfg, quantize_acts_kernel<FRONTS, NT_>, inl, table, n_entries, total_tokens, \
-                                            zp, zero_vecs, h_cap_vecs); \
+        cudaError_t le = cudaLaunchKernelEx(&cfg, quantize_acts_kernel<FRONTS, NT_, kCacheShort>, inl, table, n_entries, \
+                                            total_tokens, zp, zero_vecs, h_cap_vecs); \
         if (le != cudaSuccess) return le; \
     } while (0)
 #define BITLINEAR_LAUNCH_BOTH(NT_) \
@@ -517,6 +531,14 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
         default: BITLINEAR_LAUNCH_QUANTISER(3, NT_); break; \
         } \
     } while (0)
+    if ((fronts & 3) == 0 && n_vec > 256 * kCacheShort && n_vec <= 256 * kCacheLong) {
+        // long tokens of the plain quantiser: twice the vectors in registers, so that the token is read once
+        // (CTAs of 512 threads with four vectors each were slower: 4.7 against 5.8 TB/s on 8192 x 13824)
+        cfg.blockDim = dim3(256);
+        cudaError_t le = cudaLaunchKernelEx(&cfg, quantize_acts_kernel<0, 256, kCacheLong>, inl, table, n_entries, total_tokens,
+                                            zp, zero_vecs, h_cap_vecs);
+        return le != cudaSuccess ? le : cudaGetLastError();
+    }
     switch (nt) {
     case 64: BITLINEAR_LAUNCH_BOTH(64); break;
     case 128: BITLINEAR_LAUNCH_BOTH(128); break;

@@ -205,8 +205,10 @@ def test_matmul_i32_mma_wider_batches(oracle, M, K, N):
 
 TC_SHAPES = [(128, 128, 256), (1, 16, 16), (65, 3200, 320), (200, 8640, 528), (300, 1536, 1024), (512, 5120, 256),
              (64, 4096, 4096), (129, 144, 4112),
-             # few tiles and a long K: the tiles are cut along K and summed through the int32 scratch
-             (300, 8640, 272), (40, 16384, 1040)]
+             (300, 8640, 272), (40, 16384, 1040),
+             # few tiles and a long K: the CTAs take equal shares of the k blocks of all tiles, and tiles whose k blocks
+             # lie in several shares are summed through the per-CTA slots (64-row stages, one token tile, two token tiles)
+             (20, 32768, 2560), (100, 32768, 2576), (300, 20000, 2304)]
 
 
 @pytest.mark.parametrize("M,K,N", TC_SHAPES)
@@ -314,11 +316,13 @@ def test_forward_is_deterministic(oracle):
     assert torch.equal(y1.view(torch.int16), y2.view(torch.int16))
 
 
-def test_tiles_cut_along_k_are_reusable(oracle):
-    """Few tiles and a long K: the GEMM cuts its tiles along K and sums them through an int32 scratch in the workspace.
-    The scratch is cleared by every call, so the same workspace gives the same (oracle) result twice: as a single
-    matmul, and as a sequence whose matmuls all have a long K (table-driven launch)."""
-    specs = [(48, 8640, 272), (300, 16384, 528)]
+def test_tiles_cut_along_k_are_reusable():
+    """Few tiles and a long K: the GEMM deals equal shares of the k blocks of all tiles, and the partial sums of tiles
+    that lie in several shares travel through flags and per-CTA slots in the workspace.  The flags are cleared by every
+    call, so the same workspace gives the same (oracle) result again and again: as single matmuls (the third one deals
+    shares by itself), and as a sequence whose matmuls have different K (table-driven launch, shares across matmuls)."""
+    oracle = load_timing_oracle()
+    specs = [(40, 20000, 1280), (64, 32768, 1552), (300, 20000, 2304)]
     layers, refs = [], []
     for i, (M, K, N) in enumerate(specs):
         W = S.latent_weights(N, K, 60 + i)
@@ -335,16 +339,17 @@ def test_tiles_cut_along_k_are_reusable(oracle):
             B.forward(packed, gamma, X, N, Y=Y, workspace=ws)
             assert B.poll_status(ws) == 0
             assert np.array_equal(torch_bf16_to_bits(Y), ref)
-    seq = B.Sequence(layers)
-    for _ in range(3):
-        for l in layers:
-            l[3].zero_()
-        seq.forward()
-        torch.cuda.synchronize()
-        assert B.poll_status(seq.workspace) == 0
-        for l, ref in zip(layers, refs):
-            assert np.array_equal(torch_bf16_to_bits(l[3]), ref)
-    seq.close()
+    for part in (layers[:2], layers):  # 64-row stages; two token tiles per CTA tile
+        seq = B.Sequence(part)
+        for _ in range(3):
+            for l in part:
+                l[3].zero_()
+            seq.forward()
+            torch.cuda.synchronize()
+            assert B.poll_status(seq.workspace) == 0
+            for l, ref in zip(part, refs):
+                assert np.array_equal(torch_bf16_to_bits(l[3]), ref)
+        seq.close()
 
 
 def test_forward_sequence_matches_single_calls(oracle):
