@@ -27,6 +27,7 @@
  *   R8  output is round-to-nearest-even bfloat16 of float(acc)*scale.
  *   R9  storage layout of the 2-bit codes (see oracle_pack_weights).
  *   R10 one gamma per weight matrix.
+ *   T1  a second storage format with five weights per byte in base 3 (see oracle_pack_weights_trits).
  *
  * Parity pins (tests/test_oracle_pins.py): hand-worked cases for Eq. 1-3 and
  * the activation quantiser including rounding ties, closed-form Gaussian
@@ -220,6 +221,78 @@ int oracle_unpack_weights(const uint8_t *packed, int64_t N, int64_t K, int8_t *T
             if (code == 3)
                 return ORACLE_ERR_ARG;
             T[n * K + k] = (int8_t)(code - 1);
+        }
+    }
+    return ORACLE_OK;
+}
+
+/* ---------- base-3 storage: five weights per byte (1.6 bits per weight) ----------
+ *
+ * A ternary weight carries log2 3 = 1.58 bits (the paper's title; Section 1), and the paper notes that its 2-bit kernel
+ * leaves room (Section 3, "Memory and Latency").  Reading T1: five codes c = t + 1 in {0, 1, 2} share one byte as the
+ * base-3 number c0 + 3 c1 + 9 c2 + 27 c3 + 81 c4 (0..242).  The matrix is cut into tiles of 80 rows by 64 columns, 1024
+ * bytes each, stored one after another with the column-tile index running fastest.  Within a tile, with r = n mod 80
+ * and c = k mod 64, split
+ *     r = 16*f + 8*h + g          (f = 0..4, h = 0..1, g = 0..7)
+ *     c = 16*tq + 8*s + 4*hi + b  (tq = 0..3, s = 0..1, hi = 0..1, b = 0..3)
+ * and the weight is digit f of byte 512*s + 16*(4*g + tq) + 4*(2*hi + h) + b of the tile (the byte positions of the
+ * 2-bit format; the five rows of a byte are 16 apart).  Rows N..(multiple of 80) and columns K..(multiple of 64) hold
+ * code 1 (weight zero), so a byte of padding is 121.
+ */
+static int64_t trit_row_blocks(int64_t N) { return (N + 79) / 80; }
+
+int64_t oracle_packed_bytes_trits(int64_t N, int64_t K)
+{
+    if (N <= 0 || K <= 0 || (N % 16) != 0)
+        return -1;
+    return trit_row_blocks(N) * col_tiles(K) * 1024;
+}
+
+static const int POW3[5] = {1, 3, 9, 27, 81};
+
+static void locate_trit(int64_t n, int64_t k, int64_t KB, int64_t *byte_index, int *digit)
+{
+    int64_t tile = (n / 80) * KB + (k / 64);
+    int r = (int)(n % 80), c = (int)(k % 64);
+    int f = r / 16, h = (r % 16) / 8, g = r % 8;
+    int tq = c / 16, s = (c % 16) / 8, hi = (c % 8) / 4, b = c % 4;
+    *byte_index = tile * 1024 + 512 * s + 16 * (4 * g + tq) + 4 * (2 * hi + h) + b;
+    *digit = f;
+}
+
+int oracle_pack_weights_trits(const int8_t *T, int64_t N, int64_t K, uint8_t *packed)
+{
+    if (!T || !packed || N <= 0 || K <= 0 || (N % 16) != 0)
+        return ORACLE_ERR_ARG;
+    int64_t KB = col_tiles(K), NB = trit_row_blocks(N);
+    memset(packed, 0, (size_t)(NB * KB * 1024));
+    for (int64_t n = 0; n < NB * 80; ++n) {
+        for (int64_t k = 0; k < KB * 64; ++k) {
+            int t = (n < N && k < K) ? T[n * K + k] : 0;
+            if (t < -1 || t > 1)
+                return ORACLE_ERR_ARG;
+            int64_t at;
+            int digit;
+            locate_trit(n, k, KB, &at, &digit);
+            packed[at] = (uint8_t)(packed[at] + (t + 1) * POW3[digit]);
+        }
+    }
+    return ORACLE_OK;
+}
+
+int oracle_unpack_weights_trits(const uint8_t *packed, int64_t N, int64_t K, int8_t *T)
+{
+    if (!T || !packed || N <= 0 || K <= 0 || (N % 16) != 0)
+        return ORACLE_ERR_ARG;
+    int64_t KB = col_tiles(K);
+    for (int64_t n = 0; n < N; ++n) {
+        for (int64_t k = 0; k < K; ++k) {
+            int64_t at;
+            int digit;
+            locate_trit(n, k, KB, &at, &digit);
+            if (packed[at] > 242)
+                return ORACLE_ERR_ARG;
+            T[n * K + k] = (int8_t)((packed[at] / POW3[digit]) % 3 - 1);
         }
     }
     return ORACLE_OK;

@@ -269,3 +269,30 @@ def pack_weights(T) -> np.ndarray:
                             out[at] = v
                             at += 1
     return out
+
+
+def pack_weights_trits(T) -> np.ndarray:
+    """The base-3 storage (five weights per byte), walked from the storage side like pack_weights: tile -> slab -> slot
+    -> word -> byte -> base-3 digit, fetching the weight each digit holds.  Row blocks have 80 rows."""
+    T = np.asarray(T, np.int8)
+    N, K = T.shape
+    assert N % 16 == 0
+    row_blocks, col_tiles = (N + 79) // 80, (K + 63) // 64
+    out = np.zeros(row_blocks * col_tiles * 1024, np.uint8)
+    at = 0
+    for row_block in range(row_blocks):
+        for col_tile in range(col_tiles):
+            for slab in range(2):
+                for slot in range(32):
+                    row_low, col_group = slot // 4, slot % 4
+                    for word in range(4):
+                        for byte in range(4):
+                            v = 0
+                            for digit in range(4, -1, -1):      # Horner: the last row group is the leading digit
+                                n = 80 * row_block + 16 * digit + 8 * (word % 2) + row_low
+                                k = 64 * col_tile + 16 * col_group + 8 * slab + 4 * (word // 2) + byte
+                                code = int(T[n, k]) + 1 if (n < N and k < K) else 1
+                                v = 3 * v + code
+                            out[at] = v
+                            at += 1
+    return out

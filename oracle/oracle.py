@@ -55,6 +55,10 @@ class Oracle:
         L.oracle_packed_bytes.restype = _i64
         L.oracle_pack_weights.argtypes = [_p, _i64, _i64, _p]
         L.oracle_unpack_weights.argtypes = [_p, _i64, _i64, _p]
+        L.oracle_packed_bytes_trits.argtypes = [_i64, _i64]
+        L.oracle_packed_bytes_trits.restype = _i64
+        L.oracle_pack_weights_trits.argtypes = [_p, _i64, _i64, _p]
+        L.oracle_unpack_weights_trits.argtypes = [_p, _i64, _i64, _p]
         L.oracle_quantize_acts.argtypes = [_p, _i64, _i64, _p, _p, _p]
         L.oracle_rmsnorm_quantize_acts.argtypes = [_p, _p, ctypes.c_float, _i64, _i64, _p, _p, _p, _p]
         L.oracle_rmsnorm_mean_square.argtypes = [_p, _i64, _i64, _p]
@@ -122,6 +126,26 @@ class Oracle:
         packed = self._c(packed, np.uint8)
         T = np.empty((N, K), np.int8)
         self._check(self.lib.oracle_unpack_weights(self._ptr(packed), N, K, self._ptr(T)), "unpack_weights")
+        return T
+
+    def packed_bytes_trits(self, N: int, K: int) -> int:
+        return int(self.lib.oracle_packed_bytes_trits(N, K))
+
+    def pack_weights_trits(self, T: np.ndarray) -> np.ndarray:
+        """The base-3 storage: five weights per byte, tiles of 80 rows x 64 columns."""
+        T = self._c(T, np.int8)
+        N, K = T.shape
+        nbytes = self.packed_bytes_trits(N, K)
+        if nbytes < 0:
+            raise ValueError("N must be a positive multiple of 16")
+        out = np.empty(nbytes, np.uint8)
+        self._check(self.lib.oracle_pack_weights_trits(self._ptr(T), N, K, self._ptr(out)), "pack_weights_trits")
+        return out
+
+    def unpack_weights_trits(self, packed: np.ndarray, N: int, K: int) -> np.ndarray:
+        packed = self._c(packed, np.uint8)
+        T = np.empty((N, K), np.int8)
+        self._check(self.lib.oracle_unpack_weights_trits(self._ptr(packed), N, K, self._ptr(T)), "unpack_weights_trits")
         return T
 
     def quantize_acts(self, X_bf16_bits: np.ndarray):

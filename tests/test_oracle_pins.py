@@ -588,3 +588,38 @@ def test_c_oracle_equals_python_restatement_of_the_fronts(oracle):
         q2, beta2, rs2 = R.quantize_acts_bits(xb, bits)
         assert np.array_equal(q, q2) and np.array_equal(beta, beta2) and np.array_equal(rs, rs2)
         assert np.array_equal(oracle.dequant_bits(acc, beta, 0.0173, bits), R.dequant_bits(acc, beta, 0.0173, bits))
+
+
+# ---- base-3 storage: five weights per byte ----
+
+def test_hand_cases_layout_trits(oracle, golden):
+    lay = golden["layout_trits"]
+    N, K = lay["N"], lay["K"]
+    base = oracle.pack_weights_trits(np.zeros((N, K), np.int8))
+    assert base.size == lay["packed_bytes"] == oracle.packed_bytes_trits(N, K) and np.all(base == 121)
+    for c in lay["cases"]:
+        T = np.zeros((N, K), np.int8)
+        T[c["n"], c["k"]] = c["t"]
+        p = oracle.pack_weights_trits(T)
+        diff = np.nonzero(p != 121)[0]
+        assert diff.tolist() == [c["byte_index"]], (c, lay["citation"])
+        assert int(p[c["byte_index"]]) == c["byte_value"], c
+
+
+def test_trit_storage_properties(oracle):
+    rng = np.random.default_rng(9)
+    for N, K in [(16, 16), (80, 64), (96, 144), (176, 200), (3200, 320)]:
+        T = rng.integers(-1, 2, (N, K)).astype(np.int8)
+        p = oracle.pack_weights_trits(T)
+        assert p.size == -(-N // 80) * -(-K // 64) * 1024      # 80 x 64 weights per KiB: 1.6 bits per weight
+        assert p.max() <= 242                                    # 3^5 - 1: every byte is a five-digit base-3 number
+        assert np.array_equal(oracle.unpack_weights_trits(p, N, K), T)
+        if N * K <= 40000:
+            assert np.array_equal(p, R.pack_weights_trits(T))
+    # five weights per byte against four: the same matrix takes 4/5 of the bytes when N is a multiple of 80 and 64
+    assert oracle.packed_bytes_trits(320, 640) * 5 == oracle.packed_bytes(320, 640) * 4
+    # an all-ones matrix fills every digit with 2 (byte 242) where weights exist; minus ones give 0 there
+    p = oracle.pack_weights_trits(np.ones((80, 64), np.int8))
+    assert np.all(p == 242) and not oracle.pack_weights_trits(-np.ones((80, 64), np.int8)).any()
+    with pytest.raises(ValueError):
+        oracle.unpack_weights_trits(np.full(1024, 243, np.uint8), 80, 64)
