@@ -131,27 +131,32 @@ class ClockSampler:
 class Weights:
     """Resident packed weights (and their gammas) of a list of BitLinear matrices."""
 
-    def __init__(self, layer_shapes, n_layers, copies=1, seed_base=0):
+    def __init__(self, layer_shapes, n_layers, copies=1, seed_base=0, trits=False):
         import torch
         from paper_2402_17764_b200 import binding as B
         from paper_2402_17764_b200 import synthetic as S
+        self.trits = trits   # the base-3 format, five weights per byte
+        nbytes = B.packed_bytes_trits if trits else B.packed_bytes
+        quantize = B.quantize_weights_trits if trits else B.quantize_weights
         self.entries = [(li, mi, sh) for li in range(n_layers * copies) for mi, sh in enumerate(layer_shapes)]
         a256 = lambda n: (n + 255) // 256 * 256
-        sizes = [a256(B.packed_bytes(sh.N, sh.K)) for _, _, sh in self.entries]
+        sizes = [a256(nbytes(sh.N, sh.K)) for _, _, sh in self.entries]
         self.packed_all = torch.empty(sum(sizes), dtype=torch.uint8, device="cuda")
         self.gammas = torch.empty(len(self.entries), dtype=torch.float32, device="cuda")
         self.packed, self.seeds = [], []
-        self.algorithmic_bytes = 0
+        self.algorithmic_bytes = 0   # of the 2-bit format (N K / 4), whatever the stored format
+        self.stored_bytes = 0
         po = 0
         for i, (li, mi, sh) in enumerate(self.entries):
             seed = seed_base + li * 16 + mi
             W = S.latent_weights(sh.N, sh.K, seed, device="cuda")
-            packed = self.packed_all[po:po + B.packed_bytes(sh.N, sh.K)]
-            B.quantize_weights(W, 1e-5, packed=packed, gamma=self.gammas[i:i + 1])
+            packed = self.packed_all[po:po + nbytes(sh.N, sh.K)]
+            quantize(W, 1e-5, packed=packed, gamma=self.gammas[i:i + 1])
             del W
             self.packed.append(packed)
             self.seeds.append(seed)
             self.algorithmic_bytes += S.packed_weight_bytes(sh.N, sh.K)
+            self.stored_bytes += nbytes(sh.N, sh.K)
             po += sizes[i]
         torch.cuda.synchronize()
 
@@ -192,7 +197,7 @@ def time_sequence(stack, steps, warmup, dist_barrier=None, kernel_steps=None, mi
     pass with events around that launch."""
     import torch
     from paper_2402_17764_b200 import binding as B
-    seq = B.Sequence(stack.layers)
+    seq = B.Sequence(stack.layers, trits=stack.weights.trits)
     for _ in range(warmup):
         seq.forward()
     rounds, total_ms = [], 0.0
@@ -550,6 +555,21 @@ def extras(peaks, int8_peak, weights70):
     seq.close()
     del st, seq
 
+    # the 3B-shaped step on the base-3 format (five weights per byte: 4/5 of the bytes, a table look-up per stored byte)
+    # beside the 2-bit step
+    cfg = S.CONFIGS["3b_decode"]
+    res = {}
+    for trits in (False, True):
+        st = Stack(cfg["layers"], cfg["n_layers"], 1, weights=Weights(cfg["layers"], cfg["n_layers"], trits=trits))
+        t = time_sequence(st, 200, 20, min_timed_s=0.2)
+        res["base3_1.6bit" if trits else "2bit"] = {
+            "ms_per_step": round(t["ms"], 4), "ms_min": round(t["ms_min"], 4), "stored_bytes": st.weights.stored_bytes,
+            "stored_GB/s": round(st.weights.stored_bytes / t["ms"] / 1e6, 1),
+            "GB/s_of_2bit_bytes": round(st.algorithmic_bytes / t["ms"] / 1e6, 1)}
+        del st
+        torch.cuda.empty_cache()
+    out["3b_decode_step_trits"] = res
+
     # 70B-shaped step at more tokens: 16 (the benchmark definition) and 176 (the batch size of the paper's throughput
     # comparison on the 70B model, Table 3; tensor-core GEMM).  Each against the roof that binds it: streaming the
     # packed weights once (HBM) or 2*M*N*K integer operations (tensor cores), whichever takes longer.
@@ -822,12 +842,14 @@ def profile_case(name: str):
     torch.cuda.set_device(0)
     build.build()
     if name.startswith("decode"):
-        # 48 distinct 11008x4096 matrices (541 MB of packed weights) at M = 1; decode:M[:copies] overrides
+        # 48 distinct 11008x4096 matrices (541 MB of packed weights) at M = 1; decode:M[:copies] overrides;
+        # decode-trits[:M[:copies]]: the same matrices in the base-3 format (433 MB)
         parts = name.split(":")
         M = int(parts[1]) if len(parts) > 1 else 1
         copies = int(parts[2]) if len(parts) > 2 else 48
-        st = Stack([S.LayerShape("up", 11008, 4096)], 1, M, copies=copies)
-        seq = B.Sequence(st.layers)
+        trits = name.startswith("decode-trits")
+        st = Stack([S.LayerShape("up", 11008, 4096)], 1, M, weights=Weights([S.LayerShape("up", 11008, 4096)], 1, copies=copies, trits=trits))
+        seq = B.Sequence(st.layers, trits=trits)
         for _ in range(3):
             seq.forward()
         torch.cuda.synchronize()
@@ -841,8 +863,8 @@ def profile_case(name: str):
         torch.cuda.synchronize()
         assert B.poll_status(seq.workspace) == 0
         ms = sum(a.elapsed_time(b) for a, b in pairs) / len(pairs)
-        print(json.dumps({"case": name, "packed_bytes_per_launch": st.algorithmic_bytes,
-                          "matmul_kernel_ms": round(ms, 4), "GB/s": round(st.algorithmic_bytes / ms / 1e6, 1)}))
+        print(json.dumps({"case": name, "packed_bytes_per_launch": st.weights.stored_bytes,
+                          "matmul_kernel_ms": round(ms, 4), "GB/s": round(st.weights.stored_bytes / ms / 1e6, 1)}))
     elif name.startswith("prefill"):
         # 13824x5120 at M = 2048 (or prefill:M): 290 G integer operations per launch
         M = int(name.split(":")[1]) if ":" in name else 2048
@@ -893,7 +915,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | prefill[:M] | quantiser[:norm|:swiglu] | peak[:iters]) and exit")
+    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | decode-trits[:M[:copies]] | prefill[:M] | quantiser[:norm|:swiglu] | peak[:iters]) and exit")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)

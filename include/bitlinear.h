@@ -191,6 +191,30 @@ bitlinear_status bitlinear_forward_act_bits(const void *packed, const float *gam
                                             void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * A second storage format: five weights per byte (1.6 bits per weight).  A ternary weight carries log2 3 = 1.58 bits
+ * (the paper's title, Section 1), and Section 3 ("Memory and Latency") notes that the 2-bit kernel leaves room: this
+ * format moves 4/5 of the bytes and pays for it with a table look-up per stored byte.  The codes c = T + 1 of five rows at
+ * one column share a byte as the base-3 number c0 + 3 c1 + 9 c2 + 27 c3 + 81 c4 (0..242).  Tiles are 80 rows x 64 columns
+ * = 1024 bytes, stored like the 2-bit tiles (column-tile index fastest; padding rows and columns hold code 1, a padding
+ * byte is 121); with r = n % 80 = 16 f + 8 h + g (f = 0..4) and c = k % 64 = 16 tq + 8 s + 4 hi + b, the weight is digit f
+ * of byte 512 s + 16 (4 g + tq) + 4 (2 hi + h) + b: the byte positions of the 2-bit format, five rows 16 apart per byte.
+ * Eq. 1-3, gamma and every result are those of the 2-bit path bit for bit; only the stored bytes differ.
+ *   bitlinear_packed_bytes_trits     bytes of the buffer: ceil(N / 80) * ceil(K / 64) * 1024 (0 for rejected shapes)
+ *   bitlinear_quantize_weights_trits as bitlinear_quantize_weights, writing this format
+ *   bitlinear_forward_trits          as bitlinear_forward on such a buffer, for M <= 8 tokens (the weight-streaming kernel;
+ *                                    more tokens give BITLINEAR_ERR_SHAPE: with many tokens the weights' bytes no longer
+ *                                    bound the time, and the 2-bit format is the one to use)
+ *   bitlinear_sequence_create_trits  as bitlinear_sequence_create for entries whose weights are all in this format and
+ *                                    whose M are all <= 8; run and destroyed like any sequence
+ */
+size_t bitlinear_packed_bytes_trits(int64_t N, int64_t K);
+bitlinear_status bitlinear_quantize_weights_trits(const float *W, int64_t N, int64_t K, float eps,
+                                                  void *packed, float *gamma, void *stream);
+bitlinear_status bitlinear_forward_trits(const void *packed, const float *gamma, const void *X,
+                                         int64_t M, int64_t K, int64_t N, void *Y,
+                                         void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * The same forward for callers that cannot give it a workspace.  (The paper has no counterpart: this is a
  * convenience of the library.)  Some code that wants to run a BitLinear layer is not allowed to allocate
  * device memory at the point of the call -- a plug-in that runs inside another framework's memory pool, a
@@ -260,6 +284,10 @@ bitlinear_status bitlinear_sequence_create_swiglu(const bitlinear_layer_desc *la
                                                   const void *const *ups, float norm_eps, int n, void *workspace,
                                                   size_t workspace_bytes, bitlinear_sequence **out);
 
+/* The same for weights in the base-3 format (see bitlinear_quantize_weights_trits); every M at most 8. */
+bitlinear_status bitlinear_sequence_create_trits(const bitlinear_layer_desc *layers, int n, void *workspace,
+                                                 size_t workspace_bytes, bitlinear_sequence **out);
+
 /* Enqueues the whole sequence on `stream`: one batched activation-quantiser launch, one persistent matmul
  * launch that starts while the quantiser is still running (programmatic dependent launch) and one very small
  * finishing launch.  Calls on the same sequence must be stream-ordered, not concurrent.  Once a sequence has run once
@@ -284,6 +312,10 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
                                       int32_t *acc, int path, void *workspace, size_t workspace_bytes,
                                       void *stream);
 bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream);
+/* The same two hooks for the base-3 format (the matmul on the weight-streaming kernel, M <= 8). */
+bitlinear_status bitlinear_matmul_i32_trits(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
+                                            int32_t *acc, void *workspace, size_t workspace_bytes, void *stream);
+bitlinear_status bitlinear_unpack_weights_trits(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream);
 
 /*
  * Checks a packed weight buffer (Section 3, "Memory and Latency": 2-bit storage; a weight is -1, 0 or 1, so the

@@ -43,6 +43,12 @@ EXPORTS = [
     "bitlinear_matmul_i32",
     "bitlinear_unpack_weights",
     "bitlinear_validate_packed",
+    "bitlinear_packed_bytes_trits",
+    "bitlinear_quantize_weights_trits",
+    "bitlinear_forward_trits",
+    "bitlinear_sequence_create_trits",
+    "bitlinear_matmul_i32_trits",
+    "bitlinear_unpack_weights_trits",
     "bitlinear_probe_int8_peak",
     "bitlinear_test_expire_next_wait",
     "bitlinear_poll_status",
@@ -112,6 +118,13 @@ def load_library() -> ctypes.CDLL:
     L.bitlinear_unpack_weights.argtypes = [vp, i64, i64, vp, vp]
     L.bitlinear_poll_status.argtypes = [vp, vp, ctypes.POINTER(ci)]
     L.bitlinear_validate_packed.argtypes = [vp, i64, i64, vp, vp]
+    L.bitlinear_packed_bytes_trits.argtypes = [i64, i64]
+    L.bitlinear_packed_bytes_trits.restype = sz
+    L.bitlinear_quantize_weights_trits.argtypes = [vp, i64, i64, cf, vp, vp, vp]
+    L.bitlinear_forward_trits.argtypes = [vp, vp, vp, i64, i64, i64, vp, vp, sz, vp]
+    L.bitlinear_sequence_create_trits.argtypes = [ctypes.POINTER(LayerDesc), ci, vp, sz, ctypes.POINTER(vp)]
+    L.bitlinear_matmul_i32_trits.argtypes = [vp, vp, i64, i64, i64, vp, vp, sz, vp]
+    L.bitlinear_unpack_weights_trits.argtypes = [vp, i64, i64, vp, vp]
     L.bitlinear_probe_int8_peak.argtypes = [ci, vp, ctypes.POINTER(i64), vp]
     L.bitlinear_test_expire_next_wait.argtypes = [ctypes.c_uint32, ci]
     L.bitlinear_test_expire_next_wait.restype = None
@@ -164,6 +177,58 @@ def quantize_weights(W: torch.Tensor, eps: float = 1e-5, packed: torch.Tensor | 
     st = load_library().bitlinear_quantize_weights(_ptr(W), N, K, float(eps), _ptr(packed), _ptr(gamma), _stream(stream))
     _check(st, "bitlinear_quantize_weights")
     return packed, gamma
+
+
+def packed_bytes_trits(N: int, K: int) -> int:
+    return int(load_library().bitlinear_packed_bytes_trits(N, K))
+
+
+def quantize_weights_trits(W: torch.Tensor, eps: float = 1e-5, packed: torch.Tensor | None = None,
+                           gamma: torch.Tensor | None = None, stream=None):
+    """bitlinear_quantize_weights_trits: fp32 [N, K] -> (base-3 packed uint8 buffer, gamma fp32[1])."""
+    N, K = W.shape
+    if packed is None:
+        packed = torch.empty(packed_bytes_trits(N, K), dtype=torch.uint8, device=W.device)
+    if gamma is None:
+        gamma = torch.empty(1, dtype=torch.float32, device=W.device)
+    st = load_library().bitlinear_quantize_weights_trits(_ptr(W), N, K, float(eps), _ptr(packed), _ptr(gamma), _stream(stream))
+    _check(st, "bitlinear_quantize_weights_trits")
+    return packed, gamma
+
+
+def forward_trits(packed: torch.Tensor, gamma: torch.Tensor, X: torch.Tensor, N: int, Y: torch.Tensor | None = None,
+                  workspace: torch.Tensor | None = None, stream=None) -> torch.Tensor:
+    """bitlinear_forward_trits: bf16 [M, K] (M <= 8) -> bf16 [M, N] on base-3 packed weights."""
+    M, K = X.shape
+    if Y is None:
+        Y = torch.empty((M, N), dtype=torch.bfloat16, device=X.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, X.device)
+    st = load_library().bitlinear_forward_trits(_ptr(packed), _ptr(gamma), _ptr(X), M, K, N, _ptr(Y), _ptr(workspace),
+                                                workspace.numel(), _stream(stream))
+    _check(st, "bitlinear_forward_trits")
+    return Y
+
+
+def matmul_i32_trits(packed: torch.Tensor, Xq: torch.Tensor, N: int, workspace: torch.Tensor | None = None,
+                     stream=None) -> torch.Tensor:
+    """bitlinear_matmul_i32_trits (test hook): int8 [M, K] x base-3 packed [N, K] -> int32 [M, N]."""
+    M, K = Xq.shape
+    acc = torch.empty((M, N), dtype=torch.int32, device=Xq.device)
+    if workspace is None:
+        workspace = alloc_workspace(M, N, K, Xq.device)
+    st = load_library().bitlinear_matmul_i32_trits(_ptr(packed), _ptr(Xq), M, K, N, _ptr(acc), _ptr(workspace),
+                                                   workspace.numel(), _stream(stream))
+    _check(st, "bitlinear_matmul_i32_trits")
+    return acc
+
+
+def unpack_weights_trits(packed: torch.Tensor, N: int, K: int, stream=None) -> torch.Tensor:
+    """bitlinear_unpack_weights_trits (test hook): -> int8 [N, K] in {-1, 0, 1}."""
+    T = torch.empty((N, K), dtype=torch.int8, device=packed.device)
+    st = load_library().bitlinear_unpack_weights_trits(_ptr(packed), N, K, _ptr(T), _stream(stream))
+    _check(st, "bitlinear_unpack_weights_trits")
+    return T
 
 
 def quantize_acts(X: torch.Tensor, stream=None):
@@ -338,9 +403,10 @@ class Sequence:
     of their activation quantiser (bitlinear_sequence_create_rmsnorm).
     `ups` (optional): one bf16 tensor [M, K] or None per layer; those layers quantise silu(X) * up
     (bitlinear_sequence_create_swiglu).
+    `trits`: the packed weights are in the base-3 format (bitlinear_sequence_create_trits).
     """
 
-    def __init__(self, layers, device="cuda", gains=None, norm_eps: float = 1e-5, ups=None):
+    def __init__(self, layers, device="cuda", gains=None, norm_eps: float = 1e-5, ups=None, trits: bool = False):
         L = load_library()
         self._keep = list(layers)
         self._gains = list(gains) if gains is not None else None
@@ -359,7 +425,10 @@ class Sequence:
             assert len(tensors) == n
             return (ctypes.c_void_p * n)(*[(_ptr(x) if x is not None else None) for x in tensors])
 
-        if self._ups is not None:
+        if trits:
+            assert self._ups is None and self._gains is None
+            st = L.bitlinear_sequence_create_trits(arr, n, _ptr(self.workspace), nbytes, ctypes.byref(handle))
+        elif self._ups is not None:
             st = L.bitlinear_sequence_create_swiglu(arr, pointers(self._gains) if self._gains is not None else None,
                                                     pointers(self._ups), float(norm_eps), n, _ptr(self.workspace), nbytes,
                                                     ctypes.byref(handle))

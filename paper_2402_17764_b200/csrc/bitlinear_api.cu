@@ -84,6 +84,8 @@ inline int64_t row_blocks(int64_t N) { return (N + kTileRows - 1) / kTileRows; }
 inline int64_t col_tiles(int64_t K) { return (K + kTileCols - 1) / kTileCols; }
 
 inline int64_t gemm_k_blocks(int64_t K) { return (K + 127) / 128; }
+constexpr int kMaxTritM = 8; // the base-3 format runs on the weight-streaming kernel for up to 8 tokens only
+inline int64_t trit_row_blocks(int64_t N) { return (N + 79) / 80; }
 
 // Workspace of one matmul: [header | int32 scratch | per-warp lists | Xq | beta | rowsum].  The scratch serves the
 // weight-streaming kernel (sums of row blocks shared by several warps, at most 64 tokens) or the GEMM (flags and a slot
@@ -137,7 +139,7 @@ bool use_tcgen05_for(int64_t M)
 
 // Fills one DecodeEntry for a matmul whose workspace part starts at `base`.
 void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
-                int64_t N, void *out, int out_i32, char *base, const Layout &L)
+                int64_t N, void *out, int out_i32, char *base, const Layout &L, bool trits = false)
 {
     e.packed = reinterpret_cast<const uint4 *>(packed);
     e.gamma = gamma;
@@ -151,7 +153,7 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
     e.N = (int)N;
     e.K = (int)K;
     e.KB = (int)col_tiles(K);
-    e.NB = (int)row_blocks(N);
+    e.NB = (int)(trits ? trit_row_blocks(N) : row_blocks(N));
     e.tile_begin = 0;
     e.token_begin = 0;
     e.out_i32 = out_i32;
@@ -166,11 +168,11 @@ void fill_entry(DecodeEntry &e, const void *packed, const float *gamma, const vo
 // x_rows: rows of int8 activations that exist behind e.Xq (>= e.M; the rows past e.M may hold anything).
 // split_scratch: the GEMM's scratch with its flags zeroed, or null (then it deals whole tiles only).
 bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offset, int64_t x_rows, void *split_scratch,
-                            cudaStream_t stream)
+                            cudaStream_t stream, bool trits = false)
 {
     WorkspaceHeader *hdr = reinterpret_cast<WorkspaceHeader *>(ws);
     OwnedList *lists = reinterpret_cast<OwnedList *>(ws + lists_offset);
-    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M));
+    const bool tc = !trits && ((path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(e.M)));
     if (tc) {
         cudaError_t err = launch_prefill(e.packed, e.gamma, e.Xq, e.beta, e.rowsum, e.M, x_rows, e.K, e.N, e.out, e.out_i32,
                                          e.qb, hdr, split_scratch, stream);
@@ -180,7 +182,7 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
     InlineTable inl{};
     inl.e[0] = e;
     cudaError_t err = launch_decode(inl, nullptr, 1, decode_items(e.NB, e.KB, decode_is_wide(e.M)), e.M,
-                                    path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream);
+                                    path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream, trits);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;
 }
@@ -215,22 +217,42 @@ size_t bitlinear_packed_bytes(int64_t N, int64_t K)
     return (size_t)(row_blocks(N) * col_tiles(K)) * kTileBytes;
 }
 
+size_t bitlinear_packed_bytes_trits(int64_t N, int64_t K)
+{
+    if (check_shape(0, N, K) != BITLINEAR_OK) return 0;
+    return (size_t)(trit_row_blocks(N) * col_tiles(K)) * kTileBytes;
+}
+
 size_t bitlinear_workspace_bytes(int64_t M, int64_t N, int64_t K)
 {
     if (check_shape(M, N, K) != BITLINEAR_OK) return 0;
     return single_layout(M, N, K).total;
 }
 
-bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K, float eps, void *packed,
-                                            float *gamma, void *stream)
+namespace {
+bitlinear_status quantize_weights_impl(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
+                                       void *stream, bool trits)
 {
     if (!W || !packed || !gamma || !(eps >= 0.0f)) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(0, N, K);
     if (st != BITLINEAR_OK) return st;
     if (!aligned(W, 16) || !aligned(packed, 16) || !aligned(gamma, 4)) return BITLINEAR_ERR_ALIGN;
     if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
-    cudaError_t err = launch_absmean_and_pack(W, N, K, eps, packed, gamma, (cudaStream_t)stream);
+    cudaError_t err = launch_absmean_and_pack(W, N, K, eps, packed, gamma, (cudaStream_t)stream, trits);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+} // namespace
+
+bitlinear_status bitlinear_quantize_weights(const float *W, int64_t N, int64_t K, float eps, void *packed,
+                                            float *gamma, void *stream)
+{
+    return quantize_weights_impl(W, N, K, eps, packed, gamma, stream, false);
+}
+
+bitlinear_status bitlinear_quantize_weights_trits(const float *W, int64_t N, int64_t K, float eps, void *packed,
+                                                  float *gamma, void *stream)
+{
+    return quantize_weights_impl(W, N, K, eps, packed, gamma, stream, true);
 }
 
 namespace {
@@ -295,7 +317,7 @@ bitlinear_status bitlinear_swiglu_quantize_acts(const void *gate, const void *up
 namespace {
 bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const void *up, const float *gain,
                               float norm_eps, int act_bits, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
-                              size_t workspace_bytes, void *stream);
+                              size_t workspace_bytes, void *stream, bool trits = false);
 }
 
 bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
@@ -322,6 +344,12 @@ bitlinear_status bitlinear_forward_swiglu(const void *packed, const float *gamma
     return forward_impl(packed, gamma, gate, up, nullptr, 0.0f, 8, M, K, N, Y, workspace, workspace_bytes, stream);
 }
 
+bitlinear_status bitlinear_forward_trits(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
+                                         int64_t N, void *Y, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return forward_impl(packed, gamma, X, nullptr, nullptr, 0.0f, 8, M, K, N, Y, workspace, workspace_bytes, stream, true);
+}
+
 bitlinear_status bitlinear_forward_act_bits(const void *packed, const float *gamma, const void *X, int64_t M, int64_t K,
                                             int64_t N, int act_bits, void *Y, void *workspace, size_t workspace_bytes,
                                             void *stream)
@@ -333,9 +361,10 @@ namespace {
 // gain == null: no normalisation in front of the quantiser; up != null: X is the gate of a SwiGLU in front of it
 bitlinear_status forward_impl(const void *packed, const float *gamma, const void *X, const void *up, const float *gain,
                               float norm_eps, int act_bits, int64_t M, int64_t K, int64_t N, void *Y, void *workspace,
-                              size_t workspace_bytes, void *stream)
+                              size_t workspace_bytes, void *stream, bool trits)
 {
     if (act_bits < 2 || act_bits > 8) return BITLINEAR_ERR_ARG;
+    if (trits && M > kMaxTritM) return BITLINEAR_ERR_SHAPE;
     if (!packed || !gamma || !workspace || (M > 0 && (!X || !Y))) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(M, N, K);
     if (st != BITLINEAR_OK) return st;
@@ -347,8 +376,8 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     if (M == 0) return BITLINEAR_OK;
     char *ws = reinterpret_cast<char *>(workspace);
     InlineTable inl{};
-    fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L);
-    const bool tc = use_tcgen05_for(M);
+    fill_entry(inl.e[0], packed, gamma, X, M, K, N, Y, 0, ws, L, trits);
+    const bool tc = !trits && use_tcgen05_for(M);
     inl.e[0].xq_tiled = tc ? 0 : 1;
     inl.e[0].gain = gain;
     inl.e[0].norm_eps = norm_eps;
@@ -362,12 +391,31 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
                                            (cudaStream_t)stream);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return run_matmul(inl.e[0], BITLINEAR_PATH_AUTO, ws, L.lists, M < kMinGemmRows ? kMinGemmRows : M,
-                      split ? ws + L.acc32 : nullptr, (cudaStream_t)stream);
+                      split ? ws + L.acc32 : nullptr, (cudaStream_t)stream, trits);
 }
 } // namespace
 
+namespace {
+bitlinear_status matmul_i32_impl(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N, int32_t *acc,
+                                 int path, void *workspace, size_t workspace_bytes, void *stream, bool trits);
+}
+
 bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
                                       int32_t *acc, int path, void *workspace, size_t workspace_bytes, void *stream)
+{
+    return matmul_i32_impl(packed, Xq, M, K, N, acc, path, workspace, workspace_bytes, stream, false);
+}
+
+bitlinear_status bitlinear_matmul_i32_trits(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N,
+                                            int32_t *acc, void *workspace, size_t workspace_bytes, void *stream)
+{
+    if (M > kMaxTritM) return BITLINEAR_ERR_SHAPE;
+    return matmul_i32_impl(packed, Xq, M, K, N, acc, BITLINEAR_PATH_MMA, workspace, workspace_bytes, stream, true);
+}
+
+namespace {
+bitlinear_status matmul_i32_impl(const void *packed, const int8_t *Xq, int64_t M, int64_t K, int64_t N, int32_t *acc,
+                                 int path, void *workspace, size_t workspace_bytes, void *stream, bool trits)
 {
     if (!packed || !workspace || (M > 0 && (!Xq || !acc))) return BITLINEAR_ERR_ARG;
     if (path < BITLINEAR_PATH_AUTO || path > BITLINEAR_PATH_TCGEN05) return BITLINEAR_ERR_ARG;
@@ -383,9 +431,9 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     if (M == 0) return BITLINEAR_OK;
     char *ws = reinterpret_cast<char *>(workspace);
     cudaStream_t s = (cudaStream_t)stream;
-    const bool tc = (path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M));
+    const bool tc = !trits && ((path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M)));
     InlineTable inl{};
-    fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L);
+    fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L, trits);
     const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M)) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
@@ -399,18 +447,31 @@ bitlinear_status bitlinear_matmul_i32(const void *packed, const int8_t *Xq, int6
     }
     rowsum_kernel<<<(unsigned)M, 256, 0, s>>>(Xq, (int)K, inl.e[0].rowsum);
     if (cudaGetLastError() != cudaSuccess) return BITLINEAR_ERR_CUDA;
-    return run_matmul(inl.e[0], path, ws, L.lists, M, split ? ws + L.acc32 : nullptr, s); // (the caller's rows: exactly M)
+    return run_matmul(inl.e[0], path, ws, L.lists, M, split ? ws + L.acc32 : nullptr, s, trits); // (the caller's rows: exactly M)
 }
+} // namespace
 
-bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)
+namespace {
+bitlinear_status unpack_impl(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream, bool trits)
 {
     if (!packed || !T) return BITLINEAR_ERR_ARG;
     bitlinear_status st = check_shape(0, N, K);
     if (st != BITLINEAR_OK) return st;
     if (!aligned(packed, 16)) return BITLINEAR_ERR_ALIGN;
     if (!device_is_sm100()) return BITLINEAR_ERR_ARCH;
-    cudaError_t err = launch_unpack(packed, N, K, T, (cudaStream_t)stream);
+    cudaError_t err = launch_unpack(packed, N, K, T, (cudaStream_t)stream, trits);
     return err == cudaSuccess ? BITLINEAR_OK : BITLINEAR_ERR_CUDA;
+}
+} // namespace
+
+bitlinear_status bitlinear_unpack_weights(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)
+{
+    return unpack_impl(packed, N, K, T, stream, false);
+}
+
+bitlinear_status bitlinear_unpack_weights_trits(const void *packed, int64_t N, int64_t K, int8_t *T, void *stream)
+{
+    return unpack_impl(packed, N, K, T, stream, true);
 }
 
 bitlinear_status bitlinear_validate_packed(const void *packed, int64_t N, int64_t K, int32_t *bad_fields, void *stream)
@@ -506,6 +567,7 @@ struct bitlinear_sequence {
     int64_t gemm_total_kb;
     int fronts;             // bit 0: some entry has an RMSNorm in front of the quantiser, bit 1: some entry a SwiGLU
     void *split_scratch;    // inside the workspace; null: the GEMM deals this sequence's tiles whole
+    bool trits;             // the weights are in the base-3 format
 };
 
 namespace {
@@ -578,13 +640,22 @@ size_t bitlinear_sequence_workspace_bytes(const bitlinear_layer_desc *layers, in
 namespace {
 bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains,
                                       const void *const *ups, float norm_eps, int n, void *workspace,
-                                      size_t workspace_bytes, bitlinear_sequence **out);
+                                      size_t workspace_bytes, bitlinear_sequence **out, bool trits = false);
 }
 
 bitlinear_status bitlinear_sequence_create(const bitlinear_layer_desc *layers, int n, void *workspace,
                                            size_t workspace_bytes, bitlinear_sequence **out)
 {
     return sequence_create_impl(layers, nullptr, nullptr, 0.0f, n, workspace, workspace_bytes, out);
+}
+
+bitlinear_status bitlinear_sequence_create_trits(const bitlinear_layer_desc *layers, int n, void *workspace,
+                                                 size_t workspace_bytes, bitlinear_sequence **out)
+{
+    if (!layers || n <= 0) return BITLINEAR_ERR_ARG;
+    for (int i = 0; i < n; ++i)
+        if (layers[i].M > kMaxTritM) return BITLINEAR_ERR_SHAPE;
+    return sequence_create_impl(layers, nullptr, nullptr, 0.0f, n, workspace, workspace_bytes, out, true);
 }
 
 bitlinear_status bitlinear_sequence_create_rmsnorm(const bitlinear_layer_desc *layers, const float *const *gains,
@@ -613,7 +684,7 @@ namespace {
 // gains == null: no entry is normalised; gains[i] == null: entry i is not; ups likewise (SwiGLU in front)
 bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const float *const *gains,
                                       const void *const *ups, float norm_eps, int n, void *workspace,
-                                      size_t workspace_bytes, bitlinear_sequence **out)
+                                      size_t workspace_bytes, bitlinear_sequence **out, bool trits)
 {
     if (!layers || !workspace || !out || n <= 0) return BITLINEAR_ERR_ARG;
     *out = nullptr;
@@ -652,7 +723,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
         L.rowsum = L.beta + align_up((size_t)d.M * 4, 256);
         if (!gemm) a_off += align_up((size_t)d.M * d.N * 4, 256);
         DecodeEntry &e = table[(size_t)i];
-        fill_entry(e, d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L);
+        fill_entry(e, d.packed, d.gamma, d.X, d.M, d.K, d.N, d.Y, 0, ws, L, trits);
         e.xq_tiled = gemm ? 0 : 1;
         e.gain = gains ? gains[i] : nullptr;
         e.norm_eps = norm_eps;
@@ -691,6 +762,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     seq->gemm_tiles = gemm_tiles;
     seq->gemm_total_kb = gemm_kb;
     seq->fronts = fronts;
+    seq->trits = trits;
     seq->split_scratch = split ? ws + S.acc32 : nullptr;
     if (gemm) {
         if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -728,7 +800,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
             seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->gemm_total_kb, seq->max_M,
                                                  seq->split_scratch, s)
                             : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
-                                            reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s);
+                                            reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s, seq->trits);
         if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
     return BITLINEAR_OK;

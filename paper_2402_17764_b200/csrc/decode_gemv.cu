@@ -41,6 +41,12 @@
 // block.  Because codes are T + 1, the per-token sum of q is subtracted once at the end.
 //
 // Roofline: HBM.  Algorithmic bytes = N*K/4 per matrix (activations and outputs are < 0.1 % at M = 1).
+//
+// The same kernel streams the base-3 format (five weights per byte, tiles of 80 rows: N*K/5 bytes per matrix).  A
+// stored byte is then a number 0..242 and has to be decoded: a table in shared memory (243 entries, one copy per lane
+// so that a warp's look-ups never share a bank) turns it into the byte of four 2-bit fields the MMAs above take (rows
+// 16 f + r, f = 0..3) plus the code of the fifth row (64 + r), which feeds a fifth MMA as it is.  One look-up per
+// stored byte is what this format costs: about 19 instructions per 20 weights where the 2-bit fields cost 3 per 16.
 #include <cstdlib>
 
 #include "internal.cuh"
@@ -79,7 +85,13 @@ struct Ring {
     static constexpr int kAbortOffset = kBarsOffset + kWarps * kStages * 8;
     static constexpr int kSmem = kAbortOffset + 16;
     static_assert(kSmem * (NT <= 2 ? kCtasPerSm : 1) <= 227 * 1024, "ring does not fit the SM's shared memory");
+    // base-3 format: the decoding table behind the ring, entry v of lane l at 128 v + 4 l
+    static constexpr int kLutOffset = (kSmem + 127) / 128 * 128;
+    static constexpr int kLutBytes = 243 * 128;
+    static constexpr int kSmemTrits = kLutOffset + kLutBytes;
+    static_assert(NT != 1 || kSmemTrits <= 227 * 1024, "ring and table do not fit the SM's shared memory");
 };
+constexpr int kTritRows = 80; // rows of a tile of the base-3 format
 #ifndef BITLINEAR_DECODE_STATIC_PERCENT
 #define BITLINEAR_DECODE_STATIC_PERCENT 80
 #endif
@@ -182,31 +194,34 @@ __device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete
 // costs two memory round trips per batch and token group rather than two per row block and token.
 // `word` is the lane's 32-bit word of the warp's 128-byte list (one load for the count and all items: every round
 // trip of this launch is on the critical path of the step): word 0 the count, words 2 i + 2 and 2 i + 3 item i.
-template <int TG> // tokens handled together: 1 (single-token steps), or 4
+template <int TG, int ROWS> // tokens handled together: 1 (single-token steps), or 4; rows of a row block: 64, or 80
 __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint32_t word, int n_owned, int lane)
 {
     constexpr int kBatch = 4;
+    constexpr int kParts = (ROWS + 31) / 32; // rows per lane
     for (int b0 = 0; b0 < n_owned; b0 += kBatch) {
         const DecodeEntry *e[kBatch];
         int32_t *acc[kBatch];
-        int r0[kBatch], N[kBatch], M[kBatch], max_M = 0;
+        int r0[kBatch], rend[kBatch], N[kBatch], M[kBatch], max_M = 0;
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             const int item = min(b0 + b, n_owned - 1); // slots past the end repeat the last one and store nothing
             const uint2 o = make_uint2(__shfl_sync(0xffffffffu, word, 2 * item + 2), __shfl_sync(0xffffffffu, word, 2 * item + 3));
             e[b] = tab + o.x;
-            r0[b] = (int)o.y * kTileRows + lane;
+            r0[b] = (int)o.y * ROWS + lane;
+            rend[b] = ((int)o.y + 1) * ROWS;
         }
 #pragma unroll
         for (int b = 0; b < kBatch; ++b) {
             acc[b] = e[b]->acc32;
             N[b] = (b0 + b < n_owned) ? e[b]->N : 0;
+            rend[b] = min(rend[b], N[b]); // rows of this row block that exist
             M[b] = e[b]->M;
             if (N[b] > 0) max_M = max(max_M, M[b]);
         }
         // TG tokens of every row block of the batch at a time: all loads first, then all stores
         for (int t0 = 0; t0 < max_M; t0 += TG) {
-            int v[kBatch][TG][kTileRows / 32], rowsum[kBatch][TG];
+            int v[kBatch][TG][kParts], rowsum[kBatch][TG];
             float scale[kBatch][TG];
 #pragma unroll
             for (int b = 0; b < kBatch; ++b) {
@@ -214,8 +229,8 @@ __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint
                 for (int i = 0; i < TG; ++i) {
                     const int t = min(t0 + i, M[b] - 1); // slots past the last token repeat it and store nothing
 #pragma unroll
-                    for (int h = 0; h < kTileRows / 32; ++h)
-                        v[b][i][h] = (r0[b] + 32 * h < N[b]) ? __ldcg(acc[b] + (size_t)t * N[b] + r0[b] + 32 * h) : 0;
+                    for (int h = 0; h < kParts; ++h)
+                        v[b][i][h] = (r0[b] + 32 * h < rend[b]) ? __ldcg(acc[b] + (size_t)t * N[b] + r0[b] + 32 * h) : 0;
                     rowsum[b][i] = e[b]->rowsum[t];
                     scale[b][i] = token_scale(*e[b], t);
                 }
@@ -227,9 +242,9 @@ __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint
                     const int t = t0 + i;
                     if (t >= M[b]) continue;
 #pragma unroll
-                    for (int h = 0; h < kTileRows / 32; ++h) {
+                    for (int h = 0; h < kParts; ++h) {
                         const int r = r0[b] + 32 * h;
-                        if (r < N[b]) {
+                        if (r < rend[b]) {
                             __stcg(acc[b] + (size_t)t * N[b] + r, 0);
                             store_result(*e[b], t, r, v[b][i][h], rowsum[b][i], scale[b][i]);
                         }
@@ -259,10 +274,40 @@ __device__ __forceinline__ void mma_slab(int (&acc)[4][4], const uint4 &w, uint3
 }
 
 
+// Base-3 format: the four words of a lane's 16 bytes go through the table (entry: bits 0..7 the byte of four 2-bit
+// fields, bits 8..9 the fifth code), then four MMAs on the fields as above and a fifth on the fifth codes.
+__device__ __forceinline__ void decode_word(uint32_t w, uint32_t lut_lane, uint32_t &fields, uint32_t &fifth)
+{
+    uint32_t e[4];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint32_t v = __byte_perm(w, 0u, 0x4440u + i); // byte i, zero-extended
+        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(e[i]) : "r"(lut_lane + v * 128u));
+    }
+    const uint32_t t01 = __byte_perm(e[0], e[1], 0x5140u), t23 = __byte_perm(e[2], e[3], 0x5140u);
+    fields = __byte_perm(t01, t23, 0x5410u);
+    fifth = __byte_perm(t01, t23, 0x7632u);
+}
+
+__device__ __forceinline__ void mma_slab_trits(int (&acc)[5][4], const uint4 &stored, uint32_t lut_lane, uint32_t b0, uint32_t b1)
+{
+    uint4 w, f;
+    decode_word(stored.x, lut_lane, w.x, f.x);
+    decode_word(stored.y, lut_lane, w.y, f.y);
+    decode_word(stored.z, lut_lane, w.z, f.z);
+    decode_word(stored.w, lut_lane, w.w, f.w);
+    mma_u8s8(acc[0], w.x, w.y, w.z, w.w, b0, b1);
+    mma_u8s8(acc[1], w.x & 0xFCFCFCFCu, w.y & 0xFCFCFCFCu, w.z & 0xFCFCFCFCu, w.w & 0xFCFCFCFCu, b0, b1);
+    mma_u8s8(acc[2], w.x & 0xF0F0F0F0u, w.y & 0xF0F0F0F0u, w.z & 0xF0F0F0F0u, w.w & 0xF0F0F0F0u, b0, b1);
+    mma_u8s8(acc[3], w.x & 0xC0C0C0C0u, w.y & 0xC0C0C0C0u, w.z & 0xC0C0C0C0u, w.w & 0xC0C0C0C0u, b0, b1);
+    mma_u8s8(acc[4], f.x, f.y, f.z, f.w, b0, b1);
+}
+
 // Un-mixes the four scaled accumulators of every (row, token) this lane holds and hands the row sums to fn.
 // C fragment of field f: c0 (row 16f + g, token 2tq), c1 (same row, 2tq + 1), c2 (row 16f + 8 + g, 2tq), c3.
-template <int NT, class Begin, class Fn>
-__device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, int N, int row0, int tq, Begin begin, Fn fn)
+// NF = 5: the base-3 format's fifth accumulator holds the sums of rows 64 + r as they are.
+template <int NT, int NF, class Begin, class Fn>
+__device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, int N, int row0, int tq, Begin begin, Fn fn)
 {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -277,9 +322,9 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, i
                 const int t1 = acc[nt][1][c] >> 2; // S1 + 4 S2 + 16 S3   (exact shifts)
                 const int t2 = acc[nt][2][c] >> 4; // S2 + 4 S3
                 const int t3 = acc[nt][3][c] >> 6; // S3
-                const int S[4] = {acc[nt][0][c] - 4 * t1, t1 - 4 * t2, t2 - 4 * t3, t3};
+                const int S[5] = {acc[nt][0][c] - 4 * t1, t1 - 4 * t2, t2 - 4 * t3, t3, acc[nt][NF - 1][c]};
 #pragma unroll
-                for (int f = 0; f < 4; ++f) {
+                for (int f = 0; f < NF; ++f) {
                     const int r = row0 + 16 * f + 8 * h;
                     if (r < N) fn(terms, token, r, S[f]);
                 }
@@ -288,7 +333,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][4][4], int M, i
     }
 }
 
-template <int NT>
+template <int NT, bool kTrits>
 __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
     uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr, OwnedList *lists, const WaitHooks hooks)
@@ -305,6 +350,17 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     int n_owned = 0;
     volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + R::kAbortOffset);
 
+    constexpr int kFields = kTrits ? 5 : 4, kRows = kTrits ? kTritRows : kTileRows;
+    const uint32_t lut_lane = ptx::smem_u32(dsmem + R::kLutOffset) + lane * 4;
+    if (kTrits) {
+        // entry v of every lane's copy: the byte of four 2-bit fields c0 + 4 c1 + 16 c2 + 64 c3, and c4 << 8
+        uint32_t *lut = reinterpret_cast<uint32_t *>(dsmem + R::kLutOffset);
+        for (int v = threadIdx.x; v < 243; v += kWarps * 32) {
+            const uint32_t c0 = v % 3, c1 = (v / 3) % 3, c2 = (v / 9) % 3, c3 = (v / 27) % 3, c4 = v / 81;
+            const uint32_t entry = c0 | (c1 << 2) | (c2 << 4) | (c3 << 6) | (c4 << 8);
+            for (int l = 0; l < 32; ++l) lut[v * 32 + l] = entry;
+        }
+    }
     if (threadIdx.x == 0) *abort_flag = 0;
     if (lane == 0) {
         // two arrivals per phase: one announces the weight bytes of a chunk, one its activation bytes
@@ -497,12 +553,12 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
         }
         // ---- one row block (or the part of it that lies in this piece)
         const int M = e->M;
-        int acc[NT][4][4]; // [token tile][field][C fragment]
+        int acc[NT][kFields][4]; // [token tile][field][C fragment]
         uint32_t xlane[NT]; // offset of this lane's B-fragment token (lanes without a token read the last one) and columns
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt) {
 #pragma unroll
-            for (int f = 0; f < 4; ++f) acc[nt][f][0] = acc[nt][f][1] = acc[nt][f][2] = acc[nt][f][3] = 0;
+            for (int f = 0; f < kFields; ++f) acc[nt][f][0] = acc[nt][f][1] = acc[nt][f][2] = acc[nt][f][3] = 0;
             xlane[nt] = (uint32_t)(R::kWeightBytes + min(8 * nt + g, M - 1) * kXTileBytes + 16 * tq);
         }
         const uint32_t xtile = (uint32_t)(M * kXTileBytes); // activation bytes per column tile in the slot
@@ -521,8 +577,13 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 #pragma unroll
                     for (int nt = 0; nt < NT; ++nt) {
                         const uint4 x = lds128(slot + t * xtile + xlane[nt]);
-                        mma_slab(acc[nt], w0, x.x, x.y);
-                        mma_slab(acc[nt], w1, x.z, x.w);
+                        if constexpr (kTrits) {
+                            mma_slab_trits(acc[nt], w0, lut_lane, x.x, x.y);
+                            mma_slab_trits(acc[nt], w1, lut_lane, x.z, x.w);
+                        } else {
+                            mma_slab(acc[nt], w0, x.x, x.y);
+                            mma_slab(acc[nt], w1, x.z, x.w);
+                        }
                     }
                 }
             } else {
@@ -534,8 +595,13 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 #pragma unroll
                         for (int nt = 0; nt < NT; ++nt) {
                             const uint4 x = lds128(slot + t * xtile + xlane[nt]);
-                            mma_slab(acc[nt], w0, x.x, x.y);
-                            mma_slab(acc[nt], w1, x.z, x.w);
+                            if constexpr (kTrits) {
+                                mma_slab_trits(acc[nt], w0, lut_lane, x.x, x.y);
+                                mma_slab_trits(acc[nt], w1, lut_lane, x.z, x.w);
+                            } else {
+                                mma_slab(acc[nt], w0, x.x, x.y);
+                                mma_slab(acc[nt], w1, x.z, x.w);
+                            }
                         }
                     }
                 }
@@ -556,7 +622,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             if (lane == 0) owned[n_owned] = make_uint2((uint32_t)(e - tab), (uint32_t)rb);
             ++n_owned; // cannot exceed kMaxOwned: see next_piece
         }
-        finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, begin, fn); });
+        finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT, kFields>(acc, M, e->N, rb * kRows + g, tq, begin, fn); });
 
         // next row block, or next matrix
         if (kt == KB) {
@@ -809,7 +875,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
                     ++n_owned;
                 }
             }
-            finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT>(acc, M, e->N, rb * kTileRows + g, tq, begin, fn); });
+            finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT, 4>(acc, M, e->N, rb * kTileRows + g, tq, begin, fn); });
         }
     }
     }();
@@ -828,7 +894,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
 __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constant__ InlineTable inl,
                                                             const DecodeEntry *__restrict__ table,
                                                             const OwnedList *__restrict__ lists, uint32_t n_lists,
-                                                            int staged_entries, int single_token)
+                                                            int staged_entries, int single_token, int trits)
 {
     extern __shared__ uint4 staged_table[];
     const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -848,10 +914,17 @@ __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constan
     const uint32_t word = __ldcg(reinterpret_cast<const uint32_t *>(&lists[w]) + lane);
     const int n = (int)__shfl_sync(0xffffffffu, word, 0);
     if (n == 0) return;
-    if (single_token)
-        finish_owned_blocks<1>(table ? table : inl.e, word, n, lane);
-    else
-        finish_owned_blocks<4>(table ? table : inl.e, word, n, lane);
+    const DecodeEntry *tab = table ? table : inl.e;
+    if (trits) {
+        if (single_token)
+            finish_owned_blocks<1, kTritRows>(tab, word, n, lane);
+        else
+            finish_owned_blocks<4, kTritRows>(tab, word, n, lane);
+    } else if (single_token) {
+        finish_owned_blocks<1, kTileRows>(tab, word, n, lane);
+    } else {
+        finish_owned_blocks<4, kTileRows>(tab, word, n, lane);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -944,30 +1017,34 @@ static cudaError_t launch_dependent(const void *kernel, dim3 grid, dim3 block, s
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
-template <int NT>
+template <int NT, bool kTrits>
 static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, const DecodeEntry *table, int n_entries,
                               uint32_t total_tiles, uint32_t share, uint32_t dyn, int max_M, WorkspaceHeader *hdr,
                               OwnedList *lists, cudaStream_t stream)
 {
     WaitHooks hooks = take_wait_hooks();
     int single_token = max_M == 1 ? 1 : 0;
+    int trits = kTrits ? 1 : 0;
+    constexpr int kSmemBytes = kTrits ? Ring<NT>::kSmemTrits : Ring<NT>::kSmem;
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, Ring<NT>::kSmem);
+        cudaError_t e = cudaFuncSetAttribute(decode_mma_kernel<NT, kTrits>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
         if (e != cudaSuccess) return e;
         attr_set[dev] = true;
     }
     static const bool early = tuning_from_env("BITLINEAR_DECODE_EARLY_LAUNCH", 1, 2) == 1; // 2 = off
     void *args[] = {(void *)&inl, (void *)&table, (void *)&n_entries, (void *)&total_tiles, (void *)&share,
                     (void *)&dyn, (void *)&hdr, (void *)&lists, (void *)&hooks};
-    cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT>, grid, block, Ring<NT>::kSmem, args, early, stream);
+    cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT, kTrits>, grid, block, kSmemBytes, args, early, stream);
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
     // a table that fits beside the matmul's ring (one CTA of each per SM) is staged in the finishing CTAs' shared memory
-    int staged = (table && (size_t)n_entries * sizeof(DecodeEntry) <= kStagedTableBytes) ? n_entries : 0;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token};
+    // (the base-3 form's decoding table takes that room: its finishing CTAs read the table from global memory)
+    int staged = (!kTrits && table && (size_t)n_entries * sizeof(DecodeEntry) <= kStagedTableBytes) ? n_entries : 0;
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token,
+                     (void *)&trits};
     return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256),
                             (size_t)staged * sizeof(DecodeEntry), fargs, early, stream);
 }
@@ -993,15 +1070,17 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * kWarps;
     int staged = 0; // (this kernel's rings leave no room beside them)
-    int single_token = 0;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token};
+    int single_token = 0, trits = 0;
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token,
+                     (void *)&trits};
     return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
 }
 
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
-                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream)
+                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream, bool trits)
 {
     if (total_tiles == 0) return cudaSuccess;
+    if (trits && (max_M > 8 || path == BITLINEAR_PATH_DP4A)) return cudaErrorInvalidValue;
     const dim3 block(kWarps * 32);
     if (path != BITLINEAR_PATH_DP4A && decode_is_wide(max_M)) {
         // total_tiles counts group tiles here; one CTA per SM, equal contiguous shares, at least 4 items each
@@ -1044,7 +1123,8 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     } else {
         share = (total_tiles + n_warps - 1) / n_warps; // all static: the last warps may get less, or nothing
     }
-    return launch_mma<1>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
+    if (trits) return launch_mma<1, true>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
+    return launch_mma<1, false>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
 }
 
 } // namespace bitlinear

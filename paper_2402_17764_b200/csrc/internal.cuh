@@ -50,7 +50,7 @@ struct DecodeEntry {
     void *out;             // bf16 [M, N], or int32 [M, N] when out_i32
     int32_t *acc32;        // scratch [M, N] for row blocks shared by several warps (zero before and after a launch)
     int M, N, K;
-    int KB, NB;            // column tiles = ceil(K / 64), row blocks = ceil(N / 64)
+    int KB, NB;            // column tiles = ceil(K / 64), row blocks = ceil(N / 64) (base-3 format: ceil(N / 80))
     uint32_t tile_begin;   // index of this entry's first work item in the launch-wide sequence: tiles (NB * KB per
                            // entry) for up to 8 tokens, group tiles (ceil(NB / 8) * KB per entry) beyond: see below
     int token_begin;       // first token of this entry in the batched quantiser's grid
@@ -71,9 +71,10 @@ static inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; 
 
 // ---- kernel launchers (host side, each defined next to its kernel) ----
 
+// trits: the base-3 format (five weights per byte, tiles of 80 rows) instead of 2-bit codes
 cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
-                                    cudaStream_t stream);
-cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream);
+                                    cudaStream_t stream, bool trits = false);
+cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream, bool trits = false);
 // *bad (device) = number of 2-bit fields among the `bytes` bytes of a packed buffer that hold the unused code 3.
 cudaError_t launch_count_bad_codes(const void *packed, size_t bytes, int32_t *bad, cudaStream_t stream);
 // Copies row-major int8 activations [M, K] into the tiled layout [KB][M][64] (columns >= K become 0).
@@ -94,8 +95,10 @@ inline uint32_t decode_items(int NB, int KB, bool wide) { return (uint32_t)(wide
 // Persistent weight-streaming matmul over the entries (total_tiles = sum of decode_items over the entries).
 // path: BITLINEAR_PATH_MMA, or BITLINEAR_PATH_DP4A (first entry only).
 // `lists` is scratch of kOwnedListsBytes (no need to clear it).
+// trits: the entries' weights are in the base-3 format (five per byte, row blocks of 80 rows: NB = ceil(N / 80)); at
+// most 8 tokens then.
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
-                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream);
+                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream, bool trits = false);
 
 // Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) (by gamma * beta_t / qb) or raw int32.  x_rows >= M rows of K bytes exist behind
 // Xq; the rows past M may hold anything (they only reach accumulator rows that are never stored).

@@ -120,6 +120,69 @@ __global__ void __launch_bounds__(256) ternarize_pack_kernel(const float *__rest
     }
 }
 
+// The same for the base-3 format: one warp per tile of 80 rows x 64 columns (still 1 KiB).  The byte positions are
+// those above; a byte holds the codes of the FIVE rows 16 f + 8 h + g, f = 0..4, as the number sum_f 3^f code_f.
+__global__ void __launch_bounds__(256) ternarize_pack_trits_kernel(const float *__restrict__ W, int N, int K, int NB, int KB,
+                                                                   float eps, const float *__restrict__ gamma,
+                                                                   uint4 *__restrict__ packed)
+{
+    const long long n_tiles = (long long)NB * KB;
+    const int lane = threadIdx.x & 31;
+    const int g = lane >> 2, tq = lane & 3;
+    const float denom = __fadd_rn(*gamma, eps); // Eq. 1: gamma + eps
+    for (long long tile = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); tile < n_tiles;
+         tile += (long long)gridDim.x * (blockDim.x >> 5)) {
+        const int rb = (int)(tile / KB), kb = (int)(tile % KB);
+        uint32_t words[2][4] = {{0u, 0u, 0u, 0u}, {0u, 0u, 0u, 0u}};
+        const int col0 = kb * kTileCols + 16 * tq;
+        uint32_t weight = 1u; // 3^f
+#pragma unroll
+        for (int f = 0; f < 5; ++f) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int n = rb * 80 + 16 * f + 8 * h + g;
+                const float *row = W + (size_t)n * K;
+#pragma unroll
+                for (int v = 0; v < 4; ++v) { // four float4 = 16 columns; v = 2 s + hi
+                    const int col = col0 + 4 * v;
+                    uint32_t codes = 0x01010101u; // padding: weight 0
+                    if (n < N && col < K) {
+                        float4 w = __ldg(reinterpret_cast<const float4 *>(row + col));
+                        const float x[4] = {w.x, w.y, w.z, w.w};
+                        codes = 0;
+#pragma unroll
+                        for (int b = 0; b < 4; ++b) {
+                            int t = __float2int_rn(__fdiv_rn(x[b], denom)); // round half to even (Eq. 2)
+                            t = max(-1, min(1, t));
+                            codes |= (uint32_t)(t + 1) << (8 * b);
+                        }
+                    }
+                    words[v >> 1][2 * (v & 1) + h] += codes * weight; // (no byte exceeds 242: no carry between bytes)
+                }
+            }
+            weight *= 3u;
+        }
+        packed[tile * 64 + lane] = make_uint4(words[0][0], words[0][1], words[0][2], words[0][3]);
+        packed[tile * 64 + 32 + lane] = make_uint4(words[1][0], words[1][1], words[1][2], words[1][3]);
+    }
+}
+
+__global__ void __launch_bounds__(256) unpack_trits_kernel(const uint8_t *__restrict__ packed, int N, int K, int KB,
+                                                           int8_t *__restrict__ T)
+{
+    const size_t total = (size_t)N * K;
+    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const int n = (int)(idx / K), k = (int)(idx % K);
+        const size_t tile = (size_t)(n / 80) * KB + k / kTileCols;
+        const int r = n % 80, c = k % kTileCols;
+        const int f = r / 16, h = (r % 16) / 8, g = r % 8;
+        const int tq = c / 16, s = (c % 16) / 8, hi = (c % 8) / 4, b = c % 4;
+        int v = packed[tile * kTileBytes + s * 512 + (4 * g + tq) * 16 + 4 * (2 * hi + h) + b];
+        for (int i = 0; i < f; ++i) v /= 3;
+        T[idx] = (int8_t)(v % 3 - 1);
+    }
+}
+
 __global__ void __launch_bounds__(256) unpack_kernel(const uint8_t *__restrict__ packed, int N, int K, int KB,
                                                      int8_t *__restrict__ T)
 {
@@ -165,7 +228,7 @@ cudaError_t launch_count_bad_codes(const void *packed, size_t bytes, int32_t *ba
 }
 
 cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float eps, void *packed, float *gamma,
-                                    cudaStream_t stream)
+                                    cudaStream_t stream, bool trits)
 {
     cudaError_t err = cudaMemsetAsync(packed, 0, 32, stream);
     if (err != cudaSuccess) return err;
@@ -178,22 +241,29 @@ cudaError_t launch_absmean_and_pack(const float *W, int64_t N, int64_t K, float 
     err = cudaGetLastError();
     if (err != cudaSuccess) return err;
     const int KB = (int)((K + kTileCols - 1) / kTileCols);
-    const int NB = (int)((N + kTileRows - 1) / kTileRows);
+    const int NB = trits ? (int)((N + 79) / 80) : (int)((N + kTileRows - 1) / kTileRows);
     const long long n_tiles = (long long)NB * KB;
     long long pblocks = (n_tiles + 7) / 8;
     if (pblocks > (long long)sm_count() * 16) pblocks = (long long)sm_count() * 16;
-    ternarize_pack_kernel<<<(int)pblocks, 256, 0, stream>>>(W, (int)N, (int)K, NB, KB, eps, gamma,
-                                                            reinterpret_cast<uint4 *>(packed));
+    if (trits)
+        ternarize_pack_trits_kernel<<<(int)pblocks, 256, 0, stream>>>(W, (int)N, (int)K, NB, KB, eps, gamma,
+                                                                      reinterpret_cast<uint4 *>(packed));
+    else
+        ternarize_pack_kernel<<<(int)pblocks, 256, 0, stream>>>(W, (int)N, (int)K, NB, KB, eps, gamma,
+                                                                reinterpret_cast<uint4 *>(packed));
     return cudaGetLastError();
 }
 
-cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream)
+cudaError_t launch_unpack(const void *packed, int64_t N, int64_t K, int8_t *T, cudaStream_t stream, bool trits)
 {
     const int KB = (int)((K + kTileCols - 1) / kTileCols);
     size_t total = (size_t)N * K;
     size_t blocks = (total + 255) / 256;
     if (blocks > (size_t)sm_count() * 32) blocks = (size_t)sm_count() * 32;
-    unpack_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint8_t *>(packed), (int)N, (int)K, KB, T);
+    if (trits)
+        unpack_trits_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint8_t *>(packed), (int)N, (int)K, KB, T);
+    else
+        unpack_kernel<<<(int)blocks, 256, 0, stream>>>(reinterpret_cast<const uint8_t *>(packed), (int)N, (int)K, KB, T);
     return cudaGetLastError();
 }
 
