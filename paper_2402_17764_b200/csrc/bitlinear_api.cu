@@ -181,7 +181,7 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
     InlineTable inl{};
     inl.e[0] = e;
-    cudaError_t err = launch_decode(inl, nullptr, 1, decode_items(e.NB, e.KB, decode_is_wide(e.M)), e.M,
+    cudaError_t err = launch_decode(inl, nullptr, 1, decode_items(e.NB, e.KB, e.M), e.M,
                                     path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream, trits);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;
@@ -708,7 +708,6 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     int tokens = 0, max_M = 0;
     for (int i = 0; i < n; ++i)
         if ((int)layers[i].M > max_M) max_M = (int)layers[i].M;
-    const bool wide = decode_is_wide(max_M); // one kernel serves the whole sequence
     const bool gemm = S.use_gemm;
     std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
     int gemm_tiles = 0;
@@ -731,7 +730,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
         fronts |= (e.gain ? 1 : 0) | (e.up ? 2 : 0);
         e.tile_begin = tiles;
         e.token_begin = tokens;
-        tiles += decode_items(e.NB, e.KB, wide);
+        tiles += decode_items(e.NB, e.KB, max_M); // (one kernel serves the whole sequence)
         tokens += (int)d.M;
         if (gemm) {
             int nt = 0;

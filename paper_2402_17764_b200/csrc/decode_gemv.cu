@@ -315,7 +315,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, 
         for (int tb = 0; tb < 2; ++tb) {
             const int token = 8 * nt + 2 * tq + tb;
             if (token >= M) continue;
-            const auto terms = begin(token);
+            const auto terms = begin(token); // (fetching the terms of all the lane's tokens first was measured: no gain)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int c = 2 * h + tb;
@@ -648,8 +648,8 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 
 // ---------------------------------------------------------------------------------------------
 // The same matmul for 9 to 64 tokens.  With many tokens the activations of a chunk are as large as, or
-// larger than, its weights, so here the eight warps of a CTA share them: the CTA walks a sequence of
-// GROUP tiles (eight consecutive row blocks x one column tile), warp i streams row block 8 * group + i
+// larger than, its weights, so here the eight warps of a CTA share them: the CTA walks a
+// sequence of GROUP tiles (one row block per warp x one column tile), warp i streams row block warps * group + i
 // through its own ring exactly as above, and the activations of a chunk are fetched ONCE per CTA into a
 // shared ring.  Two barriers per activation slot keep the warps together: `xfull` (the copy has landed) and
 // `xempty` (all eight warps are done with the slot; only then does warp 0 refill it), so the warps of a CTA
@@ -657,36 +657,37 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 // sequence; cut row blocks go through the scratch and the per-warp lists as above.
 template <int NT>
 struct WideRing {
+    static constexpr int kW = decode_wide_warps(8 * NT);           // warps per CTA = row blocks per group tile
     static constexpr int kTiles = NT == 2 ? 8 : (NT == 4 ? 6 : 4); // column tiles per chunk
     static constexpr int kDepth = NT == 8 ? 4 : 3;                  // chunks in flight
     static constexpr int kWeightBytes = kTiles * kTileBytes;
     static constexpr int kXSlotBytes = kTiles * 8 * NT * kXTileBytes;
-    static constexpr int kXOffset = kWarps * kDepth * kWeightBytes;
+    static constexpr int kXOffset = kW * kDepth * kWeightBytes;
     static constexpr int kBarsOffset = kXOffset + kDepth * kXSlotBytes;
-    static constexpr int kAbortOffset = kBarsOffset + (kWarps + 2) * kDepth * 8;
+    static constexpr int kAbortOffset = kBarsOffset + (kW + 2) * kDepth * 8;
     static constexpr int kSmem = kAbortOffset + 16;
     static_assert(kSmem <= 227 * 1024, "rings do not fit the SM's shared memory");
 };
 
 template <int NT>
-__global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
+__global__ void __launch_bounds__(WideRing<NT>::kW * 32, 1) decode_wide_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
     uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists, const WaitHooks hooks)
 {
     extern __shared__ __align__(128) uint8_t dsmem[];
     ptx::griddep_launch_dependents();
     using R = WideRing<NT>;
-    constexpr int kChunkTiles = R::kTiles, kDepth = R::kDepth;
+    constexpr int kChunkTiles = R::kTiles, kDepth = R::kDepth, kW = R::kW;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int g = lane >> 2, tq = lane & 3;
     const uint32_t wring = ptx::smem_u32(dsmem) + warp * (kDepth * R::kWeightBytes);
     const uint32_t xring = ptx::smem_u32(dsmem + R::kXOffset);
     const uint32_t wbars = ptx::smem_u32(dsmem + R::kBarsOffset) + warp * (kDepth * 8); // this warp's weights have landed
-    const uint32_t xfull = ptx::smem_u32(dsmem + R::kBarsOffset) + kWarps * kDepth * 8; // the CTA's activations have landed
+    const uint32_t xfull = ptx::smem_u32(dsmem + R::kBarsOffset) + kW * kDepth * 8; // the CTA's activations have landed
     const uint32_t xempty = xfull + kDepth * 8;                                         // all warps are done with them
     volatile int *abort_flag = reinterpret_cast<volatile int *>(dsmem + R::kAbortOffset);
-    const uint32_t w = blockIdx.x * kWarps + warp;
+    const uint32_t w = blockIdx.x * kW + warp;
     uint2 *owned = lists[w].item;
     int n_owned = 0;
 
@@ -695,7 +696,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
 #pragma unroll
         for (int s = 0; s < kDepth; ++s) {
             ptx::mbar_init(xfull + 8 * s, 1);
-            ptx::mbar_init(xempty + 8 * s, kWarps);
+            ptx::mbar_init(xempty + 8 * s, kW);
         }
     }
     if (lane == 0) {
@@ -733,7 +734,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
             if (++p.group == p.groups && p.left > 0) {
                 ++p.e;
                 p.KB = p.e->KB;
-                p.groups = (p.e->NB + kWarps - 1) / kWarps;
+                p.groups = (p.e->NB + kW - 1) / kW;
                 p.group = 0;
             }
         }
@@ -748,7 +749,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
     Walker prod;
     prod.e = tab + find_entry(tab, n_entries, (uint32_t)i0, lane);
     prod.KB = prod.e->KB;
-    prod.groups = (prod.e->NB + kWarps - 1) / kWarps;
+    prod.groups = (prod.e->NB + kW - 1) / kW;
     {
         const uint32_t local = (uint32_t)i0 - prod.e->tile_begin;
         prod.group = (int)(local / (uint32_t)prod.KB);
@@ -775,7 +776,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
                 }
             }
             const Chunk c = step(prod);
-            const int rb = c.group * kWarps + warp;
+            const int rb = c.group * kW + warp;
             const int xb = c.e->M * kXTileBytes;
             const int8_t *xsrc = c.e->Xq + (size_t)c.kt * xb;
             const uint32_t xbytes = (uint32_t)(c.n * xb);
@@ -820,7 +821,7 @@ __global__ void __launch_bounds__(kWarps * 32, 1) decode_wide_kernel(
         // ---- one group of row blocks (or the part of it that lies in this share); this warp's row block is rb
         const DecodeEntry *e = cons.e;
         const int M = e->M, KB = cons.KB;
-        const int rb = cons.group * kWarps + warp;
+        const int rb = cons.group * kW + warp;
         const bool active = rb < e->NB; // the last group of a matrix may have fewer than eight row blocks
         int acc[NT][4][4];
         uint32_t xlane[NT];
@@ -1068,7 +1069,7 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
                     (void *)&hdr, (void *)&lists, (void *)&hooks};
     cudaError_t err = launch_dependent((const void *)decode_wide_kernel<NT>, grid, block, WideRing<NT>::kSmem, args, early, stream);
     if (err != cudaSuccess) return err;
-    uint32_t n_lists = grid.x * kWarps;
+    uint32_t n_lists = grid.x * WideRing<NT>::kW;
     int staged = 0; // (this kernel's rings leave no room beside them)
     int single_token = 0, trits = 0;
     void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token,
@@ -1084,15 +1085,16 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     const dim3 block(kWarps * 32);
     if (path != BITLINEAR_PATH_DP4A && decode_is_wide(max_M)) {
         // total_tiles counts group tiles here; one CTA per SM, equal contiguous shares, at least 4 items each
+        const uint32_t warps = (uint32_t)decode_wide_warps(max_M);
         uint32_t ctas = (total_tiles + 3) / 4;
         uint32_t cap = (uint32_t)sm_count();
-        if (cap > kMaxDecodeWarps / kWarps) cap = kMaxDecodeWarps / kWarps;
+        if (cap > kMaxDecodeWarps / warps) cap = kMaxDecodeWarps / warps;
         if (ctas > cap) ctas = cap;
         const uint32_t share = (total_tiles + ctas - 1) / ctas;
-        const dim3 grid(ctas);
-        if (max_M <= 16) return launch_wide<2>(grid, block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
-        if (max_M <= 32) return launch_wide<4>(grid, block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
-        return launch_wide<8>(grid, block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+        const dim3 grid(ctas), wide_block(warps * 32);
+        if (max_M <= 16) return launch_wide<2>(grid, wide_block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+        if (max_M <= 32) return launch_wide<4>(grid, wide_block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+        return launch_wide<8>(grid, wide_block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
     }
     if (path == BITLINEAR_PATH_DP4A) {
         int ctas = (inl.e[0].NB + kWarps - 1) / kWarps;
