@@ -167,35 +167,50 @@ __device__ __forceinline__ float token_scale(const DecodeEntry &e, int token)
     return __fdiv_rn(__fmul_rn(*e.gamma, e.beta[token]), e.qb); // (gamma * beta_t) / Qb
 }
 
-// What the epilogue needs of a token, fetched once per token and lane: the stores of a lane's outputs may alias
-// these loads as far as the compiler knows, so asking per output would reload (and divide) every time.
+// What the epilogue needs of a token: its row sum and its scale.  A lane holds outputs of two tokens per 8-token tile
+// (2 tq + tb), and it fetches their terms when its warp ENTERS a matrix, not at the end of every row block: there the
+// loads (and the division behind them) were a round trip to L2 that the warp sat through before it could store, once
+// per token, and a warp that stalls does not catch up with its stream again.
 struct TokenTerms {
     int rowsum;
     float scale;
 };
 
-// End of a row block.  `each(begin, fn)` calls begin(token) once for every token this lane holds outputs of and then
-// fn(terms, token, row, partial row sum) for each of them.  If all KB column tiles went into the sums they are final;
-// otherwise they are added to the int32 scratch.
-template <class Each>
-__device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete, Each each)
+template <int NT>
+__device__ __forceinline__ void load_terms(const DecodeEntry &e, int tq, TokenTerms (&tt)[NT][2])
+{
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+#pragma unroll
+        for (int tb = 0; tb < 2; ++tb) {
+            const int token = 8 * nt + 2 * tq + tb;
+            tt[nt][tb] = token < e.M ? TokenTerms{e.rowsum[token], token_scale(e, token)} : TokenTerms{0, 0.0f};
+        }
+    }
+}
+
+// End of a row block.  `each(fn)` calls fn(nt, tb, token, row, partial row sum) for every output this lane holds (token
+// = 8 nt + 2 tq + tb).  If all KB column tiles went into the sums they are final; otherwise they are added to the
+// int32 scratch.
+template <int NT, class Each>
+__device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete, const TokenTerms (&tt)[NT][2], Each each)
 {
     if (complete)
-        each([&](int token) { return TokenTerms{e.rowsum[token], token_scale(e, token)}; },
-             [&](const TokenTerms &tt, int token, int row, int v) { store_result(e, token, row, v, tt.rowsum, tt.scale); });
+        each([&](int nt, int tb, int token, int row, int v) { store_result(e, token, row, v, tt[nt][tb].rowsum, tt[nt][tb].scale); });
     else
-        each([&](int) { return TokenTerms{0, 0.0f}; },
-             [&](const TokenTerms &, int token, int row, int v) { atomicAdd(&e.acc32[(size_t)token * e.N + row], v); });
+        each([&](int, int, int token, int row, int v) { atomicAdd(&e.acc32[(size_t)token * e.N + row], v); });
 }
 
 // Finishing launch: dequantises the row blocks on one list from the scratch and leaves the scratch clean for
 // the next launch.  owned[i] = (entry index, row block).  Up to four row blocks are
 // handled at a time, and up to four tokens of each, with all loads of one kind issued together, so that the pass
 // costs two memory round trips per batch and token group rather than two per row block and token.
+// Every list is served by one warp per group of TG tokens (warp (list, group) takes tokens TG * group ..), so that the
+// launch takes as long with eight tokens as with one.
 // `word` is the lane's 32-bit word of the warp's 128-byte list (one load for the count and all items: every round
 // trip of this launch is on the critical path of the step): word 0 the count, words 2 i + 2 and 2 i + 3 item i.
 template <int TG, int ROWS> // tokens handled together: 1 (single-token steps), or 4; rows of a row block: 64, or 80
-__device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint32_t word, int n_owned, int lane)
+__device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint32_t word, int n_owned, int lane, int t0)
 {
     constexpr int kBatch = 4;
     constexpr int kParts = (ROWS + 31) / 32; // rows per lane
@@ -219,8 +234,8 @@ __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint
             M[b] = e[b]->M;
             if (N[b] > 0) max_M = max(max_M, M[b]);
         }
-        // TG tokens of every row block of the batch at a time: all loads first, then all stores
-        for (int t0 = 0; t0 < max_M; t0 += TG) {
+        // this warp's TG tokens (t0 ..) of every row block of the batch: all loads first, then all stores
+        if (t0 < max_M) {
             int v[kBatch][TG][kParts], rowsum[kBatch][TG];
             float scale[kBatch][TG];
 #pragma unroll
@@ -306,8 +321,8 @@ __device__ __forceinline__ void mma_slab_trits(int (&acc)[5][4], const uint4 &st
 // Un-mixes the four scaled accumulators of every (row, token) this lane holds and hands the row sums to fn.
 // C fragment of field f: c0 (row 16f + g, token 2tq), c1 (same row, 2tq + 1), c2 (row 16f + 8 + g, 2tq), c3.
 // NF = 5: the base-3 format's fifth accumulator holds the sums of rows 64 + r as they are.
-template <int NT, int NF, class Begin, class Fn>
-__device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, int N, int row0, int tq, Begin begin, Fn fn)
+template <int NT, int NF, class Fn>
+__device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, int N, int row0, int tq, Fn fn)
 {
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -315,7 +330,6 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, 
         for (int tb = 0; tb < 2; ++tb) {
             const int token = 8 * nt + 2 * tq + tb;
             if (token >= M) continue;
-            const auto terms = begin(token); // (fetching the terms of all the lane's tokens first was measured: no gain)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int c = 2 * h + tb;
@@ -326,7 +340,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, 
 #pragma unroll
                 for (int f = 0; f < NF; ++f) {
                     const int r = row0 + 16 * f + 8 * h;
-                    if (r < N) fn(terms, token, r, S[f]);
+                    if (r < N) fn(nt, tb, token, r, S[f]);
                 }
             }
         }
@@ -535,6 +549,8 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     // consumer
     const DecodeEntry *e = cur.e;
     int KB = e->KB, rb = cur.rb, kt = cur.kt, left = cur.left;
+    TokenTerms terms[NT][2];
+    load_terms<NT>(*e, tq, terms);
 
     bool alive = true;
     while (alive) {
@@ -543,6 +559,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             if (nxt.left == 0) break;
             if (!p_on_next) producer_start(nxt);
             p_on_next = false;
+            if (nxt.e != e) load_terms<NT>(*nxt.e, tq, terms);
             e = nxt.e;
             KB = e->KB;
             rb = nxt.rb;
@@ -622,7 +639,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
             if (lane == 0) owned[n_owned] = make_uint2((uint32_t)(e - tab), (uint32_t)rb);
             ++n_owned; // cannot exceed kMaxOwned: see next_piece
         }
-        finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT, kFields>(acc, M, e->N, rb * kRows + g, tq, begin, fn); });
+        finish_block<NT>(*e, complete, terms, [&](auto fn) { each_output<NT, kFields>(acc, M, e->N, rb * kRows + g, tq, fn); });
 
         // next row block, or next matrix
         if (kt == KB) {
@@ -631,6 +648,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
                 ++e;
                 rb = 0;
                 KB = e->KB;
+                load_terms<NT>(*e, tq, terms);
             }
         }
     }
@@ -817,9 +835,15 @@ __global__ void __launch_bounds__(WideRing<NT>::kW * 32, 1) decode_wide_kernel(
         }
     }
 
+    const DecodeEntry *terms_of = nullptr; // the matrix whose token terms this lane holds
+    TokenTerms terms[NT][2];
     while (alive && cons.left > 0) {
         // ---- one group of row blocks (or the part of it that lies in this share); this warp's row block is rb
         const DecodeEntry *e = cons.e;
+        if (e != terms_of) {
+            load_terms<NT>(*e, tq, terms);
+            terms_of = e;
+        }
         const int M = e->M, KB = cons.KB;
         const int rb = cons.group * kW + warp;
         const bool active = rb < e->NB; // the last group of a matrix may have fewer than eight row blocks
@@ -876,7 +900,7 @@ __global__ void __launch_bounds__(WideRing<NT>::kW * 32, 1) decode_wide_kernel(
                     ++n_owned;
                 }
             }
-            finish_block(*e, complete, [&](auto begin, auto fn) { each_output<NT, 4>(acc, M, e->N, rb * kTileRows + g, tq, begin, fn); });
+            finish_block<NT>(*e, complete, terms, [&](auto fn) { each_output<NT, 4>(acc, M, e->N, rb * kTileRows + g, tq, fn); });
         }
     }
     }();
@@ -892,13 +916,21 @@ __global__ void __launch_bounds__(WideRing<NT>::kW * 32, 1) decode_wide_kernel(
 // The finishing launch: warp w takes the list of warp w of the kernel above.
 // staged_entries > 0: the CTA copies that many entries of the table (all of them) into its shared memory while the
 // matmul is still running, which takes the table's round trip to L2 off the chain list -> entry -> sums -> stores.
-__global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constant__ InlineTable inl,
-                                                            const DecodeEntry *__restrict__ table,
-                                                            const OwnedList *__restrict__ lists, uint32_t n_lists,
-                                                            int staged_entries, int single_token, int trits)
+// (One instance per form, so that each takes only the registers it needs: beside a CTA of the matmul an SM has room
+// for a finishing CTA of at most 130 registers per thread, and a finishing CTA that is not resident, waiting, when the
+// matmul ends costs the step several microseconds.)
+template <int TG, int ROWS>
+__global__ void __launch_bounds__(256, 2) decode_finish_kernel(const __grid_constant__ InlineTable inl,
+                                                               const DecodeEntry *__restrict__ table,
+                                                               const OwnedList *__restrict__ lists, uint32_t n_lists,
+                                                               int staged_entries, int token_groups)
 {
     extern __shared__ uint4 staged_table[];
-    const uint32_t w = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    // warp (list w, token group tg)
+    const uint32_t gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    const uint32_t groups = (uint32_t)token_groups;
+    const uint32_t w = gw / groups;
+    const int t0 = (int)(gw - w * groups) * TG;
     // The quantiser of a step that follows may become resident at once; it waits for this grid to end before it
     // touches anything, and the matmul behind it streams weights (never written) until that quantiser has ended.
     ptx::griddep_launch_dependents();
@@ -915,17 +947,7 @@ __global__ void __launch_bounds__(256) decode_finish_kernel(const __grid_constan
     const uint32_t word = __ldcg(reinterpret_cast<const uint32_t *>(&lists[w]) + lane);
     const int n = (int)__shfl_sync(0xffffffffu, word, 0);
     if (n == 0) return;
-    const DecodeEntry *tab = table ? table : inl.e;
-    if (trits) {
-        if (single_token)
-            finish_owned_blocks<1, kTritRows>(tab, word, n, lane);
-        else
-            finish_owned_blocks<4, kTritRows>(tab, word, n, lane);
-    } else if (single_token) {
-        finish_owned_blocks<1, kTileRows>(tab, word, n, lane);
-    } else {
-        finish_owned_blocks<4, kTileRows>(tab, word, n, lane);
-    }
+    finish_owned_blocks<TG, ROWS>(table ? table : inl.e, word, n, lane, t0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -1018,14 +1040,27 @@ static cudaError_t launch_dependent(const void *kernel, dim3 grid, dim3 block, s
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 
+// Launches the finishing kernel for n_lists lists of a launch whose largest token count is max_M.
+static cudaError_t launch_finish(const InlineTable &inl, const DecodeEntry *table, const OwnedList *lists, uint32_t n_lists,
+                                 int staged, int max_M, bool trits, bool early, cudaStream_t stream)
+{
+    const bool single = max_M == 1;
+    int token_groups = single ? 1 : (max_M + 3) / 4; // warps per list
+    const void *kernel = trits ? (single ? (const void *)decode_finish_kernel<1, kTritRows> : (const void *)decode_finish_kernel<4, kTritRows>)
+                               : (single ? (const void *)decode_finish_kernel<1, kTileRows> : (const void *)decode_finish_kernel<4, kTileRows>);
+    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&token_groups};
+    const uint32_t finish_warps = n_lists * (uint32_t)token_groups;
+    return launch_dependent(kernel, dim3((finish_warps + 7) / 8), dim3(256), (size_t)staged * sizeof(DecodeEntry), fargs, early,
+                            stream);
+}
+
 template <int NT, bool kTrits>
 static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, const DecodeEntry *table, int n_entries,
                               uint32_t total_tiles, uint32_t share, uint32_t dyn, int max_M, WorkspaceHeader *hdr,
                               OwnedList *lists, cudaStream_t stream)
 {
     WaitHooks hooks = take_wait_hooks();
-    int single_token = max_M == 1 ? 1 : 0;
-    int trits = kTrits ? 1 : 0;
+
     constexpr int kSmemBytes = kTrits ? Ring<NT>::kSmemTrits : Ring<NT>::kSmem;
     static bool attr_set[64] = {false};
     int dev = 0;
@@ -1044,15 +1079,12 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
     // a table that fits beside the matmul's ring (one CTA of each per SM) is staged in the finishing CTAs' shared memory
     // (the base-3 form's decoding table takes that room: its finishing CTAs read the table from global memory)
     int staged = (!kTrits && table && (size_t)n_entries * sizeof(DecodeEntry) <= kStagedTableBytes) ? n_entries : 0;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token,
-                     (void *)&trits};
-    return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256),
-                            (size_t)staged * sizeof(DecodeEntry), fargs, early, stream);
+    return launch_finish(inl, table, lists, n_lists, staged, max_M, kTrits, early, stream);
 }
 
 template <int NT>
 static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, const DecodeEntry *table, int n_entries,
-                               uint32_t total_items, uint32_t share, WorkspaceHeader *hdr, OwnedList *lists,
+                               uint32_t total_items, uint32_t share, int max_M, WorkspaceHeader *hdr, OwnedList *lists,
                                cudaStream_t stream)
 {
     WaitHooks hooks = take_wait_hooks();
@@ -1071,10 +1103,7 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
     if (err != cudaSuccess) return err;
     uint32_t n_lists = grid.x * WideRing<NT>::kW;
     int staged = 0; // (this kernel's rings leave no room beside them)
-    int single_token = 0, trits = 0;
-    void *fargs[] = {(void *)&inl, (void *)&table, (void *)&lists, (void *)&n_lists, (void *)&staged, (void *)&single_token,
-                     (void *)&trits};
-    return launch_dependent((const void *)decode_finish_kernel, dim3((n_lists + 7) / 8), dim3(256), 0, fargs, early, stream);
+    return launch_finish(inl, table, lists, n_lists, staged, max_M, false, early, stream);
 }
 
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
@@ -1092,9 +1121,9 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
         if (ctas > cap) ctas = cap;
         const uint32_t share = (total_tiles + ctas - 1) / ctas;
         const dim3 grid(ctas), wide_block(warps * 32);
-        if (max_M <= 16) return launch_wide<2>(grid, wide_block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
-        if (max_M <= 32) return launch_wide<4>(grid, wide_block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
-        return launch_wide<8>(grid, wide_block, inl, table, n_entries, total_tiles, share, hdr, lists, stream);
+        if (max_M <= 16) return launch_wide<2>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
+        if (max_M <= 32) return launch_wide<4>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
+        return launch_wide<8>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
     }
     if (path == BITLINEAR_PATH_DP4A) {
         int ctas = (inl.e[0].NB + kWarps - 1) / kWarps;
