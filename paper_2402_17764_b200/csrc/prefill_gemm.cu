@@ -726,7 +726,7 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
 // end, so they are chosen only where whole tiles would leave a good part of the last round idle: the idle k blocks of
 // that round, spread over all SMs, must come to at least kMinIdleKb (about 8 us) per SM, and a share must have at
 // least kMinShareKb k blocks.
-constexpr long long kMinIdleKb = 12, kMinShareKb = 16;
+constexpr long long kMinIdleKb = 12, kMinShareKb = 16, kMaxShareRounds = 6;
 static bool deals_shares(long long n_tiles, long long total_kb, int sms)
 {
 #ifdef BITLINEAR_TUNING // measurement aid, not compiled into the library as build.py builds it
@@ -737,6 +737,10 @@ static bool deals_shares(long long n_tiles, long long total_kb, int sms)
     if (!enabled) return false;
 #endif
     if (n_tiles <= 0 || total_kb < kMinShareKb * sms) return false;
+    // Only launches of a few rounds: with many rounds the idle part of the last one is a small share of the whole, and
+    // whole tiles dealt round-robin keep neighbouring CTAs on neighbouring tiles of one matmul (measured: the 70B-shaped
+    // step at 176 tokens, 177 rounds, took 15.0 ms with shares against 11.9 ms with whole tiles).
+    if (n_tiles > kMaxShareRounds * sms) return false;
     const long long r = n_tiles % sms;
     if (r == 0) return false;
     const long long idle_kb = (sms - r) * (total_kb / n_tiles) / sms;

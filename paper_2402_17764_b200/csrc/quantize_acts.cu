@@ -254,18 +254,26 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
             }
         };
         uint32_t mx = 0; // |x| as an unsigned integer is monotone in the magnitude
-        auto absmax8 = [&](const uint4 &v, int i) {
-            float x[8];
-            normalised(v, i, x);
+        auto absmax8 = [&](const float (&x)[8]) {
 #pragma unroll
             for (int j = 0; j < 8; ++j) mx = max(mx, __float_as_uint(x[j]) & 0x7FFFFFFFu);
         };
+        // the normalised values of the cached vectors stay in registers for the last pass (forming them a second time,
+        // gain loads included, was a quarter of the kernel's instructions)
+        float xs[kCache][8];
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
             const int i = threadIdx.x + c * NT;
-            if (i < n_vec) absmax8(cache[c], i);
+            if (i < n_vec) {
+                normalised(cache[c], i, xs[c]);
+                absmax8(xs[c]);
+            }
         }
-        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) absmax8(__ldg(row + i), i);
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
+            float x[8];
+            normalised(__ldg(row + i), i, x);
+            absmax8(x);
+        }
         mx = __reduce_max_sync(0xffffffffu, mx);
         if (lane == 0) s_max[warp] = mx;
         __syncthreads();
@@ -276,9 +284,7 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
         const float s = __fdiv_rn(e.qb, b);
 
         int sum = 0;
-        auto quantise8 = [&](const uint4 &v, int i) {
-            float x[8];
-            normalised(v, i, x);
+        auto quantise8 = [&](const float (&x)[8], int i) {
             uint2 o;
             o.x = pack4(__fmul_rn(x[0], s), __fmul_rn(x[1], s), __fmul_rn(x[2], s), __fmul_rn(x[3], s));
             o.y = pack4(__fmul_rn(x[4], s), __fmul_rn(x[5], s), __fmul_rn(x[6], s), __fmul_rn(x[7], s));
@@ -288,9 +294,13 @@ __global__ void __launch_bounds__(NT, ((kFronts & 1) ? 768 : 1024) / NT) quantiz
 #pragma unroll
         for (int c = 0; c < kCache; ++c) {
             const int i = threadIdx.x + c * NT;
-            if (i < n_vec) quantise8(cache[c], i);
+            if (i < n_vec) quantise8(xs[c], i);
         }
-        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) quantise8(__ldg(row + i), i);
+        for (int i = threadIdx.x + kCache * NT; i < n_vec; i += NT) {
+            float x[8];
+            normalised(__ldg(row + i), i, x);
+            quantise8(x, i);
+        }
         if (tiled) // the last column tile is filled up with zeros
             for (int i = n_vec + threadIdx.x; i < e.KB * 8; i += NT) out_at(i) = make_uint2(0u, 0u);
         sum = __reduce_add_sync(0xffffffffu, sum);
