@@ -218,9 +218,7 @@ def time_sequence(stack, steps, warmup, dist_barrier=None, kernel_steps=None, mi
         total_ms += ms
         enough = total_ms >= min_timed_s * 1e3 or len(rounds) >= MAX_ROUNDS
         if dist_barrier:   # every rank must take the same number of rounds
-            flag = torch.tensor([1.0 if enough else 0.0], device="cuda")
-            torch.distributed.all_reduce(flag, op=torch.distributed.ReduceOp.MIN)
-            enough = bool(flag.item() > 0.5) or len(rounds) >= MAX_ROUNDS
+            enough = all_ranks_agree(torch.distributed, enough, "cuda") or len(rounds) >= MAX_ROUNDS
         if enough:
             break
     status = B.poll_status(seq.workspace)
@@ -726,6 +724,17 @@ def max_over_ranks(dist, values, device):
     t = torch.tensor(list(values), device=device, dtype=torch.float64)
     dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return t.tolist()
+
+
+def all_ranks_agree(dist, mine: bool, device) -> bool:
+    """True only if every rank says so: the ranks repeat their timed rounds until ALL of them have measured enough, so
+    that every rank enters the same barriers the same number of times."""
+    if dist is None:
+        return bool(mine)
+    import torch
+    flag = torch.tensor([1.0 if mine else 0.0], device=device)
+    dist.all_reduce(flag, op=dist.ReduceOp.MIN)
+    return bool(flag.item() > 0.5)
 
 
 def aggregate_throughput(bytes_per_rank, n_ranks, ms):

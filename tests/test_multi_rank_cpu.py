@@ -30,9 +30,11 @@ def _worker(rank, world, port, out):
     dist.init_process_group("gloo", rank=rank, world_size=world)
     mine = [0.150 + 0.010 * rank, 0.140 - 0.005 * rank, 0.300 + 0.020 * rank]  # step, kernel, e2e in ms
     got = bench.max_over_ranks(dist, mine, "cpu")
+    # the ranks go on with their timed rounds until ALL have measured enough: rank 1 is not done in the first poll
+    polls = [bench.all_ranks_agree(dist, rank == 0, "cpu"), bench.all_ranks_agree(dist, True, "cpu")]
     dist.barrier()
     if rank == 0:
-        out.put(got)
+        out.put(got + polls)
     dist.destroy_process_group()
 
 
@@ -47,12 +49,15 @@ def test_timings_are_reduced_with_max_over_two_gloo_ranks():
         p.join(120)
         assert p.exitcode == 0
     got = out.get()
+    assert got[3:] == [False, True]
+    got = got[:3]
     assert got == [0.160, 0.140, 0.320]
     sys.path.insert(0, str(ROOT))
     import bench
     # two replicas of 805,376,000 bytes in 0.160 ms: the slower rank sets the time, the bytes add up
     assert abs(bench.aggregate_throughput(805_376_000, 2, got[0]) - 2 * 805_376_000 / 0.160e-3 / 1e9) < 1e-6
     assert bench.max_over_ranks(None, [1.0, 2.0], "cpu") == [1.0, 2.0]
+    assert bench.all_ranks_agree(None, True, "cpu") and not bench.all_ranks_agree(None, False, "cpu")
 
 
 def test_reference_arm_prints_nothing_on_other_ranks():
