@@ -4,9 +4,12 @@
 // The cost of decode is moving the weights from HBM once (Section 1: loading weights from DRAM is
 // the expensive part; Section 3: time per output token).  All matrices of a launch form ONE sequence
 // of 1 KiB tiles (64 output rows x 64 columns each, row block after row block, matrix after matrix).
-// Most of the sequence is split into one equal, contiguous share per warp; the rest is cut into small
-// pieces that the warps draw from a counter when their share is done, so that SMs that happen to run
-// faster take more (the memory system does not serve all SMs equally).  A warp streams its pieces
+// The sequence is split into one equal, contiguous share per warp.  (The kernel can also hold back a part of the
+// sequence and cut it into small pieces that the warps draw from a counter when their share is done, so that SMs that
+// happen to run faster take more; with the costs of a piece as they are now -- two more row blocks cut and finished by
+// the second launch, per piece -- dealing everything statically measured faster on every workload: 68 against 76 us
+// on the 7B-shaped up projection set at one token, 75 against 87 us at four, 134 against 138 us on the 3B-shaped
+// step, no difference on the 70B-shaped one.  BITLINEAR_DECODE_STATIC_PERCENT below 100 brings the pieces back.)  A warp streams its pieces
 // through a private shared-memory ring filled by bulk copies (cp.async.bulk), so the HBM latency is
 // covered by the copy engine and not by registers, and the stream never drains at a row-block, matrix
 // or piece boundary.  Row blocks that lie completely inside a piece are finished by that warp alone.
@@ -93,7 +96,7 @@ struct Ring {
 };
 constexpr int kTritRows = 80; // rows of a tile of the base-3 format
 #ifndef BITLINEAR_DECODE_STATIC_PERCENT
-#define BITLINEAR_DECODE_STATIC_PERCENT 80
+#define BITLINEAR_DECODE_STATIC_PERCENT 100
 #endif
 #ifndef BITLINEAR_DECODE_PIECES_PER_WARP
 #define BITLINEAR_DECODE_PIECES_PER_WARP 3
