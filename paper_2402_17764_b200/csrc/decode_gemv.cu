@@ -72,6 +72,9 @@ namespace {
 #ifndef BITLINEAR_DECODE_CTAS_PER_SM
 #define BITLINEAR_DECODE_CTAS_PER_SM 1
 #endif
+#ifndef BITLINEAR_DECODE_STAGES_NT2
+#define BITLINEAR_DECODE_STAGES_NT2 3
+#endif
 constexpr int kWarps = BITLINEAR_DECODE_WARPS;             // warps per CTA, each independent
 constexpr int kStages = BITLINEAR_DECODE_STAGES;           // chunks in flight per warp
 constexpr int kCtasPerSm = BITLINEAR_DECODE_CTAS_PER_SM;
@@ -82,10 +85,11 @@ constexpr int kXTileBytes = 64;                            // int8 activations o
 template <int NT>
 struct Ring {
     static constexpr int kTiles = NT == 1 ? BITLINEAR_DECODE_CHUNK_TILES : (NT == 8 ? 2 : 4); // tiles per chunk
+    static constexpr int kDepth = NT == 2 ? BITLINEAR_DECODE_STAGES_NT2 : kStages;            // chunks in flight per warp
     static constexpr int kWeightBytes = kTiles * kTileBytes;
     static constexpr int kSlotBytes = kWeightBytes + kTiles * 8 * NT * kXTileBytes;
-    static constexpr int kBarsOffset = kWarps * kStages * kSlotBytes;
-    static constexpr int kAbortOffset = kBarsOffset + kWarps * kStages * 8;
+    static constexpr int kBarsOffset = kWarps * kDepth * kSlotBytes;
+    static constexpr int kAbortOffset = kBarsOffset + kWarps * kDepth * 8;
     static constexpr int kSmem = kAbortOffset + 16;
     static_assert(kSmem * (NT <= 2 ? kCtasPerSm : 1) <= 227 * 1024, "ring does not fit the SM's shared memory");
     // base-3 format: the decoding table behind the ring, entry v of lane l at 128 v + 4 l
@@ -205,7 +209,7 @@ __device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete
 }
 
 // Finishing launch: dequantises the row blocks on one list from the scratch and leaves the scratch clean for
-// the next launch.  owned[i] = (entry index, row block).  Up to four row blocks are
+// the next launch.  owned[i] = (entry index, row block).  Up to four row blocks (two with several tokens) are
 // handled at a time, and up to four tokens of each, with all loads of one kind issued together, so that the pass
 // costs two memory round trips per batch and token group rather than two per row block and token.
 // Every list is served by one warp per group of TG tokens (warp (list, group) takes tokens TG * group ..), so that the
@@ -215,7 +219,8 @@ __device__ __forceinline__ void finish_block(const DecodeEntry &e, bool complete
 template <int TG, int ROWS> // tokens handled together: 1 (single-token steps), or 4; rows of a row block: 64, or 80
 __device__ __forceinline__ void finish_owned_blocks(const DecodeEntry *tab, uint32_t word, int n_owned, int lane, int t0)
 {
-    constexpr int kBatch = 4;
+    // (with static shares a list has at most two row blocks: the two ends of its warp's share)
+    constexpr int kBatch = TG == 1 ? 4 : 2;
     constexpr int kParts = (ROWS + 31) / 32; // rows per lane
     for (int b0 = 0; b0 < n_owned; b0 += kBatch) {
         const DecodeEntry *e[kBatch];
@@ -350,6 +355,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, 
     }
 }
 
+// (Two token tiles take 138 registers; held to 128 the kernel was 4 % slower.)
 template <int NT, bool kTrits>
 __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
@@ -362,6 +368,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     const int g = lane >> 2, tq = lane & 3;
     using R = Ring<NT>;
     constexpr int kChunkTiles = R::kTiles;
+    constexpr int kStages = R::kDepth; // (the ring depth of this form)
     const uint32_t ring = ptx::smem_u32(dsmem) + warp * (kStages * R::kSlotBytes);
     const uint32_t bars = ptx::smem_u32(dsmem + R::kBarsOffset) + warp * (kStages * 8);
     int n_owned = 0;
@@ -668,7 +675,9 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same matmul for 9 to 64 tokens.  With many tokens the activations of a chunk are as large as, or
+// The same matmul for 17 to 64 tokens (reached through the test hook only: the library sends 17 tokens and more to the
+// tensor-core GEMM, and 9 to 16 tokens to the kernel above with two token tiles per warp, which measured faster than this
+// one there: 110 against 122 us on the 7B-shaped up projection set at 16 tokens).  With many tokens the activations of a chunk are as large as, or
 // larger than, its weights, so here the eight warps of a CTA share them: the CTA walks a
 // sequence of GROUP tiles (one row block per warp x one column tile), warp i streams row block warps * group + i
 // through its own ring exactly as above, and the activations of a chunk are fetched ONCE per CTA into a
@@ -1124,7 +1133,6 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
         if (ctas > cap) ctas = cap;
         const uint32_t share = (total_tiles + ctas - 1) / ctas;
         const dim3 grid(ctas), wide_block(warps * 32);
-        if (max_M <= 16) return launch_wide<2>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
         if (max_M <= 32) return launch_wide<4>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
         return launch_wide<8>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
     }
@@ -1158,6 +1166,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
         share = (total_tiles + n_warps - 1) / n_warps; // all static: the last warps may get less, or nothing
     }
     if (trits) return launch_mma<1, true>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
+    if (max_M > 8) return launch_mma<2, false>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
     return launch_mma<1, false>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
 }
 

@@ -86,12 +86,11 @@ cudaError_t launch_retile_acts(const int8_t *Xq, int64_t M, int64_t K, int8_t *t
 cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *table, int n_entries, int total_tokens,
                                  void *zero_ptr, size_t zero_bytes, int fronts, int max_K, cudaStream_t stream);
 
-// The weight-streaming matmul has two kernels: up to 8 tokens every warp streams tiles on its own; from 9
-// tokens the warps of a CTA share the activations and the CTA walks group tiles (one row block per warp x 1 column
-// tile).  The sequence of work items of a launch is counted accordingly, for the largest token count max_M of the launch.
-// (Eight warps for every token count: sixteen warps with chunks of four tiles, which is what then fits the shared
-// memory, were measured slower up to 16 tokens: 2.7 against 3.0 TB/s on the 7B-shaped up projection.)
-inline bool decode_is_wide(int max_M) { return max_M > 8; }
+// The weight-streaming matmul has two kernels: up to 16 tokens every warp streams tiles on its own (one 8-token tile
+// per MMA up to 8 tokens, two beyond); from 17 tokens (test hook only) the eight warps of a CTA share the activations and
+// the CTA walks group tiles (one row block per warp x 1 column tile).  The sequence of work items of a launch is counted
+// accordingly, for the largest token count max_M of the launch.
+inline bool decode_is_wide(int max_M) { return max_M > 16; }
 constexpr int decode_wide_warps(int max_M) { return max_M <= 16 ? 8 : 8; }
 inline uint32_t decode_items(int NB, int KB, int max_M)
 {
