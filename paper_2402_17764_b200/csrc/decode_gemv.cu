@@ -75,6 +75,9 @@ namespace {
 #ifndef BITLINEAR_DECODE_STAGES_NT2
 #define BITLINEAR_DECODE_STAGES_NT2 2
 #endif
+#ifndef BITLINEAR_DECODE_WARPS_NT2
+#define BITLINEAR_DECODE_WARPS_NT2 8
+#endif
 #ifndef BITLINEAR_DECODE_CHUNK_TILES_NT2
 #define BITLINEAR_DECODE_CHUNK_TILES_NT2 6
 #endif
@@ -94,8 +97,9 @@ struct Ring {
     static constexpr int kDepth = NT == 2 ? BITLINEAR_DECODE_STAGES_NT2 : kStages;            // chunks in flight per warp
     static constexpr int kWeightBytes = kTiles * kTileBytes;
     static constexpr int kSlotBytes = kWeightBytes + kTiles * 8 * NT * kXTileBytes;
-    static constexpr int kBarsOffset = kWarps * kDepth * kSlotBytes;
-    static constexpr int kAbortOffset = kBarsOffset + kWarps * kDepth * 8;
+    static constexpr int kW = NT == 2 ? BITLINEAR_DECODE_WARPS_NT2 : kWarps; // warps per CTA
+    static constexpr int kBarsOffset = kW * kDepth * kSlotBytes;
+    static constexpr int kAbortOffset = kBarsOffset + kW * kDepth * 8;
     static constexpr int kSmem = kAbortOffset + 16;
     static_assert(kSmem * (NT <= 2 ? kCtasPerSm : 1) <= 227 * 1024, "ring does not fit the SM's shared memory");
     // base-3 format: the decoding table behind the ring, entry v of lane l at 128 v + 4 l
@@ -363,7 +367,7 @@ __device__ __forceinline__ void each_output(const int (&acc)[NT][NF][4], int M, 
 
 // (Two token tiles take 138 registers; held to 128 the kernel was 4 % slower.)
 template <int NT, bool kTrits>
-__global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
+__global__ void __launch_bounds__(Ring<NT>::kW * 32, (NT <= 2) ? kCtasPerSm : 1) decode_mma_kernel(
     const __grid_constant__ InlineTable inl, const DecodeEntry *__restrict__ table, int n_entries,
     uint32_t total_tiles, uint32_t share, uint32_t dyn, WorkspaceHeader *hdr, OwnedList *lists, const WaitHooks hooks)
 {
@@ -385,7 +389,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
     if (kTrits) {
         // entry v of every lane's copy: the byte of four 2-bit fields c0 + 4 c1 + 16 c2 + 64 c3, and c4 << 8
         uint32_t *lut = reinterpret_cast<uint32_t *>(dsmem + R::kLutOffset);
-        for (int v = threadIdx.x; v < 243; v += kWarps * 32) {
+        for (int v = threadIdx.x; v < 243; v += R::kW * 32) {
             const uint32_t c0 = v % 3, c1 = (v / 3) % 3, c2 = (v / 9) % 3, c3 = (v / 27) % 3, c4 = v / 81;
             const uint32_t entry = c0 | (c1 << 2) | (c2 << 4) | (c3 << 6) | (c4 << 8);
             for (int l = 0; l < 32; ++l) lut[v * 32 + l] = entry;
@@ -404,7 +408,7 @@ __global__ void __launch_bounds__(kWarps * 32, (NT <= 2) ? kCtasPerSm : 1) decod
 
     // A piece is a contiguous range of the tile sequence.  Piece w (w < n_warps) is warp w's own share of
     // `share` tiles; the tiles after the shares form pieces of `dyn` tiles dealt through hdr->piece_counter.
-    const uint32_t n_warps = gridDim.x * kWarps, w = blockIdx.x * kWarps + warp;
+    const uint32_t n_warps = gridDim.x * R::kW, w = blockIdx.x * R::kW + warp;
     uint2 *owned = lists[w].item;
     struct Piece {
         const DecodeEntry *e;
@@ -1093,7 +1097,7 @@ static cudaError_t launch_mma(dim3 grid, dim3 block, const InlineTable &inl, con
                     (void *)&dyn, (void *)&hdr, (void *)&lists, (void *)&hooks};
     cudaError_t err = launch_dependent((const void *)decode_mma_kernel<NT, kTrits>, grid, block, kSmemBytes, args, early, stream);
     if (err != cudaSuccess) return err;
-    uint32_t n_lists = grid.x * kWarps;
+    uint32_t n_lists = grid.x * Ring<NT>::kW;
     // a table that fits beside the matmul's ring (one CTA of each per SM) is staged in the finishing CTAs' shared memory
     // (the base-3 form's decoding table takes that room: its finishing CTAs read the table from global memory)
     int staged = (!kTrits && table && (size_t)n_entries * sizeof(DecodeEntry) <= kStagedTableBytes) ? n_entries : 0;
@@ -1151,16 +1155,17 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
     }
     // every warp should have at least kMinTilesPerWarp tiles; beyond that, fill the machine
     constexpr uint32_t kMinTilesPerWarp = 4;
-    uint32_t ctas = (total_tiles + kMinTilesPerWarp * kWarps - 1) / (kMinTilesPerWarp * kWarps);
+    const uint32_t warps = (max_M > 8 && !trits) ? (uint32_t)Ring<2>::kW : (uint32_t)kWarps;
+    uint32_t ctas = (total_tiles + kMinTilesPerWarp * warps - 1) / (kMinTilesPerWarp * warps);
     uint32_t cap = (uint32_t)sm_count() * kCtasPerSm;
-    if (cap > kMaxDecodeWarps / kWarps) cap = kMaxDecodeWarps / kWarps;
+    if (cap > kMaxDecodeWarps / warps) cap = kMaxDecodeWarps / warps;
     if (ctas > cap) ctas = cap;
     const dim3 grid(ctas);
     // Static shares take kStaticPercent of the tiles; the rest is dealt in pieces of `dyn` tiles, about
     // kPiecesPerWarp per warp, none shorter than kMinPieceTiles.  Small launches have no dynamic part.
     static const uint32_t static_percent = tuning_from_env("BITLINEAR_DECODE_STATIC_PERCENT", kStaticPercent, 100);
     static const uint32_t pieces_per_warp = tuning_from_env("BITLINEAR_DECODE_PIECES_PER_WARP", kPiecesPerWarp, 8);
-    const uint32_t n_warps = ctas * kWarps;
+    const uint32_t n_warps = ctas * warps;
     uint32_t share = total_tiles / n_warps, dyn = 0;
     if (share >= 4 * kMinPieceTiles && static_percent < 100) {
         share = (uint32_t)((uint64_t)total_tiles * static_percent / 100 / n_warps);
@@ -1172,7 +1177,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
         share = (total_tiles + n_warps - 1) / n_warps; // all static: the last warps may get less, or nothing
     }
     if (trits) return launch_mma<1, true>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
-    if (max_M > 8) return launch_mma<2, false>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
+    if (max_M > 8) return launch_mma<2, false>(grid, dim3(warps * 32), inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
     return launch_mma<1, false>(grid, block, inl, table, n_entries, total_tiles, share, dyn, max_M, hdr, lists, stream);
 }
 
