@@ -181,8 +181,9 @@ bitlinear_status run_matmul(DecodeEntry e, int path, char *ws, size_t lists_offs
     if (e.M > kMaxDecodeM) return BITLINEAR_ERR_SHAPE; // the weight-streaming kernel takes at most 64 tokens
     InlineTable inl{};
     inl.e[0] = e;
-    cudaError_t err = launch_decode(inl, nullptr, 1, decode_items(e.NB, e.KB, e.M), e.M,
-                                    path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream, trits);
+    const bool wide = !trits && decode_is_wide(e.M, (uint64_t)e.NB * (uint64_t)e.KB);
+    cudaError_t err = launch_decode(inl, nullptr, 1, decode_items(e.NB, e.KB, wide, e.M), e.M,
+                                    path == BITLINEAR_PATH_DP4A ? path : BITLINEAR_PATH_MMA, hdr, lists, stream, trits, wide);
     if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     return BITLINEAR_OK;
 }
@@ -568,6 +569,7 @@ struct bitlinear_sequence {
     int fronts;             // bit 0: some entry has an RMSNorm in front of the quantiser, bit 1: some entry a SwiGLU
     void *split_scratch;    // inside the workspace; null: the GEMM deals this sequence's tiles whole
     bool trits;             // the weights are in the base-3 format
+    bool wide;              // the streaming kernel that runs it: the lockstep one (see decode_is_wide)
 };
 
 namespace {
@@ -709,6 +711,10 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     for (int i = 0; i < n; ++i)
         if ((int)layers[i].M > max_M) max_M = (int)layers[i].M;
     const bool gemm = S.use_gemm;
+    uint64_t plain_tiles = 0;
+    for (int i = 0; i < n; ++i)
+        plain_tiles += (uint64_t)(trits ? trit_row_blocks(layers[i].N) : row_blocks(layers[i].N)) * (uint64_t)col_tiles(layers[i].K);
+    const bool wide = !trits && !gemm && decode_is_wide(max_M, plain_tiles); // which streaming kernel serves the sequence
     std::vector<unsigned char> gemm_table(gemm ? (size_t)n * kGemmProblemBytes : 0);
     int gemm_tiles = 0;
     int64_t gemm_kb = 0;
@@ -730,7 +736,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
         fronts |= (e.gain ? 1 : 0) | (e.up ? 2 : 0);
         e.tile_begin = tiles;
         e.token_begin = tokens;
-        tiles += decode_items(e.NB, e.KB, max_M); // (one kernel serves the whole sequence)
+        tiles += decode_items(e.NB, e.KB, wide, max_M); // (one kernel serves the whole sequence)
         tokens += (int)d.M;
         if (gemm) {
             int nt = 0;
@@ -762,6 +768,7 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     seq->gemm_total_kb = gemm_kb;
     seq->fronts = fronts;
     seq->trits = trits;
+    seq->wide = wide;
     seq->split_scratch = split ? ws + S.acc32 : nullptr;
     if (gemm) {
         if (cudaMemcpy(ws + S.gemm, gemm_table.data(), gemm_table.size(), cudaMemcpyHostToDevice) != cudaSuccess) {
@@ -799,7 +806,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
             seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->gemm_total_kb, seq->max_M,
                                                  seq->split_scratch, s)
                             : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
-                                            reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s, seq->trits);
+                                            reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s, seq->trits, seq->wide);
         if (err != cudaSuccess) return BITLINEAR_ERR_CUDA;
     }
     return BITLINEAR_OK;

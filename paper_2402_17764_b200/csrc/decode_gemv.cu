@@ -685,9 +685,10 @@ __global__ void __launch_bounds__(Ring<NT>::kW * 32, (NT <= 2) ? kCtasPerSm : 1)
 }
 
 // ---------------------------------------------------------------------------------------------
-// The same matmul for 17 to 64 tokens (reached through the test hook only: the library sends 17 tokens and more to the
-// tensor-core GEMM, and 9 to 16 tokens to the kernel above with two token tiles per warp, which measured faster than this
-// one there: 110 against 122 us on the 7B-shaped up projection set at 16 tokens).  With many tokens the activations of a chunk are as large as, or
+// The same matmul for 13 to 64 tokens: 13 to 16 tokens when a launch streams 1.5 GB of weights or more (see
+// decode_is_wide: the kernel above with two token tiles per warp is faster on shorter launches, 104 against 122 us on the
+// 7B-shaped up projection set at 16 tokens, and slower on the 70B-shaped step), 17 to 64 tokens through the test hook
+// only (the library sends those to the tensor-core GEMM).  With many tokens the activations of a chunk are as large as, or
 // larger than, its weights, so here the eight warps of a CTA share them: the CTA walks a
 // sequence of GROUP tiles (one row block per warp x one column tile), warp i streams row block warps * group + i
 // through its own ring exactly as above, and the activations of a chunk are fetched ONCE per CTA into a
@@ -1129,12 +1130,13 @@ static cudaError_t launch_wide(dim3 grid, dim3 block, const InlineTable &inl, co
 }
 
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
-                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream, bool trits)
+                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream, bool trits, bool wide)
 {
     if (total_tiles == 0) return cudaSuccess;
     if (trits && (max_M > 8 || path == BITLINEAR_PATH_DP4A)) return cudaErrorInvalidValue;
     const dim3 block(kWarps * 32);
-    if (path != BITLINEAR_PATH_DP4A && decode_is_wide(max_M)) {
+    if (max_M > 16) wide = true; // (beyond 16 tokens only the lockstep kernel exists)
+    if (path != BITLINEAR_PATH_DP4A && wide && !trits) {
         // total_tiles counts group tiles here; one CTA per SM, equal contiguous shares, at least 4 items each
         const uint32_t warps = (uint32_t)decode_wide_warps(max_M);
         uint32_t ctas = (total_tiles + 3) / 4;
@@ -1143,6 +1145,7 @@ cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int 
         if (ctas > cap) ctas = cap;
         const uint32_t share = (total_tiles + ctas - 1) / ctas;
         const dim3 grid(ctas), wide_block(warps * 32);
+        if (max_M <= 16) return launch_wide<2>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
         if (max_M <= 32) return launch_wide<4>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
         return launch_wide<8>(grid, wide_block, inl, table, n_entries, total_tiles, share, max_M, hdr, lists, stream);
     }

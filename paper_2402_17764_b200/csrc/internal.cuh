@@ -90,21 +90,30 @@ cudaError_t launch_quantize_acts(const InlineTable &inl, const DecodeEntry *tabl
 // per MMA up to 8 tokens, two beyond); from 17 tokens (test hook only) the eight warps of a CTA share the activations and
 // the CTA walks group tiles (one row block per warp x 1 column tile).  The sequence of work items of a launch is counted
 // accordingly, for the largest token count max_M of the launch.
-inline bool decode_is_wide(int max_M) { return max_M > 16; }
+// Which of the two runs a launch whose largest token count is max_M and whose matmuls have plain_tiles tiles of 64 x 64
+// weights (= KiB of packed weights) in all.  Beyond 16 tokens only the lockstep kernel exists.  From 13 to 16 tokens the
+// independent warps fetch nearly a KiB of activations per KiB of weights each, which caps them near 4.3 TB/s on the
+// path from L2 to the SMs, while the lockstep kernel streams 4.6 TB/s once it runs but takes about 25 us longer to get
+// going: it wins from about 1.5 GB of weights per launch on (70B-shaped step at 16 tokens: 3.75 against 3.99 ms; 7B-shaped
+// sets of 400 MB: 122 against 104 us).
+constexpr uint64_t kWideMinTiles = 1500000;
+inline bool decode_is_wide(int max_M, uint64_t plain_tiles) { return max_M > 16 || (max_M >= 13 && plain_tiles >= kWideMinTiles); }
 constexpr int decode_wide_warps(int max_M) { return max_M <= 16 ? 8 : 8; }
-inline uint32_t decode_items(int NB, int KB, int max_M)
+inline uint32_t decode_items(int NB, int KB, bool wide, int max_M)
 {
     const int w = decode_wide_warps(max_M);
-    return (uint32_t)(decode_is_wide(max_M) ? (NB + w - 1) / w : NB) * (uint32_t)KB;
+    return (uint32_t)(wide ? (NB + w - 1) / w : NB) * (uint32_t)KB;
 }
 
-// Persistent weight-streaming matmul over the entries (total_tiles = sum of decode_items over the entries).
+// Persistent weight-streaming matmul over the entries (total_tiles = sum of decode_items over the entries, counted for
+// the kernel `wide` names: decode_is_wide).
 // path: BITLINEAR_PATH_MMA, or BITLINEAR_PATH_DP4A (first entry only).
 // `lists` is scratch of kOwnedListsBytes (no need to clear it).
 // trits: the entries' weights are in the base-3 format (five per byte, row blocks of 80 rows: NB = ceil(N / 80)); at
 // most 8 tokens then.
 cudaError_t launch_decode(const InlineTable &inl, const DecodeEntry *table, int n_entries, uint32_t total_tiles,
-                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream, bool trits = false);
+                          int max_M, int path, WorkspaceHeader *hdr, OwnedList *lists, cudaStream_t stream, bool trits = false,
+                          bool wide = false);
 
 // Tensor-core GEMM (tcgen05): out = dequant(Xq x T^T) (by gamma * beta_t / qb) or raw int32.  x_rows >= M rows of K bytes exist behind
 // Xq; the rows past M may hold anything (they only reach accumulator rows that are never stored).
