@@ -9,7 +9,7 @@ from pathlib import Path
 PKG = Path(__file__).resolve().parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libbitlinear_b200.so"
-SOURCES = ["bitlinear_api.cu", "pack_weights.cu", "quantize_acts.cu", "decode_gemv.cu", "prefill_gemm.cu", "peak_probe.cu"]
+SOURCES = ["bitlinear_api.cu", "pack_weights.cu", "quantize_acts.cu", "decode_gemv.cu", "prefill_gemm.cu", "decode_tc.cu", "peak_probe.cu"]
 
 
 def _nvcc() -> str:

@@ -36,6 +36,7 @@
 #include <cstdlib>
 #include <cstring>
 
+#include "gemm_problem.cuh"
 #include "internal.cuh"
 #include "ptx.cuh"
 #include "tma_host.cuh"
@@ -46,9 +47,8 @@ namespace {
 
 using namespace ptx;
 
-constexpr int BM = 128;      // tokens per MMA (MMA M, TMEM lanes); a CTA tile has MT of them
-constexpr int BN = 256;      // features per tile (MMA N, TMEM columns per accumulator)
-constexpr int BK = 128;      // int8 elements (= bytes) of K per stage
+// BM = 128 tokens per MMA (MMA M, TMEM lanes), BN = 256 features per tile (MMA N, TMEM columns per accumulator),
+// BK = 128 bytes of K per stage: gemm_problem.cuh
 constexpr int kMaxStages = 12; // ring of TMA stages (activations + packed weights); its depth is chosen at launch
 constexpr int kMaxBSlots = 3;  // ring of expanded weight tiles (its depth: Cfg)
 constexpr int kTmemCols = 512;
@@ -161,52 +161,6 @@ struct RingPos {
             s = 0;
             ++round;
         }
-    }
-};
-
-struct Params {
-    const float *gamma;
-    const float *beta;
-    const int32_t *rowsum;
-    void *out;
-    int M, N, KB; // KB = k blocks of 128 columns
-    int tiles_m, tiles_n; // CTA tiles: MT * 128 tokens x 256 features
-    int out_i32;
-    int out_32b_aligned; // rows of the bf16 output start on 32-byte boundaries
-    int tile_begin;      // first CTA tile of this matmul in the launch-wide tile sequence
-    long long kb_begin;  // first k block of this matmul in the launch-wide sequence of k blocks (all tiles)
-    float qb;            // largest activation code (127, or less for activations of fewer bits)
-    int32_t *status;
-};
-
-// One matmul of a launch: its two tensor maps and its parameters.  A single matmul travels as a kernel
-// parameter; the matmuls of a sequence stand in a table in device memory (written once, by the host).
-struct alignas(64) GemmProblem {
-    CUtensorMap tmap_x, tmap_w;
-    Params p;
-};
-static_assert(sizeof(GemmProblem) == kGemmProblemBytes, "internal.cuh states the size of a table entry");
-
-// The matmul a tile, or a k block of the launch-wide sequence, belongs to.  A CTA's work only goes up, so the search
-// resumes where it stopped.
-template <bool kTable>
-struct ProblemCursor {
-    const GemmProblem *table;
-    int n, i;
-    __device__ ProblemCursor(const GemmProblem &one, const GemmProblem *t, int n_) : table(kTable ? t : &one), n(n_), i(0) {}
-    __device__ const GemmProblem &seek(int tile)
-    {
-        if (kTable) {
-            while (i + 1 < n && tile >= table[i + 1].p.tile_begin) ++i;
-        }
-        return table[i];
-    }
-    __device__ const GemmProblem &seek_kb(long long pos)
-    {
-        if (kTable) {
-            while (i + 1 < n && pos >= table[i + 1].p.kb_begin) ++i;
-        }
-        return table[i];
     }
 };
 
@@ -699,8 +653,10 @@ static cudaError_t fill_problem(GemmProblem &g, const void *packed, const float 
     if (!encode_tiled_fn()) return cudaErrorNotSupported;
     if (x_rows < M) return cudaErrorInvalidValue;
     // activations: box of a_rows rows; weights: box of 4 row blocks x 2 column tiles
+    // (up to 64 tokens: the weight-stationary form reads the weights through the swizzled map)
     if (!encode_activation_map(&g.tmap_x, Xq, x_rows, K, a_rows) ||
-        !encode_packed_weight_map(&g.tmap_w, packed, N, K, BN / kTileRows))
+        !(a_rows == 64 ? encode_packed_weight_map_swizzled(&g.tmap_w, packed, N, K, BN / kTileRows)
+                       : encode_packed_weight_map(&g.tmap_w, packed, N, K, BN / kTileRows)))
         return cudaErrorInvalidValue;
     Params &p = g.p;
     p.gamma = gamma;
@@ -768,6 +724,7 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
         attr_set[dev] = true;
     }
     if (n_tiles <= 0) return cudaSuccess;
+    if (a_rows == 64) return launch_decode_tc(one, table, n, n_tiles, stream); // 17 to 64 tokens: decode_tc.cu
     const int sms = sm_count();
     Schedule sc;
     sc.stream_k = (scratch && deals_shares(n_tiles, total_kb, sms)) ? 1 : 0;

@@ -64,4 +64,23 @@ inline bool encode_packed_weight_map(CUtensorMap *map, const void *packed, int64
                   CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The same packed weights as rows of 128 bytes (eight per tile) with the 128-byte swizzle: the box (two column tiles
+// x four row blocks = 8 KiB) lands with the byte order of the plain map above, except that the 16-byte piece at offset o
+// stands at o ^ (((o >> 7) & 7) << 4).  A warp that reads the pieces (slab s, slot 4 g + tq) of the eight g at once then
+// touches eight different bank groups (decode_tc.cu).
+inline bool encode_packed_weight_map_swizzled(CUtensorMap *map, const void *packed, int64_t N, int64_t K, int box_row_blocks)
+{
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return false;
+    const cuuint64_t tiles_k = (cuuint64_t)((K + kTileCols - 1) / kTileCols);
+    const cuuint64_t tiles_n = (cuuint64_t)((N + kTileRows - 1) / kTileRows);
+    const cuuint64_t dims[3] = {128u, tiles_k * (kTileBytes / 128), tiles_n};
+    const cuuint64_t strides[2] = {128u, tiles_k * kTileBytes};
+    const cuuint32_t box[3] = {128u, 2u * (kTileBytes / 128), (cuuint32_t)box_row_blocks};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void *>(packed), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 } // namespace bitlinear

@@ -30,7 +30,8 @@ def _lib():
 
 # (M, K, N, kernel that runs): all of them one CTA
 CASES = [(1, 128, 64, "decode_mma_kernel"), (12, 128, 512, "decode_wide_kernel"),
-         (40, 128, 256, "prefill_gemm_kernel, one token tile"), (200, 128, 256, "prefill_gemm_kernel, two token tiles")]
+         (40, 128, 256, "decode_tc_kernel"), (100, 128, 256, "prefill_gemm_kernel, one token tile"),
+         (200, 128, 256, "prefill_gemm_kernel, two token tiles")]
 
 
 @pytest.mark.parametrize("M,K,N,kernel", CASES)
