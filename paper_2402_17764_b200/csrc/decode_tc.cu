@@ -70,8 +70,8 @@ constexpr uint32_t kSmemLimit = 232448; // 227 KiB
 struct Barriers {
     uint64_t full[kMaxStages];        // TMA bytes landed (activations + packed weights)
     uint64_t stage_empty[kMaxStages]; // the MMAs of both feature blocks have read the stage (passed on by an expander warp)
-    uint64_t a_full[kASlots];         // A operands of a k block written (four lane quarters)
-    uint64_t a_empty[kASlots];        // the MMAs that read them have completed (both feature blocks)
+    uint64_t a_full[kAUnits];         // A operand of (slot, feature block) written (four lane quarters)
+    uint64_t a_empty[kAUnits];        // the MMAs that read it have completed
     uint64_t acc_full[2];             // accumulators of a tile complete (four MMA threads)
     uint64_t acc_empty[2];            // drained and zeroed (four epilogue warps)
     uint32_t tmem_base;
@@ -142,7 +142,7 @@ __device__ __forceinline__ void store_unit(const uint32_t (&x)[4][2], uint32_t t
 template <bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems, int n_tiles,
-                 int n_stages, const WaitHooks hooks)
+                 int n_stages, int mma_n, const WaitHooks hooks)
 {
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -158,11 +158,11 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
     if (threadIdx.x == 0) {
         for (int s = 0; s < n_stages; ++s) {
             mbar_init(smem_u32(&bars->full[s]), 1);
-            mbar_init(smem_u32(&bars->stage_empty[s]), 1);
+            mbar_init(smem_u32(&bars->stage_empty[s]), kFeatureBlocks);
         }
-        for (int u = 0; u < kASlots; ++u) {
+        for (int u = 0; u < kAUnits; ++u) {
             mbar_init(smem_u32(&bars->a_full[u]), 4);
-            mbar_init(smem_u32(&bars->a_empty[u]), kFeatureBlocks);
+            mbar_init(smem_u32(&bars->a_empty[u]), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(smem_u32(&bars->acc_full[b]), 4);
@@ -240,7 +240,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
             const int j = warp - kFirstMmaWarp;
             const int fb = j & 1;
             const uint32_t par = (uint32_t)(j >> 1);
-            const uint32_t idesc = idesc_i8(128, kTokens, /*a_signed=*/0, /*b_signed=*/1);
+            const uint32_t idesc = idesc_i8(128, mma_n, /*a_signed=*/0, /*b_signed=*/1); // (32 tokens at most: MMAs of half the width)
             const uint32_t desc_hi = (uint32_t)(smem_desc_k_sw128(0) >> 32);
             const uint32_t b_lo0 = (uint32_t)smem_desc_k_sw128(base);
             ProblemCursor<kTable> cur(one, table, n_problems);
@@ -255,18 +255,18 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
                 const uint32_t d_tmem = tmem_base + (buf * kFeatureBlocks + (uint32_t)fb) * kAccCols;
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     if ((it & 1u) == par) {
-                        const uint32_t slot = it & (kASlots - 1);
-                        if (!mbar_wait_bounded(smem_u32(&bars->a_full[slot]), (it / kASlots) & 1, abort_flag, hooks.limit_us)) {
+                        const uint32_t unit = (it & (kASlots - 1)) * kFeatureBlocks + (uint32_t)fb;
+                        if (!mbar_wait_bounded(smem_u32(&bars->a_full[unit]), (it / kASlots) & 1, abort_flag, hooks.limit_us)) {
                             ok = false;
                             break;
                         }
                         tc_fence_after_sync();
-                        const uint32_t a_tmem = tmem_base + kAColumn0 + (slot * kFeatureBlocks + (uint32_t)fb) * 32u;
+                        const uint32_t a_tmem = tmem_base + kAColumn0 + unit * 32u;
                         const uint32_t b_lo = b_lo0 + (((uint32_t)s * kStageBytes) >> 4);
 #pragma unroll
                         for (int k4 = 0; k4 < BK / 32; ++k4) // 32 bytes of K: 8 columns of A, 2 descriptor units of B
                             mma_i8_ts(d_tmem, a_tmem + 8u * k4, ((uint64_t)desc_hi << 32) | (b_lo + 2u * k4), idesc, 1u);
-                        mma_commit(smem_u32(&bars->a_empty[slot])); // (one commit: it costs the thread as much as an MMA)
+                        mma_commit(smem_u32(&bars->a_empty[unit])); // (one commit: it costs the thread as much as an MMA)
                     }
                     if (++s == n_stages) s = 0;
                 }
@@ -274,57 +274,53 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
             }
         }
     } else if (warp >= kFirstExpanderWarp) {
-        // Expander warp (lane quarter q, slot c): both feature blocks of the k blocks it % 4 == c.  One wait for the stores
-        // of both (a store and its wait take about 300 cycles).  The MMAs of the k block that stood in this slot before
-        // have completed once `a_empty` lets the warp pass: the warp of quarter 0 hands that k block's stage back to the
-        // producer, which spares the MMA threads a second commit.
-        const uint32_t c = (uint32_t)(warp - kFirstExpanderWarp) >> 2; // (warp % 4 is the lane quarter)
+        // Expander warp (lane quarter q, feature block fb, parity par): its 32 rows of feature block fb in the k blocks of
+        // parity par, i.e. in slots par and par + 2 of the A ring in turn.  Every (slot, feature block) unit has barriers
+        // of its own, so that the MMAs of one feature block never wait for the expansion of the other.  The packed words
+        // are loaded before the warp waits for the unit to be free: only the masks, the stores and their wait stand
+        // between the MMAs that free a unit and the MMAs that use it next.  Those MMAs, of the k block four back, have
+        // completed once `a_empty` lets the warp pass: the warps of quarter 0 hand that k block's stage back to the
+        // producer (one arrival per feature block), which spares the MMA threads a second commit.
+        const int e = (warp - kFirstExpanderWarp) >> 2; // (warp % 4 is the lane quarter)
+        const int fb = e & 1;
+        const uint32_t par = (uint32_t)(e >> 1);
         const int j = lane >> 2, kq = lane & 3, h = q & 1, t = q >> 1;
         const int g8 = (j >> 1) + 4 * (j & 1), sl = kq & 1;
-        const uint32_t lane_off = kActBytes + (uint32_t)(t * 2 * kTileBytes) + 512u * (uint32_t)sl + 128u * (uint32_t)(g8 >> 1) +
+        const uint32_t lane_off = kActBytes + (uint32_t)((2 * fb + t) * 2 * kTileBytes) + 512u * (uint32_t)sl + 128u * (uint32_t)(g8 >> 1) +
                                   64u * (uint32_t)((g8 & 1) ^ sl);
         const uint32_t off_e[2] = {16u * (uint32_t)((kq >> 1) ^ (g8 >> 1)), 16u * (uint32_t)((2 + (kq >> 1)) ^ (g8 >> 1))};
         ProblemCursor<kTable> cur(one, table, n_problems);
         uint32_t it = 0, round = 0;
-        int s = 0, s_before = 0; // stage of this k block and of the one four k blocks back
+        int s = 0, s_two_back = 0, s_four_back = 0; // stages of this k block and of this warp's last two
         bool ok = true;
         for (int tile = (int)blockIdx.x; ok && tile < n_tiles; tile += (int)gridDim.x) {
             const int KB = cur.seek(tile).p.KB;
             for (int kb = 0; kb < KB; ++kb, ++it) {
-                if ((it & (kASlots - 1)) == c) {
+                if ((it & 1u) == par) {
+                    const uint32_t unit = (it & (kASlots - 1)) * kFeatureBlocks + (uint32_t)fb;
                     const uint32_t a_use = it / kASlots;
                     if (!mbar_wait_bounded(smem_u32(&bars->full[s]), round & 1, abort_flag, hooks.limit_us)) {
                         ok = false;
                         break;
                     }
-                    // the first feature block's words wait in registers for the slot
-                    const uint8_t *w = smem + (uint32_t)s * kStageBytes + lane_off;
-                    const uint32_t taddr = lane_addr + kAColumn0 + c * (kFeatureBlocks * 32u);
                     uint32_t x[4][2];
                     if (h)
-                        load_unit<1>(x, w, off_e);
+                        load_unit<1>(x, smem + (uint32_t)s * kStageBytes + lane_off, off_e);
                     else
-                        load_unit<0>(x, w, off_e);
-                    if (a_use > 0 && !mbar_wait_bounded(smem_u32(&bars->a_empty[c]), (a_use - 1) & 1, abort_flag, hooks.limit_us)) {
+                        load_unit<0>(x, smem + (uint32_t)s * kStageBytes + lane_off, off_e);
+                    if (a_use > 0 && !mbar_wait_bounded(smem_u32(&bars->a_empty[unit]), (a_use - 1) & 1, abort_flag, hooks.limit_us)) {
                         ok = false;
                         break;
                     }
-                    if (a_use > 0 && q == 0 && lane == 0) mbar_arrive(smem_u32(&bars->stage_empty[s_before]));
+                    if (a_use > 0 && q == 0 && lane == 0) mbar_arrive(smem_u32(&bars->stage_empty[s_four_back]));
                     tc_fence_after_sync();
-                    store_unit(x, taddr);
-#pragma unroll
-                    for (int fb = 1; fb < kFeatureBlocks; ++fb) {
-                        if (h)
-                            load_unit<1>(x, w + fb * 4 * kTileBytes, off_e);
-                        else
-                            load_unit<0>(x, w + fb * 4 * kTileBytes, off_e);
-                        store_unit(x, taddr + 32u * fb);
-                    }
+                    store_unit(x, lane_addr + kAColumn0 + unit * 32u);
                     tmem_st_wait();
                     tc_fence_before_sync();
                     __syncwarp();
-                    if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[c]));
-                    s_before = s;
+                    if (lane == 0) mbar_arrive(smem_u32(&bars->a_full[unit]));
+                    s_four_back = s_two_back;
+                    s_two_back = s;
                 }
                 if (++s == n_stages) {
                     s = 0;
@@ -369,7 +365,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
                 const int n = n0 + 128 * fb + row_in_block;
                 const uint32_t acc = lane_addr + (buf * kFeatureBlocks + (uint32_t)fb) * kAccCols;
 #pragma unroll 1
-                for (int half = 0; half < kTokens / 32; ++half) {
+                for (int half = 0; half < mma_n / 32; ++half) { // (columns no MMA wrote stay zero)
                     uint32_t v[32];
                     tmem_ld_32x32(acc + 32u * half, v);
                     tmem_ld_wait();
@@ -382,6 +378,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
                         const int count = p.M - 32 * half; // tokens of this half that exist (may be <= 0 or > 32)
 #pragma unroll
                         for (int i0 = 0; i0 < 32; i0 += 16) {
+                            if (i0 >= count) break; // (the same for the whole warp)
                             if (p.out_i32) {
                                 int32_t *dst = reinterpret_cast<int32_t *>(p.out) + (size_t)(32 * half + i0) * p.N + n;
                                 int a[16];
@@ -432,7 +429,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
 } // namespace
 
 
-cudaError_t launch_decode_tc(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, cudaStream_t stream)
+cudaError_t launch_decode_tc(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int max_M, cudaStream_t stream)
 {
     const void *kernel = table ? (const void *)decode_tc_kernel<true> : (const void *)decode_tc_kernel<false>;
     int n_stages = stages_that_fit();
@@ -462,7 +459,8 @@ cudaError_t launch_decode_tc(const GemmProblem &one, const GemmProblem *table, i
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     WaitHooks hooks = take_wait_hooks();
-    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles, (void *)&n_stages, (void *)&hooks};
+    int mma_n = max_M <= 32 ? 32 : kTokens;
+    void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles, (void *)&n_stages, (void *)&mma_n, (void *)&hooks};
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }
 

@@ -62,7 +62,8 @@ struct ProblemCursor {
 };
 
 // The weight-stationary form for 17 to 64 tokens (decode_tc.cu) over the CTA tiles of `one`, or of the `n` matmuls of a
-// device table; the tensor map of the weights must be the swizzled one (tma_host.cuh).
-cudaError_t launch_decode_tc(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, cudaStream_t stream);
+// device table; the tensor map of the weights must be the swizzled one (tma_host.cuh).  max_M: the largest M of the
+// launch (at most 64).
+cudaError_t launch_decode_tc(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, int max_M, cudaStream_t stream);
 
 } // namespace bitlinear

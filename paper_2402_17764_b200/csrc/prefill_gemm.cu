@@ -705,7 +705,7 @@ static bool deals_shares(long long n_tiles, long long total_kb, int sms)
 
 // Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
 static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, long long total_kb, int mt,
-                               int a_rows, void *scratch, cudaStream_t stream)
+                               int a_rows, int max_M, void *scratch, cudaStream_t stream)
 {
     const void *kernel = table ? (mt == 2 ? (const void *)prefill_gemm_kernel<2, true> : (const void *)prefill_gemm_kernel<1, true>)
                                : (mt == 2 ? (const void *)prefill_gemm_kernel<2, false> : (const void *)prefill_gemm_kernel<1, false>);
@@ -724,7 +724,7 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
         attr_set[dev] = true;
     }
     if (n_tiles <= 0) return cudaSuccess;
-    if (a_rows == 64) return launch_decode_tc(one, table, n, n_tiles, stream); // 17 to 64 tokens: decode_tc.cu
+    if (a_rows == 64) return launch_decode_tc(one, table, n, n_tiles, max_M, stream); // 17 to 64 tokens: decode_tc.cu
     const int sms = sm_count();
     Schedule sc;
     sc.stream_k = (scratch && deals_shares(n_tiles, total_kb, sms)) ? 1 : 0;
@@ -787,7 +787,7 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
                                  &hdr->status);
     if (e != cudaSuccess) return e;
     const int n_tiles = g.p.tiles_m * g.p.tiles_n;
-    return launch_gemm(g, nullptr, 1, n_tiles, (long long)n_tiles * g.p.KB, mt, a_rows, scratch, stream);
+    return launch_gemm(g, nullptr, 1, n_tiles, (long long)n_tiles * g.p.KB, mt, a_rows, (int)M, scratch, stream);
 }
 
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
@@ -808,7 +808,7 @@ cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int6
 {
     GemmProblem unused{};
     return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, total_kb,
-                       prefill_token_tiles(max_M), prefill_a_rows(max_M), scratch, stream);
+                       prefill_token_tiles(max_M), prefill_a_rows(max_M), (int)max_M, scratch, stream);
 }
 
 } // namespace bitlinear

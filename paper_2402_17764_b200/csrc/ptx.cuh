@@ -63,7 +63,13 @@ __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t byt
 
 // One try: the hardware may keep the thread suspended, without issuing instructions, until the phase completes or about
 // `suspend_ns` have passed.  A polling loop of tries without that hint takes issue slots from the warps that have work.
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_ns = 2000u)
+#ifndef BITLINEAR_WAIT_PAUSE_NS
+#define BITLINEAR_WAIT_PAUSE_NS 32u
+#endif
+#ifndef BITLINEAR_SUSPEND_NS
+#define BITLINEAR_SUSPEND_NS 2000u
+#endif
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity, uint32_t suspend_ns = BITLINEAR_SUSPEND_NS)
 {
     uint32_t ok;
     asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
@@ -88,6 +94,9 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
     const uint64_t limit_ns = (uint64_t)limit_us * 1000ull;
     for (uint32_t spin = 1;; ++spin) {
         if (mbar_try_wait(bar, parity)) return true;
+        // (a failed try returns at once on this part, whatever the hint: without a pause the waiting warps of a CTA take
+        // most of the issue slots from the warps that have work)
+        if (spin > 2u) __nanosleep(BITLINEAR_WAIT_PAUSE_NS);
         if ((spin & 0x1Fu) == 0u) {
             if (*abort_flag) return false;
             const uint64_t now = globaltimer_ns();
