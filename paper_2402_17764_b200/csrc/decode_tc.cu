@@ -66,6 +66,7 @@ constexpr uint32_t kPackedBytes = 8192;        // 4 row blocks x 2 column tiles
 constexpr uint32_t kStageBytes = kActBytes + kPackedBytes;
 constexpr int kMaxStages = 13;
 constexpr uint32_t kSmemLimit = 232448; // 227 KiB
+constexpr uint32_t kLongPauseNs = 400;  // between the polls of the roles that wait long and are not on the critical path
 
 struct Barriers {
     uint64_t full[kMaxStages];        // TMA bytes landed (activations + packed weights)
@@ -213,7 +214,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
                 for (int kb = 0; kb < KB; ++kb, ++it) {
                     if ((it & (kProducerWarps - 1)) == (uint32_t)warp) {
                         if (round > 0 &&
-                            !mbar_wait_bounded(smem_u32(&bars->stage_empty[s]), (round - 1) & 1, abort_flag, hooks.limit_us)) {
+                            !mbar_wait_bounded(smem_u32(&bars->stage_empty[s]), (round - 1) & 1, abort_flag, hooks.limit_us, kLongPauseNs)) {
                             ok = false;
                             break;
                         }
@@ -240,7 +241,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
             const int j = warp - kFirstMmaWarp;
             const int fb = j & 1;
             const uint32_t par = (uint32_t)(j >> 1);
-            const uint32_t idesc = idesc_i8(128, mma_n, /*a_signed=*/0, /*b_signed=*/1); // (32 tokens at most: MMAs of half the width)
+            const uint32_t idesc = idesc_i8(128, mma_n, /*a_signed=*/0, /*b_signed=*/1); // (fewer tokens: narrower, shorter MMAs)
             const uint32_t desc_hi = (uint32_t)(smem_desc_k_sw128(0) >> 32);
             const uint32_t b_lo0 = (uint32_t)smem_desc_k_sw128(base);
             ProblemCursor<kTable> cur(one, table, n_problems);
@@ -355,7 +356,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
                 scale[m] = sc;
             }
             __syncwarp();
-            if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), (tile_it >> 1) & 1, abort_flag, hooks.limit_us)) break;
+            if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), (tile_it >> 1) & 1, abort_flag, hooks.limit_us, kLongPauseNs)) break;
             tc_fence_after_sync();
             uint32_t z[16];
 #pragma unroll
@@ -365,7 +366,7 @@ decode_tc_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__r
                 const int n = n0 + 128 * fb + row_in_block;
                 const uint32_t acc = lane_addr + (buf * kFeatureBlocks + (uint32_t)fb) * kAccCols;
 #pragma unroll 1
-                for (int half = 0; half < mma_n / 32; ++half) { // (columns no MMA wrote stay zero)
+                for (int half = 0; 32 * half < mma_n; ++half) { // (columns no MMA wrote stay zero)
                     uint32_t v[32];
                     tmem_ld_32x32(acc + 32u * half, v);
                     tmem_ld_wait();
@@ -459,7 +460,7 @@ cudaError_t launch_decode_tc(const GemmProblem &one, const GemmProblem *table, i
     cfg.attrs = &attr;
     cfg.numAttrs = 1;
     WaitHooks hooks = take_wait_hooks();
-    int mma_n = max_M <= 32 ? 32 : kTokens;
+    int mma_n = max_M <= 32 ? 32 : (max_M <= 48 ? 48 : kTokens); // columns of the MMAs: the tokens, rounded up to 16
     void *args[] = {(void *)&one, (void *)&table, (void *)&n, (void *)&n_tiles, (void *)&n_stages, (void *)&mma_n, (void *)&hooks};
     return cudaLaunchKernelExC(&cfg, kernel, args);
 }

@@ -1,8 +1,9 @@
-// Kernel (d): ternary x int8 GEMM for 17 tokens and more on the tcgen05 tensor cores.
+// Kernel (d): ternary x int8 GEMM for 65 tokens and more on the tcgen05 tensor cores (17 to 64 tokens: decode_tc.cu,
+// which this file's launchers hand those launches to).
 //
 // With hundreds of tokens every weight is reused hundreds of times, so the integer matmul
 // (Section 1 / Section 3 "Energy": matrix multiplication dominates) is a dense contraction and
-// belongs on the tensor cores; from 17 to 128 tokens the same kernel streams the weights faster than the
+// belongs on the tensor cores; from 65 to 128 tokens the same kernel streams the weights faster than the
 // warp-level MMAs of the decode kernel can.  Per CTA tile of 128 tokens x 256 output features, per 128-wide
 // k block:
 //   producer warp  : TMA loads the int8 activation tile (128 x 128 B, 128-byte swizzle) and the
@@ -80,8 +81,8 @@ struct Cfg {
 // What waits on memory (the TMA stages) and what the expander hands to the tensor core (the expanded tiles)
 // have rings of their own: the expanded tile is four times the packed one, and with one ring the 227 KiB held
 // three or four k blocks in flight, too few to cover the latency of HBM when the weights are streamed once
-// (few tokens).  A stage's activation part is a_rows rows of 128 bytes per token tile: 128, or 64 when no matmul
-// of the launch has more than 64 tokens (the MMAs then have M = 64).
+// (few tokens).  A stage's activation part is a_rows = 128 rows of 128 bytes per token tile (launches whose largest M
+// is 64 or less ask for 64 rows and go to the weight-stationary kernel of decode_tc.cu instead).
 constexpr uint32_t kSmemLimit = 232448; // 227 KiB
 constexpr uint32_t kBarrierBytes = 512;
 __host__ __device__ constexpr uint32_t stage_bytes(int mt, int a_rows) { return (uint32_t)(mt * a_rows * BK) + kPBytes; }
@@ -308,9 +309,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         // so there is one wait and one commit per k block: `expanded` implies `full` (the expander warps waited for
         // the stage before they arrived), and `empty` also tells the expander that the expanded tile was read.
         if (lane == 0) {
-            // With 64 activation rows per stage the MMA has M = 64: half the operand reads from shared memory.  Its
-            // accumulator rows 16 i .. 16 i + 15 stand in TMEM lanes 32 i .. 32 i + 15.
-            const uint32_t idesc = idesc_i8(a_rows == 64 ? 64 : BM, BN, /*a_signed=*/1, /*b_signed=*/0);
+            const uint32_t idesc = idesc_i8(BM, BN, /*a_signed=*/1, /*b_signed=*/0);
             UnitWalker<kTable> walk(sc, one, table, n_problems);
             uint32_t tile_it = 0;
             bool ok = true;
@@ -498,7 +497,6 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             };
             // the token whose sums this thread's TMEM lane holds (past M: none)
             auto token_of_lane = [&](int half) {
-                if (MT == 1 && a_rows == 64) return lane < 16 ? m0 + 16 * q + lane : 0x7FFFFFFF; // M = 64 MMA: see above
                 return m0 + half * BM + 32 * q + lane;
             };
             auto token_scale = [&](int t, int &rowsum, float &scale) {

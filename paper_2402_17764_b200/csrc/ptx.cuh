@@ -85,7 +85,10 @@ constexpr uint32_t kWaitLimitUs = 2000000u; // 2 s
 
 // Waits for the phase with the given parity to complete.  Returns false if another thread already
 // raised the CTA's abort flag or if the limit expired (then raises the flag itself).
-__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t limit_us)
+// pause_ns: how long the thread sleeps between two tries (roles whose waits are long and not on the critical path pass
+// a long pause: every poll takes issue slots from the warps that have work).
+__device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity, volatile int *abort_flag, uint32_t limit_us,
+                                                  uint32_t pause_ns = BITLINEAR_WAIT_PAUSE_NS)
 {
     if (mbar_try_wait(bar, parity)) return true;
     // The global timer is read only every 32nd failed try (a read costs far more than a try), so the limit counts
@@ -96,7 +99,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
         if (mbar_try_wait(bar, parity)) return true;
         // (a failed try returns at once on this part, whatever the hint: without a pause the waiting warps of a CTA take
         // most of the issue slots from the warps that have work)
-        if (spin > 2u) __nanosleep(BITLINEAR_WAIT_PAUSE_NS);
+        if (pause_ns != 0u && (spin > 2u || pause_ns > BITLINEAR_WAIT_PAUSE_NS)) __nanosleep(pause_ns);
         if ((spin & 0x1Fu) == 0u) {
             if (*abort_flag) return false;
             const uint64_t now = globaltimer_ns();
