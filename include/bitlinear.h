@@ -60,7 +60,7 @@ enum {
     BITLINEAR_PATH_AUTO = 0,
     BITLINEAR_PATH_DP4A = 1,   /* scalar dp4a, M <= 8 */
     BITLINEAR_PATH_MMA = 2,    /* warp-level integer MMA on register-unpacked weights, M <= 64 */
-    BITLINEAR_PATH_TCGEN05 = 3 /* TMA + tcgen05 int8 tensor-core GEMM with TMEM accumulators, any M */
+    BITLINEAR_PATH_TCGEN05 = 3 /* TMA + tcgen05 int8 tensor cores, any M: up to 64 tokens the weight-stationary kernel, beyond it the GEMM */
 };
 
 /* Human-readable name of a status code; never NULL. (host) */
@@ -240,8 +240,9 @@ bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma
  * A list of independent BitLinear forwards executed by one persistent launch (the seven projections of
  * every decoder layer of a decode step, Section 2 "LLaMA-alike Components").  All inputs X must be
  * ready when the call is enqueued: entries do not depend on each other.  The entries may have different M;
- * the largest decides the kernel for all of them: up to 16 tokens the weight-streaming kernel, from 17 on the
- * tensor-core GEMM walking the CTA tiles of all matmuls in one launch.
+ * the largest decides the kernel for all of them: up to 16 tokens the weight-streaming kernel, from 17 on a
+ * tensor-core kernel (weights stationary in tensor memory up to 64 tokens, the GEMM beyond) walking the CTA tiles
+ * of all matmuls in one launch.
  */
 typedef struct {
     const void *packed; /* device */
