@@ -96,7 +96,7 @@ Layout single_layout(int64_t M, int64_t N, int64_t K)
     size_t off = sizeof(WorkspaceHeader);
     L.acc32 = off;
     const size_t decode_scratch = (size_t)(M < kMaxDecodeM ? M : kMaxDecodeM) * N * 4;
-    const size_t gemm_scratch = M > 0 ? prefill_scratch_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M), M) : 0;
+    const size_t gemm_scratch = M > 0 ? prefill_scratch_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M), gemm_k_blocks(K), M) : 0;
     off += align_up(decode_scratch > gemm_scratch ? decode_scratch : gemm_scratch, 256);
     L.table = off; // end of what is cleared before every call
     L.lists = off;
@@ -385,7 +385,7 @@ bitlinear_status forward_impl(const void *packed, const float *gamma, const void
     inl.e[0].up = reinterpret_cast<const __nv_bfloat16 *>(up);
     inl.e[0].qb = (float)((1 << (act_bits - 1)) - 1);
     // quantise the tokens; the same launch clears the header and the scratch of the kernel that follows, if it uses it
-    const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M)) : 0;
+    const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, (int)M, ws, zero_bytes, (gain ? 1 : 0) | (up ? 2 : 0), (int)K,
@@ -435,7 +435,7 @@ bitlinear_status matmul_i32_impl(const void *packed, const int8_t *Xq, int64_t M
     const bool tc = !trits && ((path == BITLINEAR_PATH_TCGEN05) || (path == BITLINEAR_PATH_AUTO && use_tcgen05_for(M)));
     InlineTable inl{};
     fill_entry(inl.e[0], packed, nullptr, nullptr, M, K, N, acc, 1, ws, L, trits);
-    const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M)) : 0;
+    const size_t clear = tc ? prefill_scratch_clear_bytes(prefill_tile_count(M, N, M), prefill_kb_count(M, N, K, M), gemm_k_blocks(K), M) : 0;
     const bool split = clear > 0;
     const size_t zero_bytes = tc ? L.acc32 + align_up(clear, 256) : L.table;
     cudaError_t err = launch_quantize_acts(inl, nullptr, 1, 0, ws, zero_bytes, false, (int)K, s);
@@ -565,7 +565,7 @@ struct bitlinear_sequence {
     bitlinear::InlineTable inl;
     const void *gemm_table; // inside the workspace; null: the weight-streaming kernel runs the sequence
     int gemm_tiles;
-    int64_t gemm_total_kb;
+    int64_t gemm_total_kb, gemm_min_kb;
     int fronts;             // bit 0: some entry has an RMSNorm in front of the quantiser, bit 1: some entry a SwiGLU
     void *split_scratch;    // inside the workspace; null: the GEMM deals this sequence's tiles whole
     bool trits;             // the weights are in the base-3 format
@@ -577,6 +577,7 @@ struct SeqLayout {
     size_t acc32, table, lists, gemm, data, total;
     bool use_gemm;
     int64_t gemm_tiles, gemm_total_kb; // CTA tiles and k blocks (tiles x k blocks each) of all matmuls on the GEMM
+    int64_t gemm_min_kb;               // the fewest k blocks any of them has
 };
 
 inline size_t seq_xq_bytes(int64_t M, int64_t K, bool gemm)
@@ -608,13 +609,15 @@ bool seq_layout(const bitlinear_layer_desc *layers, int n, SeqLayout &S, std::ve
     if (tiles > 0xFFFFFFFFull) return false; // the tile sequence is indexed with 32 bits (4 TiB of weights)
     if (tokens > 0x3FFFFFFFull) return false; // tokens (plus the clearing CTAs) index the quantiser's grid with an int
     if (gemm && gemm_tiles > 0x7FFFFFFFull) return false;
-    S.gemm_tiles = S.gemm_total_kb = 0;
+    S.gemm_tiles = S.gemm_total_kb = S.gemm_min_kb = 0;
     if (gemm) { // the GEMM's scratch, where the streaming kernel has its int32 scratch
         for (int i = 0; i < n; ++i) {
             S.gemm_tiles += prefill_tile_count(layers[i].M, layers[i].N, max_M);
             S.gemm_total_kb += prefill_kb_count(layers[i].M, layers[i].N, layers[i].K, max_M);
+            const int64_t kb = gemm_k_blocks(layers[i].K);
+            if (i == 0 || kb < S.gemm_min_kb) S.gemm_min_kb = kb;
         }
-        acc = align_up(prefill_scratch_bytes(S.gemm_tiles, S.gemm_total_kb, max_M), 256);
+        acc = align_up(prefill_scratch_bytes(S.gemm_tiles, S.gemm_total_kb, S.gemm_min_kb, max_M), 256);
     }
     size_t off = sizeof(WorkspaceHeader);
     S.acc32 = off;
@@ -759,13 +762,14 @@ bitlinear_status sequence_create_impl(const bitlinear_layer_desc *layers, const 
     seq->max_K = 0;
     for (int i = 0; i < n; ++i)
         if ((int)layers[i].K > seq->max_K) seq->max_K = (int)layers[i].K;
-    const size_t clear = gemm ? prefill_scratch_clear_bytes(gemm_tiles, gemm_kb) : 0;
+    const size_t clear = gemm ? prefill_scratch_clear_bytes(gemm_tiles, gemm_kb, S.gemm_min_kb, max_M) : 0;
     const bool split = clear > 0;
     seq->zero_bytes = gemm ? S.acc32 + align_up(clear, 256) : S.table; // header and the int32 scratch in use
     seq->dev_table = nullptr;
     seq->gemm_table = nullptr;
     seq->gemm_tiles = gemm_tiles;
     seq->gemm_total_kb = gemm_kb;
+    seq->gemm_min_kb = S.gemm_min_kb;
     seq->fronts = fronts;
     seq->trits = trits;
     seq->wide = wide;
@@ -803,7 +807,7 @@ bitlinear_status bitlinear_forward_sequence_stage(const bitlinear_sequence *seq,
         return BITLINEAR_ERR_CUDA;
     if (stage != 1) {
         const cudaError_t err =
-            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->gemm_total_kb, seq->max_M,
+            seq->gemm_table ? launch_prefill_table(seq->gemm_table, seq->n, seq->gemm_tiles, seq->gemm_total_kb, seq->gemm_min_kb, seq->max_M,
                                                  seq->split_scratch, s)
                             : launch_decode(seq->inl, seq->dev_table, seq->n, seq->tiles, seq->max_M, BITLINEAR_PATH_MMA,
                                             reinterpret_cast<WorkspaceHeader *>(seq->workspace), seq->lists, s, seq->trits, seq->wide);

@@ -130,8 +130,10 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
 // many bytes at the start of that scratch must be zero when the launch starts.
 int64_t prefill_tile_count(int64_t M, int64_t N, int64_t max_M);
 int64_t prefill_kb_count(int64_t M, int64_t N, int64_t K, int64_t max_M); // tiles x k blocks of one matmul
-size_t prefill_scratch_bytes(int64_t n_tiles, int64_t total_kb, int64_t max_M);
-size_t prefill_scratch_clear_bytes(int64_t n_tiles, int64_t total_kb);
+// min_kb: the fewest k blocks any matmul of the launch has (a launch of few tiles splits every tile among several CTAs
+// along K when all its matmuls are long enough for that).
+size_t prefill_scratch_bytes(int64_t n_tiles, int64_t total_kb, int64_t min_kb, int64_t max_M);
+size_t prefill_scratch_clear_bytes(int64_t n_tiles, int64_t total_kb, int64_t min_kb, int64_t max_M);
 
 // The same kernel over the matmuls of a sequence in ONE launch.  The host fills a table of kGemmProblemBytes-sized
 // entries (tensor maps + parameters) with prefill_table_entry, copies it to device memory (64-byte aligned) once, and
@@ -143,8 +145,8 @@ int prefill_token_tiles(int64_t max_M);
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
                                 const int32_t *rowsum, int64_t M, int64_t x_rows, int64_t K, int64_t N, void *out,
                                 float qb, int64_t max_M, int tile_begin, int64_t kb_begin, WorkspaceHeader *hdr, int *n_tiles);
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t total_kb, int64_t max_M, void *scratch,
-                                 cudaStream_t stream);
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t total_kb, int64_t min_kb, int64_t max_M,
+                                 void *scratch, cudaStream_t stream);
 
 // What a matmul launch is told about its bounded device-side waits.  limit_us: how long a wait may last (2 s unless
 // a test shortened it).  skip_arrive != 0 is a test device: ONE producer thread of the launch (in CTA 0) leaves out ONE

@@ -25,7 +25,9 @@
 // memory): the CTAs walk one launch-wide sequence of CTA tiles.  When whole tiles would leave many SMs idle in the
 // last round (160 tiles on 148 SMs), the launch instead gives every CTA an equal, contiguous share of the sequence of
 // K BLOCKS of all tiles: a CTA's share then begins and ends inside tiles, the tile it begins in is finished by the CTA
-// in front of it, and partial sums travel through a scratch slot per CTA (see Schedule below).
+// in front of it, and partial sums travel through a scratch slot per CTA (see Schedule below).  With at most half as many
+// tiles as SMs every tile is split along K among several CTAs, each of which then finishes its part of the tile's outputs
+// (split_factor below).
 // The kernel is a programmatic dependent of the activation quantiser: set-up (barriers, tensor memory,
 // descriptor prefetch) runs while the quantiser finishes; the producer waits for it before the first load.
 // All waits are bounded; on expiry the CTA sets the workspace status to BITLINEAR_ERR_TIMEOUT,
@@ -121,8 +123,11 @@ static_assert(sizeof(Barriers) <= kBarrierBytes, "barrier block");
 //     CTA that holds the tile's last k block), which were those CTAs' first work and are long done; the finisher waits
 //     for their flags (a bounded wait), adds their slots to its own sums and dequantises.  No CTA ever waits for work
 //     that itself waits, flags must be zero when the launch starts, slots need no clearing.
+//   split tiles (stream_k == 2): tile t belongs to CTAs s t .. s t + s - 1, each with 1/s of its k blocks (its only
+//     unit) and 1/s of its outputs to finish: see split_factor.
 struct Schedule {
-    int stream_k;
+    int stream_k; // 0: whole tiles, 1: k-block shares, 2: split tiles
+    int split;    // split tiles: CTAs per tile
     int n_tiles;
     long long total_kb;
     uint32_t *flags; // one word per CTA
@@ -142,11 +147,12 @@ static_assert(4 * kFetchBufs * kFetchBytes <= 3 * 64 * 1024, "the fetch buffers 
 // have this layout (they reach shared memory by bulk copies, as they are).
 __device__ __forceinline__ uint32_t slot_piece(int lane, int piece) { return (uint32_t)(lane * 128 + ((piece ^ (lane & 7)) << 4)); }
 
-enum UnitKind { kWholeTile = 0, kContribution = 1, kFinisher = 2 };
+enum UnitKind { kWholeTile = 0, kContribution = 1, kFinisher = 2, kSplit = 3 };
 
 struct Unit {
     int tile, kb0, kb1, kind;
     int last_contributor; // finisher: the contributions are the first units of CTAs blockIdx.x + 1 .. last_contributor
+    int split_s, split_r; // split tile: the tile belongs to split_s CTAs, this one is number split_r of them
 };
 
 // Position in the ring of TMA stages and in the ring of expanded tiles after `it` k blocks.
@@ -175,7 +181,7 @@ struct UnitWalker {
     __device__ UnitWalker(const Schedule &sc_, const GemmProblem &one, const GemmProblem *t, int n)
         : sc(sc_), cur(one, t, n), next_tile((int)blockIdx.x), pos(0), end(0)
     {
-        if (sc.stream_k) {
+        if (sc.stream_k == 1) {
             pos = (long long)blockIdx.x * sc.total_kb / (long long)gridDim.x;
             end = (long long)(blockIdx.x + 1) * sc.total_kb / (long long)gridDim.x;
         }
@@ -183,6 +189,23 @@ struct UnitWalker {
     // the next unit and its matmul; false: none is left
     __device__ bool next(Unit &u, const GemmProblem *&g)
     {
+        u.split_s = 1;
+        u.split_r = 0;
+        if (sc.stream_k == 2) { // split tiles: CTA b is number b % s of the s CTAs of tile b / s, its only unit
+            if (next_tile < 0) return false;
+            const int s = sc.split;
+            u.tile = (int)blockIdx.x / s;
+            u.split_s = s;
+            u.split_r = (int)blockIdx.x % s;
+            g = &cur.seek(u.tile);
+            const int KB = g->p.KB;
+            u.kb0 = (int)((long long)u.split_r * KB / s);
+            u.kb1 = (int)((long long)(u.split_r + 1) * KB / s);
+            u.kind = kSplit;
+            u.last_contributor = 0;
+            next_tile = -1;
+            return true;
+        }
         if (!sc.stream_k) {
             if (next_tile >= sc.n_tiles) return false;
             g = &cur.seek(next_tile);
@@ -514,13 +537,30 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                        (size_t)((half * 4 + q) * (BN / 32) + c) * 4096;
             };
 
-            if (unit.kind == kContribution) {
-                // partial sums of a tile that another CTA finishes: to this CTA's slot as they are, then the flag
+            // The sums of a tile are handled as jobs: (token tile, pair of chunks of 32 features), this warp's lane quarter
+            // of each.  A whole tile: the CTA finishes all jobs, nothing to fetch.  A contribution: all jobs go to the
+            // CTA's slot.  A finisher: all jobs, with the slots of the CTAs behind it added.  A split tile: the CTA
+            // finishes the jobs r, r + s, ... with the slots of the other CTAs of its tile added, and writes the rest.
+            constexpr int kPairs = BN / 32 / (int)kFetchChunks;
+            const int n_jobs_tile = halves * kPairs;
+            const bool split = unit.kind == kSplit;
+            const int job_start = split ? unit.split_r : 0, job_stride = split ? unit.split_s : 1;
+            const int n_contrib = unit.kind == kFinisher ? unit.last_contributor - (int)blockIdx.x : (split ? unit.split_s - 1 : 0);
+            // the CTA whose slot holds the j-th contribution
+            auto contributor = [&](int j) {
+                if (split) return (int)blockIdx.x - unit.split_r + (j < unit.split_r ? j : j + 1);
+                return (int)blockIdx.x + 1 + j;
+            };
+
+            if (unit.kind == kContribution || split) {
+                // partial sums that another CTA finishes: to this CTA's slot as they are, then the flag
 #pragma unroll 1
-                for (int half = 0; half < halves; ++half) {
+                for (int jb = 0; jb < n_jobs_tile; ++jb) {
+                    if (split && jb % job_stride == job_start) continue; // (finished here: stays in tensor memory)
+                    const int half = jb / kPairs;
                     const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
 #pragma unroll 1
-                    for (int c = 0; c < BN / 32; ++c) {
+                    for (int c = (jb % kPairs) * (int)kFetchChunks; c < (jb % kPairs + 1) * (int)kFetchChunks; ++c) {
                         uint32_t v[32];
                         tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)(c * 32), v);
                         tmem_ld_wait();
@@ -535,39 +575,37 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 __threadfence(); // this thread's stores are visible to the whole GPU before the flag can be
                 __syncwarp();
                 if (lane == 0) {
-                    mbar_arrive(smem_u32(&bars->acc_empty[buf]));
+                    if (!split) mbar_arrive(smem_u32(&bars->acc_empty[buf]));
                     mbar_arrive(smem_u32(&bars->epilogue_met));
                 }
-                // the four epilogue warps meet (a contribution is the CTA's first unit: phase 0 of this barrier), then
-                // one thread raises the flag
+                // the four epilogue warps meet (a contribution is the CTA's first unit, a split tile its only one: phase 0
+                // of this barrier), then one thread raises the flag
                 if (!mbar_wait_bounded(smem_u32(&bars->epilogue_met), 0, abort_flag, hooks.limit_us)) break;
                 if (warp == 2 && lane == 0) st_release_gpu(sc.flags + blockIdx.x, 1u);
-                continue;
+                if (!split) continue;
             }
 
-            // The other parts of a finisher's tile are in the slots of the CTAs behind this one, once their flags are up.
-            // They are fetched piece by piece (kFetchChunks chunks of one contribution) into this warp's buffers, in
-            // the order in which they are added: token tile, chunk pair, contribution.
-            const int n_contrib = unit.kind == kFinisher ? unit.last_contributor - (int)blockIdx.x : 0;
-            const int n_jobs = n_contrib * halves * (BN / 32 / (int)kFetchChunks);
+            // The jobs this CTA finishes.  The parts of other CTAs are in their slots once their flags are up.  They are
+            // fetched piece by piece (the kFetchChunks chunks of one job of one contribution) into this warp's buffers,
+            // in the order in which they are added: job, contribution.
+            const int n_mine = job_start < n_jobs_tile ? (n_jobs_tile - job_start + job_stride - 1) / job_stride : 0;
+            const int n_fetches = n_contrib * n_mine;
             uint8_t *fetch_base = smem + q * (kFetchBufs * kFetchBytes);
             int issued = 0, taken = 0;
             auto issue_fetches = [&]() { // lane 0 only
-                while (issued < n_jobs && issued - taken < kFetchBufs) {
-                    const int j = issued % n_contrib, pair = (issued / n_contrib) % (BN / 32 / (int)kFetchChunks),
-                              half = issued / (n_contrib * (BN / 32 / (int)kFetchChunks));
+                while (issued < n_fetches && issued - taken < kFetchBufs) {
+                    const int j = issued % n_contrib, jb = job_start + (issued / n_contrib) * job_stride;
                     const int b = issued % kFetchBufs;
                     const uint32_t bar = smem_u32(&bars->fetched[q][b]);
                     mbar_arrive_expect_tx(bar, kFetchBytes);
                     bulk_copy_g2s(smem_u32(fetch_base + b * kFetchBytes),
-                                  slot_chunk((int)blockIdx.x + 1 + j, half, pair * (int)kFetchChunks), kFetchBytes, bar);
+                                  slot_chunk(contributor(j), jb / kPairs, (jb % kPairs) * (int)kFetchChunks), kFetchBytes, bar);
                     ++issued;
                 }
             };
-            if (n_contrib > 0) {
+            if (n_fetches > 0) {
                 bool ok = true;
-                for (int cta = (int)blockIdx.x + 1; cta <= unit.last_contributor && ok; ++cta)
-                    ok = flag_wait_bounded(sc.flags + cta, abort_flag, hooks.limit_us);
+                for (int j = 0; j < n_contrib && ok; ++j) ok = flag_wait_bounded(sc.flags + contributor(j), abort_flag, hooks.limit_us);
                 if (!ok) break;
                 fence_proxy_async_smem(); // (the buffers were last touched through the generic proxy or by the tensor core)
                 __syncwarp();
@@ -575,46 +613,45 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             }
             bool alive = true;
 #pragma unroll 1
-            for (int half = 0; half < halves && alive; ++half) {
+            for (int mj = 0; mj < n_mine && alive; ++mj) {
+                const int jb = job_start + mj * job_stride;
+                const int half = jb / kPairs, c0 = (jb % kPairs) * (int)kFetchChunks;
                 const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
                 const int t = token_of_lane(half);
                 int rowsum;
                 float scale;
                 token_scale(t, rowsum, scale);
-#pragma unroll 1
-                for (int c0 = 0; c0 < BN / 32 && alive; c0 += (int)kFetchChunks) {
-                    uint32_t v[kFetchChunks][32];
+                uint32_t v[kFetchChunks][32];
 #pragma unroll
-                    for (int cc = 0; cc < (int)kFetchChunks; ++cc)
-                        tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)((c0 + cc) * 32), v[cc]);
-                    tmem_ld_wait();
-                    for (int j = 0; j < n_contrib; ++j) {
-                        const int b = taken % kFetchBufs;
-                        if (!mbar_wait_bounded(smem_u32(&bars->fetched[q][b]), (uint32_t)(taken / kFetchBufs) & 1u, abort_flag,
-                                               hooks.limit_us)) {
-                            alive = false;
-                            break;
-                        }
-                        const uint8_t *src = fetch_base + b * kFetchBytes;
-#pragma unroll
-                        for (int cc = 0; cc < (int)kFetchChunks; ++cc) {
-#pragma unroll
-                            for (int pc = 0; pc < 8; ++pc) {
-                                const uint4 w = *reinterpret_cast<const uint4 *>(src + cc * 4096 + slot_piece(lane, pc));
-                                v[cc][4 * pc] += w.x;
-                                v[cc][4 * pc + 1] += w.y;
-                                v[cc][4 * pc + 2] += w.z;
-                                v[cc][4 * pc + 3] += w.w;
-                            }
-                        }
-                        __syncwarp(); // every lane has read the buffer before lane 0 refills it
-                        ++taken;
-                        if (lane == 0) issue_fetches();
+                for (int cc = 0; cc < (int)kFetchChunks; ++cc)
+                    tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)((c0 + cc) * 32), v[cc]);
+                tmem_ld_wait();
+                for (int j = 0; j < n_contrib; ++j) {
+                    const int b = taken % kFetchBufs;
+                    if (!mbar_wait_bounded(smem_u32(&bars->fetched[q][b]), (uint32_t)(taken / kFetchBufs) & 1u, abort_flag,
+                                           hooks.limit_us)) {
+                        alive = false;
+                        break;
                     }
-                    if (!alive) break;
+                    const uint8_t *src = fetch_base + b * kFetchBytes;
 #pragma unroll
-                    for (int cc = 0; cc < (int)kFetchChunks; ++cc) emit(v[cc], c0 + cc, t, rowsum, scale);
+                    for (int cc = 0; cc < (int)kFetchChunks; ++cc) {
+#pragma unroll
+                        for (int pc = 0; pc < 8; ++pc) {
+                            const uint4 w = *reinterpret_cast<const uint4 *>(src + cc * 4096 + slot_piece(lane, pc));
+                            v[cc][4 * pc] += w.x;
+                            v[cc][4 * pc + 1] += w.y;
+                            v[cc][4 * pc + 2] += w.z;
+                            v[cc][4 * pc + 3] += w.w;
+                        }
+                    }
+                    __syncwarp(); // every lane has read the buffer before lane 0 refills it
+                    ++taken;
+                    if (lane == 0) issue_fetches();
                 }
+                if (!alive) break;
+#pragma unroll
+                for (int cc = 0; cc < (int)kFetchChunks; ++cc) emit(v[cc], c0 + cc, t, rowsum, scale);
             }
             if (!alive) break;
             tc_fence_before_sync();
@@ -701,9 +738,32 @@ static bool deals_shares(long long n_tiles, long long total_kb, int sms)
     return idle_kb >= kMinIdleKb;
 }
 
+// Split tiles.  A launch with so few CTA tiles that at least half of the SMs would have none gives every tile to s CTAs,
+// each with 1/s of the tile's k blocks and, afterwards, 1/s of its outputs to finish: every CTA writes the partial sums of
+// the jobs it does not finish to its slot, raises its flag, waits for the flags of the other CTAs of its tile and adds
+// their parts of its own jobs.  All CTAs are resident at once (grid = n_tiles * s <= SMs, one CTA per SM) and every CTA
+// raises its flag before it waits, so the waits end.  s is the largest number with n_tiles * s <= SMs that leaves every
+// CTA kMinSplitKb k blocks of the shortest matmul (and at most kMaxSplit: what a CTA writes and fetches grows with s).
+constexpr long long kMinSplitKb = 8, kMaxSplit = 8;
+static int split_factor(long long n_tiles, long long min_kb, int sms)
+{
+#ifdef BITLINEAR_TUNING // measurement aid, not compiled into the library as build.py builds it
+    static const int enabled = [] {
+        const char *v = std::getenv("BITLINEAR_PREFILL_SPLIT_TILES");
+        return (v && *v) ? std::atoi(v) : 1;
+    }();
+    if (!enabled) return 1;
+#endif
+    if (n_tiles <= 0) return 1;
+    long long s = sms / n_tiles;
+    if (s > min_kb / kMinSplitKb) s = min_kb / kMinSplitKb;
+    if (s > kMaxSplit) s = kMaxSplit;
+    return s >= 2 ? (int)s : 1;
+}
+
 // Launches the kernel over `n_tiles` CTA tiles: of `one`, or of the `n` matmuls of a device table.
-static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, long long total_kb, int mt,
-                               int a_rows, int max_M, void *scratch, cudaStream_t stream)
+static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table, int n, int n_tiles, long long total_kb,
+                               long long min_kb, int mt, int a_rows, int max_M, void *scratch, cudaStream_t stream)
 {
     const void *kernel = table ? (mt == 2 ? (const void *)prefill_gemm_kernel<2, true> : (const void *)prefill_gemm_kernel<1, true>)
                                : (mt == 2 ? (const void *)prefill_gemm_kernel<2, false> : (const void *)prefill_gemm_kernel<1, false>);
@@ -725,12 +785,13 @@ static cudaError_t launch_gemm(const GemmProblem &one, const GemmProblem *table,
     if (a_rows == 64) return launch_decode_tc(one, table, n, n_tiles, max_M, stream); // 17 to 64 tokens: decode_tc.cu
     const int sms = sm_count();
     Schedule sc;
-    sc.stream_k = (scratch && deals_shares(n_tiles, total_kb, sms)) ? 1 : 0;
+    sc.split = scratch ? split_factor(n_tiles, min_kb, sms) : 1;
+    sc.stream_k = sc.split > 1 ? 2 : ((scratch && deals_shares(n_tiles, total_kb, sms)) ? 1 : 0);
     sc.n_tiles = n_tiles;
     sc.total_kb = total_kb;
     sc.flags = reinterpret_cast<uint32_t *>(scratch);
     sc.slots = reinterpret_cast<int32_t *>(reinterpret_cast<char *>(scratch) + kFlagBytes);
-    int grid = sc.stream_k ? sms : (n_tiles < sms ? n_tiles : sms);
+    int grid = sc.stream_k == 2 ? n_tiles * sc.split : (sc.stream_k ? sms : (n_tiles < sms ? n_tiles : sms));
     // programmatic dependent launch: see the head of this file
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
@@ -759,17 +820,20 @@ int64_t prefill_tile_count(int64_t M, int64_t N, int64_t max_M)
 
 int64_t prefill_kb_count(int64_t M, int64_t N, int64_t K, int64_t max_M) { return prefill_tile_count(M, N, max_M) * ((K + BK - 1) / BK); }
 
-size_t prefill_scratch_bytes(int64_t n_tiles, int64_t total_kb, int64_t max_M)
+size_t prefill_scratch_bytes(int64_t n_tiles, int64_t total_kb, int64_t min_kb, int64_t max_M)
 {
     static_assert(kFlagBytes >= 4 * 148, "one flag per CTA");
+    if (max_M <= 64) return 0; // (the weight-stationary kernel deals whole tiles)
     const int sms = sm_count();
-    if (!deals_shares(n_tiles, total_kb, sms)) return 0;
-    return kFlagBytes + (size_t)sms * (size_t)prefill_token_tiles(max_M) * kSlotTileBytes;
+    const int s = split_factor(n_tiles, min_kb, sms);
+    if (s < 2 && !deals_shares(n_tiles, total_kb, sms)) return 0;
+    const size_t ctas = s >= 2 ? (size_t)n_tiles * (size_t)s : (size_t)sms; // one slot per CTA of the launch
+    return kFlagBytes + ctas * (size_t)prefill_token_tiles(max_M) * kSlotTileBytes;
 }
 
-size_t prefill_scratch_clear_bytes(int64_t n_tiles, int64_t total_kb)
+size_t prefill_scratch_clear_bytes(int64_t n_tiles, int64_t total_kb, int64_t min_kb, int64_t max_M)
 {
-    return deals_shares(n_tiles, total_kb, sm_count()) ? kFlagBytes : 0;
+    return prefill_scratch_bytes(n_tiles, total_kb, min_kb, max_M) > 0 ? kFlagBytes : 0;
 }
 
 // rows of activations per token tile in a TMA stage, for the largest M of a launch
@@ -785,7 +849,7 @@ cudaError_t launch_prefill(const void *packed, const float *gamma, const int8_t 
                                  &hdr->status);
     if (e != cudaSuccess) return e;
     const int n_tiles = g.p.tiles_m * g.p.tiles_n;
-    return launch_gemm(g, nullptr, 1, n_tiles, (long long)n_tiles * g.p.KB, mt, a_rows, (int)M, scratch, stream);
+    return launch_gemm(g, nullptr, 1, n_tiles, (long long)n_tiles * g.p.KB, g.p.KB, mt, a_rows, (int)M, scratch, stream);
 }
 
 cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gamma, const int8_t *Xq, const float *beta,
@@ -801,11 +865,11 @@ cudaError_t prefill_table_entry(void *slot, const void *packed, const float *gam
     return cudaSuccess;
 }
 
-cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t total_kb, int64_t max_M, void *scratch,
-                                 cudaStream_t stream)
+cudaError_t launch_prefill_table(const void *dev_table, int n, int n_tiles, int64_t total_kb, int64_t min_kb, int64_t max_M,
+                                 void *scratch, cudaStream_t stream)
 {
     GemmProblem unused{};
-    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, total_kb,
+    return launch_gemm(unused, reinterpret_cast<const GemmProblem *>(dev_table), n, n_tiles, total_kb, min_kb,
                        prefill_token_tiles(max_M), prefill_a_rows(max_M), (int)max_M, scratch, stream);
 }
 

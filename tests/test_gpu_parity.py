@@ -208,7 +208,10 @@ TC_SHAPES = [(128, 128, 256), (1, 16, 16), (65, 3200, 320), (200, 8640, 528), (3
              (300, 8640, 272), (40, 16384, 1040),
              # few tiles and a long K: the CTAs take equal shares of the k blocks of all tiles, and tiles whose k blocks
              # lie in several shares are summed through the per-CTA slots (64-row stages, one token tile, two token tiles)
-             (20, 32768, 2560), (100, 32768, 2576), (300, 20000, 2304)]
+             (20, 32768, 2560), (100, 32768, 2576), (300, 20000, 2304),
+             # at most half as many tiles as SMs: every tile is split along K among 2, 3 or 8 CTAs, each of which finishes
+             # its share of the tile's outputs; ragged M, K and N; and one launch that still deals k-block shares
+             (200, 2048, 6400), (512, 3200, 5120), (70, 2096, 528), (300, 4800, 12800)]
 
 
 @pytest.mark.parametrize("M,K,N", TC_SHAPES)
