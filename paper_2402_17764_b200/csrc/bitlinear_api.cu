@@ -128,8 +128,9 @@ __global__ void rowsum_kernel(const int8_t *__restrict__ Xq, int K, int32_t *__r
     }
 }
 
-// From 17 tokens on a single matmul goes to the tensor-core GEMM: measured on 110080 x 4096, the GEMM takes the
-// same 52 us from 17 to 128 tokens, the weight-streaming kernel 59 us at 16 tokens, 92 us at 32 and 174 us at 64.
+// From 17 tokens on a matmul goes to the tensor cores (the launchers of prefill_gemm.cu pick the weight-stationary kernel
+// up to 64 tokens and the GEMM beyond): measured on 110080 x 4096, the weight-streaming kernel takes 59 us at 16 tokens,
+// 92 us at 32 and 174 us at 64, the tensor-core kernels between 45 and 52 us from 17 to 128 tokens.
 // (In a -DBITLINEAR_TUNING build BITLINEAR_TCGEN05_MIN_M moves the switch-over point.)
 bool use_tcgen05_for(int64_t M)
 {
@@ -551,9 +552,9 @@ bitlinear_status bitlinear_forward_static(const void *packed, const float *gamma
 
 // ---- sequences -------------------------------------------------------------------------------
 // Workspace: [header | all acc32 | descriptor table | per-warp lists | GEMM table | per-entry Xq, beta, rowsum]
-// A sequence whose largest matmul has 17 tokens or more runs all its matmuls in one launch of the tensor-core
-// GEMM (no int32 scratch, row-major activations with at least kMinGemmRows rows each); otherwise in one launch
-// of the weight-streaming kernel.
+// A sequence whose largest matmul has 17 tokens or more runs all its matmuls in one launch on the tensor cores (up to 64
+// tokens the weight-stationary kernel of decode_tc.cu, beyond it the GEMM; no int32 scratch, row-major activations with at
+// least kMinGemmRows rows each); otherwise in one launch of the weight-streaming kernel.
 
 struct bitlinear_sequence {
     char *workspace;
