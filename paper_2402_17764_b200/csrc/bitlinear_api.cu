@@ -129,8 +129,9 @@ __global__ void rowsum_kernel(const int8_t *__restrict__ Xq, int K, int32_t *__r
 }
 
 // From 17 tokens on a matmul goes to the tensor cores (the launchers of prefill_gemm.cu pick the weight-stationary kernel
-// up to 64 tokens and the GEMM beyond): measured on 110080 x 4096, the weight-streaming kernel takes 59 us at 16 tokens,
-// 92 us at 32 and 174 us at 64, the tensor-core kernels between 45 and 52 us from 17 to 128 tokens.
+// up to 64 tokens and the GEMM beyond): measured on 110080 x 4096 (whole forward, the 113 MB of weights resident in L2),
+// the weight-streaming kernel takes 48 us at 16 tokens, 92 us at 32 and 174 us at 64; the weight-stationary kernel 39, 40
+// and 42 us at 17, 32 and 64 tokens, the GEMM 57 us at 128.
 // (In a -DBITLINEAR_TUNING build BITLINEAR_TCGEN05_MIN_M moves the switch-over point.)
 bool use_tcgen05_for(int64_t M)
 {
