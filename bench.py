@@ -875,17 +875,19 @@ def profile_case(name: str):
         print(json.dumps({"case": name, "packed_bytes_per_launch": st.weights.stored_bytes,
                           "matmul_kernel_ms": round(ms, 4), "GB/s": round(st.weights.stored_bytes / ms / 1e6, 1)}))
     elif name.startswith("prefill"):
-        # 13824x5120 at M = 2048 (or prefill:M): 290 G integer operations per launch
-        M = int(name.split(":")[1]) if ":" in name else 2048
-        W = S.latent_weights(13824, 5120, 0, device="cuda")
+        # 13824x5120 at M = 2048 (290 G integer operations per launch), or prefill:M, or prefill:M:N:K
+        parts = name.split(":")
+        M = int(parts[1]) if len(parts) > 1 else 2048
+        N, K = (int(parts[2]), int(parts[3])) if len(parts) > 3 else (13824, 5120)
+        W = S.latent_weights(N, K, 0, device="cuda")
         packed, gamma = B.quantize_weights(W)
-        X = S.activations(M, 5120, 0, device="cuda")
-        ws = B.alloc_workspace(M, 13824, 5120)
+        X = S.activations(M, K, 0, device="cuda")
+        ws = B.alloc_workspace(M, N, K)
         for _ in range(3):
-            B.forward(packed, gamma, X, 13824, workspace=ws)
+            B.forward(packed, gamma, X, N, workspace=ws)
         torch.cuda.synchronize()
-        ms = time_forward_calls(lambda: B.forward(packed, gamma, X, 13824, workspace=ws), 20)
-        ops = 2 * M * 13824 * 5120
+        ms = time_forward_calls(lambda: B.forward(packed, gamma, X, N, workspace=ws), 20)
+        ops = 2 * M * N * K
         print(json.dumps({"case": name, "int_ops_per_launch": ops, "forward_ms": round(ms, 4),
                           "TOPS": round(ops / ms / 1e9, 1)}))
     elif name.startswith("quantiser"):
@@ -924,7 +926,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-extras", action="store_true")
-    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | decode-trits[:M[:copies]] | prefill[:M] | quantiser[:norm|:swiglu] | peak[:iters]) and exit")
+    ap.add_argument("--profile-case", default=None, help="run a small fixed case (decode[:M[:copies]] | decode-trits[:M[:copies]] | prefill[:M[:N:K]] | quantiser[:norm|:swiglu] | peak[:iters]) and exit")
     args = ap.parse_args()
     if args.profile_case:
         profile_case(args.profile_case)
