@@ -296,6 +296,21 @@ def test_forward_prefill_shapes(oracle, M, K, N, seed):
     assert same == 1.0
 
 
+def _ragged_shapes(seed, count, m_range):
+    """Seeded shapes with ragged M, K and N (K and N multiples of 16, the library's rule)."""
+    rng = np.random.default_rng(seed)
+    return [(int(rng.integers(m_range[0], m_range[1] + 1)), 16 * int(rng.integers(1, 260)), 16 * int(rng.integers(1, 130)), 100 + i)
+            for i in range(count)]
+
+
+# (the last two: several CTA tiles per CTA, i.e. both accumulator buffers in turn and rings that wrap, with short tiles)
+@pytest.mark.parametrize("M,K,N,seed", _ragged_shapes(17, 12, (17, 64)) + [(40, 1024, 65536, 200), (33, 256, 131072, 201)])
+def test_forward_weight_stationary_kernel_ragged_shapes(oracle, M, K, N, seed):
+    """17 to 64 tokens (MMAs of 32, 48 and 64 columns), K from one ragged k block to 32, N from one partly filled tile up."""
+    same = run_forward_case(oracle, M, K, N, seed, frac=0.01, scale=20.0, big=True)
+    assert same == 1.0
+
+
 def test_forward_empty_batch_and_errors():
     W = S.latent_weights(16, 16, 0)
     packed, gamma = B.quantize_weights(dev(W))
