@@ -19,9 +19,10 @@ def _lib():
     torch.cuda.synchronize()
 
 
-@pytest.mark.parametrize("M", [1, 12, 40])
+@pytest.mark.parametrize("M", [1, 12, 40, 130])
 def test_sequence_replays_in_a_cuda_graph(M):
-    """1 and 12 tokens: the weight-streaming kernels; 40 tokens: the table-driven tensor-core GEMM."""
+    """1 and 12 tokens: the weight-streaming kernels; 40 tokens: the table-driven weight-stationary tensor-core kernel;
+    130 tokens: the table-driven tensor-core GEMM."""
     shapes = S.decoder_layer_shapes(512, 1408, kv_dim=128)
     layers = []
     for mi, sh in enumerate(shapes * 2):
