@@ -9,15 +9,16 @@
 //   producer threads: four, each every fourth k block (an issued copy costs its thread 100 to 150 cycles): TMA loads 64
 //                     rows of int8 activations (128-byte swizzle, the MMA's B operand) and 8 KiB of packed weights (four
 //                     row blocks x two column tiles, 128-byte swizzle) into a ring of stages;
-//   expander warps  : sixteen, one per (lane quarter of tensor memory, slot of the A ring): every thread loads ONE
-//                     16-byte piece of packed words per MMA k step, keeps the fields of four output rows with one mask
+//   expander warps  : sixteen, one per (lane quarter of tensor memory, feature block, parity of the k block): every thread
+//                     loads ONE 16-byte piece of packed words per MMA k step, keeps the fields of four output rows with one mask
 //                     each (the byte is code * 4^f) and writes them with tcgen05.st.16x256b straight into TENSOR memory
 //                     as the A operand of the MMAs (lane = output row, 32 columns = the k block): the expanded weights
 //                     never touch shared memory, and no packed byte is fetched twice by a warp (store_unit below);
 //   MMA threads     : four, one per (feature block of 128, parity of the k block), because one thread issues a
 //                     tcgen05.mma only every 110 cycles whatever its size, and an MMA of 128 x 64 x 32 takes 36: each
 //                     issues the four MMAs of its k blocks (A from tensor memory, B from the stage) and commits to the
-//                     barrier that frees the slot of the A ring.  The two threads of a feature block add into the SAME
+//                     barrier that frees the unit of the A ring (the MMAs' N is 32, 48 or 64: the largest M of the launch
+//                     rounded up to 16).  The two threads of a feature block add into the SAME
 //                     accumulator, which the epilogue left zeroed, so that no MMA has to be the first (measured on
 //                     B200: sums of MMAs issued by four threads into one accumulator are exact);
 //   epilogue warps  : four: tcgen05.ld the finished sums (lane = feature, column = token), undo the 4^f of their row
