@@ -153,7 +153,8 @@ bitlinear_status bitlinear_swiglu_quantize_acts(const void *gate, const void *up
  *   Y               out  bf16 [M, N]
  *   workspace       scratch, >= bitlinear_workspace_bytes(M, N, K); contents undefined afterwards.
  *                   Two calls that run concurrently must not share a workspace.
- * M <= 16 runs the weight-streaming decode kernel, larger M the tensor-core GEMM.
+ * M <= 16 runs the weight-streaming decode kernel, 17 <= M <= 64 the weight-stationary tensor-core kernel, larger M the
+ * tensor-core GEMM.
  */
 bitlinear_status bitlinear_forward(const void *packed, const float *gamma, const void *X,
                                    int64_t M, int64_t K, int64_t N, void *Y,
