@@ -106,6 +106,7 @@ struct Barriers {
     uint64_t acc_full[2];        // accumulator(s) of a tile complete
     uint64_t acc_empty[2];       // drained by the epilogue
     uint64_t epilogue_met;       // rendezvous of the four epilogue warps (after a contribution)
+    uint64_t last_full;          // the accumulators of the CTA's last unit are complete (for the warps that only help there)
     uint64_t fetched[4][kFetchBufs]; // finisher: a piece of a contribution has landed in an epilogue warp's buffer
     uint32_t tmem_base;
     int abort_flag;
@@ -186,6 +187,12 @@ struct UnitWalker {
             end = (long long)(blockIdx.x + 1) * sc.total_kb / (long long)gridDim.x;
         }
     }
+    // whether another unit follows the one `next` returned last
+    __device__ bool more() const
+    {
+        if (sc.stream_k == 2) return false;
+        return sc.stream_k ? pos < end : next_tile < sc.n_tiles;
+    }
     // the next unit and its matmul; false: none is left
     __device__ bool next(Unit &u, const GemmProblem *&g)
     {
@@ -241,6 +248,83 @@ struct UnitWalker {
     }
 };
 
+// Shift, subtract, scale, round and store the 32 sums `v` of chunk c (features n0 + 32 c ..) of token t.
+__device__ __forceinline__ void emit_chunk(const Params &p, int n0, const uint32_t (&v)[32], int c, int t, int rowsum, float scale)
+{
+    const int n = n0 + c * 32;
+    // output row n + i carries the factor 4^f, f = ((n + i) % 64) / 16 = 2 (c % 2) + i / 16
+    const int sh_lo = 4 * (c & 1), sh_hi = sh_lo + 2;
+    int a[32];
+#pragma unroll
+    for (int i = 0; i < 32; ++i) a[i] = ((int)v[i] >> (i < 16 ? sh_lo : sh_hi)) - rowsum;
+    if (t >= p.M) return;
+    if (p.out_i32) {
+        int32_t *dst = reinterpret_cast<int32_t *>(p.out) + (size_t)t * p.N + n;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4)
+            if (n + i < p.N) *reinterpret_cast<int4 *>(dst + i) = make_int4(a[i], a[i + 1], a[i + 2], a[i + 3]);
+    } else {
+        __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)t * p.N + n;
+#pragma unroll
+        for (int i = 0; i < 32; i += 16) { // N is a multiple of 16: 16 features are in or out together
+            if (n + i < p.N) {
+                uint32_t o[8];
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    const float x0 = __fmul_rn((float)a[i + 2 * h], scale);
+                    const float x1 = __fmul_rn((float)a[i + 2 * h + 1], scale);
+                    const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
+                    o[h] = *reinterpret_cast<const uint32_t *>(&pr);
+                }
+                if (p.out_32b_aligned) {
+                    st_global_v8(dst + i, o);
+                } else {
+                    *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
+                    *reinterpret_cast<uint4 *>(dst + i + 8) = make_uint4(o[4], o[5], o[6], o[7]);
+                }
+            }
+        }
+    }
+}
+
+// The sum of q and the scale gamma * beta_t / Q_b of token t (past M: zeros).
+__device__ __forceinline__ void token_terms(const Params &p, float gamma, int t, int &rowsum, float &scale)
+{
+    rowsum = 0;
+    scale = 0.0f;
+    if (t < p.M) {
+        rowsum = p.rowsum[t];
+        if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), p.qb);
+    }
+}
+
+// Jobs first, first + step, ... of a tile whose sums are complete in tensor memory (nothing to add): this warp's lane
+// quarter q of (token tile, pair of 32-feature chunks).  The epilogue warps run this for every whole tile; for the last
+// tile of a CTA, whose epilogue nothing overlaps, the two expander warps of the same lane quarter take two thirds of the jobs.
+template <int MT>
+__device__ __forceinline__ void finish_whole_jobs(const Params &p, uint32_t tmem_base, int q, int lane, int buf, int m0, int n0,
+                                                  int halves, int first, int step)
+{
+    constexpr int kPairs = BN / 32 / (int)kFetchChunks;
+    const float gamma = p.out_i32 ? 0.0f : *p.gamma;
+#pragma unroll 1
+    for (int jb = first; jb < halves * kPairs; jb += step) {
+        const int half = jb / kPairs, c0 = (jb % kPairs) * (int)kFetchChunks;
+        const uint32_t acc_col = (uint32_t)((buf * MT + half) * BN);
+        const int t = m0 + half * BM + 32 * q + lane;
+        int rowsum;
+        float scale;
+        token_terms(p, gamma, t, rowsum, scale);
+        uint32_t v[kFetchChunks][32];
+#pragma unroll
+        for (int cc = 0; cc < (int)kFetchChunks; ++cc)
+            tmem_ld_32x32(tmem_base + ((uint32_t)(32 * q) << 16) + acc_col + (uint32_t)((c0 + cc) * 32), v[cc]);
+        tmem_ld_wait();
+#pragma unroll
+        for (int cc = 0; cc < (int)kFetchChunks; ++cc) emit_chunk(p, n0, v[cc], c0 + cc, t, rowsum, scale);
+    }
+}
+
 template <int MT, bool kTable>
 __global__ void __launch_bounds__(kThreads, 1)
 prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *__restrict__ table, int n_problems,
@@ -272,6 +356,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             mbar_init(smem_u32(&bars->acc_empty[b]), 4);
         }
         mbar_init(smem_u32(&bars->epilogue_met), 4);
+        mbar_init(smem_u32(&bars->last_full), 1);
         for (int w = 0; w < 4; ++w)
             for (int b = 0; b < kFetchBufs; ++b) mbar_init(smem_u32(&bars->fetched[w][b]), 1);
         bars->abort_flag = 0;
@@ -392,6 +477,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                     }
                 }
                 if (ok) mma_commit(smem_u32(&bars->acc_full[buf]));
+                if (ok && !walk.more()) mma_commit(smem_u32(&bars->last_full));
             }
         }
     } else if (warp >= kFirstExpanderWarp) {
@@ -414,8 +500,10 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
         RingPos pos, reader; // reader: the k block kBSlots steps back, whose MMAs read the expanded tile written next
         bool ok = true;
         Unit unit;
-        const GemmProblem *gp;
+        const GemmProblem *gp = nullptr;
+        uint32_t n_units = 0;
         while (ok && walk.next(unit, gp)) {
+            ++n_units;
             const int kb_end = unit.kb1;
             for (int kb = unit.kb0; kb < kb_end; ++kb, pos.advance(n_stages)) {
                 const int s = pos.s, b = (int)(pos.it % kBSlots);
@@ -461,6 +549,21 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 if (lane == 0) mbar_arrive(smem_u32(&bars->expanded[b]));
             }
         }
+        // The CTA's last unit, when it is a whole tile: this warp takes a third of the jobs of its lane quarter (see the
+        // epilogue warps below, which take the jobs 0, 3, 6, ...).
+        if (ok && n_units > 0 && unit.kind == kWholeTile) {
+            const Params &p = gp->p;
+            const int local = unit.tile - p.tile_begin;
+            const int m0 = (local % p.tiles_m) * (MT * BM), n0 = (local / p.tiles_m) * BN;
+            const int halves = (MT == 2 && m0 + BM < p.M) ? 2 : 1;
+            const int buf = (int)((n_units - 1) % kAccBufs);
+            // (not `acc_full`: this warp may be several tiles ahead of the MMAs, and a wait on a phase's parity only
+            // works for a waiter that is at most one phase behind)
+            if (mbar_wait_bounded(smem_u32(&bars->last_full), 0, abort_flag, hooks.limit_us)) {
+                tc_fence_after_sync();
+                finish_whole_jobs<MT>(p, tmem_base, warp & 3, lane, buf, m0, n0, halves, 1 + (ew >> 2), 3);
+            }
+        }
     } else {
         // epilogue: warp w may touch TMEM lanes 32*(w % 4) .. +31
         const int q = warp & 3;
@@ -481,54 +584,9 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             if (!mbar_wait_bounded(smem_u32(&bars->acc_full[buf]), parity, abort_flag, hooks.limit_us)) break;
             tc_fence_after_sync();
 
-            // shift, subtract, scale, round and store the 32 sums `v` of chunk c (features n0 + 32 c ..) of token t
-            auto emit = [&](const uint32_t (&v)[32], int c, int t, int rowsum, float scale) {
-                const int n = n0 + c * 32;
-                // output row n + i carries the factor 4^f, f = ((n + i) % 64) / 16 = 2 (c % 2) + i / 16
-                const int sh_lo = 4 * (c & 1), sh_hi = sh_lo + 2;
-                int a[32];
-#pragma unroll
-                for (int i = 0; i < 32; ++i) a[i] = ((int)v[i] >> (i < 16 ? sh_lo : sh_hi)) - rowsum;
-                if (t >= p.M) return;
-                if (p.out_i32) {
-                    int32_t *dst = reinterpret_cast<int32_t *>(p.out) + (size_t)t * p.N + n;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 4)
-                        if (n + i < p.N) *reinterpret_cast<int4 *>(dst + i) = make_int4(a[i], a[i + 1], a[i + 2], a[i + 3]);
-                } else {
-                    __nv_bfloat16 *dst = reinterpret_cast<__nv_bfloat16 *>(p.out) + (size_t)t * p.N + n;
-#pragma unroll
-                    for (int i = 0; i < 32; i += 16) { // N is a multiple of 16: 16 features are in or out together
-                        if (n + i < p.N) {
-                            uint32_t o[8];
-#pragma unroll
-                            for (int h = 0; h < 8; ++h) {
-                                const float x0 = __fmul_rn((float)a[i + 2 * h], scale);
-                                const float x1 = __fmul_rn((float)a[i + 2 * h + 1], scale);
-                                const __nv_bfloat162 pr = __floats2bfloat162_rn(x0, x1);
-                                o[h] = *reinterpret_cast<const uint32_t *>(&pr);
-                            }
-                            if (p.out_32b_aligned) {
-                                st_global_v8(dst + i, o);
-                            } else {
-                                *reinterpret_cast<uint4 *>(dst + i) = make_uint4(o[0], o[1], o[2], o[3]);
-                                *reinterpret_cast<uint4 *>(dst + i + 8) = make_uint4(o[4], o[5], o[6], o[7]);
-                            }
-                        }
-                    }
-                }
-            };
             // the token whose sums this thread's TMEM lane holds (past M: none)
             auto token_of_lane = [&](int half) {
                 return m0 + half * BM + 32 * q + lane;
-            };
-            auto token_scale = [&](int t, int &rowsum, float &scale) {
-                rowsum = 0;
-                scale = 0.0f;
-                if (t < p.M) {
-                    rowsum = p.rowsum[t];
-                    if (!p.out_i32) scale = __fdiv_rn(__fmul_rn(gamma, p.beta[t]), p.qb);
-                }
             };
             // the 4 KiB that hold this warp's 32 x 32 sums of chunk c of token tile `half` in the slot of CTA `cta` (the
             // chunks of a warp follow each other)
@@ -544,7 +602,10 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
             constexpr int kPairs = BN / 32 / (int)kFetchChunks;
             const int n_jobs_tile = halves * kPairs;
             const bool split = unit.kind == kSplit;
-            const int job_start = split ? unit.split_r : 0, job_stride = split ? unit.split_s : 1;
+            // (the last unit of the CTA, when it is a whole tile: the two expander warps of this lane quarter, idle by then,
+            // take the jobs 1, 4, 7, ... and 2, 5, 8, ...: nothing overlaps this epilogue)
+            const bool shared_last = unit.kind == kWholeTile && !walk.more();
+            const int job_start = split ? unit.split_r : 0, job_stride = split ? unit.split_s : (shared_last ? 3 : 1);
             const int n_contrib = unit.kind == kFinisher ? unit.last_contributor - (int)blockIdx.x : (split ? unit.split_s - 1 : 0);
             // the CTA whose slot holds the j-th contribution
             auto contributor = [&](int j) {
@@ -620,7 +681,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 const int t = token_of_lane(half);
                 int rowsum;
                 float scale;
-                token_scale(t, rowsum, scale);
+                token_terms(p, gamma, t, rowsum, scale);
                 uint32_t v[kFetchChunks][32];
 #pragma unroll
                 for (int cc = 0; cc < (int)kFetchChunks; ++cc)
@@ -651,7 +712,7 @@ prefill_gemm_kernel(const __grid_constant__ GemmProblem one, const GemmProblem *
                 }
                 if (!alive) break;
 #pragma unroll
-                for (int cc = 0; cc < (int)kFetchChunks; ++cc) emit(v[cc], c0 + cc, t, rowsum, scale);
+                for (int cc = 0; cc < (int)kFetchChunks; ++cc) emit_chunk(p, n0, v[cc], c0 + cc, t, rowsum, scale);
             }
             if (!alive) break;
             tc_fence_before_sync();
