@@ -143,10 +143,12 @@ constexpr uint32_t kFetchChunks = 2;                    // chunks of 32 features
 constexpr uint32_t kFetchBytes = kFetchChunks * 4096;   // 8 KiB
 static_assert(4 * kFetchBufs * kFetchBytes <= 3 * 64 * 1024, "the fetch buffers lie inside the idle rings");
 
-// Byte offset of 16-byte piece `piece` (of 8) of lane `lane` inside a chunk of 32 lanes x 128 bytes: pieces are
-// swizzled by lane so that 16-byte shared-memory loads of a warp are free of bank conflicts.  The slots in global memory
-// have this layout (they reach shared memory by bulk copies, as they are).
-__device__ __forceinline__ uint32_t slot_piece(int lane, int piece) { return (uint32_t)(lane * 128 + ((piece ^ (lane & 7)) << 4)); }
+// Byte offset of 16-byte piece `piece` (of 8) of lane `lane` inside a chunk of 32 lanes x 128 bytes: piece-major, so that
+// the 32 lanes of a warp write (global memory) and read (shared memory, after the bulk copy) 512 consecutive bytes per
+// instruction -- four full lines per store (lane-major rows made every store instruction touch 32 lines, 16 bytes of
+// each), no bank conflicts per load.  The slots in global memory have this layout (they reach shared memory by bulk
+// copies, as they are).
+__device__ __forceinline__ uint32_t slot_piece(int lane, int piece) { return (uint32_t)(piece * 512 + lane * 16); }
 
 enum UnitKind { kWholeTile = 0, kContribution = 1, kFinisher = 2, kSplit = 3 };
 
